@@ -1,0 +1,197 @@
+/*
+ * flexdraft.h -- C ABI of the FlexDraft decode-step hot path for NVIDIA B200 (sm_100a).
+ *
+ * One decode step of FlexDraft's parallel draft-and-verify decoding (paper Sec. 4.1,
+ * "Inference"; Sec. 3 for the verification rule) is, per attention layer and per
+ * sequence b, the attention of a query block
+ *
+ *        [ bonus token | k_b draft tokens | M_b mask tokens ]
+ *          \____ C_b = k_b + 1 candidate rows ____/
+ *
+ * against that sequence's paged KV cache under the hybrid mask, followed, once per
+ * step, by lossless verification of the drafts and by the commit / rollback of the KV
+ * positions written for this block.  This library exports exactly those three
+ * operations.  Everything runs in hand-written CUDA kernels; there is no CPU fallback.
+ *
+ * Conventions (all entry points)
+ *   - "device pointer": memory on the GPU that is current when fd_create() ran, owned
+ *     by the caller.  "host pointer": ordinary host memory, owned by the caller.
+ *   - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream) and ordered by it.  Calls that share one fd_ctx
+ *     must be issued on one stream, or be ordered by the caller: they share the context's
+ *     scratch memory.
+ *   - The hot calls (fd_attn_draft_verify, fd_verify_accept, fd_kv_commit) never allocate
+ *     and never synchronise; all scratch memory is sized by fd_create() from fd_config.
+ *   - Errors the host can see (NULL pointer, size beyond the configured maximum,
+ *     unsupported shape, misaligned pointer) return a code and launch nothing.
+ *   - Errors only the device can see (lengths that contradict each other, a page id
+ *     outside the pool, ...) never trap: the kernels skip the work, write a defined
+ *     value (documented per call) and OR a FD_DEV_* bit into a sticky status word that
+ *     fd_last_device_status() reads.
+ *
+ * Notation: B sequences; Hq q-heads, Hkv kv-heads, G = Hq/Hkv; d = head_dim; P = page_size
+ * (16 tokens); V = vocab.  n_b = prefix_lens[b]; Lq_b = q_lens[b]; M_b = n_mask[b];
+ * C_b = Lq_b - M_b; kv_len_b = n_b + Lq_b; T = sum_b Lq_b; R = sum_b C_b.
+ */
+#ifndef FLEXDRAFT_H
+#define FLEXDRAFT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fd_ctx fd_ctx; /* opaque; owns scratch memory and the device status word */
+
+typedef enum {
+    FD_OK = 0,
+    FD_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, size beyond fd_config maximum */
+    FD_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels implement */
+    FD_ERR_WORKSPACE = 3,     /* scratch memory could not be allocated */
+    FD_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
+    FD_ERR_DEVICE_STATUS = 5  /* reserved */
+} fd_status;
+
+/* Bits of the sticky device status word. */
+enum {
+    FD_DEV_BAD_LENGTHS = 1,   /* lengths negative, n_mask > q_len, q_len > max_q_len, kv_len beyond the
+                                 page table, or row totals that do not match the call's row count */
+    FD_DEV_BAD_PAGE = 2,      /* a page id needed by a sequence is outside [0, num_pages) */
+    FD_DEV_TIMEOUT = 4,       /* a bounded device-side wait ran out; the kernel returned early */
+    FD_DEV_BAD_ACCEPT = 8     /* fd_kv_commit: accepted_len[b] >= q_lens[b] */
+};
+
+/* Which attention kernel fd_attn_draft_verify launches. */
+enum {
+    FD_ATTN_AUTO = 0,         /* tensor-core kernel when the shape allows it, else the SIMT kernel */
+    FD_ATTN_SIMT = 1,         /* CUDA-core split-KV kernel (any supported shape) */
+    FD_ATTN_TCGEN05 = 2       /* tcgen05 / TMEM / TMA split-KV kernel (head_dim 64 or 128) */
+};
+
+typedef struct {
+    int n_q_heads;            /* Hq */
+    int n_kv_heads;           /* Hkv, divides Hq */
+    int head_dim;             /* d: 64 or 128 */
+    int page_size;            /* P: 16 */
+    int vocab;                /* V >= 1 */
+    int max_batch;            /* largest B of any call */
+    int max_q_len;            /* largest Lq_b; G * max_q_len <= 128 */
+    int max_pages_per_seq;    /* row length of page_table */
+    float softmax_scale;      /* 0 selects 1/sqrt(d) */
+    int attn_path;            /* FD_ATTN_* */
+} fd_config;
+
+/* Create a context on the current CUDA device.  Allocates all scratch memory (a few tens
+ * of MB).  *ctx is NULL on failure. */
+fd_status fd_create(fd_ctx** ctx, const fd_config* cfg);
+
+/* Free a context.  Synchronises the device first.  NULL is accepted. */
+fd_status fd_destroy(fd_ctx* ctx);
+
+/*
+ * Attention of one target forward pass over the ragged query blocks (Sec. 4.1,
+ * "Inference"; hybrid mask of Sec. 4.1 and the Fig. 2 caption).  For sequence b, q-head
+ * h, block row i:
+ *
+ *     out[row0_b + i, h, :] = sum_{j in A_b(i)} softmax_j( scale * <q[row0_b+i, h], K_b[j, h/G]> ) V_b[j, h/G]
+ *
+ *     A_b(i), i <  C_b (candidate row): { j < n_b } U { n_b + t : t <= i }        causal; no mask token
+ *     A_b(i), i >= C_b (mask row):      { j < kv_len_b }                          prefix, all candidates,
+ *                                                                                 whole mask block
+ *     K_b[j], V_b[j] = kv_cache[ page_table[b][j / P], 0 | 1, h / G, j % P, : ]
+ *
+ * The caller has already written K/V of all Lq_b query tokens (candidates first, then
+ * mask tokens) at logical positions n_b .. n_b + Lq_b - 1 ("append, then attend"), with
+ * positional encoding and norms applied.  Slots that no valid token owns may hold any
+ * bit pattern (NaN included); they never influence the result.
+ *
+ *   batch          B, 0 <= B <= max_batch (B = 0 is a no-op)
+ *   total_q_rows   T; must equal sum_b q_lens[b]
+ *   q              device, [T, Hq, d] bf16, 16-byte aligned, sequence-major rows
+ *   kv_cache       device, [num_pages, 2, Hkv, P, d] bf16, 128-byte aligned
+ *   num_pages      size of the page pool
+ *   page_table     device, [B, max_pages_per_seq] int32; entries beyond ceil(kv_len_b/P) are ignored
+ *   prefix_lens, q_lens, n_mask   device, [B] int32
+ *   out            device, [T, Hq, d] bf16, 16-byte aligned; fully overwritten
+ *   stream         cudaStream_t
+ *
+ * Device-detected errors: a sequence with a page id outside the pool gets zeros in its
+ * out rows (FD_DEV_BAD_PAGE); inconsistent lengths zero all T rows (FD_DEV_BAD_LENGTHS).
+ * Arithmetic: bf16 inputs, fp32 scores / softmax / accumulation, bf16 output.
+ */
+fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
+                               const void* q, const void* kv_cache, int num_pages,
+                               const int32_t* page_table, const int32_t* prefix_lens,
+                               const int32_t* q_lens, const int32_t* n_mask,
+                               void* out, void* stream);
+
+/*
+ * Lossless verification at temperature 0 (Sec. 3: draft tokens are accepted up to the
+ * first rejection, the token produced there is the bonus token, committed length
+ * L_acc = r_acc + 1).  With am[r] = argmax_v logits[r, v] (larger value wins, equal
+ * values: lower index wins; inputs must be NaN-free) and r0_b the first candidate row of
+ * sequence b:
+ *
+ *     accepted_len[b] = number of leading j < k_b with am[r0_b + j] == draft_tokens[r0_b + j + 1]
+ *     bonus_token[b]  = am[r0_b + accepted_len[b]]
+ *
+ * so 0 <= accepted_len[b] <= k_b = C_b - 1 (this is the paper's r_acc).  A sequence with
+ * C_b = 0 gets accepted_len = bonus_token = -1.
+ *
+ *   total_cand_rows  R; must equal sum_b (q_lens[b] - n_mask[b])
+ *   logits           device, [R, V] fp32, candidate rows only, sequence-major
+ *   draft_tokens     device, [R] int32: the token fed at each candidate row (row 0 of a
+ *                    sequence is the previous bonus token and is never compared)
+ *   q_lens, n_mask   device, [B] int32
+ *   accepted_len, bonus_token   device, [B] int32, overwritten
+ *
+ * Inconsistent lengths: every accepted_len / bonus_token is set to -1 (FD_DEV_BAD_LENGTHS).
+ */
+fd_status fd_verify_accept(fd_ctx* ctx, int batch, int total_cand_rows,
+                           const float* logits, const int32_t* draft_tokens,
+                           const int32_t* q_lens, const int32_t* n_mask,
+                           int32_t* accepted_len, int32_t* bonus_token, void* stream);
+
+/*
+ * KV commit / rollback.  The paper implies it (the clean-prefix KV cache is reused by
+ * every later step, Sec. 4.1 "Inference" and Sec. 4.3 "Decoupled execution"; mask tokens
+ * are invisible to clean tokens) without spelling it out; the reading implemented: the
+ * bonus row and the accepted drafts stay, every later position of the block (rejected
+ * drafts, mask tokens) is dropped by truncating the length and releasing the pages that
+ * no kept token lives in.  For b ascending, with new_len = n_b + accepted_len[b] + 1:
+ *
+ *     for p = ceil(new_len / P) .. ceil((n_b + Lq_b) / P) - 1 ascending:
+ *         append page_table[b][p] to freed_pages; page_table[b][p] = -1
+ *     prefix_lens[b] = new_len
+ *
+ * KV bytes are not touched.  Sequences with accepted_len[b] < 0 are left unchanged; one with
+ * accepted_len[b] >= q_lens[b] is left unchanged and raises FD_DEV_BAD_ACCEPT.
+ *
+ *   page_table    device, [B, max_pages_per_seq] int32, in/out
+ *   prefix_lens   device, [B] int32, in/out
+ *   q_lens, accepted_len   device, [B] int32
+ *   freed_pages   device, int32, capacity >= B * (ceil(max_q_len / P) + 1), packed output
+ *   n_freed       device, [1] int32, output
+ */
+fd_status fd_kv_commit(fd_ctx* ctx, int batch, int32_t* page_table, int32_t* prefix_lens,
+                       const int32_t* q_lens, const int32_t* accepted_len,
+                       int32_t* freed_pages, int32_t* n_freed, void* stream);
+
+/* Read and clear the sticky device status word (an OR of FD_DEV_* bits) into *code (host
+ * pointer).  Synchronises `stream` first. */
+fd_status fd_last_device_status(fd_ctx* ctx, int32_t* code, void* stream);
+
+/* Which attention kernel the context resolved to: FD_ATTN_SIMT or FD_ATTN_TCGEN05. */
+int fd_attn_path(const fd_ctx* ctx);
+
+/* Number of CUDA kernels this library has launched through `ctx` since fd_create. */
+int64_t fd_launch_count(const fd_ctx* ctx);
+
+/* Static string for a status code. */
+const char* fd_status_string(fd_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLEXDRAFT_H */

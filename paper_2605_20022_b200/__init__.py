@@ -1,0 +1,145 @@
+"""Python binding of libflexdraft (argument marshalling only).
+
+Every function has the name and the argument order of its C entry point in
+``include/flexdraft.h``; tensors are torch CUDA tensors whose ``data_ptr()`` is
+handed through unchanged.  All arithmetic runs inside the library's CUDA kernels.
+If the library has not been built, or no CUDA device is present, the calls raise:
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+from . import _build
+
+FD_OK = 0
+FD_ERR_INVALID_ARG, FD_ERR_UNSUPPORTED, FD_ERR_WORKSPACE, FD_ERR_CUDA, FD_ERR_DEVICE_STATUS = 1, 2, 3, 4, 5
+FD_DEV_BAD_LENGTHS, FD_DEV_BAD_PAGE, FD_DEV_TIMEOUT, FD_DEV_BAD_ACCEPT = 1, 2, 4, 8
+FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
+
+EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
+           "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string"]
+
+
+class fd_config(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int), ("n_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int),
+                ("page_size", ctypes.c_int), ("vocab", ctypes.c_int), ("max_batch", ctypes.c_int),
+                ("max_q_len", ctypes.c_int), ("max_pages_per_seq", ctypes.c_int),
+                ("softmax_scale", ctypes.c_float), ("attn_path", ctypes.c_int)]
+
+
+class FlexDraftError(RuntimeError):
+    def __init__(self, where: str, code: int):
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.SO
+
+
+def load() -> ctypes.CDLL:
+    """dlopen libflexdraft.so (built in-tree by ``_build.build()``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_build.SO):
+            raise FileNotFoundError(f"{_build.SO} is not built: run `python -m paper_2605_20022_b200._build`")
+        lib = ctypes.CDLL(_build.SO)
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        lib.fd_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(fd_config)]
+        lib.fd_destroy.argtypes = [vp]
+        lib.fd_attn_draft_verify.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp]
+        lib.fd_verify_accept.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_kv_commit.argtypes = [vp, ci, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+        lib.fd_attn_path.argtypes = [vp]
+        lib.fd_launch_count.argtypes = [vp]
+        lib.fd_launch_count.restype = ctypes.c_int64
+        lib.fd_status_string.argtypes = [ci]
+        lib.fd_status_string.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().fd_status_string(int(code)).decode()
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _check(where: str, code: int, raise_on_error: bool) -> int:
+    if code != FD_OK and raise_on_error:
+        raise FlexDraftError(where, code)
+    return code
+
+
+def fd_create(n_q_heads: int, n_kv_heads: int, head_dim: int, vocab: int, max_batch: int, max_q_len: int,
+              max_pages_per_seq: int, page_size: int = 16, softmax_scale: float = 0.0,
+              attn_path: int = FD_ATTN_AUTO) -> int:
+    """Returns the opaque context handle (an integer address)."""
+    cfg = fd_config(n_q_heads, n_kv_heads, head_dim, page_size, vocab, max_batch, max_q_len, max_pages_per_seq,
+                    softmax_scale, attn_path)
+    ctx = ctypes.c_void_p()
+    code = load().fd_create(ctypes.byref(ctx), ctypes.byref(cfg))
+    _check("fd_create", code, True)
+    return ctx.value
+
+
+def fd_destroy(ctx: int) -> None:
+    load().fd_destroy(ctx)
+
+
+def fd_attn_draft_verify(ctx, batch, total_q_rows, q, kv_cache, num_pages, page_table, prefix_lens, q_lens, n_mask,
+                         out, stream=None, raise_on_error=True) -> int:
+    code = load().fd_attn_draft_verify(ctx, batch, total_q_rows, _ptr(q), _ptr(kv_cache), num_pages,
+                                       _ptr(page_table), _ptr(prefix_lens), _ptr(q_lens), _ptr(n_mask), _ptr(out),
+                                       _stream(stream))
+    return _check("fd_attn_draft_verify", code, raise_on_error)
+
+
+def fd_verify_accept(ctx, batch, total_cand_rows, logits, draft_tokens, q_lens, n_mask, accepted_len, bonus_token,
+                     stream=None, raise_on_error=True) -> int:
+    code = load().fd_verify_accept(ctx, batch, total_cand_rows, _ptr(logits), _ptr(draft_tokens), _ptr(q_lens),
+                                   _ptr(n_mask), _ptr(accepted_len), _ptr(bonus_token), _stream(stream))
+    return _check("fd_verify_accept", code, raise_on_error)
+
+
+def fd_kv_commit(ctx, batch, page_table, prefix_lens, q_lens, accepted_len, freed_pages, n_freed, stream=None,
+                 raise_on_error=True) -> int:
+    code = load().fd_kv_commit(ctx, batch, _ptr(page_table), _ptr(prefix_lens), _ptr(q_lens), _ptr(accepted_len),
+                               _ptr(freed_pages), _ptr(n_freed), _stream(stream))
+    return _check("fd_kv_commit", code, raise_on_error)
+
+
+def fd_last_device_status(ctx, stream=None) -> int:
+    code = ctypes.c_int32(0)
+    _check("fd_last_device_status", load().fd_last_device_status(ctx, ctypes.byref(code), _stream(stream)), True)
+    return code.value
+
+
+def fd_attn_path(ctx) -> int:
+    return load().fd_attn_path(ctx)
+
+
+def fd_launch_count(ctx) -> int:
+    return int(load().fd_launch_count(ctx))

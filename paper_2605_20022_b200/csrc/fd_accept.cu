@@ -1,0 +1,132 @@
+// Greedy verification: vocab argmax of every candidate row fused with the accept scan.
+//
+// The [R, V] fp32 logits are swept once.  Each CTA reduces one 8192-logit chunk of one row
+// to a 64-bit key (order-preserving image of the float in the high word, ~index in the low
+// word, so an unsigned max picks the larger value and, on equal values, the lower index)
+// and folds it into the row's running key with atomicMax -- an exact, order-independent
+// reduction, so the result is deterministic.  The CTA that finishes last (a ticket counter,
+// no spinning) runs the per-sequence accept scan and re-zeroes the keys for the next call.
+#include "fd_internal.cuh"
+
+namespace fd {
+
+__device__ inline unsigned long long make_key(float v, unsigned idx) {
+    v += 0.0f;  // -0.0 -> +0.0: they compare equal, so the lower index must decide
+    unsigned u = __float_as_uint(v);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - idx);
+}
+
+__device__ inline void fold(float& bv, unsigned& bi, float v, unsigned i) {
+    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+}
+
+__global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_per_row) {
+    const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
+    const float* base = p.logits + (long long)row * p.vocab;
+    const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
+    const int tid = threadIdx.x;
+
+    float bv = -INFINITY;
+    unsigned bi = 0xffffffffu;
+    // scalar head up to the first 16-byte boundary, float4 body, scalar tail
+    const int mis = (int)((reinterpret_cast<uintptr_t>(base + c0) >> 2) & 3);
+    const int head = min(c1 - c0, (4 - mis) & 3);
+    const int nvec = (c1 - c0 - head) >> 2;
+    if (tid < head) fold(bv, bi, base[c0 + tid], c0 + tid);
+    const float4* vp = reinterpret_cast<const float4*>(base + c0 + head);
+    float4 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int e = tid + k * 256;
+        v[k] = (e < nvec) ? __ldcs(vp + e) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const unsigned i0 = c0 + head + 4 * (tid + k * 256);
+        if (tid + k * 256 < nvec) {
+            fold(bv, bi, v[k].x, i0);
+            fold(bv, bi, v[k].y, i0 + 1);
+            fold(bv, bi, v[k].z, i0 + 2);
+            fold(bv, bi, v[k].w, i0 + 3);
+        }
+    }
+    const int tail0 = c0 + head + 4 * nvec;
+    if (tail0 + tid < c1) fold(bv, bi, base[tail0 + tid], tail0 + tid);
+
+    unsigned long long key = (bi == 0xffffffffu) ? 0ull : make_key(bv, bi);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+    }
+    __shared__ unsigned long long wkey[8];
+    __shared__ bool last;
+    if ((tid & 31) == 0) wkey[tid >> 5] = key;
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll
+        for (int w = 1; w < 8; ++w) key = wkey[w] > key ? wkey[w] : key;
+        atomicMax(p.keys + row, key);
+        __threadfence();
+        last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+
+    // ---- accept scan, one CTA, after every row key is final ----
+    extern __shared__ int cu_c[];  // [B+1] first candidate row of each sequence
+    __shared__ int s_bad;
+    if (tid == 0) {
+        long long rows = 0;
+        cu_c[0] = 0;
+        for (int b = 0; b < p.batch; ++b) {
+            const int C = p.q_lens[b] - p.n_mask[b];
+            if (C < 0 || p.n_mask[b] < 0) { rows = -1; break; }
+            rows += C;
+            if (rows > p.total_rows) break;
+            cu_c[b + 1] = (int)rows;
+        }
+        s_bad = rows != p.total_rows;
+        if (s_bad) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+    }
+    __syncthreads();
+    if (s_bad) {
+        for (int b = tid; b < p.batch; b += blockDim.x) { p.accepted[b] = -1; p.bonus[b] = -1; }
+    } else {
+        // thread b walks the candidate rows of sequence b
+        for (int b = tid; b < p.batch; b += blockDim.x) {
+            const int r0 = cu_c[b], C = cu_c[b + 1] - r0;
+            if (C == 0) { p.accepted[b] = -1; p.bonus[b] = -1; continue; }
+            int a = 0;
+            int am = (int)(0xffffffffu - (unsigned)(__ldcg(p.keys + r0) & 0xffffffffull));
+            while (a < C - 1 && am == p.drafts[r0 + a + 1]) {
+                ++a;
+                am = (int)(0xffffffffu - (unsigned)(__ldcg(p.keys + r0 + a) & 0xffffffffull));
+            }
+            p.accepted[b] = a;
+            p.bonus[b] = am;
+        }
+    }
+    __syncthreads();
+    for (int r = tid; r < p.total_rows; r += blockDim.x) p.keys[r] = 0ull;
+    if (tid == 0) *p.ticket = 0u;
+}
+
+// R = 0: nothing to sweep, but the outputs are still defined (-1 everywhere).
+__global__ void accept_empty_kernel(AcceptParams p) {
+    bool bad = false;
+    for (int b = 0; b < p.batch; ++b) bad |= (p.q_lens[b] - p.n_mask[b]) != 0;
+    if (threadIdx.x == 0 && bad) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) { p.accepted[b] = -1; p.bonus[b] = -1; }
+}
+
+void launch_accept(const AcceptParams& p, cudaStream_t s) {
+    if (p.batch == 0) return;
+    if (p.total_rows == 0) { accept_empty_kernel<<<1, 256, 0, s>>>(p); return; }
+    const int chunks = (p.vocab + kAcceptChunk - 1) / kAcceptChunk;
+    accept_kernel<<<p.total_rows * chunks, 256, (p.batch + 1) * sizeof(int), s>>>(p, chunks);
+}
+
+}  // namespace fd

@@ -1,0 +1,206 @@
+// C ABI of libflexdraft: context, argument checks, launch sequencing.
+#include <math.h>
+#include <new>
+
+#include "fd_internal.cuh"
+
+struct fd_ctx {
+    fd_config cfg;
+    int device;
+    int n_sms;
+    int n_ctas;        // attention grid
+    int attn_path;     // resolved FD_ATTN_*
+    float scale_log2e;
+    // scratch (device)
+    unsigned char* pool;
+    fd::Plan plan;
+    fd::PartialView part;
+    unsigned long long* keys;
+    unsigned int* ticket;
+    int* status;
+    int max_rows;      // capacity of keys
+    void* tc_state;
+    long long launches;
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char* fd_status_string(fd_status s) {
+    switch (s) {
+        case FD_OK: return "FD_OK";
+        case FD_ERR_INVALID_ARG: return "FD_ERR_INVALID_ARG";
+        case FD_ERR_UNSUPPORTED: return "FD_ERR_UNSUPPORTED";
+        case FD_ERR_WORKSPACE: return "FD_ERR_WORKSPACE";
+        case FD_ERR_CUDA: return "FD_ERR_CUDA";
+        case FD_ERR_DEVICE_STATUS: return "FD_ERR_DEVICE_STATUS";
+    }
+    return "FD_UNKNOWN";
+}
+
+fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
+    if (!out) return FD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return FD_ERR_INVALID_ARG;
+    if (cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->vocab <= 0 || cfg->max_batch <= 0 ||
+        cfg->max_q_len <= 0 || cfg->max_pages_per_seq <= 0 || cfg->softmax_scale < 0.f)
+        return FD_ERR_INVALID_ARG;
+    if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FD_ERR_INVALID_ARG;
+    if (cfg->attn_path < FD_ATTN_AUTO || cfg->attn_path > FD_ATTN_TCGEN05) return FD_ERR_INVALID_ARG;
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return FD_ERR_UNSUPPORTED;
+    if ((long long)G * cfg->max_q_len > fd::kMaxRows) return FD_ERR_UNSUPPORTED;
+    if ((long long)cfg->max_pages_per_seq * 16 > 0x3fffffffLL || cfg->max_batch > (1 << 20)) return FD_ERR_UNSUPPORTED;
+
+    fd_ctx* c = new (std::nothrow) fd_ctx();
+    if (!c) return FD_ERR_WORKSPACE;
+    c->cfg = *cfg;
+    c->launches = 0;
+    c->tc_state = nullptr;
+    if (cudaGetDevice(&c->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
+        delete c;
+        return FD_ERR_CUDA;
+    }
+    const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+    c->scale_log2e = scale * 1.4426950408889634f;
+
+    const bool tc_ok = fd::attn_tc_supported(cfg->head_dim, G, cfg->max_q_len);
+    if (cfg->attn_path == FD_ATTN_TCGEN05 && !tc_ok) { delete c; return FD_ERR_UNSUPPORTED; }
+    c->attn_path = (cfg->attn_path == FD_ATTN_SIMT || !tc_ok) ? FD_ATTN_SIMT : FD_ATTN_TCGEN05;
+    // SIMT kernel: two 74 KB CTAs fit an SM; tensor-core kernel: one persistent CTA per SM
+    c->n_ctas = c->attn_path == FD_ATTN_SIMT ? 2 * c->n_sms : c->n_sms;
+
+    const int B = cfg->max_batch, d = cfg->head_dim;
+    const size_t slots = 2 * (size_t)c->n_ctas;
+    c->max_rows = (int)std::min<long long>((long long)B * cfg->max_q_len, 0x7fffffffLL);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t o_hdr = take(sizeof(fd::PlanHeader));
+    const size_t o_cuq = take((B + 1) * sizeof(int));
+    const size_t o_cut = take((B + 1) * sizeof(int));
+    const size_t o_ok = take(B * sizeof(int));
+    const size_t o_po = take(slots * d * fd::kMaxRows * sizeof(float));
+    const size_t o_pm = take(slots * fd::kMaxRows * sizeof(float));
+    const size_t o_pl = take(slots * fd::kMaxRows * sizeof(float));
+    const size_t o_keys = take((size_t)c->max_rows * sizeof(unsigned long long));
+    const size_t o_tick = take(sizeof(unsigned int));
+    const size_t o_stat = take(sizeof(int));
+    if (cudaMalloc(&c->pool, off) != cudaSuccess) { cudaGetLastError(); delete c; return FD_ERR_WORKSPACE; }
+    if (cudaMemset(c->pool, 0, off) != cudaSuccess) { cudaFree(c->pool); delete c; return FD_ERR_CUDA; }
+    c->plan.hdr = reinterpret_cast<fd::PlanHeader*>(c->pool + o_hdr);
+    c->plan.cu_q = reinterpret_cast<int*>(c->pool + o_cuq);
+    c->plan.cu_tiles = reinterpret_cast<int*>(c->pool + o_cut);
+    c->plan.seq_ok = reinterpret_cast<int*>(c->pool + o_ok);
+    c->part.o = reinterpret_cast<float*>(c->pool + o_po);
+    c->part.m = reinterpret_cast<float*>(c->pool + o_pm);
+    c->part.l = reinterpret_cast<float*>(c->pool + o_pl);
+    c->keys = reinterpret_cast<unsigned long long*>(c->pool + o_keys);
+    c->ticket = reinterpret_cast<unsigned int*>(c->pool + o_tick);
+    c->status = reinterpret_cast<int*>(c->pool + o_stat);
+    *out = c;
+    return FD_OK;
+}
+
+fd_status fd_destroy(fd_ctx* c) {
+    if (!c) return FD_OK;
+    cudaDeviceSynchronize();
+    fd::attn_tc_free(c->tc_state);
+    cudaFree(c->pool);
+    delete c;
+    return FD_OK;
+}
+
+int fd_attn_path(const fd_ctx* c) { return c ? c->attn_path : -1; }
+
+int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
+
+fd_status fd_attn_draft_verify(fd_ctx* c, int batch, int total_q_rows, const void* q, const void* kv_cache,
+                               int num_pages, const int32_t* page_table, const int32_t* prefix_lens,
+                               const int32_t* q_lens, const int32_t* n_mask, void* out, void* stream) {
+    if (!c || batch < 0 || total_q_rows < 0 || num_pages < 0) return FD_ERR_INVALID_ARG;
+    if (batch > c->cfg.max_batch || (long long)total_q_rows > (long long)batch * c->cfg.max_q_len)
+        return FD_ERR_INVALID_ARG;
+    if (batch == 0) return total_q_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
+    if (!page_table || !prefix_lens || !q_lens || !n_mask) return FD_ERR_INVALID_ARG;
+    if (total_q_rows > 0 && (!q || !out)) return FD_ERR_INVALID_ARG;
+    if (!kv_cache || num_pages == 0) return FD_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(kv_cache, 128) || !aligned(page_table, 4)) return FD_ERR_INVALID_ARG;
+    if ((long long)num_pages * 2 * c->cfg.n_kv_heads * 16 > 0x7fffffffLL) return FD_ERR_UNSUPPORTED;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    fd::AttnParams p;
+    p.batch = batch; p.total_q_rows = total_q_rows; p.num_pages = num_pages;
+    p.Hq = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.Hq / p.Hkv; p.d = c->cfg.head_dim;
+    p.max_pages = c->cfg.max_pages_per_seq; p.max_q_len = c->cfg.max_q_len;
+    p.scale_log2e = c->scale_log2e;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.kv = static_cast<const __nv_bfloat16*>(kv_cache);
+    p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.n_mask = n_mask;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
+
+    if (c->attn_path == FD_ATTN_TCGEN05) {
+        if (fd::attn_tc_prepare(&c->tc_state, p) != cudaSuccess) { cudaGetLastError(); return FD_ERR_CUDA; }
+    }
+    fd::launch_plan(p, s);
+    if (c->attn_path == FD_ATTN_TCGEN05) fd::launch_attn_tc(c->tc_state, p, s);
+    else fd::launch_attn_simt(p, s);
+    fd::launch_merge(p, s);
+    c->launches += 3;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const float* logits,
+                           const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask,
+                           int32_t* accepted_len, int32_t* bonus_token, void* stream) {
+    if (!c || batch < 0 || total_cand_rows < 0) return FD_ERR_INVALID_ARG;
+    if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
+    if (batch == 0) return total_cand_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
+    if (!q_lens || !n_mask || !accepted_len || !bonus_token) return FD_ERR_INVALID_ARG;
+    if (total_cand_rows > 0 && (!logits || !draft_tokens)) return FD_ERR_INVALID_ARG;
+    if (!aligned(logits, 4)) return FD_ERR_INVALID_ARG;
+    const long long ctas = (long long)total_cand_rows * ((c->cfg.vocab + fd::kAcceptChunk - 1) / fd::kAcceptChunk);
+    if (ctas > 0x7fffffffLL) return FD_ERR_UNSUPPORTED;
+    fd::AcceptParams p;
+    p.batch = batch; p.total_rows = total_cand_rows; p.vocab = c->cfg.vocab;
+    p.logits = logits; p.drafts = draft_tokens; p.q_lens = q_lens; p.n_mask = n_mask;
+    p.accepted = accepted_len; p.bonus = bonus_token;
+    p.keys = c->keys; p.ticket = c->ticket; p.status = c->status;
+    fd::launch_accept(p, static_cast<cudaStream_t>(stream));
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefix_lens, const int32_t* q_lens,
+                       const int32_t* accepted_len, int32_t* freed_pages, int32_t* n_freed, void* stream) {
+    if (!c || batch < 0 || batch > c->cfg.max_batch || !n_freed) return FD_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (batch == 0) return cudaMemsetAsync(n_freed, 0, sizeof(int32_t), s) == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+    if (!page_table || !prefix_lens || !q_lens || !accepted_len || !freed_pages) return FD_ERR_INVALID_ARG;
+    fd::CommitParams p;
+    p.batch = batch; p.max_pages = c->cfg.max_pages_per_seq; p.page_size = c->cfg.page_size;
+    p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.accepted = accepted_len;
+    p.freed = freed_pages; p.n_freed = n_freed; p.status = c->status;
+    fd::launch_commit(p, s);
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_last_device_status(fd_ctx* c, int32_t* code, void* stream) {
+    if (!c || !code) return FD_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(code, c->status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return FD_ERR_CUDA;
+    if (cudaMemsetAsync(c->status, 0, sizeof(int), s) != cudaSuccess) return FD_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FD_ERR_CUDA;
+    return FD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,137 @@
+// Plan (work list of the split-KV attention) and split merge.
+//
+// The attention of one call is cut into tiles of 128 KV tokens.  Tiles are numbered
+// sequence-major, then kv-head, then position, and the numbered list is cut into one
+// contiguous range per CTA of the attention grid ("stream-K"), so every CTA streams the
+// same number of KV bytes whatever the mix of prefix lengths.  A (sequence, kv-head)
+// segment that falls into several ranges leaves one partial result per range; the merge
+// kernel combines them in range order, which makes the result independent of timing.
+#include "fd_internal.cuh"
+
+namespace fd {
+
+__global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
+    __shared__ int s_fatal;
+    const int B = p.batch, tid = threadIdx.x;
+    if (tid == 0) s_fatal = 0;
+    __syncthreads();
+    const int P = 16;
+    for (int b = tid; b < B; b += blockDim.x) {
+        const long long n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
+        const bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || Lq * p.G > kMaxRows ||
+                         n + Lq > (long long)p.max_pages * P;
+        if (bad) atomicOr(&s_fatal, 1);
+        p.plan.seq_ok[b] = 1;
+    }
+    __syncthreads();
+    if (!s_fatal) {
+        for (int b = 0; b < B; ++b) {
+            const int Lq = p.q_lens[b];
+            const int need = Lq > 0 ? (p.prefix_lens[b] + Lq + P - 1) / P : 0;
+            for (int pg = tid; pg < need; pg += blockDim.x) {
+                const int id = p.page_table[(long long)b * p.max_pages + pg];
+                if (id < 0 || id >= p.num_pages) {
+                    p.plan.seq_ok[b] = 0;
+                    atomicOr(p.status, FD_DEV_BAD_PAGE);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        long long rows = 0, tiles = 0;
+        int fatal = s_fatal;
+        p.plan.cu_q[0] = 0;
+        p.plan.cu_tiles[0] = 0;
+        if (!fatal) {
+            for (int b = 0; b < B; ++b) {
+                const int Lq = p.q_lens[b];
+                rows += Lq;
+                if (Lq > 0 && p.plan.seq_ok[b]) tiles += (p.prefix_lens[b] + Lq + kTileTokens - 1) / kTileTokens;
+                p.plan.cu_q[b + 1] = (int)rows;
+                p.plan.cu_tiles[b + 1] = (int)tiles;
+            }
+            if (rows != p.total_q_rows || tiles * p.Hkv > 0x7fffffffLL) fatal = 1;
+        }
+        if (fatal) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        p.plan.hdr->fatal = fatal;
+        p.plan.hdr->total_tiles = fatal ? 0 : (int)(tiles * p.Hkv);
+    }
+}
+
+void launch_plan(const AttnParams& p, cudaStream_t s) { plan_kernel<<<1, 256, 0, s>>>(p); }
+
+template <int D>
+__device__ inline void store_row_bf16(__nv_bfloat16* dst, const float* o, float inv) {
+#pragma unroll
+    for (int c = 0; c < D; c += 8) {
+        __align__(16) __nv_bfloat162 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v[k] = __floats2bfloat162_rn(o[c + 2 * k] * inv, o[c + 2 * k + 1] * inv);
+        *reinterpret_cast<uint4*>(dst + c) = *reinterpret_cast<const uint4*>(v);
+    }
+}
+
+// One CTA per (sequence, kv-head) segment, one thread per query row of the segment.
+template <int D>
+__global__ void __launch_bounds__(kMaxRows) merge_kernel(AttnParams p) {
+    const PlanHeader hdr = *p.plan.hdr;
+    if (hdr.fatal) {  // defined output for an undefined request: zeros
+        const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
+        uint4* o = reinterpret_cast<uint4*>(p.out);
+        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16;
+             i += (long long)gridDim.x * blockDim.x)
+            o[i] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    const int row0 = p.plan.cu_q[b], Lq = p.plan.cu_q[b + 1] - row0;
+    const int rows = Lq * p.G, r = threadIdx.x;
+    if (r >= rows) return;
+    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D;
+    float acc[D];
+    if (!p.plan.seq_ok[b]) {
+#pragma unroll
+        for (int c = 0; c < D; ++c) acc[c] = 0.f;
+        store_row_bf16<D>(dst, acc, 0.f);
+        return;
+    }
+    const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
+    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles, t1 = t0 + ntiles;
+    const int c_first = range_owner(t0, hdr.total_tiles, p.n_ctas);
+    const int c_last = range_owner(t1 - 1, hdr.total_tiles, p.n_ctas);
+    if (c_first == c_last) return;  // one CTA held the whole segment and wrote the final rows itself
+
+    float m = -INFINITY;
+    for (int c = c_first; c <= c_last; ++c) {
+        const int sc = range_begin(c, hdr.total_tiles, p.n_ctas), ec = range_begin(c + 1, hdr.total_tiles, p.n_ctas);
+        if (max(sc, t0) >= min(ec, t1)) continue;
+        const int slot = 2 * c + (sc >= t0 ? 0 : 1);
+        m = fmaxf(m, p.part.m[slot * kMaxRows + r]);
+    }
+#pragma unroll
+    for (int c = 0; c < D; ++c) acc[c] = 0.f;
+    float l = 0.f;
+    for (int c = c_first; c <= c_last; ++c) {
+        const int sc = range_begin(c, hdr.total_tiles, p.n_ctas), ec = range_begin(c + 1, hdr.total_tiles, p.n_ctas);
+        if (max(sc, t0) >= min(ec, t1)) continue;
+        const int slot = 2 * c + (sc >= t0 ? 0 : 1);
+        const float mp = p.part.m[slot * kMaxRows + r];
+        if (mp == -INFINITY) continue;  // this piece saw no visible key for the row
+        const float w = exp2f(mp - m);
+        l += w * p.part.l[slot * kMaxRows + r];
+        const float* o = p.part.o + (long long)slot * D * kMaxRows + r;
+#pragma unroll
+        for (int col = 0; col < D; ++col) acc[col] += w * o[col * kMaxRows];
+    }
+    store_row_bf16<D>(dst, acc, 1.f / l);
+}
+
+void launch_merge(const AttnParams& p, cudaStream_t s) {
+    const int grid = p.batch * p.Hkv;
+    if (grid == 0) return;
+    if (p.d == 64) merge_kernel<64><<<grid, kMaxRows, 0, s>>>(p);
+    else merge_kernel<128><<<grid, kMaxRows, 0, s>>>(p);
+}
+
+}  // namespace fd

@@ -1,0 +1,233 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Attention within |err| <= 2e-2 + 2e-2 |ref|; accept and commit bit-exact."""
+import zlib
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_20022_b200 as fd
+from paper_2605_20022_b200 import workload as wl
+from helpers import Ctx, assert_close, gpu_accept, gpu_attn, gpu_commit
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [fd.FD_ATTN_SIMT, fd.FD_ATTN_AUTO]
+
+
+def oracle_attn(step, q, kv):
+    return oracle.attn(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_attention_workloads(idx, path):
+    step = wl.workload(idx)
+    q, kv = wl.make_q(step), wl.make_kv(step)
+    with Ctx(step, path) as ctx:
+        got, status = gpu_attn(ctx, step, q, kv)
+    assert status == 0
+    assert_close(got.numpy(), oracle_attn(step, q, kv), step.name)
+
+
+EDGE = {
+    # name: (Hq, Hkv, d, prefix_lens, q_lens, n_mask)
+    "prefix0_and_single_row": (8, 2, 128, [0, 0, 1, 15], [1, 9, 1, 1], [0, 4, 0, 1]),
+    "page_boundaries": (8, 2, 128, [16, 15, 17, 112, 127, 128, 129, 240], [16, 17, 15, 16, 1, 32, 31, 32],
+                        [0, 1, 15, 16, 0, 16, 16, 16]),
+    "mask_only_and_one_candidate": (8, 2, 128, [300, 77, 5], [16, 17, 4], [16, 16, 4]),
+    "all_mask_counts": (4, 1, 128, [100 + 3 * m for m in range(17)], [16 + m for m in range(17)], list(range(17))),
+    "empty_sequences_inside_batch": (8, 2, 128, [40, 90, 0, 260], [0, 5, 0, 32], [0, 2, 0, 16]),
+    "head_dim64_gqa8": (16, 2, 64, [200, 31, 1000], [16, 3, 9], [8, 0, 4]),
+    "mha_group1": (4, 4, 64, [130, 257], [32, 20], [16, 4]),
+    "one_long_sequence_many_splits": (8, 1, 128, [20000], [32], [16]),
+    "ragged_mix": (32, 8, 128, [5000, 13, 700, 2047, 2049, 129], [32, 1, 20, 9, 32, 16], [16, 0, 16, 0, 16, 8]),
+}
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name", sorted(EDGE))
+def test_attention_edge_cases(name, path):
+    Hq, Hkv, d, pl, ql, nm = EDGE[name]
+    step = wl.make_step(name, wl.Shape(Hq, Hkv, d, 1000), pl, ql, nm, seed=zlib.crc32(name.encode()) % 10000, extra_table_cols=2)
+    q, kv = wl.make_q(step), wl.make_kv(step, poison=float("nan"))     # NaN in every slot no token owns
+    with Ctx(step, path) as ctx:
+        got, status = gpu_attn(ctx, step, q, kv)
+        again, _ = gpu_attn(ctx, step, q, kv)
+    assert status == 0
+    assert_close(got.numpy(), oracle_attn(step, q, kv), name)
+    assert torch.equal(got, again), "two runs on the same inputs differ bitwise"
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_attention_custom_scale_and_empty_batch(path):
+    step = wl.make_step("scale", wl.Shape(8, 2, 128, 1000), [333, 40], [12, 32], [4, 16], seed=5)
+    q, kv = wl.make_q(step), wl.make_kv(step)
+    with Ctx(step, path, scale=0.05) as ctx:
+        got, status = gpu_attn(ctx, step, q, kv)
+        assert status == 0
+        ref = oracle.attn(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, scale=0.05)
+        assert_close(got.numpy(), ref, "scale")
+        empty = torch.zeros((0,), dtype=torch.int32)
+        code = fd.fd_attn_draft_verify(ctx.h, 0, 0, None, None, 0, None, None, None, None, None)
+        assert code == fd.FD_OK and fd.fd_last_device_status(ctx.h) == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_attention_device_detected_errors(path):
+    step = wl.make_step("err", wl.Shape(8, 2, 128, 1000), [100, 200, 50], [8, 8, 8], [4, 4, 4], seed=6)
+    q, kv = wl.make_q(step), wl.make_kv(step)
+    ref = oracle_attn(step, q, kv)
+    with Ctx(step, path) as ctx:
+        bad = step.page_table.clone()
+        bad[1, 3] = step.num_pages + 5                      # a page id outside the pool
+        got, status = gpu_attn(ctx, step, q, kv, page_table=bad)
+        assert status == fd.FD_DEV_BAD_PAGE
+        assert_close(got[:8].numpy(), ref[:8], "seq0"); assert_close(got[16:].numpy(), ref[16:], "seq2")
+        assert (got[8:16] == 0).all()
+        for lens in [(step.prefix_lens, torch.tensor([8, 9, 8], dtype=torch.int32), step.n_mask),   # rows != T
+                     (step.prefix_lens, step.q_lens, torch.tensor([4, 9, 4], dtype=torch.int32)),   # n_mask > q_len
+                     (torch.tensor([100, -1, 50], dtype=torch.int32), step.q_lens, step.n_mask),
+                     (torch.tensor([100, 10 ** 6, 50], dtype=torch.int32), step.q_lens, step.n_mask)]:
+            got, status = gpu_attn(ctx, step, q, kv, lens=lens)
+            assert status == fd.FD_DEV_BAD_LENGTHS and (got == 0).all()
+        got, status = gpu_attn(ctx, step, q, kv)             # the context still works
+        assert status == 0
+        assert_close(got.numpy(), ref, "after errors")
+
+
+def test_host_detected_errors_launch_nothing():
+    step = wl.workload(0)
+    with Ctx(step) as ctx:
+        q = torch.zeros((9, 4, 64), dtype=torch.bfloat16, device="cuda")
+        before = fd.fd_launch_count(ctx.h)
+        assert fd.fd_attn_draft_verify(ctx.h, 1, 9, None, q, 4, q, q, q, q, q, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        assert fd.fd_attn_draft_verify(ctx.h, 2, 9, q, q, 4, q, q, q, q, q, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        assert fd.fd_verify_accept(ctx.h, 1, 5, None, q, q, q, q, q, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        assert fd.fd_kv_commit(ctx.h, 1, q, q, q, q, q, None, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        assert fd.fd_launch_count(ctx.h) == before
+    with pytest.raises(fd.FlexDraftError):
+        fd.fd_create(32, 8, 96, 1000, 1, 32, 8)             # head_dim 96
+    with pytest.raises(fd.FlexDraftError):
+        fd.fd_create(32, 8, 128, 1000, 1, 33, 8)            # G * max_q_len > 128
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
+def test_accept_and_commit_workloads(idx):
+    step = wl.workload(idx)
+    logits, drafts, target = wl.make_logits(step)
+    exp_acc, exp_bon, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    with Ctx(step) as ctx:
+        acc, bon, status = gpu_accept(ctx, step, logits, drafts)
+        assert status == 0
+        np.testing.assert_array_equal(acc, exp_acc)
+        np.testing.assert_array_equal(bon, exp_bon)
+        acc2, bon2, _ = gpu_accept(ctx, step, logits, drafts)      # scratch keys were re-zeroed
+        np.testing.assert_array_equal(acc2, exp_acc); np.testing.assert_array_equal(bon2, exp_bon)
+        pt, pl, freed, status = gpu_commit(ctx, step, acc)
+        assert status == 0
+    ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, exp_acc)
+    np.testing.assert_array_equal(pt, ept)
+    np.testing.assert_array_equal(pl, epl)
+    np.testing.assert_array_equal(freed, efreed)
+
+
+@pytest.mark.parametrize("V", [1, 3, 17, 1000, 4097, 8191, 8192, 8193, 151937, 200003])
+def test_accept_vocab_sizes_ties_and_alignment(V):
+    g = torch.Generator().manual_seed(V)
+    ql = [1, 4, 16, 2, 7, 0, 16]
+    nm = [0, 0, 0, 1, 3, 0, 16]
+    step = wl.make_step("acc", wl.Shape(4, 2, 64, V), [5] * len(ql), ql, nm, seed=V, p_match=0.85)
+    logits, drafts, _ = wl.make_logits(step)
+    logits = torch.round(logits * 2) / 2                       # coarse grid: many exact ties, planted peak kept
+    R = logits.shape[0]
+    logits[0] = 0.25                                           # a flat row -> index 0
+    if V > 2:
+        logits[1, V - 1] = 9.0; logits[1, V // 2] = 9.0        # two-way tie for the maximum
+        logits[2, :] = -float("inf"); logits[2, V - 2] = -3e38
+        logits[3, 1] = float("inf"); logits[3, V - 1] = float("inf")
+        logits[4, 0] = -0.0; logits[4, 1:] = -1.0; logits[4, V - 1] = 0.0   # -0.0 ties with +0.0
+    exp_acc, exp_bon, exp_am = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    drafts2 = drafts.clone()                                   # make the drafts agree with the tied rows too
+    r0 = 0
+    for b, C in enumerate(step.cand_rows.tolist()):
+        for j in range(C - 1):
+            if (r0 + j) % 3 != 2:
+                drafts2[r0 + j + 1] = int(exp_am[r0 + j])
+        r0 += C
+    with Ctx(step) as ctx:
+        for d_ in (drafts, drafts2):
+            e_acc, e_bon, _ = oracle.accept(logits, d_, step.q_lens, step.n_mask)
+            acc, bon, status = gpu_accept(ctx, step, logits, d_)
+            assert status == 0
+            np.testing.assert_array_equal(acc, e_acc)
+            np.testing.assert_array_equal(bon, e_bon)
+
+
+def test_accept_bad_lengths_and_no_candidates():
+    step = wl.make_step("acc", wl.Shape(4, 2, 64, 500), [5, 5], [4, 16], [0, 16], seed=3)
+    logits, drafts, _ = wl.make_logits(step)
+    with Ctx(step) as ctx:
+        acc, bon, status = gpu_accept(ctx, step, logits, drafts,
+                                      lens=(torch.tensor([5, 16], dtype=torch.int32), step.n_mask))
+        assert status == fd.FD_DEV_BAD_LENGTHS and (acc == -1).all() and (bon == -1).all()
+        acc, bon, status = gpu_accept(ctx, step, logits, drafts)
+        e_acc, e_bon, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+        assert status == 0
+        np.testing.assert_array_equal(acc, e_acc); np.testing.assert_array_equal(bon, e_bon)
+        none = wl.make_step("none", wl.Shape(4, 2, 64, 500), [5, 5], [16, 16], [16, 16], seed=3)
+        lg, dr, _ = wl.make_logits(none)
+        acc, bon, status = gpu_accept(ctx, none, lg, dr)
+        assert status == 0 and (acc == -1).all() and (bon == -1).all()
+
+
+def test_commit_random_and_degenerate():
+    g = torch.Generator().manual_seed(9)
+    B = 300
+    n = torch.randint(0, 400, (B,), generator=g)
+    C = torch.randint(0, 17, (B,), generator=g)
+    M = torch.randint(0, 2, (B,), generator=g) * 16
+    step = wl.make_step("commit", wl.Shape(4, 2, 64, 100), n.tolist(), (C + M).tolist(), M.tolist(), seed=10,
+                        extra_table_cols=2)
+    acc = np.array([int(torch.randint(0, int(c), (1,), generator=g)) if c > 0 else -1 for c in C], np.int32)
+    with Ctx(step) as ctx:
+        pt, pl, freed, status = gpu_commit(ctx, step, acc)
+        assert status == 0
+        ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, acc)
+        np.testing.assert_array_equal(pt, ept); np.testing.assert_array_equal(pl, epl)
+        np.testing.assert_array_equal(freed, efreed)
+        bad = acc.copy()
+        k = int(np.argmax(acc >= 0))
+        bad[k] = int(step.q_lens[k])                            # accepted_len >= q_len: left unchanged, flagged
+        pt, pl, freed, status = gpu_commit(ctx, step, bad)
+        assert status == fd.FD_DEV_BAD_ACCEPT
+        skip = acc.copy(); skip[k] = -1
+        ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, skip)
+        np.testing.assert_array_equal(pt, ept); np.testing.assert_array_equal(pl, epl)
+        np.testing.assert_array_equal(freed, efreed)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_long_context_full_size_sampled(path):
+    """Workload 5 at its full per-layer size (16 x 32 800 tokens, 2.15 GB of KV per layer, two
+    layers with distinct pools), in the launch configuration the benchmark times; the oracle
+    computes sampled output rows one by one."""
+    step = wl.workload(4, n_layers=2)
+    dpt, dpl, dql, dnm = (t.cuda() for t in (step.page_table, step.prefix_lens, step.q_lens, step.n_mask))
+    g = torch.Generator().manual_seed(1)
+    with Ctx(step, path) as ctx:
+        for layer in range(2):
+            q = wl.make_q(step, layer, device="cuda")
+            kv = wl.make_kv(step, layer, device="cuda")
+            out = torch.empty_like(q)
+            fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, q, kv, step.num_pages, dpt, dpl, dql, dnm, out)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            qc, kvc, outc = q.cpu(), kv.cpu(), out.float().cpu().numpy()
+            assert np.isfinite(outc).all()
+            for _ in range(24):
+                b = int(torch.randint(0, 16, (1,), generator=g)); i = int(torch.randint(0, 32, (1,), generator=g))
+                h = int(torch.randint(0, 32, (1,), generator=g))
+                ref = oracle.attn_row(qc, kvc, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, b, i, h)
+                assert_close(outc[b * 32 + i, h], ref, f"layer {layer} b {b} row {i} head {h}")
+            del q, kv, out
