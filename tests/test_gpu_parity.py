@@ -41,7 +41,7 @@ EDGE = {
     "empty_sequences_inside_batch": (8, 2, 128, [40, 90, 0, 260], [0, 5, 0, 32], [0, 2, 0, 16]),
     "head_dim64_gqa8": (16, 2, 64, [200, 31, 1000], [16, 3, 9], [8, 0, 4]),
     "mha_group1": (4, 4, 64, [130, 257], [32, 20], [16, 4]),
-    "one_long_sequence_many_splits": (8, 1, 128, [20000], [32], [16]),
+    "one_long_sequence_many_splits": (4, 1, 128, [20000], [32], [16]),
     "ragged_mix": (32, 8, 128, [5000, 13, 700, 2047, 2049, 129], [32, 1, 20, 9, 32, 16], [16, 0, 16, 0, 16, 8]),
 }
 
