@@ -1,8 +1,460 @@
-// placeholder: the tensor-core attention kernel is added in a later step
+// Tensor-core split-KV attention under the hybrid mask for sm_100a: TMA-staged KV pages,
+// tcgen05 MMAs with accumulators in tensor memory, softmax in registers.
+//
+// Work decomposition.  The plan kernel numbers all 128-token KV tiles of the call
+// (sequence-major, then kv-head, then position) and each of the n_ctas persistent CTAs takes
+// one contiguous range, so every SM streams the same number of KV bytes.  A range is walked
+// piece by piece, a piece being its intersection with one (sequence b, kv-head) segment.
+//
+// One piece.  The G * Lq_b <= 128 query rows that share the kv-head (row r = block row
+// r / G of q-head kvh * G + r % G) form the M = 128 operand of every MMA, so each KV tile is
+// read from HBM once for all of them.  Per tile j of the piece:
+//     producer warp : 32 lanes issue one 2 KB TMA box each (8 pages x {K,V} x two 64-wide
+//                     halves of d) into a 128B-swizzled stage of a 3-deep ring;
+//     MMA warp      : S_s = Q K^T (tcgen05.mma, A and B from shared memory, S in TMEM), and
+//                     after the softmax O_s += P_s V (A = P from TMEM, B = V MN-major);
+//     softmax group : 128 threads, one query row each: tcgen05.ld the row of S, hybrid mask
+//                     from the row's (kind, index) -> first invisible key position, online
+//                     softmax in the log2 domain, bf16 P written back over S in TMEM.
+// Tiles alternate between two independent streams s = j & 1, each with its own softmax
+// group, S/P buffer, (m, l) state and O accumulator in TMEM, so the tensor pipe works on one
+// stream while the other is in its softmax; the two streams are merged in the epilogue.  O is
+// rescaled lazily (only when a row maximum grows by more than 2^8), which is exact because
+// the same reference maximum is used for P, l and O.
+//
+// TMEM columns: S0/P0 [0,128)  S1/P1 [128,256)  O0 [256,256+d)  O1 [384,384+d).
+//
+// Every wait is bounded.  A wait that runs out raises a CTA-wide abort flag: all roles leave
+// their loops, in-flight TMA copies are drained, TMEM is released and FD_DEV_TIMEOUT is set.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "fd_internal.cuh"
+#include "fd_sm100.cuh"
+
 namespace fd {
-bool attn_tc_supported(int, int, int) { return false; }
-cudaError_t attn_tc_prepare(void**, const AttnParams&) { return cudaErrorNotSupported; }
-void launch_attn_tc(void*, const AttnParams&, cudaStream_t) {}
-void attn_tc_free(void*) {}
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kThreads = 320;  // warps 0-3 softmax group 0, 4-7 softmax group 1, 8 producer, 9 MMA
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+template <int D>
+struct Cfg {
+    static constexpr int kStages = (D == 128) ? 3 : 4;
+    static constexpr int kQBytes = kMaxRows * D * 2;
+    static constexpr int kKBytes = kTileTokens * D * 2;
+    static constexpr int kStageBytes = 2 * kKBytes;
+    static constexpr int kBarOffset = kQBytes + kStages * kStageBytes;
+    static constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // + barriers + slack for 1024-byte alignment
+    static constexpr int kKSteps = D / 16;
+    static constexpr int kHalves = D / 64;
+};
+
+struct Bars {
+    uint64_t kv_full[4], kv_empty[4];
+    uint64_t s_full[2], p_full[2], pv_done[2];
+    uint64_t all_done;
+    uint32_t tmem_base;
+    int abort;
+};
+
+struct Piece {
+    int b, kvh, tile0, nt, n, Lq, M, kv_len, rows, row0, slot;
+    bool complete;
+};
+
+__device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_c, int e_c, int cta) {
+    Piece pc;
+    int lo = 0, hi = p.batch;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (p.Hkv * p.plan.cu_tiles[mid] <= t) lo = mid; else hi = mid;
+    }
+    pc.b = lo;
+    const int ntiles = p.plan.cu_tiles[lo + 1] - p.plan.cu_tiles[lo];
+    const int rem = t - p.Hkv * p.plan.cu_tiles[lo];
+    pc.kvh = rem / ntiles;
+    pc.tile0 = rem % ntiles;
+    const int seg_start = t - pc.tile0, seg_end = seg_start + ntiles;
+    const int t_end = min(e_c, seg_end);
+    pc.nt = t_end - t;
+    pc.n = p.prefix_lens[lo];
+    pc.Lq = p.q_lens[lo];
+    pc.M = p.n_mask[lo];
+    pc.kv_len = pc.n + pc.Lq;
+    pc.rows = pc.Lq * p.G;
+    pc.row0 = p.plan.cu_q[lo];
+    pc.complete = (t == seg_start) && (t_end == seg_end);
+    pc.slot = 2 * cta + (t == s_c ? 0 : 1);
+    return pc;
+}
+
+// Warp-uniform bounded wait.
+__device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    const bool ok = mbar_wait(bar, parity, abort);
+    return __all_sync(0xffffffffu, ok);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, AttnParams p) {
+    using C = Cfg<D>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* sq = smem;
+    unsigned char* sstage = smem + C::kQBytes;
+    Bars* bars = reinterpret_cast<Bars*>(smem + C::kBarOffset);
+    float* ex_m = reinterpret_cast<float*>(sq);          // [2][128], aliases Q after the last MMA of a piece
+    float* ex_l = ex_m + 2 * kMaxRows;
+    volatile int* abort = &bars->abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const PlanHeader hdr = *p.plan.hdr;
+    const int total = hdr.total_tiles;
+    if (total == 0) return;  // uniform: nothing allocated yet
+    const int cta = blockIdx.x;
+    const int s_c = range_begin(cta, total, p.n_ctas), e_c = range_begin(cta + 1, total, p.n_ctas);
+    if (s_c >= e_c) return;
+
+    if (tid == 0) {
+        for (int i = 0; i < C::kStages; ++i) { mbar_init(&bars->kv_full[i], 1); mbar_init(&bars->kv_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->s_full[i], 1);
+            mbar_init(&bars->p_full[i], 128);
+            mbar_init(&bars->pv_done[i], 1);
+        }
+        mbar_init(&bars->all_done, 1);
+        bars->abort = 0;
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
+    if (warp == kProducerWarp && lane == 0) prefetch_tmap(&tmap);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    const uint32_t col_s[2] = {0u, 128u};
+    const uint32_t col_o[2] = {256u, 384u};
+
+    int g0 = 0;            // KV tiles this CTA has pushed through the stage ring so far
+    int u_base[2] = {0, 0};  // tiles each stream has processed so far
+    int piece_idx = 0;
+    int issued = 0;        // producer: tiles whose loads were issued
+
+    for (int t = s_c; t < e_c;) {
+        const Piece pc = decode_piece(p, t, s_c, e_c, cta);
+
+        // ---- Q tile -> shared memory, K-major, 128-byte swizzle; rows beyond the block are zero
+        for (int idx = tid; idx < kMaxRows * (D / 8); idx += kThreads) {
+            const int r = idx / (D / 8), ch = idx % (D / 8);
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (r < pc.rows)
+                v = *reinterpret_cast<const uint4*>(p.q + ((long long)(pc.row0 + r / p.G) * p.Hq + pc.kvh * p.G + r % p.G) * D + ch * 8);
+            const int half = ch >> 3, c16 = ch & 7;
+            *reinterpret_cast<uint4*>(sq + half * (kMaxRows * 128) + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
+        }
+        fence_proxy_async_smem();
+        __syncthreads();
+
+        if (warp == kProducerWarp) {
+            // ============================== TMA producer ==============================
+            constexpr int kOps = 8 * 2 * C::kHalves;
+            const int pg = lane / (2 * C::kHalves), which = (lane / C::kHalves) & 1, half = lane % C::kHalves;
+            for (int j = 0; j < pc.nt; ++j) {
+                const int g = g0 + j, st = g % C::kStages, use = g / C::kStages;
+                if (!wait_all(&bars->kv_empty[st], (use & 1) ^ 1, abort)) break;
+                const int pos0 = (pc.tile0 + j) * kTileTokens;
+                const int npg = min(8, (pc.kv_len - pos0 + 15) >> 4);
+                if (lane == 0) mbar_arrive_expect_tx(&bars->kv_full[st], npg * (2 * 16 * D * 2));
+                __syncwarp();
+                if (lane < kOps && pg < npg) {
+                    const int phys = p.page_table[(long long)pc.b * p.max_pages + (pos0 >> 4) + pg];
+                    unsigned char* dst = sstage + st * C::kStageBytes + which * C::kKBytes + half * (kTileTokens * 128) + pg * 2048;
+                    tma_load_2d(dst, &tmap, half * 64, ((phys * 2 + which) * p.Hkv + pc.kvh) * 16, &bars->kv_full[st]);
+                }
+                issued = g + 1;
+            }
+        } else if (warp == kMmaWarp) {
+            // ============================== MMA issuer ==============================
+            constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
+            const uint32_t q_addr = smem_u32(sq);
+            bool ok = true;
+            auto issue_pv = [&](int jj) {
+                const int s = jj & 1, st = (g0 + jj) % C::kStages, u = u_base[s] + (jj >> 1);
+                if (!wait_all(&bars->p_full[s], u & 1, abort)) { ok = false; return; }
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t v_addr = smem_u32(sstage + st * C::kStageBytes + C::kKBytes);
+#pragma unroll
+                    for (int kk = 0; kk < kTileTokens / 16; ++kk)
+                        umma_ts(tmem + col_o[s], tmem + col_s[s] + kk * 8,
+                                make_smem_desc(v_addr + kk * 2048, kTileTokens * 128, 1024), idesc_pv, jj >= 2 || kk > 0);
+                    umma_commit(&bars->kv_empty[st]);
+                    umma_commit(&bars->pv_done[s]);
+                }
+                __syncwarp();
+            };
+            for (int j = 0; j < pc.nt && ok; ++j) {
+                const int g = g0 + j, st = g % C::kStages, use = g / C::kStages;
+                const int s = j & 1, u = u_base[s] + (j >> 1);
+                if (!wait_all(&bars->kv_full[st], use & 1, abort)) { ok = false; break; }
+                const int valid = pc.kv_len - (pc.tile0 + j) * kTileTokens;
+                if (valid < kTileTokens) {
+                    // V rows no token owns may hold NaN or stale data: P is 0 there, but 0 * NaN is not
+                    unsigned char* sv = sstage + st * C::kStageBytes + C::kKBytes;
+                    const int nbad = kTileTokens - valid;
+                    for (int e = lane; e < nbad * 8 * C::kHalves; e += 32) {
+                        const int r = valid + e / (8 * C::kHalves), w = e % (8 * C::kHalves);
+                        *reinterpret_cast<uint4*>(sv + (w >> 3) * (kTileTokens * 128) + r * 128 + ((w & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                }
+                if (u >= 1 && !wait_all(&bars->pv_done[s], (u - 1) & 1, abort)) { ok = false; break; }
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t k_addr = smem_u32(sstage + st * C::kStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < C::kKSteps; ++kk) {
+                        const uint32_t off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
+                        umma_ss(tmem + col_s[s], make_smem_desc(q_addr + off, 16, 1024), make_smem_desc(k_addr + off, 16, 1024),
+                                idesc_qk, kk > 0);
+                    }
+                    umma_commit(&bars->s_full[s]);
+                }
+                __syncwarp();
+                if (j >= 1) issue_pv(j - 1);
+            }
+            if (ok) issue_pv(pc.nt - 1);
+            if (ok && lane == 0) umma_commit(&bars->all_done);
+            __syncwarp();
+        } else {
+            // ============================== softmax groups ==============================
+            const int s = warp >> 2;                  // stream
+            const int r = (warp & 3) * 32 + lane;     // query row == TMEM lane
+            const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+            const bool warp_active = (warp & 3) * 32 < pc.rows;
+            const int i = r / p.G;
+            const int limit = (r < pc.rows) ? ((i < pc.Lq - pc.M) ? pc.n + i + 1 : pc.kv_len) : 0;
+            const float c = p.scale_log2e;
+            float m = -INFINITY, l = 0.f;
+            bool ok = true;
+
+            for (int j = s; j < pc.nt; j += 2) {
+                const int u = u_base[s] + (j >> 1);
+                if (!wait_all(&bars->s_full[s], u & 1, abort)) { ok = false; break; }
+                tc_fence_after();
+                if (warp_active) {
+                    const int pos0 = (pc.tile0 + j) * kTileTokens;
+                    uint32_t sv[4][32];
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) tmem_ld32(tmem + lane_base + col_s[s] + ch * 32, sv[ch]);
+                    tc_wait_ld();
+                    if (pos0 + kTileTokens > pc.n) {  // tile reaches into the query block (or past kv_len)
+                        const int lim = limit - pos0;
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+                            for (int k = 0; k < 32; ++k)
+                                if (ch * 32 + k >= lim) sv[ch][k] = 0xff800000u;  // -inf, a select: S may be NaN there
+                    }
+                    float mx = -INFINITY;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(sv[ch][k]));
+                    const float m_new = fmaxf(m, mx * c);
+                    float alpha = 1.f;
+                    if (j < 2 || m == -INFINITY) {
+                        m = m_new;  // nothing accumulated yet (O is overwritten, or exactly zero)
+                    } else if (m_new > m + kRescaleThreshold) {
+                        alpha = exp2f(m - m_new);
+                        m = m_new;
+                    }
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                        // previous PV of this stream has completed (S/P buffer reuse orders it), so O is quiescent
+#pragma unroll
+                        for (int ch = 0; ch < D / 32; ++ch) {
+                            uint32_t o[32];
+                            tmem_ld32(tmem + lane_base + col_o[s] + ch * 32, o);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                            tmem_st32(tmem + lane_base + col_o[s] + ch * 32, o);
+                        }
+                        l *= alpha;
+                    }
+                    const float mc = (m == -INFINITY) ? 0.f : m;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ch += 2) {
+                        uint32_t pk[32];
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                            for (int k = 0; k < 32; k += 2) {
+                                const float p0 = exp2f(fmaf(__uint_as_float(sv[ch + hh][k]), c, -mc));
+                                const float p1 = exp2f(fmaf(__uint_as_float(sv[ch + hh][k + 1]), c, -mc));
+                                l += p0 + p1;
+                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                                pk[hh * 16 + (k >> 1)] = *reinterpret_cast<const uint32_t*>(&b2);
+                            }
+                        tmem_st32(tmem + lane_base + col_s[s] + (ch >> 1) * 32, pk);
+                    }
+                    tc_wait_st();
+                }
+                tc_fence_before();
+                mbar_arrive(&bars->p_full[s]);
+            }
+
+            // ---- epilogue: merge the two streams, then final rows or a partial for the merge kernel
+            ok = ok && wait_all(&bars->all_done, piece_idx & 1, abort);
+            tc_fence_after();
+            if (ok) {
+                ex_m[s * kMaxRows + r] = m;
+                ex_l[s * kMaxRows + r] = l;
+            }
+            named_bar_sync(1, 256);
+            if (ok && !*abort && warp_active) {
+                const bool two = pc.nt >= 2;
+                const float m0 = ex_m[r], m1 = two ? ex_m[kMaxRows + r] : -INFINITY;
+                const float mm = fmaxf(m0, m1);
+                const float a0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - mm);
+                const float a1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mm);
+                const float L = a0 * ex_l[r] + (two ? a1 * ex_l[kMaxRows + r] : 0.f);
+                const float inv = pc.complete ? 1.f / L : 1.f;
+                constexpr int kChunks = D / 64;  // 32-column chunks per softmax group
+#pragma unroll
+                for (int ch = 0; ch < kChunks; ++ch) {
+                    const int col = s * (D / 2) + ch * 32;
+                    uint32_t o0[32], o1[32];
+                    tmem_ld32(tmem + lane_base + col_o[0] + col, o0);
+                    if (two) tmem_ld32(tmem + lane_base + col_o[1] + col, o1);
+                    tc_wait_ld();
+                    float o[32];
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) {
+                        o[k] = __uint_as_float(o0[k]) * a0;
+                        if (two) o[k] = fmaf(__uint_as_float(o1[k]), a1, o[k]);
+                        o[k] *= inv;
+                    }
+                    if (r < pc.rows) {
+                        if (pc.complete) {
+                            __nv_bfloat16* dst = p.out + ((long long)(pc.row0 + i) * p.Hq + pc.kvh * p.G + r % p.G) * D + col;
+#pragma unroll
+                            for (int k = 0; k < 32; k += 8) {
+                                __align__(16) __nv_bfloat162 v[4];
+#pragma unroll
+                                for (int q2 = 0; q2 < 4; ++q2) v[q2] = __floats2bfloat162_rn(o[k + 2 * q2], o[k + 2 * q2 + 1]);
+                                *reinterpret_cast<uint4*>(dst + k) = *reinterpret_cast<const uint4*>(v);
+                            }
+                        } else {
+                            float* dst = p.part.o + ((long long)pc.slot * D + col) * kMaxRows + r;
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) dst[k * kMaxRows] = o[k];
+                        }
+                    }
+                }
+                if (!pc.complete && s == 0 && r < pc.rows) {
+                    p.part.m[pc.slot * kMaxRows + r] = mm;
+                    p.part.l[pc.slot * kMaxRows + r] = L;
+                }
+            }
+            tc_fence_before();
+        }
+
+        // ---- end of piece: everything of this piece has completed (or the CTA is aborting)
+        __syncthreads();
+        if (*abort) break;
+        g0 += pc.nt;
+        u_base[0] += (pc.nt + 1) >> 1;
+        u_base[1] += pc.nt >> 1;
+        ++piece_idx;
+        t += pc.nt;
+    }
+
+    if (*abort) {
+        // drain TMA copies still in flight before the shared memory is given back
+        if (warp == kProducerWarp) {
+            for (int g = max(0, issued - C::kStages); g < issued; ++g) {
+                const int st = g % C::kStages, use = g / C::kStages;
+                for (uint32_t it = 0; it < kSpinLimit; ++it)
+                    if (mbar_try_wait(&bars->kv_full[st], use & 1)) break;
+            }
+        }
+        if (tid == 0) atomicOr(p.status, FD_DEV_TIMEOUT);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+struct TmapEntry {
+    const void* ptr;
+    int num_pages;
+    CUtensorMap map;
+};
+
+struct TcState {
+    PFN_cuTensorMapEncodeTiled_v12000 encode;
+    TmapEntry cache[64];
+    int n_cached, next;
+    int d, hkv;
+    const CUtensorMap* current;
+};
+
+}  // namespace
+
+bool attn_tc_supported(int d, int G, int max_q_len) {
+    return (d == 64 || d == 128) && G * max_q_len <= kMaxRows;
+}
+
+// Looks up (or encodes) the tensor map of this KV pool: a 2-D view [rows = pages*2*Hkv*16, d]
+// with a 16-row x 64-element box and 128-byte swizzle.
+cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
+    TcState* st = static_cast<TcState*>(*state);
+    if (!st) {
+        st = new TcState();
+        st->n_cached = st->next = 0;
+        st->encode = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", reinterpret_cast<void**>(&st->encode), cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !st->encode) { delete st; return e != cudaSuccess ? e : cudaErrorNotSupported; }
+        st->d = p.d; st->hkv = p.Hkv;
+        if (p.d == 64) e = cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+        else e = cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+        if (e != cudaSuccess) { delete st; return e; }
+        *state = st;
+    }
+    for (int i = 0; i < st->n_cached; ++i)
+        if (st->cache[i].ptr == p.kv && st->cache[i].num_pages == p.num_pages) { st->current = &st->cache[i].map; return cudaSuccess; }
+    TmapEntry& e = st->cache[st->next];
+    cuuint64_t dims[2] = {(cuuint64_t)p.d, (cuuint64_t)p.num_pages * 2 * p.Hkv * 16};
+    cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
+    cuuint32_t box[2] = {64, 16};
+    cuuint32_t estr[2] = {1, 1};
+    const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(p.kv), dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    e.ptr = p.kv;
+    e.num_pages = p.num_pages;
+    st->current = &e.map;
+    st->next = (st->next + 1) % 64;
+    if (st->n_cached < 64) ++st->n_cached;
+    return cudaSuccess;
+}
+
+void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s) {
+    if (p.batch == 0) return;
+    const TcState* st = static_cast<const TcState*>(state);
+    if (p.d == 64) attn_tc_kernel<64><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, s>>>(*st->current, p);
+    else attn_tc_kernel<128><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, s>>>(*st->current, p);
+}
+
+void attn_tc_free(void* state) { delete static_cast<TcState*>(state); }
+
 }  // namespace fd

@@ -26,6 +26,8 @@ def test_attention_workloads(idx, path):
     step = wl.workload(idx)
     q, kv = wl.make_q(step), wl.make_kv(step)
     with Ctx(step, path) as ctx:
+        # the auto path must be the tensor-core kernel for every benchmark shape
+        assert fd.fd_attn_path(ctx.h) == (fd.FD_ATTN_SIMT if path == fd.FD_ATTN_SIMT else fd.FD_ATTN_TCGEN05)
         got, status = gpu_attn(ctx, step, q, kv)
     assert status == 0
     assert_close(got.numpy(), oracle_attn(step, q, kv), step.name)
