@@ -93,6 +93,12 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_
     return pc;
 }
 
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // Warp-uniform bounded wait.
 __device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, volatile int* abort) {
     const bool ok = mbar_wait(bar, parity, abort);
@@ -250,24 +256,35 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                 tc_fence_after();
                 if (warp_active) {
                     const int pos0 = (pc.tile0 + j) * kTileTokens;
-                    uint32_t sv[4][32];
+                    // tile reaches into the query block (or past kv_len): columns >= lim are invisible
+                    const bool masked = pos0 + kTileTokens > pc.n;
+                    const int lim = limit - pos0;
+                    const uint32_t s_addr = tmem + lane_base + col_s[s];
+
+                    // ---- pass 1: row maximum (S is read from TMEM twice; keeping it in registers spills)
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) tmem_ld32(tmem + lane_base + col_s[s] + ch * 32, sv[ch]);
-                    tc_wait_ld();
-                    if (pos0 + kTileTokens > pc.n) {  // tile reaches into the query block (or past kv_len)
-                        const int lim = limit - pos0;
+                    for (int hp = 0; hp < 2; ++hp) {
+                        uint32_t a[32], b[32];
+                        tmem_ld32(s_addr + hp * 64, a);
+                        tmem_ld32(s_addr + hp * 64 + 32, b);
+                        tc_wait_ld();
+                        if (masked) {
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch)
+                            for (int k = 0; k < 32; ++k) {
+                                if (hp * 64 + k >= lim) a[k] = 0xff800000u;       // -inf by select: S may be NaN there
+                                if (hp * 64 + 32 + k >= lim) b[k] = 0xff800000u;
+                            }
+                        }
 #pragma unroll
-                            for (int k = 0; k < 32; ++k)
-                                if (ch * 32 + k >= lim) sv[ch][k] = 0xff800000u;  // -inf, a select: S may be NaN there
+                        for (int k = 0; k < 32; k += 2) {
+                            mx[0] = fmaxf(mx[0], __uint_as_float(a[k]));
+                            mx[1] = fmaxf(mx[1], __uint_as_float(a[k + 1]));
+                            mx[2] = fmaxf(mx[2], __uint_as_float(b[k]));
+                            mx[3] = fmaxf(mx[3], __uint_as_float(b[k + 1]));
+                        }
                     }
-                    float mx = -INFINITY;
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch)
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(sv[ch][k]));
-                    const float m_new = fmaxf(m, mx * c);
+                    const float m_new = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c);
                     float alpha = 1.f;
                     if (j < 2 || m == -INFINITY) {
                         m = m_new;  // nothing accumulated yet (O is overwritten, or exactly zero)
@@ -288,22 +305,39 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                         }
                         l *= alpha;
                     }
+
+                    // ---- pass 2: P = exp2(S * c - m), row sum, bf16 P written over S (64 tokens -> 32 columns)
                     const float mc = (m == -INFINITY) ? 0.f : m;
+                    const float2 c2 = make_float2(c, c), nm2 = make_float2(-mc, -mc);
+                    float2 sum0 = make_float2(0.f, 0.f), sum1 = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int ch = 0; ch < 4; ch += 2) {
-                        uint32_t pk[32];
+                    for (int hp = 0; hp < 2; ++hp) {
+                        uint32_t a[32], b[32], pk[32];
+                        tmem_ld32(s_addr + hp * 64, a);
+                        tmem_ld32(s_addr + hp * 64 + 32, b);
+                        tc_wait_ld();
+                        if (masked) {
 #pragma unroll
-                        for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-                            for (int k = 0; k < 32; k += 2) {
-                                const float p0 = exp2f(fmaf(__uint_as_float(sv[ch + hh][k]), c, -mc));
-                                const float p1 = exp2f(fmaf(__uint_as_float(sv[ch + hh][k + 1]), c, -mc));
-                                l += p0 + p1;
-                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                                pk[hh * 16 + (k >> 1)] = *reinterpret_cast<const uint32_t*>(&b2);
+                            for (int k = 0; k < 32; ++k) {
+                                if (hp * 64 + k >= lim) a[k] = 0xff800000u;
+                                if (hp * 64 + 32 + k >= lim) b[k] = 0xff800000u;
                             }
-                        tmem_st32(tmem + lane_base + col_s[s] + (ch >> 1) * 32, pk);
+                        }
+#pragma unroll
+                        for (int k = 0; k < 32; k += 2) {
+                            const float2 xa = __ffma2_rn(make_float2(__uint_as_float(a[k]), __uint_as_float(a[k + 1])), c2, nm2);
+                            const float2 xb = __ffma2_rn(make_float2(__uint_as_float(b[k]), __uint_as_float(b[k + 1])), c2, nm2);
+                            const float2 pa = make_float2(ex2_approx(xa.x), ex2_approx(xa.y));
+                            const float2 pb = make_float2(ex2_approx(xb.x), ex2_approx(xb.y));
+                            sum0 = __fadd2_rn(sum0, pa);
+                            sum1 = __fadd2_rn(sum1, pb);
+                            const __nv_bfloat162 ba = __floats2bfloat162_rn(pa.x, pa.y), bb = __floats2bfloat162_rn(pb.x, pb.y);
+                            pk[k >> 1] = *reinterpret_cast<const uint32_t*>(&ba);
+                            pk[16 + (k >> 1)] = *reinterpret_cast<const uint32_t*>(&bb);
+                        }
+                        tmem_st32(s_addr + hp * 32, pk);  // overwrites S columns already consumed
                     }
+                    l += (sum0.x + sum0.y) + (sum1.x + sum1.y);
                     tc_wait_st();
                 }
                 tc_fence_before();
