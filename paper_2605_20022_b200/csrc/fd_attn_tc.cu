@@ -9,8 +9,9 @@
 // One piece.  The G * Lq_b <= 128 query rows that share the kv-head (row r = block row
 // r / G of q-head kvh * G + r % G) form the M = 128 operand of every MMA, so each KV tile is
 // read from HBM once for all of them.  Per tile j of the piece:
-//     producer warp : 32 lanes issue one 2 KB TMA box each (8 pages x {K,V} x two 64-wide
-//                     halves of d) into a 128B-swizzled stage of a 3-deep ring;
+//     producer warps: one for K, one for V; 16 lanes issue one 2 KB TMA box each (8 pages x two
+//                     64-wide halves of d) into a 128B-swizzled buffer of a 3-deep ring per
+//                     operand; a K buffer is released by the QK^T commit, a V buffer by P V;
 //     MMA warp      : S_s = Q K^T (tcgen05.mma, A and B from shared memory, S in TMEM), and
 //                     after the softmax O_s += P_s V (A = P from TMEM, B = V MN-major);
 //     softmax group : 128 threads, one query row each: tcgen05.ld the row of S, hybrid mask
@@ -38,24 +39,23 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kThreads = 320;  // warps 0-3 softmax group 0, 4-7 softmax group 1, 8 producer, 9 MMA
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 384;  // warps 0-3 softmax group 0, 4-7 softmax group 1, 8 K loads, 9 V loads, 10 MMA, 11 idle
+constexpr int kKWarp = 8, kVWarp = 9, kMmaWarp = 10;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 template <int D>
 struct Cfg {
-    static constexpr int kStages = (D == 128) ? 3 : 4;
+    static constexpr int kStages = (D == 128) ? 3 : 6;   // buffers in the K ring, and again in the V ring
     static constexpr int kQBytes = kMaxRows * D * 2;
-    static constexpr int kKBytes = kTileTokens * D * 2;
-    static constexpr int kStageBytes = 2 * kKBytes;
-    static constexpr int kBarOffset = kQBytes + kStages * kStageBytes;
-    static constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // + barriers + slack for 1024-byte alignment
+    static constexpr int kKBytes = kTileTokens * D * 2;  // one K (or V) tile
+    static constexpr int kBarOffset = kQBytes + 2 * kStages * kKBytes;
+    static constexpr int kSmemBytes = kBarOffset + 512 + 1024;  // + barriers + slack for 1024-byte alignment
     static constexpr int kKSteps = D / 16;
     static constexpr int kHalves = D / 64;
 };
 
 struct Bars {
-    uint64_t kv_full[4], kv_empty[4];
+    uint64_t k_full[6], k_empty[6], v_full[6], v_empty[6];
     uint64_t s_full[2], p_full[2], pv_done[2];
     uint64_t all_done;
     uint32_t tmem_base;
@@ -93,6 +93,20 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_
     return pc;
 }
 
+#ifdef FD_TRACE
+// Debug build only: per-role timestamps of CTA 0 (role, event, tile, clock) for pipeline analysis.
+__device__ unsigned long long g_trace[4 * 8192];
+__device__ unsigned int g_trace_n;
+__device__ __forceinline__ void trace(int role, int ev, int tile) {
+    if (blockIdx.x != 0) return;
+    const unsigned int i = atomicAdd(&g_trace_n, 1u);
+    if (i < 8192) { g_trace[4 * i] = role; g_trace[4 * i + 1] = ev; g_trace[4 * i + 2] = tile; g_trace[4 * i + 3] = clock64(); }
+}
+#define TRACE(role, ev, tile) trace(role, ev, tile)
+#else
+#define TRACE(role, ev, tile)
+#endif
+
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -111,7 +125,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* sq = smem;
-    unsigned char* sstage = smem + C::kQBytes;
+    unsigned char* sk = smem + C::kQBytes;                      // K ring
+    unsigned char* sv = sk + C::kStages * C::kKBytes;           // V ring
     Bars* bars = reinterpret_cast<Bars*>(smem + C::kBarOffset);
     float* ex_m = reinterpret_cast<float*>(sq);          // [2][128], aliases Q after the last MMA of a piece
     float* ex_l = ex_m + 2 * kMaxRows;
@@ -126,7 +141,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     if (s_c >= e_c) return;
 
     if (tid == 0) {
-        for (int i = 0; i < C::kStages; ++i) { mbar_init(&bars->kv_full[i], 1); mbar_init(&bars->kv_empty[i], 1); }
+        for (int i = 0; i < C::kStages; ++i) {
+            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
+            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars->s_full[i], 1);
             mbar_init(&bars->p_full[i], 128);
@@ -137,7 +155,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         mbar_fence_init();
     }
     if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
-    if (warp == kProducerWarp && lane == 0) prefetch_tmap(&tmap);
+    if (warp == kKWarp && lane == 0) prefetch_tmap(&tmap);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -165,21 +183,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         fence_proxy_async_smem();
         __syncthreads();
 
-        if (warp == kProducerWarp) {
-            // ============================== TMA producer ==============================
-            constexpr int kOps = 8 * 2 * C::kHalves;
-            const int pg = lane / (2 * C::kHalves), which = (lane / C::kHalves) & 1, half = lane % C::kHalves;
+        if (warp == kKWarp || warp == kVWarp) {
+            // ============================== TMA producers ==============================
+            // K and V travel through separate rings: a K buffer is free again as soon as QK^T of its
+            // tile has completed, a V buffer once P V has, so loads run several tiles ahead of the MMAs.
+            const int which = (warp == kVWarp) ? 1 : 0;
+            unsigned char* ring = which ? sv : sk;
+            uint64_t* full = which ? bars->v_full : bars->k_full;
+            uint64_t* empty = which ? bars->v_empty : bars->k_empty;
+            constexpr int kOps = 8 * C::kHalves;
+            const int pg = lane / C::kHalves, half = lane % C::kHalves;
             for (int j = 0; j < pc.nt; ++j) {
                 const int g = g0 + j, st = g % C::kStages, use = g / C::kStages;
-                if (!wait_all(&bars->kv_empty[st], (use & 1) ^ 1, abort)) break;
+                if (!wait_all(&empty[st], (use & 1) ^ 1, abort)) break;
+                if (lane == 0) TRACE(which, 0, g0 + j);
                 const int pos0 = (pc.tile0 + j) * kTileTokens;
                 const int npg = min(8, (pc.kv_len - pos0 + 15) >> 4);
-                if (lane == 0) mbar_arrive_expect_tx(&bars->kv_full[st], npg * (2 * 16 * D * 2));
+                if (lane == 0) mbar_arrive_expect_tx(&full[st], npg * (16 * D * 2));
                 __syncwarp();
                 if (lane < kOps && pg < npg) {
                     const int phys = p.page_table[(long long)pc.b * p.max_pages + (pos0 >> 4) + pg];
-                    unsigned char* dst = sstage + st * C::kStageBytes + which * C::kKBytes + half * (kTileTokens * 128) + pg * 2048;
-                    tma_load_2d(dst, &tmap, half * 64, ((phys * 2 + which) * p.Hkv + pc.kvh) * 16, &bars->kv_full[st]);
+                    unsigned char* dst = ring + st * C::kKBytes + half * (kTileTokens * 128) + pg * 2048;
+                    tma_load_2d(dst, &tmap, half * 64, ((phys * 2 + which) * p.Hkv + pc.kvh) * 16, &full[st]);
                 }
                 issued = g + 1;
             }
@@ -190,16 +215,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             const uint32_t q_addr = smem_u32(sq);
             bool ok = true;
             auto issue_pv = [&](int jj) {
-                const int s = jj & 1, st = (g0 + jj) % C::kStages, u = u_base[s] + (jj >> 1);
+                const int gg = g0 + jj, s = jj & 1, st = gg % C::kStages, u = u_base[s] + (jj >> 1);
+                if (!wait_all(&bars->v_full[st], (gg / C::kStages) & 1, abort)) { ok = false; return; }
+                unsigned char* vt = sv + st * C::kKBytes;
+                const int valid = pc.kv_len - (pc.tile0 + jj) * kTileTokens;
+                if (valid < kTileTokens) {
+                    // V rows no token owns may hold NaN or stale data: P is 0 there, but 0 * NaN is not
+                    const int nbad = kTileTokens - valid;
+                    for (int e = lane; e < nbad * 8 * C::kHalves; e += 32) {
+                        const int r = valid + e / (8 * C::kHalves), w = e % (8 * C::kHalves);
+                        *reinterpret_cast<uint4*>(vt + (w >> 3) * (kTileTokens * 128) + r * 128 + ((w & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                }
                 if (!wait_all(&bars->p_full[s], u & 1, abort)) { ok = false; return; }
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t v_addr = smem_u32(sstage + st * C::kStageBytes + C::kKBytes);
+                    TRACE(2, 2, g0 + jj);
+                    const uint32_t v_addr = smem_u32(vt);
 #pragma unroll
                     for (int kk = 0; kk < kTileTokens / 16; ++kk)
                         umma_ts(tmem + col_o[s], tmem + col_s[s] + kk * 8,
                                 make_smem_desc(v_addr + kk * 2048, kTileTokens * 128, 1024), idesc_pv, jj >= 2 || kk > 0);
-                    umma_commit(&bars->kv_empty[st]);
+                    umma_commit(&bars->v_empty[st]);
                     umma_commit(&bars->pv_done[s]);
                 }
                 __syncwarp();
@@ -207,29 +246,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             for (int j = 0; j < pc.nt && ok; ++j) {
                 const int g = g0 + j, st = g % C::kStages, use = g / C::kStages;
                 const int s = j & 1, u = u_base[s] + (j >> 1);
-                if (!wait_all(&bars->kv_full[st], use & 1, abort)) { ok = false; break; }
-                const int valid = pc.kv_len - (pc.tile0 + j) * kTileTokens;
-                if (valid < kTileTokens) {
-                    // V rows no token owns may hold NaN or stale data: P is 0 there, but 0 * NaN is not
-                    unsigned char* sv = sstage + st * C::kStageBytes + C::kKBytes;
-                    const int nbad = kTileTokens - valid;
-                    for (int e = lane; e < nbad * 8 * C::kHalves; e += 32) {
-                        const int r = valid + e / (8 * C::kHalves), w = e % (8 * C::kHalves);
-                        *reinterpret_cast<uint4*>(sv + (w >> 3) * (kTileTokens * 128) + r * 128 + ((w & 7) << 4)) = make_uint4(0, 0, 0, 0);
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                }
+                if (!wait_all(&bars->k_full[st], use & 1, abort)) { ok = false; break; }
+                if (lane == 0) TRACE(2, 0, g);
                 if (u >= 1 && !wait_all(&bars->pv_done[s], (u - 1) & 1, abort)) { ok = false; break; }
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t k_addr = smem_u32(sstage + st * C::kStageBytes);
+                    TRACE(2, 1, g);
+                    const uint32_t k_addr = smem_u32(sk + st * C::kKBytes);
 #pragma unroll
                     for (int kk = 0; kk < C::kKSteps; ++kk) {
                         const uint32_t off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
                         umma_ss(tmem + col_s[s], make_smem_desc(q_addr + off, 16, 1024), make_smem_desc(k_addr + off, 16, 1024),
                                 idesc_qk, kk > 0);
                     }
+                    umma_commit(&bars->k_empty[st]);
                     umma_commit(&bars->s_full[s]);
                 }
                 __syncwarp();
@@ -238,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             if (ok) issue_pv(pc.nt - 1);
             if (ok && lane == 0) umma_commit(&bars->all_done);
             __syncwarp();
-        } else {
+        } else if (warp < 8) {
             // ============================== softmax groups ==============================
             const int s = warp >> 2;                  // stream
             const int r = (warp & 3) * 32 + lane;     // query row == TMEM lane
@@ -254,6 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                 const int u = u_base[s] + (j >> 1);
                 if (!wait_all(&bars->s_full[s], u & 1, abort)) { ok = false; break; }
                 tc_fence_after();
+                if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 0, g0 + j);
                 if (warp_active) {
                     const int pos0 = (pc.tile0 + j) * kTileTokens;
                     // tile reaches into the query block (or past kv_len): columns >= lim are invisible
@@ -285,6 +316,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                         }
                     }
                     const float m_new = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c);
+                    if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 1, g0 + j);
                     float alpha = 1.f;
                     if (j < 2 || m == -INFINITY) {
                         m = m_new;  // nothing accumulated yet (O is overwritten, or exactly zero)
@@ -342,6 +374,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                 }
                 tc_fence_before();
                 mbar_arrive(&bars->p_full[s]);
+                if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 2, g0 + j);
             }
 
             // ---- epilogue: merge the two streams, then final rows or a partial for the merge kernel
@@ -412,11 +445,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 
     if (*abort) {
         // drain TMA copies still in flight before the shared memory is given back
-        if (warp == kProducerWarp) {
+        if (warp == kKWarp || warp == kVWarp) {
+            uint64_t* full = (warp == kVWarp) ? bars->v_full : bars->k_full;
             for (int g = max(0, issued - C::kStages); g < issued; ++g) {
                 const int st = g % C::kStages, use = g / C::kStages;
                 for (uint32_t it = 0; it < kSpinLimit; ++it)
-                    if (mbar_try_wait(&bars->kv_full[st], use & 1)) break;
+                    if (mbar_try_wait(&full[st], use & 1)) break;
             }
         }
         if (tid == 0) atomicOr(p.status, FD_DEV_TIMEOUT);
@@ -490,5 +524,19 @@ void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s) {
 }
 
 void attn_tc_free(void* state) { delete static_cast<TcState*>(state); }
+
+#ifdef FD_TRACE
+extern "C" int fd_debug_read_trace(unsigned long long* dst, int max_events) {
+    unsigned int n = 0;
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n));
+    if (n > 8192) n = 8192;
+    if ((int)n > max_events) n = max_events;
+    cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * 4 * n);
+    unsigned int zero = 0;
+    cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero));
+    return (int)n;
+}
+#endif
 
 }  // namespace fd
