@@ -109,7 +109,7 @@ __device__ __forceinline__ void trace(int role, int ev, int tile) {
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
@@ -119,46 +119,20 @@ __device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, volatil
     return __all_sync(0xffffffffu, ok);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, AttnParams p) {
+// Everything after the set-up, for one role class.  The two instantiations (softmax groups /
+// producer + MMA warps) run in disjoint branches of the kernel so that each is compiled for its
+// own register budget (setmaxnreg); they meet only at the CTA-wide barriers, which both execute
+// the same number of times.
+template <int D, bool kSoftmax>
+__device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnParams& p, unsigned char* sq, unsigned char* sk,
+                                         unsigned char* sv, Bars* bars, int total, int s_c, int e_c) {
     using C = Cfg<D>;
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* sq = smem;
-    unsigned char* sk = smem + C::kQBytes;                      // K ring
-    unsigned char* sv = sk + C::kStages * C::kKBytes;           // V ring
-    Bars* bars = reinterpret_cast<Bars*>(smem + C::kBarOffset);
     float* ex_m = reinterpret_cast<float*>(sq);          // [2][128], aliases Q after the last MMA of a piece
     float* ex_l = ex_m + 2 * kMaxRows;
     volatile int* abort = &bars->abort;
-
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const PlanHeader hdr = *p.plan.hdr;
-    const int total = hdr.total_tiles;
-    if (total == 0) return;  // uniform: nothing allocated yet
     const int cta = blockIdx.x;
-    const int s_c = range_begin(cta, total, p.n_ctas), e_c = range_begin(cta + 1, total, p.n_ctas);
-    if (s_c >= e_c) return;
-
-    if (tid == 0) {
-        for (int i = 0; i < C::kStages; ++i) {
-            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
-            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&bars->s_full[i], 1);
-            mbar_init(&bars->p_full[i], 128);
-            mbar_init(&bars->pv_done[i], 1);
-        }
-        mbar_init(&bars->all_done, 1);
-        bars->abort = 0;
-        mbar_fence_init();
-    }
-    if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
-    if (warp == kKWarp && lane == 0) prefetch_tmap(&tmap);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    (void)total;
     const uint32_t tmem = bars->tmem_base;
     const uint32_t col_s[2] = {0u, 128u};
     const uint32_t col_o[2] = {256u, 384u};
@@ -183,6 +157,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         fence_proxy_async_smem();
         __syncthreads();
 
+        if constexpr (!kSoftmax) {
         if (warp == kKWarp || warp == kVWarp) {
             // ============================== TMA producers ==============================
             // K and V travel through separate rings: a K buffer is free again as soon as QK^T of its
@@ -193,19 +168,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             uint64_t* empty = which ? bars->v_empty : bars->k_empty;
             constexpr int kOps = 8 * C::kHalves;
             const int pg = lane / C::kHalves, half = lane % C::kHalves;
+            const int32_t* table = p.page_table + (long long)pc.b * p.max_pages;
+            // the page id of the next tile is fetched before waiting for a free buffer, so the
+            // table lookup never sits between a buffer becoming free and its refill
+            auto page_of = [&](int j) -> int {
+                const int pos = (pc.tile0 + j) * kTileTokens + pg * 16;
+                return (j < pc.nt && lane < kOps && pos < pc.kv_len) ? table[pos >> 4] : -1;
+            };
+            int phys = page_of(0);
             for (int j = 0; j < pc.nt; ++j) {
                 const int g = g0 + j, st = g % C::kStages, use = g / C::kStages;
+                const int phys_next = page_of(j + 1);
                 if (!wait_all(&empty[st], (use & 1) ^ 1, abort)) break;
                 if (lane == 0) TRACE(which, 0, g0 + j);
                 const int pos0 = (pc.tile0 + j) * kTileTokens;
                 const int npg = min(8, (pc.kv_len - pos0 + 15) >> 4);
                 if (lane == 0) mbar_arrive_expect_tx(&full[st], npg * (16 * D * 2));
                 __syncwarp();
-                if (lane < kOps && pg < npg) {
-                    const int phys = p.page_table[(long long)pc.b * p.max_pages + (pos0 >> 4) + pg];
+                if (phys >= 0) {
                     unsigned char* dst = ring + st * C::kKBytes + half * (kTileTokens * 128) + pg * 2048;
                     tma_load_2d(dst, &tmap, half * 64, ((phys * 2 + which) * p.Hkv + pc.kvh) * 16, &full[st]);
                 }
+                phys = phys_next;
                 issued = g + 1;
             }
         } else if (warp == kMmaWarp) {
@@ -268,7 +252,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             if (ok) issue_pv(pc.nt - 1);
             if (ok && lane == 0) umma_commit(&bars->all_done);
             __syncwarp();
-        } else if (warp < 8) {
+        }
+        } else {
             // ============================== softmax groups ==============================
             const int s = warp >> 2;                  // stream
             const int r = (warp & 3) * 32 + lane;     // query row == TMEM lane
@@ -292,29 +277,29 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                     const int lim = limit - pos0;
                     const uint32_t s_addr = tmem + lane_base + col_s[s];
 
-                    // ---- pass 1: row maximum (S is read from TMEM twice; keeping it in registers spills)
+                    // ---- the whole row of S in one round trip: TMEM loads queue behind the MMAs in flight,
+                    //      so every ld -> wait pair costs up to one MMA tile; registers come from setmaxnreg
+                    uint32_t sv[4][32];
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, sv[ch]);
+                    tc_wait_ld();
+                    if (masked) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+                            for (int k = 0; k < 32; ++k)
+                                if (ch * 32 + k >= lim) sv[ch][k] = 0xff800000u;  // -inf by select: S may be NaN there
+                    }
                     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int hp = 0; hp < 2; ++hp) {
-                        uint32_t a[32], b[32];
-                        tmem_ld32(s_addr + hp * 64, a);
-                        tmem_ld32(s_addr + hp * 64 + 32, b);
-                        tc_wait_ld();
-                        if (masked) {
+                    for (int ch = 0; ch < 4; ++ch)
 #pragma unroll
-                            for (int k = 0; k < 32; ++k) {
-                                if (hp * 64 + k >= lim) a[k] = 0xff800000u;       // -inf by select: S may be NaN there
-                                if (hp * 64 + 32 + k >= lim) b[k] = 0xff800000u;
-                            }
+                        for (int k = 0; k < 32; k += 4) {
+                            mx[0] = fmaxf(mx[0], __uint_as_float(sv[ch][k]));
+                            mx[1] = fmaxf(mx[1], __uint_as_float(sv[ch][k + 1]));
+                            mx[2] = fmaxf(mx[2], __uint_as_float(sv[ch][k + 2]));
+                            mx[3] = fmaxf(mx[3], __uint_as_float(sv[ch][k + 3]));
                         }
-#pragma unroll
-                        for (int k = 0; k < 32; k += 2) {
-                            mx[0] = fmaxf(mx[0], __uint_as_float(a[k]));
-                            mx[1] = fmaxf(mx[1], __uint_as_float(a[k + 1]));
-                            mx[2] = fmaxf(mx[2], __uint_as_float(b[k]));
-                            mx[3] = fmaxf(mx[3], __uint_as_float(b[k + 1]));
-                        }
-                    }
                     const float m_new = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c);
                     if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 1, g0 + j);
                     float alpha = 1.f;
@@ -326,39 +311,29 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                     }
                     if (__any_sync(0xffffffffu, alpha != 1.f)) {
                         // previous PV of this stream has completed (S/P buffer reuse orders it), so O is quiescent
-#pragma unroll
-                        for (int ch = 0; ch < D / 32; ++ch) {
-                            uint32_t o[32];
-                            tmem_ld32(tmem + lane_base + col_o[s] + ch * 32, o);
+#pragma unroll 1
+                        for (int ch = 0; ch < D / 16; ++ch) {
+                            uint32_t o[16];
+                            tmem_ld16(tmem + lane_base + col_o[s] + ch * 16, o);
                             tc_wait_ld();
 #pragma unroll
-                            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                            tmem_st32(tmem + lane_base + col_o[s] + ch * 32, o);
+                            for (int k = 0; k < 16; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                            tmem_st16(tmem + lane_base + col_o[s] + ch * 16, o);
                         }
                         l *= alpha;
                     }
 
-                    // ---- pass 2: P = exp2(S * c - m), row sum, bf16 P written over S (64 tokens -> 32 columns)
+                    // ---- P = exp2(S * c - m), row sum, bf16 P written over S (64 tokens -> 32 columns)
                     const float mc = (m == -INFINITY) ? 0.f : m;
                     const float2 c2 = make_float2(c, c), nm2 = make_float2(-mc, -mc);
                     float2 sum0 = make_float2(0.f, 0.f), sum1 = make_float2(0.f, 0.f);
 #pragma unroll
                     for (int hp = 0; hp < 2; ++hp) {
-                        uint32_t a[32], b[32], pk[32];
-                        tmem_ld32(s_addr + hp * 64, a);
-                        tmem_ld32(s_addr + hp * 64 + 32, b);
-                        tc_wait_ld();
-                        if (masked) {
-#pragma unroll
-                            for (int k = 0; k < 32; ++k) {
-                                if (hp * 64 + k >= lim) a[k] = 0xff800000u;
-                                if (hp * 64 + 32 + k >= lim) b[k] = 0xff800000u;
-                            }
-                        }
+                        uint32_t pk[32];
 #pragma unroll
                         for (int k = 0; k < 32; k += 2) {
-                            const float2 xa = __ffma2_rn(make_float2(__uint_as_float(a[k]), __uint_as_float(a[k + 1])), c2, nm2);
-                            const float2 xb = __ffma2_rn(make_float2(__uint_as_float(b[k]), __uint_as_float(b[k + 1])), c2, nm2);
+                            const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sv[2 * hp][k]), __uint_as_float(sv[2 * hp][k + 1])), c2, nm2);
+                            const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sv[2 * hp + 1][k]), __uint_as_float(sv[2 * hp + 1][k + 1])), c2, nm2);
                             const float2 pa = make_float2(ex2_approx(xa.x), ex2_approx(xa.y));
                             const float2 pb = make_float2(ex2_approx(xb.x), ex2_approx(xb.y));
                             sum0 = __fadd2_rn(sum0, pa);
@@ -367,7 +342,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                             pk[k >> 1] = *reinterpret_cast<const uint32_t*>(&ba);
                             pk[16 + (k >> 1)] = *reinterpret_cast<const uint32_t*>(&bb);
                         }
-                        tmem_st32(s_addr + hp * 32, pk);  // overwrites S columns already consumed
+                        tmem_st32(s_addr + hp * 32, pk);  // overwrites S columns that are already in registers
+                        asm volatile("" ::: "memory");    // keep the second half's math after this store (register pressure)
                     }
                     l += (sum0.x + sum0.y) + (sum1.x + sum1.y);
                     tc_wait_st();
@@ -449,7 +425,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             uint64_t* full = (warp == kVWarp) ? bars->v_full : bars->k_full;
             for (int g = max(0, issued - C::kStages); g < issued; ++g) {
                 const int st = g % C::kStages, use = g / C::kStages;
-                for (uint32_t it = 0; it < kSpinLimit; ++it)
+                const unsigned long long t0 = global_ns();
+                for (uint32_t it = 0; it < kSpinLimit && global_ns() - t0 < kWaitLimitNs; ++it)
                     if (mbar_try_wait(&full[st], use & 1)) break;
             }
         }
@@ -458,6 +435,55 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, AttnParams p) {
+    using C = Cfg<D>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* sq = smem;
+    unsigned char* sk = smem + C::kQBytes;                      // K ring
+    unsigned char* sv = sk + C::kStages * C::kKBytes;           // V ring
+    Bars* bars = reinterpret_cast<Bars*>(smem + C::kBarOffset);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const PlanHeader hdr = *p.plan.hdr;
+    const int total = hdr.total_tiles;
+    if (total == 0) return;  // uniform: nothing allocated yet
+    const int cta = blockIdx.x;
+    const int s_c = range_begin(cta, total, p.n_ctas), e_c = range_begin(cta + 1, total, p.n_ctas);
+    if (s_c >= e_c) return;
+
+    if (tid == 0) {
+        for (int i = 0; i < C::kStages; ++i) {
+            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
+            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->s_full[i], 1);
+            mbar_init(&bars->p_full[i], 128);
+            mbar_init(&bars->pv_done[i], 1);
+        }
+        mbar_init(&bars->all_done, 1);
+        bars->abort = 0;
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
+    if (warp == kKWarp && lane == 0) prefetch_tmap(&tmap);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // warp-specialised register budgets: the softmax groups keep a whole 128-column row of S in registers.
+    // 8 x 32 x 216 + 4 x 32 x 72 = 384 x 168: exactly what the launch allocated, so the increase can
+    // always be served by what the decrease released (asking for more than that never returns).
+    if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        run_role<D, true>(tmap, p, sq, sk, sv, bars, total, s_c, e_c);
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        run_role<D, false>(tmap, p, sq, sk, sv, bars, total, s_c, e_c);
+    }
 }
 
 struct TmapEntry {
