@@ -75,7 +75,11 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
             for (int pg = 0; pg < kTileTokens / 16; ++pg) {
                 const int pos0 = tile * kTileTokens + pg * 16;
                 if (pos0 >= kv_len) break;
-                const int phys = p.page_table[(long long)b * p.max_pages + pos0 / 16];
+                int phys = p.page_table[(long long)b * p.max_pages + pos0 / 16];
+                if ((unsigned)phys >= (unsigned)p.num_pages) {  // never form an address from a bad id
+                    if (r == 0) { p.plan.seq_ok[b] = 0; atomicOr(p.status, FD_DEV_BAD_PAGE); }
+                    phys = 0;
+                }
                 const __nv_bfloat16* kp = p.kv + (((long long)phys * 2 + 0) * p.Hkv + kvh) * 16 * D;
                 const __nv_bfloat16* vp = p.kv + (((long long)phys * 2 + 1) * p.Hkv + kvh) * 16 * D;
                 __syncthreads();  // everyone is done with the previous page

@@ -173,7 +173,14 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
             // table lookup never sits between a buffer becoming free and its refill
             auto page_of = [&](int j) -> int {
                 const int pos = (pc.tile0 + j) * kTileTokens + pg * 16;
-                return (j < pc.nt && lane < kOps && pos < pc.kv_len) ? table[pos >> 4] : -1;
+                if (!(j < pc.nt && lane < kOps && pos < pc.kv_len)) return -1;
+                int id = table[pos >> 4];
+                if ((unsigned)id >= (unsigned)p.num_pages) {  // never form an address from a bad id
+                    p.plan.seq_ok[pc.b] = 0;
+                    atomicOr(p.status, FD_DEV_BAD_PAGE);
+                    id = 0;
+                }
+                return id;
             };
             int phys = page_of(0);
             for (int j = 0; j < pc.nt; ++j) {

@@ -6,53 +6,69 @@
 // same number of KV bytes whatever the mix of prefix lengths.  A (sequence, kv-head)
 // segment that falls into several ranges leaves one partial result per range; the merge
 // kernel combines them in range order, which makes the result independent of timing.
+//
+// The plan kernel checks the lengths (O(B) work, one CTA).  Page ids are checked where they are
+// used, by the attention kernels: a sequence with an id outside the pool is flagged in seq_ok,
+// read from page 0 instead, and has its output rows zeroed by the merge kernel.
 #include "fd_internal.cuh"
 
 namespace fd {
 
+// Inclusive scan of (a, b) pairs over the 256 threads of the CTA; returns the totals in (ta, tb).
+__device__ inline void block_scan2(int& a, int& b, int& ta, int& tb, int (*wsum)[2]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int ua = __shfl_up_sync(0xffffffffu, a, o), ub = __shfl_up_sync(0xffffffffu, b, o);
+        if (lane >= o) { a += ua; b += ub; }
+    }
+    __syncthreads();  // wsum may still be read from the previous round
+    if (lane == 31) { wsum[warp][0] = a; wsum[warp][1] = b; }
+    __syncthreads();
+    int oa = 0, ob = 0;
+    ta = tb = 0;
+    for (int w = 0; w < 8; ++w) {
+        if (w < warp) { oa += wsum[w][0]; ob += wsum[w][1]; }
+        ta += wsum[w][0];
+        tb += wsum[w][1];
+    }
+    a += oa;
+    b += ob;
+}
+
 __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     __shared__ int s_fatal;
+    __shared__ int wsum[8][2];
     const int B = p.batch, tid = threadIdx.x;
     if (tid == 0) s_fatal = 0;
     __syncthreads();
     const int P = 16;
-    for (int b = tid; b < B; b += blockDim.x) {
-        const long long n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
-        const bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || Lq * p.G > kMaxRows ||
-                         n + Lq > (long long)p.max_pages * P;
-        if (bad) atomicOr(&s_fatal, 1);
-        p.plan.seq_ok[b] = 1;
-    }
-    __syncthreads();
-    if (!s_fatal) {
-        for (int b = 0; b < B; ++b) {
-            const int Lq = p.q_lens[b];
-            const int need = Lq > 0 ? (p.prefix_lens[b] + Lq + P - 1) / P : 0;
-            for (int pg = tid; pg < need; pg += blockDim.x) {
-                const int id = p.page_table[(long long)b * p.max_pages + pg];
-                if (id < 0 || id >= p.num_pages) {
-                    p.plan.seq_ok[b] = 0;
-                    atomicOr(p.status, FD_DEV_BAD_PAGE);
-                }
-            }
+    long long rows = 0, tiles = 0;  // running totals (identical in every thread)
+    for (int base = 0; base < B; base += blockDim.x) {
+        const int b = base + tid;
+        int q = 0, t = 0;
+        if (b < B) {
+            const long long n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
+            const bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || Lq * p.G > kMaxRows ||
+                             n + Lq > (long long)p.max_pages * P;
+            if (bad) atomicOr(&s_fatal, 1);
+            else { q = (int)Lq; t = Lq > 0 ? (int)((n + Lq + kTileTokens - 1) / kTileTokens) : 0; }
+            p.plan.seq_ok[b] = 1;
         }
+        int tq, tt;
+        block_scan2(q, t, tq, tt, wsum);
+        if (b < B) {
+            p.plan.cu_q[b + 1] = (int)min(rows + q, (long long)0x7fffffff);
+            p.plan.cu_tiles[b + 1] = (int)min(tiles + t, (long long)0x7fffffff);
+        }
+        rows += tq;
+        tiles += tt;
     }
     __syncthreads();
     if (tid == 0) {
-        long long rows = 0, tiles = 0;
-        int fatal = s_fatal;
+        const int fatal = s_fatal || rows != p.total_q_rows || tiles * p.Hkv > 0x7fffffffLL;
         p.plan.cu_q[0] = 0;
         p.plan.cu_tiles[0] = 0;
-        if (!fatal) {
-            for (int b = 0; b < B; ++b) {
-                const int Lq = p.q_lens[b];
-                rows += Lq;
-                if (Lq > 0 && p.plan.seq_ok[b]) tiles += (p.prefix_lens[b] + Lq + kTileTokens - 1) / kTileTokens;
-                p.plan.cu_q[b + 1] = (int)rows;
-                p.plan.cu_tiles[b + 1] = (int)tiles;
-            }
-            if (rows != p.total_q_rows || tiles * p.Hkv > 0x7fffffffLL) fatal = 1;
-        }
         if (fatal) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         p.plan.hdr->fatal = fatal;
         p.plan.hdr->total_tiles = fatal ? 0 : (int)(tiles * p.Hkv);
@@ -72,9 +88,14 @@ __device__ inline void store_row_bf16(__nv_bfloat16* dst, const float* o, float 
     }
 }
 
-// One CTA per (sequence, kv-head) segment, one thread per query row of the segment.
+// One CTA per (sequence, kv-head) segment; thread (r, cg) owns query row r = tid % 128 and the
+// column group cg = tid / 128 (a quarter of d), so the partial reads of a warp are coalesced
+// and enough loads are in flight to hide their latency.
+constexpr int kMergeThreads = 4 * kMaxRows;
+
 template <int D>
-__global__ void __launch_bounds__(kMaxRows) merge_kernel(AttnParams p) {
+__global__ void __launch_bounds__(kMergeThreads) merge_kernel(AttnParams p) {
+    constexpr int CW = D / 4;  // columns per thread
     const PlanHeader hdr = *p.plan.hdr;
     if (hdr.fatal) {  // defined output for an undefined request: zeros
         const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
@@ -86,14 +107,14 @@ __global__ void __launch_bounds__(kMaxRows) merge_kernel(AttnParams p) {
     }
     const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
     const int row0 = p.plan.cu_q[b], Lq = p.plan.cu_q[b + 1] - row0;
-    const int rows = Lq * p.G, r = threadIdx.x;
+    const int rows = Lq * p.G, r = threadIdx.x % kMaxRows, cg = threadIdx.x / kMaxRows;
     if (r >= rows) return;
-    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D;
-    float acc[D];
-    if (!p.plan.seq_ok[b]) {
+    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
+    float acc[CW];
 #pragma unroll
-        for (int c = 0; c < D; ++c) acc[c] = 0.f;
-        store_row_bf16<D>(dst, acc, 0.f);
+    for (int c = 0; c < CW; ++c) acc[c] = 0.f;
+    if (!p.plan.seq_ok[b]) {
+        store_row_bf16<CW>(dst, acc, 0.f);
         return;
     }
     const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
@@ -109,8 +130,6 @@ __global__ void __launch_bounds__(kMaxRows) merge_kernel(AttnParams p) {
         const int slot = 2 * c + (sc >= t0 ? 0 : 1);
         m = fmaxf(m, p.part.m[slot * kMaxRows + r]);
     }
-#pragma unroll
-    for (int c = 0; c < D; ++c) acc[c] = 0.f;
     float l = 0.f;
     for (int c = c_first; c <= c_last; ++c) {
         const int sc = range_begin(c, hdr.total_tiles, p.n_ctas), ec = range_begin(c + 1, hdr.total_tiles, p.n_ctas);
@@ -120,18 +139,18 @@ __global__ void __launch_bounds__(kMaxRows) merge_kernel(AttnParams p) {
         if (mp == -INFINITY) continue;  // this piece saw no visible key for the row
         const float w = exp2f(mp - m);
         l += w * p.part.l[slot * kMaxRows + r];
-        const float* o = p.part.o + (long long)slot * D * kMaxRows + r;
+        const float* o = p.part.o + ((long long)slot * D + cg * CW) * kMaxRows + r;
 #pragma unroll
-        for (int col = 0; col < D; ++col) acc[col] += w * o[col * kMaxRows];
+        for (int col = 0; col < CW; ++col) acc[col] += w * o[col * kMaxRows];
     }
-    store_row_bf16<D>(dst, acc, 1.f / l);
+    store_row_bf16<CW>(dst, acc, 1.f / l);
 }
 
 void launch_merge(const AttnParams& p, cudaStream_t s) {
     const int grid = p.batch * p.Hkv;
     if (grid == 0) return;
-    if (p.d == 64) merge_kernel<64><<<grid, kMaxRows, 0, s>>>(p);
-    else merge_kernel<128><<<grid, kMaxRows, 0, s>>>(p);
+    if (p.d == 64) merge_kernel<64><<<grid, kMergeThreads, 0, s>>>(p);
+    else merge_kernel<128><<<grid, kMergeThreads, 0, s>>>(p);
 }
 
 }  // namespace fd
