@@ -50,7 +50,8 @@ typedef enum {
     FD_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels implement */
     FD_ERR_WORKSPACE = 3,     /* scratch memory could not be allocated */
     FD_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
-    FD_ERR_DEVICE_STATUS = 5  /* reserved */
+    FD_ERR_DEVICE_STATUS = 5, /* reserved */
+    FD_ERR_STATIC_LIMIT = 6   /* fd_verify_accept_static: more rows or sequences than its fixed scratch holds */
 } fd_status;
 
 /* Bits of the sticky device status word. */
@@ -177,6 +178,44 @@ fd_status fd_verify_accept(fd_ctx* ctx, int batch, int total_cand_rows,
 fd_status fd_kv_commit(fd_ctx* ctx, int batch, int32_t* page_table, int32_t* prefix_lens,
                        const int32_t* q_lens, const int32_t* accepted_len,
                        int32_t* freed_pages, int32_t* n_freed, void* stream);
+
+/*
+ * fd_verify_accept without any allocation.  (The paper has no counterpart; this entry point
+ * exists for the callers described here.)
+ *
+ * Who needs it: code that must not call cudaMalloc -- a plugin running inside a serving
+ * process whose memory pool owns every byte of the device, a step that runs while a CUDA
+ * graph is being captured elsewhere in the process, a late-initialised worker that finds the
+ * device already full.  fd_create() is closed to such callers because it allocates the
+ * context's scratch memory.  This call needs no context: the (value, index) maxima of the
+ * vocabulary sweep and the finished-CTA counter live in a fixed array compiled into the
+ * library (FD_STATIC_MAX_ROWS * 8 bytes + 64 bytes = 32.06 KB of device memory on every GPU
+ * that loads the library, held until the process exits).
+ *
+ * Semantics, argument layout and results are those of fd_verify_accept, with these changes:
+ *   vocab           V, passed per call (there is no fd_config)
+ *   device_status   device pointer to one int32 that receives FD_DEV_* bits (OR-ed in; the
+ *                   caller clears it), or NULL to drop them
+ * Limits: total_cand_rows <= FD_STATIC_MAX_ROWS and batch <= FD_STATIC_MAX_BATCH, else
+ * FD_ERR_STATIC_LIMIT is returned and nothing is launched.
+ *
+ * The call allocates nothing: no cudaMalloc / cudaFree, no allocating library routine; it
+ * enqueues two small cudaMemsetAsync (the part of the array it is about to use keeps the
+ * previous call's contents and must start at zero) and one kernel on `stream`.
+ * First call on each device: the device address of the array is looked up once
+ * (cudaGetSymbolAddress, with that device current) and cached; make that first call outside
+ * any stream capture.
+ * Every call in the process shares the one array per device.  Calls issued on one stream are
+ * safe back to back; calls that can overlap on the GPU (different streams, different threads,
+ * different contexts of the same library image) race on it and must be serialised by the caller.
+ */
+#define FD_STATIC_MAX_ROWS 4096
+#define FD_STATIC_MAX_BATCH 4096
+fd_status fd_verify_accept_static(int vocab, int batch, int total_cand_rows,
+                                  const float* logits, const int32_t* draft_tokens,
+                                  const int32_t* q_lens, const int32_t* n_mask,
+                                  int32_t* accepted_len, int32_t* bonus_token,
+                                  int32_t* device_status, void* stream);
 
 /* Read and clear the sticky device status word (an OR of FD_DEV_* bits) into *code (host
  * pointer).  Synchronises `stream` first. */

@@ -16,11 +16,14 @@ from . import _build
 
 FD_OK = 0
 FD_ERR_INVALID_ARG, FD_ERR_UNSUPPORTED, FD_ERR_WORKSPACE, FD_ERR_CUDA, FD_ERR_DEVICE_STATUS = 1, 2, 3, 4, 5
+FD_ERR_STATIC_LIMIT = 6
+FD_STATIC_MAX_ROWS, FD_STATIC_MAX_BATCH = 4096, 4096
 FD_DEV_BAD_LENGTHS, FD_DEV_BAD_PAGE, FD_DEV_TIMEOUT, FD_DEV_BAD_ACCEPT = 1, 2, 4, 8
 FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
-           "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string"]
+           "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
+           "fd_verify_accept_static"]
 
 
 class fd_config(ctypes.Structure):
@@ -56,6 +59,7 @@ def load() -> ctypes.CDLL:
         lib.fd_attn_draft_verify.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp]
         lib.fd_verify_accept.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_kv_commit.argtypes = [vp, ci, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_verify_accept_static.argtypes = [ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         lib.fd_attn_path.argtypes = [vp]
         lib.fd_launch_count.argtypes = [vp]
@@ -122,6 +126,16 @@ def fd_verify_accept(ctx, batch, total_cand_rows, logits, draft_tokens, q_lens, 
     code = load().fd_verify_accept(ctx, batch, total_cand_rows, _ptr(logits), _ptr(draft_tokens), _ptr(q_lens),
                                    _ptr(n_mask), _ptr(accepted_len), _ptr(bonus_token), _stream(stream))
     return _check("fd_verify_accept", code, raise_on_error)
+
+
+def fd_verify_accept_static(vocab, batch, total_cand_rows, logits, draft_tokens, q_lens, n_mask, accepted_len,
+                            bonus_token, device_status=None, stream=None, raise_on_error=True) -> int:
+    """fd_verify_accept for callers that may not allocate: no context, scratch inside the library
+    (at most FD_STATIC_MAX_ROWS candidate rows).  Calls sharing a device must not overlap on the GPU."""
+    code = load().fd_verify_accept_static(vocab, batch, total_cand_rows, _ptr(logits), _ptr(draft_tokens), _ptr(q_lens),
+                                          _ptr(n_mask), _ptr(accepted_len), _ptr(bonus_token), _ptr(device_status),
+                                          _stream(stream))
+    return _check("fd_verify_accept_static", code, raise_on_error)
 
 
 def fd_kv_commit(ctx, batch, page_table, prefix_lens, q_lens, accepted_len, freed_pages, n_freed, stream=None,

@@ -41,6 +41,7 @@ const char* fd_status_string(fd_status s) {
         case FD_ERR_WORKSPACE: return "FD_ERR_WORKSPACE";
         case FD_ERR_CUDA: return "FD_ERR_CUDA";
         case FD_ERR_DEVICE_STATUS: return "FD_ERR_DEVICE_STATUS";
+        case FD_ERR_STATIC_LIMIT: return "FD_ERR_STATIC_LIMIT";
     }
     return "FD_UNKNOWN";
 }
