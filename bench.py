@@ -198,48 +198,41 @@ class DeviceStep:
 
 
 class HostStep:
-    """End-to-end leg: the step's inputs start in pinned host memory and its results end there.
-    The KV cache is decode state and stays resident; everything a step produces or consumes
-    anew (q of every layer, logits, draft tokens, lengths, page table in; attention outputs,
-    accepted lengths, bonus tokens, page table, lengths, freed pages out) crosses PCIe inside
-    the timed region."""
+    """End-to-end leg: one C-ABI call (fd_step_host) per step, every per-step input in pinned host
+    memory and every result back on the host inside the timed region.  The KV cache is decode state
+    and stays resident; q of every layer, logits, draft tokens, lengths and page table go up;
+    attention outputs, accepted lengths, bonus tokens, page table, lengths and freed pages come back.
+    The library pipelines the copies against the kernels on its own streams."""
 
     def __init__(self, ds: DeviceStep):
-        torch = ds.torch
-        pin = lambda t: t.cpu().pin_memory()
+        torch, st = ds.torch, ds.step
+        pin = lambda t: t.cpu().contiguous().pin_memory()
         self.ds = ds
-        self.h_q = [pin(t) for t in ds.q]
+        self.h_q = pin(torch.stack(ds.q))
+        self.h_out = torch.empty_like(self.h_q).pin_memory()
         self.h_logits, self.h_drafts = pin(ds.logits), pin(ds.drafts)
-        self.h_pt, self.h_pl, self.h_ql, self.h_nm = pin(ds.pt0), pin(ds.pl0), pin(ds.ql), pin(ds.nm)
-        self.h_out = [torch.empty_like(t, device="cpu").pin_memory() for t in ds.out]
+        self.pt0, self.pl0 = st.page_table.clone(), st.prefix_lens.clone()
+        self.h_pt, self.h_pl, self.h_ql, self.h_nm = pin(st.page_table), pin(st.prefix_lens), pin(st.q_lens), pin(st.n_mask)
         self.h_acc, self.h_bon = pin(ds.acc), pin(ds.bon)
-        self.h_pt_out, self.h_pl_out = pin(ds.pt), pin(ds.pl)
         self.h_freed, self.h_nfreed = pin(ds.freed), pin(ds.n_freed)
         nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
-        self.h2d = nbytes(self.h_q + [self.h_logits, self.h_drafts, self.h_pt, self.h_pl, self.h_ql, self.h_nm])
-        self.d2h = nbytes(self.h_out + [self.h_acc, self.h_bon, self.h_pt_out, self.h_pl_out, self.h_freed, self.h_nfreed])
+        self.h2d = nbytes([self.h_q, self.h_logits, self.h_drafts, self.h_pt, self.h_pl, self.h_ql, self.h_nm])
+        self.d2h = nbytes([self.h_out, self.h_acc, self.h_bon, self.h_pt, self.h_pl]) + 4 * st.batch * 3 + 4
+        ds.fd.fd_host_reserve(ds.ctx, st.total_q_rows, st.total_cand_rows)
 
     def run(self):
         ds, fd, st = self.ds, self.ds.fd, self.ds.step
-        ds.pt.copy_(self.h_pt, non_blocking=True); ds.pl.copy_(self.h_pl, non_blocking=True)
-        ds.ql.copy_(self.h_ql, non_blocking=True); ds.nm.copy_(self.h_nm, non_blocking=True)
-        for l in range(ds.L):
-            ds.q[l].copy_(self.h_q[l], non_blocking=True)
-            fd.fd_attn_draft_verify(ds.ctx, st.batch, st.total_q_rows, ds.q[l], ds.kv[l], st.num_pages, ds.pt, ds.pl,
-                                    ds.ql, ds.nm, ds.out[l])
-            self.h_out[l].copy_(ds.out[l], non_blocking=True)
-        ds.logits.copy_(self.h_logits, non_blocking=True); ds.drafts.copy_(self.h_drafts, non_blocking=True)
-        fd.fd_verify_accept(ds.ctx, st.batch, st.total_cand_rows, ds.logits, ds.drafts, ds.ql, ds.nm, ds.acc, ds.bon)
-        fd.fd_kv_commit(ds.ctx, st.batch, ds.pt, ds.pl, ds.ql, ds.acc, ds.freed, ds.n_freed)
-        for h, d in ((self.h_acc, ds.acc), (self.h_bon, ds.bon), (self.h_pt_out, ds.pt), (self.h_pl_out, ds.pl),
-                     (self.h_freed, ds.freed), (self.h_nfreed, ds.n_freed)):
-            h.copy_(d, non_blocking=True)
+        self.h_pt.copy_(self.pt0); self.h_pl.copy_(self.pl0)       # host-side reset of what the commit edited
+        fd.fd_step_host(ds.ctx, st.batch, st.total_q_rows, st.total_cand_rows, ds.kv, st.num_pages, self.h_q, self.h_out,
+                        self.h_logits, self.h_drafts, self.h_pt, self.h_pl, self.h_ql, self.h_nm, self.h_acc, self.h_bon,
+                        self.h_freed, self.h_nfreed)
+        ds.torch.cuda.current_stream().synchronize()               # the results are consumed on the host every step
 
 
 def timed_region(torch, dist, fn, steps, flush=None):
     """barrier + synchronize, `steps` x fn() between two CUDA events, synchronize + barrier."""
-    if dist is not None:
-        dist.barrier()
+    from paper_2605_20022_b200 import replicas
+    replicas.barrier(dist)
     torch.cuda.synchronize()
     if flush is None:
         e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
@@ -257,9 +250,24 @@ def timed_region(torch, dist, fn, steps, flush=None):
             e0.record(); fn(); e1.record()
             torch.cuda.synchronize()
             ms += e0.elapsed_time(e1)
-    if dist is not None:
-        dist.barrier()
+    replicas.barrier(dist)
     return ms
+
+
+def capture_step_graph(torch, ds):
+    """The whole step (attention x layers, accept, commit) as one CUDA graph on a side stream.  Only
+    used after warm-up, so every first-call set-up inside the library has already happened."""
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        ds.run()
+        side.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            ds.run()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    return g
 
 
 def check_against_oracle(ds: DeviceStep, n_rows=6):
@@ -314,21 +322,29 @@ def run_ours(args, step, rank, world, dist):
     clocks = sampler.stop()
     attn_ms = [a.elapsed_time(b) for a, b in ds.attn_events]
 
+    # the same step replayed as one CUDA graph: what the GPU needs once CPU launch cost is out of the way
+    ms_graph = None
+    if not args.no_graph:
+        graph = capture_step_graph(torch, ds)
+        for _ in range(2):
+            graph.replay()
+        ms_graph = timed_region(torch, dist, graph.replay, args.steps, flush)
+        del graph
+
     hs = HostStep(ds)
     for _ in range(2):
         hs.run()
     ms_e2e = timed_region(torch, dist, hs.run, args.steps)
     ds.close()
 
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
+    from paper_2605_20022_b200 import replicas
+    ms, ms_e2e, ms_graph_r = replicas.max_over_ranks([ms, ms_e2e, ms_graph or 0.0], dist, device)
     if rank != 0:
         return None
     # N independent replicas process N steps in the time of one: whole-job us per step = T / N
-    us_step = ms * 1e3 / args.steps / world
-    us_e2e = ms_e2e * 1e3 / args.steps / world
+    us_step = replicas.whole_job_us_per_step(ms, args.steps, world)
+    us_e2e = replicas.whole_job_us_per_step(ms_e2e, args.steps, world)
+    us_graph = replicas.whole_job_us_per_step(ms_graph_r, args.steps, world) if ms_graph is not None else None
     attn_bytes = step.attn_bytes()
     attn_avg_ms = statistics.mean(attn_ms)
     achieved = attn_bytes / (attn_avg_ms * 1e-3) / 1e9
@@ -343,7 +359,8 @@ def run_ours(args, step, rank, world, dist):
                    "attn_path": resolved,
                    "l2": "flushed between steps (512 MB write)" if small else "inputs larger than L2 (distinct KV pool per layer)",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU",
-                   "parity_vs_oracle_sampled": parity_ok, "device_status": status},
+                   "parity_vs_oracle_sampled": parity_ok, "device_status": status,
+                   "us_per_step_cuda_graph_replay": us_graph},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
                      "kernel": "fd_attn_draft_verify (plan + split-KV attention + merge launches)",
@@ -366,6 +383,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="override the layer count of workload 4")
     ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel")
     ap.add_argument("--ref-heads", type=int, default=8, help="q-heads in the oracle's timed sample")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -378,13 +396,11 @@ def main():
             print(json.dumps(run_reference(args, step)), flush=True)
         return
 
-    dist = None
+    import torch
+    from paper_2605_20022_b200 import replicas
     if world > 1:
-        import torch.distributed as dist_mod
-        import torch
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", 0)))
-        dist_mod.init_process_group("nccl")
-        dist = dist_mod
+    dist = replicas.init("nccl")
     import paper_2605_20022_b200 as fd
     fd.load()                                               # raises if the CUDA library is missing
     res = run_ours(args, step, rank, world, dist)

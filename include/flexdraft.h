@@ -180,6 +180,41 @@ fd_status fd_kv_commit(fd_ctx* ctx, int batch, int32_t* page_table, int32_t* pre
                        int32_t* freed_pages, int32_t* n_freed, void* stream);
 
 /*
+ * One whole decode step from HOST buffers: the attention of n_layers layers, the verification
+ * and the commit (the three calls above, in the order of Sec. 4.1 "Inference"), with every
+ * per-step input copied up and every result copied back by the library.  The KV caches are
+ * decode state and stay on the device; all other pointers are host pointers (pinned memory
+ * makes the copies asynchronous and lets them overlap the kernels; pageable memory works but
+ * serialises).  Copies run on two internal streams so that q of layer l+1 goes up and out of
+ * layer l-1 comes back while layer l computes; one cudaMemcpyAsync per buffer.
+ *
+ * fd_host_reserve(ctx, max_total_q_rows, max_total_cand_rows) allocates the device staging
+ * (2 x q, 2 x out, logits, small arrays) and the copy streams once; it is the only part that
+ * allocates and must precede fd_step_host.  A second call with sizes within the first is a
+ * no-op; larger sizes return FD_ERR_INVALID_ARG.
+ *
+ *   kv_caches         host array of n_layers device pointers, each [num_pages, 2, Hkv, P, d] bf16
+ *   q_host            [n_layers][T, Hq, d] bf16          out_host   [n_layers][T, Hq, d] bf16, written
+ *   logits_host       [R, V] fp32                        draft_tokens_host [R] int32
+ *   page_table_host   [B, max_pages_per_seq] int32, in/out (the commit's edits come back)
+ *   prefix_lens_host  [B] int32, in/out                  q_lens_host, n_mask_host [B] int32
+ *   accepted_len_host, bonus_token_host [B] int32, written
+ *   freed_pages_host  capacity B * (ceil(max_q_len / P) + 1) int32, written; n_freed_host [1]
+ *
+ * The call returns after enqueueing; `stream` has finished the step, results on the host
+ * included, once everything enqueued on it has completed.  The host buffers must stay valid
+ * and untouched until then.  Steps on one context must not overlap.
+ */
+fd_status fd_host_reserve(fd_ctx* ctx, int max_total_q_rows, int max_total_cand_rows);
+fd_status fd_step_host(fd_ctx* ctx, int batch, int total_q_rows, int total_cand_rows, int n_layers,
+                       const void* const* kv_caches, int num_pages, const void* q_host, void* out_host,
+                       const float* logits_host, const int32_t* draft_tokens_host,
+                       int32_t* page_table_host, int32_t* prefix_lens_host,
+                       const int32_t* q_lens_host, const int32_t* n_mask_host,
+                       int32_t* accepted_len_host, int32_t* bonus_token_host,
+                       int32_t* freed_pages_host, int32_t* n_freed_host, void* stream);
+
+/*
  * fd_verify_accept without any allocation.  (The paper has no counterpart; this entry point
  * exists for the callers described here.)
  *

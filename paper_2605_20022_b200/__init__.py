@@ -23,7 +23,7 @@ FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host"]
 
 
 class fd_config(ctypes.Structure):
@@ -60,6 +60,8 @@ def load() -> ctypes.CDLL:
         lib.fd_verify_accept.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_kv_commit.argtypes = [vp, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_verify_accept_static.argtypes = [ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_host_reserve.argtypes = [vp, ci, ci]
+        lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 13
         lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         lib.fd_attn_path.argtypes = [vp]
         lib.fd_launch_count.argtypes = [vp]
@@ -143,6 +145,24 @@ def fd_kv_commit(ctx, batch, page_table, prefix_lens, q_lens, accepted_len, free
     code = load().fd_kv_commit(ctx, batch, _ptr(page_table), _ptr(prefix_lens), _ptr(q_lens), _ptr(accepted_len),
                                _ptr(freed_pages), _ptr(n_freed), _stream(stream))
     return _check("fd_kv_commit", code, raise_on_error)
+
+
+def fd_host_reserve(ctx, max_total_q_rows, max_total_cand_rows) -> None:
+    _check("fd_host_reserve", load().fd_host_reserve(ctx, max_total_q_rows, max_total_cand_rows), True)
+
+
+def fd_step_host(ctx, batch, total_q_rows, total_cand_rows, kv_caches, num_pages, q_host, out_host, logits_host,
+                 draft_tokens_host, page_table_host, prefix_lens_host, q_lens_host, n_mask_host, accepted_len_host,
+                 bonus_token_host, freed_pages_host, n_freed_host, stream=None, raise_on_error=True) -> int:
+    """One whole step from host (CPU, ideally pinned) tensors; `kv_caches` is a list of device tensors, one per
+    layer.  `q_host` / `out_host` are [n_layers, T, Hq, d] CPU tensors."""
+    n_layers = len(kv_caches)
+    arr = (ctypes.c_void_p * n_layers)(*[_ptr(t) for t in kv_caches])
+    code = load().fd_step_host(ctx, batch, total_q_rows, total_cand_rows, n_layers, arr, num_pages, _ptr(q_host),
+                               _ptr(out_host), _ptr(logits_host), _ptr(draft_tokens_host), _ptr(page_table_host),
+                               _ptr(prefix_lens_host), _ptr(q_lens_host), _ptr(n_mask_host), _ptr(accepted_len_host),
+                               _ptr(bonus_token_host), _ptr(freed_pages_host), _ptr(n_freed_host), _stream(stream))
+    return _check("fd_step_host", code, raise_on_error)
 
 
 def fd_last_device_status(ctx, stream=None) -> int:

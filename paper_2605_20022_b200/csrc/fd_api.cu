@@ -21,6 +21,18 @@ struct fd_ctx {
     int max_rows;      // capacity of keys
     void* tc_state;
     long long launches;
+    struct HostStage* host;  // staging for fd_step_host, nullptr until fd_host_reserve
+};
+
+// Device staging + copy streams of the host-buffer step (fd_host_reserve / fd_step_host).
+struct HostStage {
+    int max_q_rows, max_cand_rows;
+    cudaStream_t h2d, d2h;
+    cudaEvent_t start, meta, logits, done, fin, q_ready[2], attn_done[2], out_copied[2];
+    unsigned char* pool;
+    void *q[2], *out[2];
+    float* lg;
+    int32_t *drafts, *pt, *pl, *ql, *nm, *acc, *bon, *freed, *nfreed;
 };
 
 namespace {
@@ -65,6 +77,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->cfg = *cfg;
     c->launches = 0;
     c->tc_state = nullptr;
+    c->host = nullptr;
     if (cudaGetDevice(&c->device) != cudaSuccess ||
         cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
         delete c;
@@ -114,8 +127,132 @@ fd_status fd_destroy(fd_ctx* c) {
     if (!c) return FD_OK;
     cudaDeviceSynchronize();
     fd::attn_tc_free(c->tc_state);
+    if (c->host) {
+        HostStage* h = c->host;
+        cudaStreamDestroy(h->h2d); cudaStreamDestroy(h->d2h);
+        cudaEvent_t evs[] = {h->start, h->meta, h->logits, h->done, h->fin, h->q_ready[0], h->q_ready[1],
+                             h->attn_done[0], h->attn_done[1], h->out_copied[0], h->out_copied[1]};
+        for (cudaEvent_t e : evs) cudaEventDestroy(e);
+        cudaFree(h->pool);
+        delete h;
+    }
     cudaFree(c->pool);
     delete c;
+    return FD_OK;
+}
+
+fd_status fd_host_reserve(fd_ctx* c, int max_total_q_rows, int max_total_cand_rows) {
+    if (!c || max_total_q_rows < 0 || max_total_cand_rows < 0) return FD_ERR_INVALID_ARG;
+    if (c->host) return (max_total_q_rows <= c->host->max_q_rows && max_total_cand_rows <= c->host->max_cand_rows)
+                            ? FD_OK : FD_ERR_INVALID_ARG;  // reserve once, with the maxima
+    HostStage* h = new (std::nothrow) HostStage();
+    if (!h) return FD_ERR_WORKSPACE;
+    h->max_q_rows = max_total_q_rows; h->max_cand_rows = max_total_cand_rows;
+    const int B = c->cfg.max_batch;
+    const size_t qb = (size_t)max_total_q_rows * c->cfg.n_q_heads * c->cfg.head_dim * 2;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t o_q0 = take(qb), o_q1 = take(qb), o_o0 = take(qb), o_o1 = take(qb);
+    const size_t o_lg = take((size_t)max_total_cand_rows * c->cfg.vocab * 4);
+    const size_t o_dr = take((size_t)max_total_cand_rows * 4);
+    const size_t o_pt = take((size_t)B * c->cfg.max_pages_per_seq * 4);
+    const size_t o_pl = take(B * 4), o_ql = take(B * 4), o_nm = take(B * 4), o_ac = take(B * 4), o_bo = take(B * 4);
+    const size_t n_fr = (size_t)B * ((c->cfg.max_q_len + 15) / 16 + 1);
+    const size_t o_fr = take(n_fr * 4), o_nf = take(4);
+    if (cudaMalloc(&h->pool, off) != cudaSuccess) { cudaGetLastError(); delete h; return FD_ERR_WORKSPACE; }
+    bool ok = cudaStreamCreateWithFlags(&h->h2d, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&h->d2h, cudaStreamNonBlocking) == cudaSuccess;
+    cudaEvent_t* evs[] = {&h->start, &h->meta, &h->logits, &h->done, &h->fin, &h->q_ready[0], &h->q_ready[1],
+                          &h->attn_done[0], &h->attn_done[1], &h->out_copied[0], &h->out_copied[1]};
+    for (cudaEvent_t* e : evs) ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); cudaFree(h->pool); delete h; return FD_ERR_CUDA; }
+    h->q[0] = h->pool + o_q0; h->q[1] = h->pool + o_q1; h->out[0] = h->pool + o_o0; h->out[1] = h->pool + o_o1;
+    h->lg = reinterpret_cast<float*>(h->pool + o_lg);
+    h->drafts = reinterpret_cast<int32_t*>(h->pool + o_dr); h->pt = reinterpret_cast<int32_t*>(h->pool + o_pt);
+    h->pl = reinterpret_cast<int32_t*>(h->pool + o_pl); h->ql = reinterpret_cast<int32_t*>(h->pool + o_ql);
+    h->nm = reinterpret_cast<int32_t*>(h->pool + o_nm); h->acc = reinterpret_cast<int32_t*>(h->pool + o_ac);
+    h->bon = reinterpret_cast<int32_t*>(h->pool + o_bo); h->freed = reinterpret_cast<int32_t*>(h->pool + o_fr);
+    h->nfreed = reinterpret_cast<int32_t*>(h->pool + o_nf);
+    c->host = h;
+    return FD_OK;
+}
+
+fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_rows, int n_layers,
+                       const void* const* kv_caches, int num_pages, const void* q_host, void* out_host,
+                       const float* logits_host, const int32_t* draft_tokens_host, int32_t* page_table_host,
+                       int32_t* prefix_lens_host, const int32_t* q_lens_host, const int32_t* n_mask_host,
+                       int32_t* accepted_len_host, int32_t* bonus_token_host, int32_t* freed_pages_host,
+                       int32_t* n_freed_host, void* stream) {
+    if (!c || !c->host) return FD_ERR_INVALID_ARG;
+    HostStage* h = c->host;
+    if (batch <= 0 || batch > c->cfg.max_batch || n_layers <= 0 || total_q_rows < 0 || total_cand_rows < 0 ||
+        total_q_rows > h->max_q_rows || total_cand_rows > h->max_cand_rows)
+        return FD_ERR_INVALID_ARG;
+    if (!kv_caches || !q_host || !out_host || !page_table_host || !prefix_lens_host || !q_lens_host || !n_mask_host ||
+        !accepted_len_host || !bonus_token_host || !freed_pages_host || !n_freed_host ||
+        (total_cand_rows > 0 && (!logits_host || !draft_tokens_host)))
+        return FD_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t qb = (size_t)total_q_rows * c->cfg.n_q_heads * c->cfg.head_dim * 2;
+    const size_t ptb = (size_t)batch * c->cfg.max_pages_per_seq * 4, lb = (size_t)batch * 4;
+    const size_t n_fr = (size_t)batch * ((c->cfg.max_q_len + 15) / 16 + 1);
+    bool ok = true;
+    auto chk = [&](cudaError_t e) { ok = ok && e == cudaSuccess; };
+    const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
+
+    // everything of this step is ordered after what the caller already put on `stream`
+    chk(cudaEventRecord(h->start, s));
+    chk(cudaStreamWaitEvent(h->h2d, h->start, 0));
+    chk(cudaStreamWaitEvent(h->d2h, h->start, 0));
+    chk(cudaMemcpyAsync(h->pt, page_table_host, ptb, H2D, h->h2d));
+    chk(cudaMemcpyAsync(h->pl, prefix_lens_host, lb, H2D, h->h2d));
+    chk(cudaMemcpyAsync(h->ql, q_lens_host, lb, H2D, h->h2d));
+    chk(cudaMemcpyAsync(h->nm, n_mask_host, lb, H2D, h->h2d));
+    chk(cudaEventRecord(h->meta, h->h2d));
+    chk(cudaStreamWaitEvent(s, h->meta, 0));
+    fd_status st = FD_OK;
+    for (int l = 0; l < n_layers && ok && st == FD_OK; ++l) {
+        const int b = l & 1;
+        // q of layer l goes up while layer l-1 computes; the staging pair is reused every other layer
+        if (l >= 2) chk(cudaStreamWaitEvent(h->h2d, h->attn_done[b], 0));
+        chk(cudaMemcpyAsync(h->q[b], static_cast<const unsigned char*>(q_host) + (size_t)l * qb, qb, H2D, h->h2d));
+        chk(cudaEventRecord(h->q_ready[b], h->h2d));
+        if (l == 1 && total_cand_rows > 0) {  // the logits follow the first two q blocks so that layer 0 starts at once
+            chk(cudaMemcpyAsync(h->lg, logits_host, (size_t)total_cand_rows * c->cfg.vocab * 4, H2D, h->h2d));
+            chk(cudaMemcpyAsync(h->drafts, draft_tokens_host, (size_t)total_cand_rows * 4, H2D, h->h2d));
+            chk(cudaEventRecord(h->logits, h->h2d));
+        }
+        chk(cudaStreamWaitEvent(s, h->q_ready[b], 0));
+        if (l >= 2) chk(cudaStreamWaitEvent(s, h->out_copied[b], 0));
+        st = fd_attn_draft_verify(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
+                                  h->out[b], s);
+        chk(cudaEventRecord(h->attn_done[b], s));
+        chk(cudaStreamWaitEvent(h->d2h, h->attn_done[b], 0));
+        chk(cudaMemcpyAsync(static_cast<unsigned char*>(out_host) + (size_t)l * qb, h->out[b], qb, D2H, h->d2h));
+        chk(cudaEventRecord(h->out_copied[b], h->d2h));
+    }
+    if (st != FD_OK) return st;
+    if (n_layers < 2 && total_cand_rows > 0) {
+        chk(cudaMemcpyAsync(h->lg, logits_host, (size_t)total_cand_rows * c->cfg.vocab * 4, H2D, h->h2d));
+        chk(cudaMemcpyAsync(h->drafts, draft_tokens_host, (size_t)total_cand_rows * 4, H2D, h->h2d));
+        chk(cudaEventRecord(h->logits, h->h2d));
+    }
+    if (total_cand_rows > 0) chk(cudaStreamWaitEvent(s, h->logits, 0));
+    st = fd_verify_accept(c, batch, total_cand_rows, h->lg, h->drafts, h->ql, h->nm, h->acc, h->bon, s);
+    if (st != FD_OK) return st;
+    st = fd_kv_commit(c, batch, h->pt, h->pl, h->ql, h->acc, h->freed, h->nfreed, s);
+    if (st != FD_OK) return st;
+    chk(cudaEventRecord(h->done, s));
+    chk(cudaStreamWaitEvent(h->d2h, h->done, 0));
+    chk(cudaMemcpyAsync(accepted_len_host, h->acc, lb, D2H, h->d2h));
+    chk(cudaMemcpyAsync(bonus_token_host, h->bon, lb, D2H, h->d2h));
+    chk(cudaMemcpyAsync(page_table_host, h->pt, ptb, D2H, h->d2h));
+    chk(cudaMemcpyAsync(prefix_lens_host, h->pl, lb, D2H, h->d2h));
+    chk(cudaMemcpyAsync(freed_pages_host, h->freed, n_fr * 4, D2H, h->d2h));
+    chk(cudaMemcpyAsync(n_freed_host, h->nfreed, 4, D2H, h->d2h));
+    chk(cudaEventRecord(h->fin, h->d2h));
+    chk(cudaStreamWaitEvent(s, h->fin, 0));  // `stream` is complete only when every result is on the host
+    if (!ok) { cudaGetLastError(); return FD_ERR_CUDA; }
     return FD_OK;
 }
 

@@ -233,3 +233,40 @@ def test_long_context_full_size_sampled(path):
                 ref = oracle.attn_row(qc, kvc, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, b, i, h)
                 assert_close(outc[b * 32 + i, h], ref, f"layer {layer} b {b} row {i} head {h}")
             del q, kv, out
+
+
+def test_host_buffer_step_matches_oracle():
+    """fd_step_host: a whole 3-layer step from pinned host buffers (copies pipelined inside the library)."""
+    shape = wl.Shape(32, 8, 128, 5000, n_layers=3)
+    step = wl.make_step("host", shape, [700, 130, 2049, 0], [32, 9, 20, 16], [16, 0, 8, 0], seed=17, p_match=0.7,
+                        extra_table_cols=1)
+    L, B, T, R = 3, step.batch, step.total_q_rows, step.total_cand_rows
+    qs = [wl.make_q(step, l) for l in range(L)]
+    kvs = [wl.make_kv(step, l) for l in range(L)]
+    logits, drafts, _ = wl.make_logits(step)
+    pin = lambda t: t.contiguous().pin_memory()
+    q_host = pin(torch.stack(qs)); out_host = pin(torch.zeros_like(q_host))
+    h_logits, h_drafts = pin(logits), pin(drafts)
+    h_pt, h_pl, h_ql, h_nm = pin(step.page_table.clone()), pin(step.prefix_lens.clone()), pin(step.q_lens), pin(step.n_mask)
+    h_acc, h_bon = pin(torch.zeros(B, dtype=torch.int32)), pin(torch.zeros(B, dtype=torch.int32))
+    h_freed, h_nf = pin(torch.full((B * 3,), -7, dtype=torch.int32)), pin(torch.zeros(1, dtype=torch.int32))
+    dkv = [t.cuda() for t in kvs]
+    with Ctx(step) as ctx:
+        assert fd.fd_step_host(ctx.h, B, T, R, dkv, step.num_pages, q_host, out_host, h_logits, h_drafts, h_pt, h_pl, h_ql,
+                               h_nm, h_acc, h_bon, h_freed, h_nf, raise_on_error=False) == fd.FD_ERR_INVALID_ARG  # not reserved
+        fd.fd_host_reserve(ctx.h, T, R)
+        for _ in range(2):                                   # twice: the second step reuses the staging buffers
+            h_pt.copy_(step.page_table); h_pl.copy_(step.prefix_lens); out_host.zero_()
+            fd.fd_step_host(ctx.h, B, T, R, dkv, step.num_pages, q_host, out_host, h_logits, h_drafts, h_pt, h_pl, h_ql,
+                            h_nm, h_acc, h_bon, h_freed, h_nf)
+            torch.cuda.current_stream().synchronize()
+            assert fd.fd_last_device_status(ctx.h) == 0
+            for l in range(L):
+                ref = oracle.attn(qs[l], kvs[l], step.page_table, step.prefix_lens, step.q_lens, step.n_mask)
+                assert_close(out_host[l].float().numpy(), ref, f"layer {l}")
+            e_acc, e_bon, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+            np.testing.assert_array_equal(h_acc.numpy(), e_acc); np.testing.assert_array_equal(h_bon.numpy(), e_bon)
+            ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, e_acc)
+            np.testing.assert_array_equal(h_pt.numpy(), ept); np.testing.assert_array_equal(h_pl.numpy(), epl)
+            assert int(h_nf) == len(efreed)
+            np.testing.assert_array_equal(h_freed.numpy()[:len(efreed)], efreed)
