@@ -76,7 +76,7 @@ typedef struct {
     int head_dim;             /* d: 64 or 128 */
     int page_size;            /* P: 16 */
     int vocab;                /* V >= 1 */
-    int max_batch;            /* largest B of any call */
+    int max_batch;            /* largest B of any call; at most 4096 */
     int max_q_len;            /* largest Lq_b; G * max_q_len <= 128 */
     int max_pages_per_seq;    /* row length of page_table */
     float softmax_scale;      /* 0 selects 1/sqrt(d) */

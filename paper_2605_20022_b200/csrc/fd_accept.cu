@@ -75,38 +75,68 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_
     if (!last) return;
     __threadfence();
 
-    // ---- accept scan, one CTA, after every row key is final ----
-    extern __shared__ int cu_c[];  // [B+1] first candidate row of each sequence
-    __shared__ int s_bad;
-    if (tid == 0) {
-        long long rows = 0;
-        cu_c[0] = 0;
-        for (int b = 0; b < p.batch; ++b) {
-            const int C = p.q_lens[b] - p.n_mask[b];
-            if (C < 0 || p.n_mask[b] < 0) { rows = -1; break; }
-            rows += C;
-            if (rows > p.total_rows) break;
-            cu_c[b + 1] = (int)rows;
+    // ---- accept scan, one CTA, after every row key is final.  Everything is one parallel round of
+    //      loads per step (serial walks over global memory would cost a DRAM/L2 latency per element):
+    //      (1) block scan of the candidate-row counts, (2) one thread per candidate row compares its
+    //      argmax with the next draft and lowers the sequence's first-mismatch index, (3) one thread
+    //      per sequence reads the argmax at that index.
+    extern __shared__ int sm[];            // cu_c [B+1], then first_mismatch [B]
+    int* cu_c = sm;
+    int* first_bad = sm + p.batch + 1;
+    __shared__ int s_bad, s_carry, s_wsum[8];
+    if (tid == 0) { s_bad = 0; s_carry = 0; cu_c[0] = 0; }
+    __syncthreads();
+    for (int base = 0; base < p.batch; base += blockDim.x) {
+        const int b = base + tid;
+        int c = 0;
+        if (b < p.batch) {
+            const int M = p.n_mask[b];
+            c = p.q_lens[b] - M;
+            if (c < 0 || M < 0) { atomicOr(&s_bad, 1); c = 0; }
         }
-        s_bad = rows != p.total_rows;
-        if (s_bad) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        int inc = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, inc, o);
+            if ((tid & 31) >= o) inc += u;
+        }
+        if ((tid & 31) == 31) s_wsum[tid >> 5] = inc;
+        __syncthreads();
+        int off = s_carry;
+        for (int w = 0; w < (tid >> 5); ++w) off += s_wsum[w];
+        if (b < p.batch) {
+            const long long end = (long long)off + inc;
+            cu_c[b + 1] = (int)min(end, (long long)0x7fffffff);
+            first_bad[b] = max(c - 1, 0);                      // k_b: "every draft matched"
+        }
+        __syncthreads();
+        if (tid == blockDim.x - 1) s_carry = min((long long)off + inc, (long long)0x7fffffff);
+        __syncthreads();
     }
+    if (tid == 0 && (s_bad || s_carry != p.total_rows)) { s_bad = 1; atomicOr(p.status, FD_DEV_BAD_LENGTHS); }
     __syncthreads();
     if (s_bad) {
         for (int b = tid; b < p.batch; b += blockDim.x) { p.accepted[b] = -1; p.bonus[b] = -1; }
     } else {
-        // thread b walks the candidate rows of sequence b
+        for (int r = tid; r < p.total_rows; r += blockDim.x) {
+            int lo = 0, hi = p.batch;                          // sequence of row r: last b with cu_c[b] <= r
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cu_c[mid] <= r) lo = mid; else hi = mid;
+            }
+            const int j = r - cu_c[lo];
+            if (r + 1 < cu_c[lo + 1]) {                        // row j has a draft after it
+                const int am = (int)(0xffffffffu - (unsigned)(__ldcg(p.keys + r) & 0xffffffffull));
+                if (am != p.drafts[r + 1]) atomicMin(&first_bad[lo], j);
+            }
+        }
+        __syncthreads();
         for (int b = tid; b < p.batch; b += blockDim.x) {
             const int r0 = cu_c[b], C = cu_c[b + 1] - r0;
             if (C == 0) { p.accepted[b] = -1; p.bonus[b] = -1; continue; }
-            int a = 0;
-            int am = (int)(0xffffffffu - (unsigned)(__ldcg(p.keys + r0) & 0xffffffffull));
-            while (a < C - 1 && am == p.drafts[r0 + a + 1]) {
-                ++a;
-                am = (int)(0xffffffffu - (unsigned)(__ldcg(p.keys + r0 + a) & 0xffffffffull));
-            }
+            const int a = first_bad[b];
             p.accepted[b] = a;
-            p.bonus[b] = am;
+            p.bonus[b] = (int)(0xffffffffu - (unsigned)(__ldcg(p.keys + r0 + a) & 0xffffffffull));
         }
     }
     __syncthreads();
@@ -126,7 +156,7 @@ void launch_accept(const AcceptParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
     if (p.total_rows == 0) { accept_empty_kernel<<<1, 256, 0, s>>>(p); return; }
     const int chunks = (p.vocab + kAcceptChunk - 1) / kAcceptChunk;
-    accept_kernel<<<p.total_rows * chunks, 256, (p.batch + 1) * sizeof(int), s>>>(p, chunks);
+    accept_kernel<<<p.total_rows * chunks, 256, (2 * p.batch + 1) * sizeof(int), s>>>(p, chunks);
 }
 
 }  // namespace fd

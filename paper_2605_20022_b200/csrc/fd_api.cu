@@ -70,7 +70,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
     if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return FD_ERR_UNSUPPORTED;
     if ((long long)G * cfg->max_q_len > fd::kMaxRows) return FD_ERR_UNSUPPORTED;
-    if ((long long)cfg->max_pages_per_seq * 16 > 0x3fffffffLL || cfg->max_batch > (1 << 20)) return FD_ERR_UNSUPPORTED;
+    if ((long long)cfg->max_pages_per_seq * 16 > 0x3fffffffLL || cfg->max_batch > 4096) return FD_ERR_UNSUPPORTED;
 
     fd_ctx* c = new (std::nothrow) fd_ctx();
     if (!c) return FD_ERR_WORKSPACE;
@@ -101,6 +101,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const size_t o_cuq = take((B + 1) * sizeof(int));
     const size_t o_cut = take((B + 1) * sizeof(int));
     const size_t o_ok = take(B * sizeof(int));
+    const size_t o_sc = take((size_t)B * cfg->n_kv_heads * sizeof(int));
     const size_t o_po = take(slots * d * fd::kMaxRows * sizeof(float));
     const size_t o_pm = take(slots * fd::kMaxRows * sizeof(float));
     const size_t o_pl = take(slots * fd::kMaxRows * sizeof(float));
@@ -113,6 +114,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->plan.cu_q = reinterpret_cast<int*>(c->pool + o_cuq);
     c->plan.cu_tiles = reinterpret_cast<int*>(c->pool + o_cut);
     c->plan.seq_ok = reinterpret_cast<int*>(c->pool + o_ok);
+    c->plan.seg_count = reinterpret_cast<int*>(c->pool + o_sc);
     c->part.o = reinterpret_cast<float*>(c->pool + o_po);
     c->part.m = reinterpret_cast<float*>(c->pool + o_pm);
     c->part.l = reinterpret_cast<float*>(c->pool + o_pl);
@@ -289,10 +291,14 @@ fd_status fd_attn_draft_verify(fd_ctx* c, int batch, int total_q_rows, const voi
         if (fd::attn_tc_prepare(&c->tc_state, p) != cudaSuccess) { cudaGetLastError(); return FD_ERR_CUDA; }
     }
     fd::launch_plan(p, s);
-    if (c->attn_path == FD_ATTN_TCGEN05) fd::launch_attn_tc(c->tc_state, p, s);
-    else fd::launch_attn_simt(p, s);
-    fd::launch_merge(p, s);
-    c->launches += 3;
+    if (c->attn_path == FD_ATTN_TCGEN05) {
+        fd::launch_attn_tc(c->tc_state, p, s);  // merges split segments in its own epilogue
+        c->launches += 2;
+    } else {
+        fd::launch_attn_simt(p, s);
+        fd::launch_merge(p, s);
+        c->launches += 3;
+    }
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }
 

@@ -19,7 +19,8 @@
 //                     softmax in the log2 domain, bf16 P written back over S in TMEM.
 // Tiles alternate between two independent streams s = j & 1, each with its own softmax
 // group, S/P buffer, (m, l) state and O accumulator in TMEM, so the tensor pipe works on one
-// stream while the other is in its softmax; the two streams are merged in the epilogue.  O is
+// stream while the other is in its softmax; the two streams are merged in the epilogue.  A segment
+// that several CTAs share is merged by whichever of them delivers its partial last (a counter, no waiting).  O is
 // rescaled lazily (only when a row maximum grows by more than 2^8), which is exact because
 // the same reference maximum is used for P, l and O.
 //
@@ -60,6 +61,7 @@ struct Bars {
     uint64_t all_done;
     uint32_t tmem_base;
     int abort;
+    int merge_flag;
 };
 
 struct Piece {
@@ -132,7 +134,6 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
     volatile int* abort = &bars->abort;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
-    (void)total;
     const uint32_t tmem = bars->tmem_base;
     const uint32_t col_s[2] = {0u, 128u};
     const uint32_t col_o[2] = {256u, 384u};
@@ -142,11 +143,18 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
     int piece_idx = 0;
     int issued = 0;        // producer: tiles whose loads were issued
 
+    // The two load warps never take part in the per-piece barriers: they walk the pieces on their own,
+    // held back only by the K / V rings, so the rings are already full when the MMAs of the next piece start.
+    const bool loader = !kSoftmax && (warp == kKWarp || warp == kVWarp);
+    const int ltid = warp < 8 ? tid : tid - 64;                 // index among the kPieceThreads other threads
+    constexpr int kPieceThreads = kThreads - 64;
+
     for (int t = s_c; t < e_c;) {
         const Piece pc = decode_piece(p, t, s_c, e_c, cta);
 
         // ---- Q tile -> shared memory, K-major, 128-byte swizzle; rows beyond the block are zero
-        for (int idx = tid; idx < kMaxRows * (D / 8); idx += kThreads) {
+        if (!loader)
+        for (int idx = ltid; idx < kMaxRows * (D / 8); idx += kPieceThreads) {
             const int r = idx / (D / 8), ch = idx % (D / 8);
             uint4 v = make_uint4(0, 0, 0, 0);
             if (r < pc.rows)
@@ -154,8 +162,10 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
             const int half = ch >> 3, c16 = ch & 7;
             *reinterpret_cast<uint4*>(sq + half * (kMaxRows * 128) + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
         }
-        fence_proxy_async_smem();
-        __syncthreads();
+        if (!loader) {
+            fence_proxy_async_smem();
+            named_bar_sync(2, kPieceThreads);
+        }
 
         if constexpr (!kSoftmax) {
         if (warp == kKWarp || warp == kVWarp) {
@@ -360,7 +370,8 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
                 if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 2, g0 + j);
             }
 
-            // ---- epilogue: merge the two streams, then final rows or a partial for the merge kernel
+            // ---- epilogue: merge the two streams, then final rows, or a partial plus -- if this CTA is the
+            //      last one to deliver a piece of the segment -- the merge of all its partials
             ok = ok && wait_all(&bars->all_done, piece_idx & 1, abort);
             tc_fence_after();
             if (ok) {
@@ -393,6 +404,11 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
                     }
                     if (r < pc.rows) {
                         if (pc.complete) {
+                            // the load warps of this CTA have seen every page id of the segment by now
+                            if (!__ldcg(p.plan.seq_ok + pc.b)) {
+#pragma unroll
+                                for (int k = 0; k < 32; ++k) o[k] = 0.f;
+                            }
                             __nv_bfloat16* dst = p.out + ((long long)(pc.row0 + i) * p.Hq + pc.kvh * p.G + r % p.G) * D + col;
 #pragma unroll
                             for (int k = 0; k < 32; k += 8) {
@@ -413,11 +429,34 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
                     p.part.l[pc.slot * kMaxRows + r] = L;
                 }
             }
+            if (!pc.complete) {
+                // Fused split merge: count the delivered pieces of the segment; whoever delivers the last
+                // one combines them all (no CTA ever waits for another).  Both barriers are taken by all
+                // 256 softmax threads whatever happened before, and thread 0 alone takes the decision.
+                __threadfence();
+                named_bar_sync(1, 256);
+                if (tid == 0) {
+                    int last = 0;
+                    if (!*abort) {
+                        const int ntiles = p.plan.cu_tiles[pc.b + 1] - p.plan.cu_tiles[pc.b];
+                        const int seg_start = t - pc.tile0;
+                        const int n = segment_pieces(seg_start, seg_start + ntiles, total, p.n_ctas);
+                        last = atomicAdd(p.plan.seg_count + pc.b * p.Hkv + pc.kvh, 1) + 1 == n;
+                    }
+                    bars->merge_flag = last;
+                }
+                named_bar_sync(1, 256);
+                if (bars->merge_flag) {
+                    __threadfence();
+                    const int rr = tid & (kMaxRows - 1), cg = tid >> 7;
+                    if (rr < pc.rows) merge_row<D, D / 2>(p, total, pc.b, pc.kvh, rr, cg);
+                }
+            }
             tc_fence_before();
         }
 
-        // ---- end of piece: everything of this piece has completed (or the CTA is aborting)
-        __syncthreads();
+        // ---- end of piece: every MMA and every epilogue read of this piece has completed (or the CTA is aborting)
+        if (!loader) named_bar_sync(2, kPieceThreads);
         if (*abort) break;
         g0 += pc.nt;
         u_base[0] += (pc.nt + 1) >> 1;
@@ -457,7 +496,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const PlanHeader hdr = *p.plan.hdr;
     const int total = hdr.total_tiles;
-    if (total == 0) return;  // uniform: nothing allocated yet
+    if (total == 0) {  // uniform: nothing allocated yet
+        if (hdr.fatal) {  // inconsistent lengths: a defined output, zeros
+            const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
+            uint4* o = reinterpret_cast<uint4*>(p.out);
+            for (long long i2 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i2 < n16; i2 += (long long)gridDim.x * blockDim.x)
+                o[i2] = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
     const int cta = blockIdx.x;
     const int s_c = range_begin(cta, total, p.n_ctas), e_c = range_begin(cta + 1, total, p.n_ctas);
     if (s_c >= e_c) return;

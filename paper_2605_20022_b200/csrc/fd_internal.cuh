@@ -25,7 +25,8 @@ struct Plan {
     PlanHeader* hdr;
     int* cu_q;      // [B+1] first query row of each sequence
     int* cu_tiles;  // [B+1] exclusive scan of tiles_b (per kv-head)
-    int* seq_ok;    // [B]   0 = skipped (bad page id), 1 = computed
+    int* seq_ok;    // [B]   0 = a page id of the sequence was outside the pool: its rows are zeroed
+    int* seg_count; // [B * Hkv] partial pieces of a segment that have been written (fused merge)
 };
 
 // Partial result of one piece of a (sequence, kv-head) segment, log2 domain:
@@ -62,6 +63,70 @@ __host__ __device__ inline int range_begin(int c, int total, int n) {
 // The CTA whose range holds tile t.
 __host__ __device__ inline int range_owner(int t, int total, int n) {
     return (int)((((long long)(t + 1)) * n + total - 1) / total) - 1;
+}
+
+// Write one row segment of `n` columns as bf16 (n a multiple of 8), scaled by inv.
+template <int N>
+__device__ inline void store_cols_bf16(__nv_bfloat16* dst, const float* o, float inv) {
+#pragma unroll
+    for (int c = 0; c < N; c += 8) {
+        __align__(16) __nv_bfloat162 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v[k] = __floats2bfloat162_rn(o[c + 2 * k] * inv, o[c + 2 * k + 1] * inv);
+        *reinterpret_cast<uint4*>(dst + c) = *reinterpret_cast<const uint4*>(v);
+    }
+}
+
+// Number of partial pieces segment [t0, t1) was cut into by the CTA ranges (0 or 1 = not split).
+__device__ inline int segment_pieces(int t0, int t1, int total, int n_ctas) {
+    const int c_first = range_owner(t0, total, n_ctas), c_last = range_owner(t1 - 1, total, n_ctas);
+    if (c_first == c_last) return 1;
+    int n = 0;
+    for (int c = c_first; c <= c_last; ++c) {
+        const int sc = range_begin(c, total, n_ctas), ec = range_begin(c + 1, total, n_ctas);
+        n += max(sc, t0) < min(ec, t1);
+    }
+    return n;
+}
+
+// Combine the partial pieces of segment (b, kvh) for query row r, columns [cg * CW, (cg + 1) * CW),
+// in CTA-range order (fixed, so the result does not depend on timing), and write the bf16 output.
+// The caller guarantees that every piece has been written and is visible.
+template <int D, int CW>
+__device__ inline void merge_row(const AttnParams& p, int total, int b, int kvh, int r, int cg) {
+    const int row0 = p.plan.cu_q[b];
+    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
+    float acc[CW];
+#pragma unroll
+    for (int c = 0; c < CW; ++c) acc[c] = 0.f;
+    if (!__ldcg(p.plan.seq_ok + b)) {  // a page id of this sequence was bad: defined output, zeros
+        store_cols_bf16<CW>(dst, acc, 0.f);
+        return;
+    }
+    const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
+    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles, t1 = t0 + ntiles;
+    const int c_first = range_owner(t0, total, p.n_ctas), c_last = range_owner(t1 - 1, total, p.n_ctas);
+    float m = -INFINITY;
+    for (int c = c_first; c <= c_last; ++c) {
+        const int sc = range_begin(c, total, p.n_ctas), ec = range_begin(c + 1, total, p.n_ctas);
+        if (max(sc, t0) >= min(ec, t1)) continue;
+        const int slot = 2 * c + (sc >= t0 ? 0 : 1);
+        m = fmaxf(m, __ldcg(p.part.m + slot * kMaxRows + r));
+    }
+    float l = 0.f;
+    for (int c = c_first; c <= c_last; ++c) {
+        const int sc = range_begin(c, total, p.n_ctas), ec = range_begin(c + 1, total, p.n_ctas);
+        if (max(sc, t0) >= min(ec, t1)) continue;
+        const int slot = 2 * c + (sc >= t0 ? 0 : 1);
+        const float mp = __ldcg(p.part.m + slot * kMaxRows + r);
+        if (mp == -INFINITY) continue;  // this piece saw no visible key for the row
+        const float w = exp2f(mp - m);
+        l += w * __ldcg(p.part.l + slot * kMaxRows + r);
+        const float* o = p.part.o + ((long long)slot * D + cg * CW) * kMaxRows + r;
+#pragma unroll
+        for (int col = 0; col < CW; ++col) acc[col] += w * __ldcg(o + col * kMaxRows);
+    }
+    store_cols_bf16<CW>(dst, acc, 1.f / l);
 }
 
 // Launchers (defined next to their kernels).

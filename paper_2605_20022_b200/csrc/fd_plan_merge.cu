@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     if (tid == 0) s_fatal = 0;
     __syncthreads();
     const int P = 16;
+    for (int i = tid; i < B * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
     long long rows = 0, tiles = 0;  // running totals (identical in every thread)
     for (int base = 0; base < B; base += blockDim.x) {
         const int b = base + tid;
@@ -77,25 +78,13 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
 
 void launch_plan(const AttnParams& p, cudaStream_t s) { plan_kernel<<<1, 256, 0, s>>>(p); }
 
-template <int D>
-__device__ inline void store_row_bf16(__nv_bfloat16* dst, const float* o, float inv) {
-#pragma unroll
-    for (int c = 0; c < D; c += 8) {
-        __align__(16) __nv_bfloat162 v[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) v[k] = __floats2bfloat162_rn(o[c + 2 * k] * inv, o[c + 2 * k + 1] * inv);
-        *reinterpret_cast<uint4*>(dst + c) = *reinterpret_cast<const uint4*>(v);
-    }
-}
-
-// One CTA per (sequence, kv-head) segment; thread (r, cg) owns query row r = tid % 128 and the
-// column group cg = tid / 128 (a quarter of d), so the partial reads of a warp are coalesced
-// and enough loads are in flight to hide their latency.
+// Separate merge pass (used with the SIMT attention kernel; the tensor-core kernel merges inside
+// its own epilogue).  One CTA per (sequence, kv-head) segment; thread (r, cg) owns query row
+// r = tid % 128 and a quarter of the columns, so partial reads are coalesced and plentiful.
 constexpr int kMergeThreads = 4 * kMaxRows;
 
 template <int D>
 __global__ void __launch_bounds__(kMergeThreads) merge_kernel(AttnParams p) {
-    constexpr int CW = D / 4;  // columns per thread
     const PlanHeader hdr = *p.plan.hdr;
     if (hdr.fatal) {  // defined output for an undefined request: zeros
         const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
@@ -106,44 +95,14 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(AttnParams p) {
         return;
     }
     const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
-    const int row0 = p.plan.cu_q[b], Lq = p.plan.cu_q[b + 1] - row0;
-    const int rows = Lq * p.G, r = threadIdx.x % kMaxRows, cg = threadIdx.x / kMaxRows;
+    const int rows = (p.plan.cu_q[b + 1] - p.plan.cu_q[b]) * p.G;
+    const int r = threadIdx.x % kMaxRows, cg = threadIdx.x / kMaxRows;
     if (r >= rows) return;
-    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
-    float acc[CW];
-#pragma unroll
-    for (int c = 0; c < CW; ++c) acc[c] = 0.f;
-    if (!p.plan.seq_ok[b]) {
-        store_row_bf16<CW>(dst, acc, 0.f);
-        return;
-    }
     const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
-    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles, t1 = t0 + ntiles;
-    const int c_first = range_owner(t0, hdr.total_tiles, p.n_ctas);
-    const int c_last = range_owner(t1 - 1, hdr.total_tiles, p.n_ctas);
-    if (c_first == c_last) return;  // one CTA held the whole segment and wrote the final rows itself
-
-    float m = -INFINITY;
-    for (int c = c_first; c <= c_last; ++c) {
-        const int sc = range_begin(c, hdr.total_tiles, p.n_ctas), ec = range_begin(c + 1, hdr.total_tiles, p.n_ctas);
-        if (max(sc, t0) >= min(ec, t1)) continue;
-        const int slot = 2 * c + (sc >= t0 ? 0 : 1);
-        m = fmaxf(m, p.part.m[slot * kMaxRows + r]);
-    }
-    float l = 0.f;
-    for (int c = c_first; c <= c_last; ++c) {
-        const int sc = range_begin(c, hdr.total_tiles, p.n_ctas), ec = range_begin(c + 1, hdr.total_tiles, p.n_ctas);
-        if (max(sc, t0) >= min(ec, t1)) continue;
-        const int slot = 2 * c + (sc >= t0 ? 0 : 1);
-        const float mp = p.part.m[slot * kMaxRows + r];
-        if (mp == -INFINITY) continue;  // this piece saw no visible key for the row
-        const float w = exp2f(mp - m);
-        l += w * p.part.l[slot * kMaxRows + r];
-        const float* o = p.part.o + ((long long)slot * D + cg * CW) * kMaxRows + r;
-#pragma unroll
-        for (int col = 0; col < CW; ++col) acc[col] += w * o[col * kMaxRows];
-    }
-    store_row_bf16<CW>(dst, acc, 1.f / l);
+    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles;
+    // an unsplit segment was written by the attention kernel itself; it is revisited only to zero it
+    if (segment_pieces(t0, t0 + ntiles, hdr.total_tiles, p.n_ctas) <= 1 && p.plan.seq_ok[b]) return;
+    merge_row<D, D / 4>(p, hdr.total_tiles, b, kvh, r, cg);
 }
 
 void launch_merge(const AttnParams& p, cudaStream_t s) {
