@@ -96,17 +96,21 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_
 }
 
 #ifdef FD_TRACE
-// Debug build only: per-role timestamps of CTA 0 (role, event, tile, clock) for pipeline analysis.
-__device__ unsigned long long g_trace[4 * 8192];
-__device__ unsigned int g_trace_n;
-__device__ __forceinline__ void trace(int role, int ev, int tile) {
-    if (blockIdx.x != 0) return;
-    const unsigned int i = atomicAdd(&g_trace_n, 1u);
-    if (i < 8192) { g_trace[4 * i] = role; g_trace[4 * i + 1] = ev; g_trace[4 * i + 2] = tile; g_trace[4 * i + 3] = clock64(); }
+// Debug build only: per-role timestamps of CTA 0 for pipeline analysis.  Each role's tracing thread
+// owns a region and a private counter, so an event costs one clock read and one store.
+constexpr int kTraceRoles = 6, kTracePerRole = 4096;
+__device__ unsigned long long g_trace[kTraceRoles * kTracePerRole];
+__device__ unsigned int g_trace_n[kTraceRoles];
+__device__ __forceinline__ void trace(int role, int ev, int tile, int& n) {
+    if (blockIdx.x != 0 || n >= kTracePerRole) return;
+    g_trace[role * kTracePerRole + n] = ((unsigned long long)clock64() & 0xffffffffffull) | ((unsigned long long)ev << 40) | ((unsigned long long)tile << 48);
+    g_trace_n[role] = ++n;
 }
-#define TRACE(role, ev, tile) trace(role, ev, tile)
+#define TRACE(role, ev, tile) trace(role, ev, tile, tr_n)
+#define TRACE_DECL int tr_n = 0
 #else
 #define TRACE(role, ev, tile)
+#define TRACE_DECL
 #endif
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -129,6 +133,7 @@ template <int D, bool kSoftmax>
 __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnParams& p, unsigned char* sq, unsigned char* sk,
                                          unsigned char* sv, Bars* bars, int total, int s_c, int e_c) {
     using C = Cfg<D>;
+    TRACE_DECL;
     float* ex_m = reinterpret_cast<float*>(sq);          // [2][128], aliases Q after the last MMA of a piece
     float* ex_l = ex_m + 2 * kMaxRows;
     volatile int* abort = &bars->abort;
@@ -151,20 +156,32 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
 
     for (int t = s_c; t < e_c;) {
         const Piece pc = decode_piece(p, t, s_c, e_c, cta);
+        if (tid == 0) TRACE(5, 2, piece_idx);
 
         // ---- Q tile -> shared memory, K-major, 128-byte swizzle; rows beyond the block are zero
-        if (!loader)
-        for (int idx = ltid; idx < kMaxRows * (D / 8); idx += kPieceThreads) {
-            const int r = idx / (D / 8), ch = idx % (D / 8);
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (r < pc.rows)
-                v = *reinterpret_cast<const uint4*>(p.q + ((long long)(pc.row0 + r / p.G) * p.Hq + pc.kvh * p.G + r % p.G) * D + ch * 8);
-            const int half = ch >> 3, c16 = ch & 7;
-            *reinterpret_cast<uint4*>(sq + half * (kMaxRows * 128) + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
+        if (!loader) {
+            constexpr int kChunks = kMaxRows * (D / 8);                               // 16-byte chunks of the tile
+            constexpr int kIters = (kChunks + kPieceThreads - 1) / kPieceThreads;
+            uint4 v[kIters];
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {                                     // all loads in flight first
+                const int idx = ltid + it * kPieceThreads, r = idx / (D / 8), ch = idx % (D / 8);
+                v[it] = make_uint4(0, 0, 0, 0);
+                if (idx < kChunks && r < pc.rows)
+                    v[it] = *reinterpret_cast<const uint4*>(p.q + ((long long)(pc.row0 + r / p.G) * p.Hq + pc.kvh * p.G + r % p.G) * D + ch * 8);
+            }
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {
+                const int idx = ltid + it * kPieceThreads, r = idx / (D / 8), ch = idx % (D / 8);
+                const int half = ch >> 3, c16 = ch & 7;
+                if (idx < kChunks)
+                    *reinterpret_cast<uint4*>(sq + half * (kMaxRows * 128) + r * 128 + ((c16 ^ (r & 7)) << 4)) = v[it];
+            }
         }
         if (!loader) {
             fence_proxy_async_smem();
             named_bar_sync(2, kPieceThreads);
+            if (tid == 0) TRACE(5, 3, piece_idx);
         }
 
         if constexpr (!kSoftmax) {
@@ -282,7 +299,10 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
             float m = -INFINITY, l = 0.f;
             bool ok = true;
 
-            for (int j = s; j < pc.nt; j += 2) {
+            // Warps whose 32 rows are all padding do nothing per tile: warp 0 of the group (always active)
+            // arrives on p_full for them, and they wait at the epilogue's hardware barrier, not by polling.
+            const int n_idle_threads = 32 * (4 - min(4, (pc.rows + 31) >> 5));
+            for (int j = s; j < pc.nt && warp_active; j += 2) {
                 const int u = u_base[s] + (j >> 1);
                 if (!wait_all(&bars->s_full[s], u & 1, abort)) { ok = false; break; }
                 tc_fence_after();
@@ -367,14 +387,16 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
                 }
                 tc_fence_before();
                 mbar_arrive(&bars->p_full[s]);
+                if ((warp & 3) == 0 && lane == 0 && n_idle_threads) mbar_arrive_cnt(&bars->p_full[s], n_idle_threads);
                 if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 2, g0 + j);
             }
 
             // ---- epilogue: merge the two streams, then final rows, or a partial plus -- if this CTA is the
             //      last one to deliver a piece of the segment -- the merge of all its partials
-            ok = ok && wait_all(&bars->all_done, piece_idx & 1, abort);
+            if (warp_active) ok = ok && wait_all(&bars->all_done, piece_idx & 1, abort);
             tc_fence_after();
-            if (ok) {
+            if (tid == 0) TRACE(5, 4, piece_idx);
+            if (ok && warp_active) {  // (idle warps have not waited for the MMAs: Q, which this aliases, may still be read)
                 ex_m[s * kMaxRows + r] = m;
                 ex_l[s * kMaxRows + r] = l;
             }
@@ -456,6 +478,7 @@ __device__ __forceinline__ void run_role(const CUtensorMap& tmap, const AttnPara
         }
 
         // ---- end of piece: every MMA and every epilogue read of this piece has completed (or the CTA is aborting)
+        if (tid == 0) TRACE(5, 5, piece_idx);
         if (!loader) named_bar_sync(2, kPieceThreads);
         if (*abort) break;
         g0 += pc.nt;
@@ -606,16 +629,14 @@ void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s) {
 void attn_tc_free(void* state) { delete static_cast<TcState*>(state); }
 
 #ifdef FD_TRACE
-extern "C" int fd_debug_read_trace(unsigned long long* dst, int max_events) {
-    unsigned int n = 0;
+// dst: [roles][per_role] packed events; counts: [roles].  Resets the counters.
+extern "C" int fd_debug_read_trace(unsigned long long* dst, unsigned int* counts) {
     cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n));
-    if (n > 8192) n = 8192;
-    if ((int)n > max_events) n = max_events;
-    cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * 4 * n);
-    unsigned int zero = 0;
-    cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero));
-    return (int)n;
+    cudaMemcpyFromSymbol(counts, g_trace_n, sizeof(unsigned int) * kTraceRoles);
+    cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * kTraceRoles * kTracePerRole);
+    unsigned int zero[kTraceRoles] = {0};
+    cudaMemcpyToSymbol(g_trace_n, zero, sizeof(zero));
+    return kTracePerRole;
 }
 #endif
 
