@@ -102,6 +102,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const size_t o_cut = take((B + 1) * sizeof(int));
     const size_t o_ok = take(B * sizeof(int));
     const size_t o_sc = take((size_t)B * cfg->n_kv_heads * sizeof(int));
+    const size_t o_cf = take((size_t)c->n_ctas * sizeof(int));
     const size_t o_po = take(slots * d * fd::kMaxRows * sizeof(float));
     const size_t o_pm = take(slots * fd::kMaxRows * sizeof(float));
     const size_t o_pl = take(slots * fd::kMaxRows * sizeof(float));
@@ -115,6 +116,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->plan.cu_tiles = reinterpret_cast<int*>(c->pool + o_cut);
     c->plan.seq_ok = reinterpret_cast<int*>(c->pool + o_ok);
     c->plan.seg_count = reinterpret_cast<int*>(c->pool + o_sc);
+    c->plan.cta_first = reinterpret_cast<int*>(c->pool + o_cf);
     c->part.o = reinterpret_cast<float*>(c->pool + o_po);
     c->part.m = reinterpret_cast<float*>(c->pool + o_pm);
     c->part.l = reinterpret_cast<float*>(c->pool + o_pl);
@@ -287,11 +289,14 @@ fd_status fd_attn_draft_verify(fd_ctx* c, int batch, int total_q_rows, const voi
     p.out = static_cast<__nv_bfloat16*>(out);
     p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
 
-    if (c->attn_path == FD_ATTN_TCGEN05) {
+    const bool tc = c->attn_path == FD_ATTN_TCGEN05 && total_q_rows > 0;  // no rows: the plan alone checks the lengths
+    if (tc) {
         if (fd::attn_tc_prepare(&c->tc_state, p) != cudaSuccess) { cudaGetLastError(); return FD_ERR_CUDA; }
     }
     fd::launch_plan(p, s);
-    if (c->attn_path == FD_ATTN_TCGEN05) {
+    if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
+        c->launches += 1;
+    } else if (tc) {
         fd::launch_attn_tc(c->tc_state, p, s);  // merges split segments in its own epilogue
         c->launches += 2;
     } else {

@@ -27,6 +27,7 @@ struct Plan {
     int* cu_tiles;  // [B+1] exclusive scan of tiles_b (per kv-head)
     int* seq_ok;    // [B]   0 = a page id of the sequence was outside the pool: its rows are zeroed
     int* seg_count; // [B * Hkv] partial pieces of a segment that have been written (fused merge)
+    int* cta_first; // [n_ctas] sequence that owns the first tile of each attention CTA's range
 };
 
 // Partial result of one piece of a (sequence, kv-head) segment, log2 domain:

@@ -66,6 +66,20 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
         tiles += tt;
     }
     __syncthreads();
+    // where each attention CTA starts: the sequence that owns the first tile of its range (the kernels
+    // then walk forward from there instead of searching the scan with dependent loads)
+    const long long total = tiles * p.Hkv;
+    if (!s_fatal && total > 0 && total <= 0x7fffffffLL) {
+        for (int c = tid; c < p.n_ctas; c += blockDim.x) {
+            const int t = range_begin(c, (int)total, p.n_ctas);
+            int lo = 0, hi = B;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (p.Hkv * __ldcg(p.plan.cu_tiles + mid) <= t) lo = mid; else hi = mid;
+            }
+            p.plan.cta_first[c] = lo;
+        }
+    }
     if (tid == 0) {
         const int fatal = s_fatal || rows != p.total_q_rows || tiles * p.Hkv > 0x7fffffffLL;
         p.plan.cu_q[0] = 0;
