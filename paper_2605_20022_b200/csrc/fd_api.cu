@@ -1,5 +1,6 @@
 // C ABI of libflexdraft: context, argument checks, launch sequencing.
 #include <math.h>
+#include <algorithm>
 #include <new>
 
 #include "fd_internal.cuh"
@@ -221,10 +222,19 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         if (l >= 2) chk(cudaStreamWaitEvent(h->h2d, h->attn_done[b], 0));
         chk(cudaMemcpyAsync(h->q[b], static_cast<const unsigned char*>(q_host) + (size_t)l * qb, qb, H2D, h->h2d));
         chk(cudaEventRecord(h->q_ready[b], h->h2d));
-        if (l == 1 && total_cand_rows > 0) {  // the logits follow the first two q blocks so that layer 0 starts at once
-            chk(cudaMemcpyAsync(h->lg, logits_host, (size_t)total_cand_rows * c->cfg.vocab * 4, H2D, h->h2d));
-            chk(cudaMemcpyAsync(h->drafts, draft_tokens_host, (size_t)total_cand_rows * 4, H2D, h->h2d));
-            chk(cudaEventRecord(h->logits, h->h2d));
+        if (l >= 1 && total_cand_rows > 0) {
+            // the logits go up in n_layers - 1 slices, one behind each later q block, so that no q block ever
+            // queues behind a large copy; each slice hides under one layer's attention
+            const size_t total = (size_t)total_cand_rows * c->cfg.vocab * 4;
+            const size_t per = ((total + (size_t)(n_layers - 1) - 1) / (size_t)(n_layers - 1) + 255) / 256 * 256;
+            const size_t lo = std::min(total, per * (size_t)(l - 1)), hi = std::min(total, per * (size_t)l);
+            if (hi > lo)
+                chk(cudaMemcpyAsync(reinterpret_cast<unsigned char*>(h->lg) + lo,
+                                    reinterpret_cast<const unsigned char*>(logits_host) + lo, hi - lo, H2D, h->h2d));
+            if (l == n_layers - 1) {
+                chk(cudaMemcpyAsync(h->drafts, draft_tokens_host, (size_t)total_cand_rows * 4, H2D, h->h2d));
+                chk(cudaEventRecord(h->logits, h->h2d));
+            }
         }
         chk(cudaStreamWaitEvent(s, h->q_ready[b], 0));
         if (l >= 2) chk(cudaStreamWaitEvent(s, h->out_copied[b], 0));
