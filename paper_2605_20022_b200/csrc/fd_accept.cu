@@ -1,6 +1,6 @@
 // Greedy verification: vocab argmax of every candidate row fused with the accept scan.
 //
-// The [R, V] fp32 logits are swept once.  Each CTA reduces one 8192-logit chunk of one row
+// The [R, V] fp32 logits are swept once.  Each CTA reduces one 4096-logit chunk of one row
 // to a 64-bit key (order-preserving image of the float in the high word, ~index in the low
 // word, so an unsigned max picks the larger value and, on equal values, the lower index)
 // and folds it into the row's running key with atomicMax -- an exact, order-independent
@@ -9,6 +9,8 @@
 #include "fd_internal.cuh"
 
 namespace fd {
+
+constexpr int kVecPerThread = kAcceptChunk / (4 * 256);  // float4 loads in flight per thread
 
 __device__ inline unsigned long long make_key(float v, unsigned idx) {
     v += 0.0f;  // -0.0 -> +0.0: they compare equal, so the lower index must decide
@@ -35,14 +37,14 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_
     const int nvec = (c1 - c0 - head) >> 2;
     if (tid < head) fold(bv, bi, base[c0 + tid], c0 + tid);
     const float4* vp = reinterpret_cast<const float4*>(base + c0 + head);
-    float4 v[8];
+    float4 v[kVecPerThread];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < kVecPerThread; ++k) {
         const int e = tid + k * 256;
         v[k] = (e < nvec) ? __ldcs(vp + e) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < kVecPerThread; ++k) {
         const unsigned i0 = c0 + head + 4 * (tid + k * 256);
         if (tid + k * 256 < nvec) {
             fold(bv, bi, v[k].x, i0);

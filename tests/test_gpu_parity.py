@@ -135,7 +135,7 @@ def test_accept_and_commit_workloads(idx):
     np.testing.assert_array_equal(freed, efreed)
 
 
-@pytest.mark.parametrize("V", [1, 3, 17, 1000, 4097, 8191, 8192, 8193, 151937, 200003])
+@pytest.mark.parametrize("V", [1, 3, 17, 1000, 4095, 4096, 4097, 8191, 8193, 151937, 200003])
 def test_accept_vocab_sizes_ties_and_alignment(V):
     g = torch.Generator().manual_seed(V)
     ql = [1, 4, 16, 2, 7, 0, 16]
