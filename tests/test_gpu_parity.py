@@ -45,6 +45,11 @@ EDGE = {
     "mha_group1": (4, 4, 64, [130, 257], [32, 20], [16, 4]),
     "one_long_sequence_many_splits": (4, 1, 128, [20000], [32], [16]),
     "ragged_mix": (32, 8, 128, [5000, 13, 700, 2047, 2049, 129], [32, 1, 20, 9, 32, 16], [16, 0, 16, 0, 16, 8]),
+    # many short segments per CTA range: every piece boundary, single-tile pieces, 1..3 active softmax warps
+    "many_tiny_sequences": (32, 8, 128, [(7 * b) % 41 for b in range(150)], [1 + (5 * b) % 24 for b in range(150)],
+                            [min(1 + (5 * b) % 24, (3 * b) % 17) for b in range(150)]),
+    # one CTA range holds the tail of a long segment, whole short ones and the head of another long one
+    "long_short_long": (32, 8, 128, [9000, 100, 37, 260, 12000, 5], [32, 4, 17, 32, 32, 9], [16, 0, 1, 16, 16, 0]),
 }
 
 
@@ -54,7 +59,7 @@ def test_attention_edge_cases(name, path):
     Hq, Hkv, d, pl, ql, nm = EDGE[name]
     step = wl.make_step(name, wl.Shape(Hq, Hkv, d, 1000), pl, ql, nm, seed=zlib.crc32(name.encode()) % 10000, extra_table_cols=2)
     q, kv = wl.make_q(step), wl.make_kv(step, poison=float("nan"))     # NaN in every slot no token owns
-    with Ctx(step, path) as ctx:
+    with Ctx(step, path, max_batch=len(pl)) as ctx:
         got, status = gpu_attn(ctx, step, q, kv)
         again, _ = gpu_attn(ctx, step, q, kv)
     assert status == 0
