@@ -545,21 +545,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     volatile int* abort = &bars->abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const PlanHeader hdr = *p.plan.hdr;
-    const int total = hdr.total_tiles;
-    if (total == 0) {  // uniform: nothing allocated yet
-        if (hdr.fatal) {  // inconsistent lengths: a defined output, zeros
-            const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
-            uint4* o = reinterpret_cast<uint4*>(p.out);
-            for (long long i2 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i2 < n16; i2 += (long long)gridDim.x * blockDim.x)
-                o[i2] = make_uint4(0, 0, 0, 0);
-        }
-        return;
-    }
-    const int cta = blockIdx.x;
-    const int s_c = range_begin(cta, total, p.n_ctas), e_c = range_begin(cta + 1, total, p.n_ctas);
-    if (s_c >= e_c) return;
 
+    // ---- set-up that needs nothing from the plan kernel: it overlaps that kernel's execution
+    //      (programmatic dependent launch); griddepcontrol.wait below is where its results are needed
     if (tid == 0) {
         for (int i = 0; i < C::kStages; ++i) {
             mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
@@ -584,6 +572,23 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the plan kernel has completed and its writes are visible
+
+    const PlanHeader hdr = *p.plan.hdr;
+    const int total = hdr.total_tiles;
+    const int cta = blockIdx.x;
+    const int s_c = total ? range_begin(cta, total, p.n_ctas) : 0, e_c = total ? range_begin(cta + 1, total, p.n_ctas) : 0;
+    if (s_c >= e_c) {  // uniform: no tile for this CTA (or nothing at all)
+        if (total == 0 && hdr.fatal) {  // inconsistent lengths: a defined output, zeros
+            const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
+            uint4* o = reinterpret_cast<uint4*>(p.out);
+            for (long long i2 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i2 < n16; i2 += (long long)gridDim.x * blockDim.x)
+                o[i2] = make_uint4(0, 0, 0, 0);
+        }
+        __syncthreads();
+        if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+        return;
+    }
     // Warp-specialised register budgets: the softmax groups keep a whole 128-column row of S in registers.
     // 8 x 32 x 216 + 4 x 32 x 72 = 384 x 168, what the launch allocated: the increase is served by what
     // the decrease released (a request for more than that did not return when it was tried).
@@ -687,8 +692,24 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
 void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
     const TcState* st = static_cast<const TcState*>(state);
-    if (p.d == 64) attn_tc_kernel<64><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, s>>>(*st->current, *st->qcurrent, p);
-    else attn_tc_kernel<128><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, s>>>(*st->current, *st->qcurrent, p);
+    // Programmatic dependent launch: the CTAs may start while the plan kernel (the previous launch on the
+    // stream) is still running; they do their set-up and then wait for it inside the kernel.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (p.d == 64) {
+        cfg.dynamicSmemBytes = Cfg<64>::kSmemBytes;
+        cudaLaunchKernelEx(&cfg, attn_tc_kernel<64>, *st->current, *st->qcurrent, p);
+    } else {
+        cfg.dynamicSmemBytes = Cfg<128>::kSmemBytes;
+        cudaLaunchKernelEx(&cfg, attn_tc_kernel<128>, *st->current, *st->qcurrent, p);
+    }
 }
 
 void attn_tc_free(void* state) { delete static_cast<TcState*>(state); }

@@ -39,6 +39,8 @@ __device__ inline void block_scan2(int& a, int& b, int& ta, int& tb, int (*wsum)
 __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     __shared__ int s_fatal;
     __shared__ int wsum[8][2];
+    // let the attention kernel behind us start its set-up now; it waits for our completion before it reads the plan
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int B = p.batch, tid = threadIdx.x;
     if (tid == 0) s_fatal = 0;
     __syncthreads();
