@@ -20,6 +20,7 @@
  *     NULL = the legacy default stream) and ordered by it.  Calls that share one fd_ctx
  *     must be issued on one stream, or be ordered by the caller: they share the context's
  *     scratch memory.
+ *     A context is not thread-safe: one host thread at a time per fd_ctx.
  *   - The hot calls (fd_attn_draft_verify, fd_verify_accept, fd_kv_commit) never allocate
  *     and never synchronise; all scratch memory is sized by fd_create() from fd_config.
  *   - Errors the host can see (NULL pointer, size beyond the configured maximum,

@@ -92,6 +92,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->attn_path = (cfg->attn_path == FD_ATTN_SIMT || !tc_ok) ? FD_ATTN_SIMT : FD_ATTN_TCGEN05;
     // SIMT kernel: two 74 KB CTAs fit an SM; tensor-core kernel: one persistent CTA per SM
     c->n_ctas = c->attn_path == FD_ATTN_SIMT ? 2 * c->n_sms : c->n_sms;
+    if (c->attn_path == FD_ATTN_SIMT && fd::attn_simt_prepare(cfg->head_dim) != cudaSuccess) { cudaGetLastError(); delete c; return FD_ERR_CUDA; }
 
     const int B = cfg->max_batch, d = cfg->head_dim;
     const size_t slots = 2 * (size_t)c->n_ctas;

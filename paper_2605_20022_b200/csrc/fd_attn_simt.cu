@@ -145,17 +145,18 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
     }
 }
 
+// 66 KB + 8 KB of dynamic shared memory needs the opt-in; a per-device attribute, set once per context at fd_create.
+cudaError_t attn_simt_prepare(int d) {
+    if (d != 128) return cudaSuccess;
+    return cudaFuncSetAttribute(attn_simt_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kMaxRows * 4 + 2 * 16 * 128 * 2);
+}
+
 void launch_attn_simt(const AttnParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
     const int smem = p.d * kMaxRows * 4 + 2 * 16 * p.d * 2;
     if (p.d == 64) {
         attn_simt_kernel<64><<<p.n_ctas, kMaxRows, smem, s>>>(p);
     } else {
-        static bool once = false;  // 66 KB + 8 KB of dynamic shared memory needs the opt-in
-        if (!once) {
-            cudaFuncSetAttribute(attn_simt_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            once = true;
-        }
         attn_simt_kernel<128><<<p.n_ctas, kMaxRows, smem, s>>>(p);
     }
 }

@@ -132,6 +132,7 @@ __device__ inline void merge_row(const AttnParams& p, int total, int b, int kvh,
 
 // Launchers (defined next to their kernels).
 void launch_plan(const AttnParams& p, cudaStream_t s);
+cudaError_t attn_simt_prepare(int d);
 void launch_attn_simt(const AttnParams& p, cudaStream_t s);
 bool attn_tc_supported(int d, int G, int max_q_len);
 cudaError_t attn_tc_prepare(void** state, const AttnParams& p);  // tensor map for this kv pool
