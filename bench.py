@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 
 # DRAM bytes (read + write) of ONE attention-kernel launch on the long-context workload, from the
 # ncu capture summarised in profiles/attn_tc_and_accept_kernels_long_context_1layer.md
-# (dram__bytes_read.sum 2 161 183 000 + dram__bytes_write.sum 16 745 728; one layer = one full-size launch).
-NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_177_928_728}
+# (dram__bytes_read.sum 2 158 917 000 + dram__bytes_write.sum 7 709 696; one layer = one full-size launch).
+NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_166_626_696}
 
 METRIC = "draft-verify attn+accept us/step"
 UNIT = "us/step"
@@ -368,7 +368,7 @@ def run_ours(args, step, rank, world, dist):
                    "us_per_step_cuda_graph_replay": us_graph},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(step.name) if resolved == "tcgen05" else None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
-                     "kernel": "fd_attn_draft_verify (plan + split-KV attention + merge launches)",
+                     "kernel": "fd_attn_draft_verify (plan launch + split-KV attention launch, merge fused)",
                      "algorithmic_bytes_per_launch": attn_bytes, "avg_launch_ms": attn_avg_ms,
                      "launches_timed": len(attn_ms)},
         "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": cpu_desc},
