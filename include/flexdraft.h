@@ -257,6 +257,13 @@ fd_status fd_verify_accept_static(int vocab, int batch, int total_cand_rows,
  * pointer).  Synchronises `stream` first. */
 fd_status fd_last_device_status(fd_ctx* ctx, int32_t* code, void* stream);
 
+/* Failure-detection self-test (no counterpart in the paper).  Every device-side wait of the
+ * attention kernel is bounded: when it runs out, the kernel stops cleanly and raises
+ * FD_DEV_TIMEOUT instead of hanging the GPU.  This call exercises exactly that mechanism on a
+ * barrier that nothing will ever signal: one warp waits for `limit_ms` (1..1000) milliseconds,
+ * gives up, sets FD_DEV_TIMEOUT in the status word and returns.  The context stays usable. */
+fd_status fd_selftest_wait_timeout(fd_ctx* ctx, int limit_ms, void* stream);
+
 /* Which attention kernel the context resolved to: FD_ATTN_SIMT or FD_ATTN_TCGEN05. */
 int fd_attn_path(const fd_ctx* ctx);
 

@@ -23,7 +23,7 @@ FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout"]
 
 
 class fd_config(ctypes.Structure):
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
         lib.fd_kv_commit.argtypes = [vp, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_verify_accept_static.argtypes = [ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_host_reserve.argtypes = [vp, ci, ci]
+        lib.fd_selftest_wait_timeout.argtypes = [vp, ci, vp]
         lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 13
         lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         lib.fd_attn_path.argtypes = [vp]
@@ -163,6 +164,10 @@ def fd_step_host(ctx, batch, total_q_rows, total_cand_rows, kv_caches, num_pages
                                _ptr(prefix_lens_host), _ptr(q_lens_host), _ptr(n_mask_host), _ptr(accepted_len_host),
                                _ptr(bonus_token_host), _ptr(freed_pages_host), _ptr(n_freed_host), _stream(stream))
     return _check("fd_step_host", code, raise_on_error)
+
+
+def fd_selftest_wait_timeout(ctx, limit_ms, stream=None) -> None:
+    _check("fd_selftest_wait_timeout", load().fd_selftest_wait_timeout(ctx, limit_ms, _stream(stream)), True)
 
 
 def fd_last_device_status(ctx, stream=None) -> int:

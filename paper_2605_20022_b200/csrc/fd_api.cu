@@ -354,6 +354,13 @@ fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefi
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }
 
+fd_status fd_selftest_wait_timeout(fd_ctx* c, int limit_ms, void* stream) {
+    if (!c || limit_ms < 1 || limit_ms > 1000) return FD_ERR_INVALID_ARG;
+    fd::launch_wait_timeout_selftest(c->status, (unsigned long long)limit_ms * 1000000ull, static_cast<cudaStream_t>(stream));
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
 fd_status fd_last_device_status(fd_ctx* c, int32_t* code, void* stream) {
     if (!c || !code) return FD_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -714,6 +714,22 @@ void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s) {
 
 void attn_tc_free(void* state) { delete static_cast<TcState*>(state); }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever arrive on.
+// The wait gives up after `limit_ns`, the kernel raises FD_DEV_TIMEOUT and returns normally.
+__global__ void wait_timeout_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0; mbar_fence_init(); }
+    __syncthreads();
+    const bool ok = mbar_wait_ns(&bar, 0, &abort_flag, limit_ns);
+    __syncwarp();
+    if (threadIdx.x == 0 && !ok) atomicOr(status, FD_DEV_TIMEOUT);
+}
+
+void launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, limit_ns);
+}
+
 #ifdef FD_TRACE
 // dst: [roles][per_role] packed events; counts: [roles].  Resets the counters.
 extern "C" int fd_debug_read_trace(unsigned long long* dst, unsigned int* counts) {

@@ -138,6 +138,7 @@ bool attn_tc_supported(int d, int G, int max_q_len);
 cudaError_t attn_tc_prepare(void** state, const AttnParams& p);  // tensor map for this kv pool
 void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s);
 void attn_tc_free(void* state);
+void launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);
 void launch_merge(const AttnParams& p, cudaStream_t s);
 
 struct AcceptParams {

@@ -48,18 +48,21 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // of the CTA has raised *abort; raises *abort itself when it gives up.  Returns false if it gave up.
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // one second
 constexpr uint32_t kSpinLimit = 1u << 20;                                  // polls of a drain loop
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait_ns(uint64_t* bar, uint32_t parity, volatile int* abort, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 0u) {
             if (*abort) return false;
-            if (global_ns() - t0 > kWaitLimitNs) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort = 1;
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    return mbar_wait_ns(bar, parity, abort, kWaitLimitNs);
 }
 
 // ---------------------------------------------------------------- proxies / fences

@@ -275,3 +275,22 @@ def test_host_buffer_step_matches_oracle():
             np.testing.assert_array_equal(h_pt.numpy(), ept); np.testing.assert_array_equal(h_pl.numpy(), epl)
             assert int(h_nf) == len(efreed)
             np.testing.assert_array_equal(h_freed.numpy()[:len(efreed)], efreed)
+
+
+def test_bounded_wait_times_out_cleanly_and_context_survives():
+    """A device-side wait that nothing will ever satisfy gives up after its limit, raises FD_DEV_TIMEOUT and
+    the kernel returns; the same context then computes a correct result."""
+    import time
+    step = wl.make_step("timeout", wl.Shape(8, 2, 128, 1000), [300], [12], [4], seed=2)
+    q, kv = wl.make_q(step), wl.make_kv(step)
+    with Ctx(step) as ctx:
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        fd.fd_selftest_wait_timeout(ctx.h, 50)
+        assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_TIMEOUT          # synchronises
+        dt = time.perf_counter() - t0
+        assert 0.04 < dt < 2.0, dt
+        assert fd.fd_last_device_status(ctx.h) == 0                           # read-and-clear
+        got, status = gpu_attn(ctx, step, q, kv)
+        assert status == 0
+        assert_close(got.numpy(), oracle_attn(step, q, kv), "after timeout")
