@@ -36,6 +36,21 @@ METRIC = "draft-verify attn+accept us/step"
 UNIT = "us/step"
 
 
+def paper_context():
+    """The paper's own end-to-end number, quoted as context only (another machine, another metric)."""
+    vals = {}
+    path = os.path.join(ROOT, "tests", "golden", "paper_context_numbers.txt")
+    if os.path.exists(path):
+        for ln in open(path):
+            ln = ln.strip()
+            if ln and not ln.startswith("#"):
+                k, v = [x.strip() for x in ln.split("=", 1)]
+                vals[k] = v
+    return {"speedup_over_autoregressive": float(vals.get("abstract_avg_speedup_qwen3_8b", 4.59)), "model": "Qwen3-8B",
+            "hardware": vals.get("hardware", "NVIDIA A100"), "batch_size": int(vals.get("batch_size", 1)),
+            "note": "the paper's end-to-end average speedup over autoregressive decoding; context only, not this metric"}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -375,6 +390,7 @@ def run_ours(args, step, rank, world, dist):
         "e2e": {"value": us_e2e, "unit": UNIT, "h2d_bytes_per_step": hs.h2d, "d2h_bytes_per_step": hs.d2h},
         "gpu_launches": int(launches),
         "clocks": clocks,
+        "paper_context": paper_context(),
     }
 
 
