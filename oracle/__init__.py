@@ -9,6 +9,8 @@ Functions
 ---------
 attn(...)        full attention under the hybrid mask (Sec. 4.1), float64 output
 attn_row(...)    one output row of the same definition (sampled checks)
+attn_blocks(...) the same with several mask blocks per sequence (all hypotheses, Eq. 2)
+select_branch(...) pick the prepared next-draft branch of the accepted length
 accept(...)      greedy verification: argmax, accepted length, bonus token (Sec. 3)
 commit(...)      KV commit / rollback by page-table truncation
 """
@@ -83,6 +85,32 @@ def attn(q, kv_cache, page_table, prefix_lens, q_lens, n_mask, scale=None) -> np
                      ctypes.c_int(P), ctypes.c_int(pt.shape[1]), _p(qb), _p(kvb), _p(pt), _p(pl), _p(ql),
                      _p(nm), ctypes.c_double(s), _p(out))
     return out
+
+
+def attn_blocks(q, kv_cache, page_table, prefix_lens, q_lens, n_mask, n_blocks, scale=None) -> np.ndarray:
+    """Attention with several mask blocks per sequence (all-hypotheses parallel drafting, Eq. 2)."""
+    qb, kvb = _bits(q), _bits(kv_cache)
+    T, Hq, d = qb.shape
+    _, two, Hkv, P, d2 = kvb.shape
+    pt, pl, ql, nm, nb = _i32(page_table), _i32(prefix_lens), _i32(q_lens), _i32(n_mask), _i32(n_blocks)
+    B = pl.shape[0]
+    assert int(ql.sum()) == T
+    out = np.zeros((T, Hq, d), dtype=np.float64)
+    s = float(scale) if scale else 1.0 / float(np.sqrt(d))
+    _load().fdo_attn_blocks(ctypes.c_int(B), ctypes.c_int(Hq), ctypes.c_int(Hkv), ctypes.c_int(d), ctypes.c_int(P),
+                            ctypes.c_int(pt.shape[1]), _p(qb), _p(kvb), _p(pt), _p(pl), _p(ql), _p(nm), _p(nb),
+                            ctypes.c_double(s), _p(out))
+    return out
+
+
+def select_branch(mask_tokens, q_lens, n_mask, n_blocks, accepted_len, max_kb):
+    """Returns (next_draft [B, max_kb] padded with -1, next_len [B])."""
+    mt, ql, nm, nb, acc = _i32(mask_tokens), _i32(q_lens), _i32(n_mask), _i32(n_blocks), _i32(accepted_len)
+    B = ql.shape[0]
+    nd = np.zeros((B, max_kb), np.int32)
+    nl = np.zeros((B,), np.int32)
+    _load().fdo_select_branch(ctypes.c_int(B), ctypes.c_int(max_kb), _p(mt), _p(ql), _p(nm), _p(nb), _p(acc), _p(nd), _p(nl))
+    return nd, nl
 
 
 def attn_row(q, kv_cache, page_table, prefix_lens, q_lens, n_mask, b, i, h, scale=None) -> np.ndarray:

@@ -46,6 +46,7 @@ static double bf16_to_f64(uint16_t bits)
 
 typedef struct {
     int Hq, Hkv, d, page_size, max_pages;
+    const int32_t *n_blocks;  /* [B] or NULL: mask blocks per sequence (0 / 1 / NULL = one block) */
     const uint16_t *q;        /* [T, Hq, d] bf16 bits */
     const uint16_t *kv;       /* [num_pages, 2, Hkv, page_size, d] bf16 bits */
     const int32_t *page_table;/* [B, max_pages] */
@@ -61,15 +62,24 @@ static const uint16_t *kv_ptr(const fdo_problem *p, int b, int j, int which, int
     return p->kv + ((((page * 2 + which) * p->Hkv + g) * p->page_size + slot) * (int64_t)p->d);
 }
 
-/* Hybrid mask (Sec. 4.1; Fig. 2 caption).  i = query row inside the block,
- * j = logical key position.  n = prefix length, C = candidate rows, M = mask rows. */
-static int allowed(int i, int j, int n, int C, int M)
+/* Hybrid mask (Sec. 4.1; Fig. 2 caption; Eq. 2 for several blocks).  i = query row inside the
+ * block, j = logical key position.  n = prefix length, C = candidate rows, M = mask rows, nb = mask
+ * blocks.  The M mask tokens form nb consecutive blocks of M / nb tokens; block g is the next-draft
+ * branch under the hypothesis that r = C - nb + g drafts are accepted (Eq. 2: conditioned on the
+ * prefix and the first r drafts), so it sees the candidates 0..r -- row 0 being the known bonus
+ * token -- and its own block in both directions; blocks never see each other, and clean rows never
+ * see a mask token.  nb = 1 is the single block that sees every candidate. */
+static int allowed(int i, int j, int n, int C, int M, int nb)
 {
     if (j < n) return 1;                    /* everyone sees the clean prefix */
     int t = j - n;                          /* index of the key inside the query block */
     if (i < C) return t <= i;               /* clean row: causal, never sees a mask token */
-    (void)M;
-    return 1;                               /* mask row: candidates + whole own block */
+    if (nb < 1) nb = 1;
+    int kb = M / nb;                        /* tokens per mask block */
+    int g = (i - C) / kb;                   /* block of this mask row */
+    int r = C - nb + g;                     /* hypothesis: candidates 0..r are the verified context */
+    if (t < C) return t <= r;               /* a candidate key */
+    return (t - C) / kb == g;               /* a mask key: own block only */
 }
 
 /* one output row out[d] for sequence b, block row i, q-head h; row0 = first q row of b */
@@ -78,12 +88,13 @@ static void attn_row(const fdo_problem *p, int b, int64_t row0, int i, int h, do
     const int d = p->d;
     const int n = p->prefix_lens[b], Lq = p->q_lens[b], M = p->n_mask[b], C = Lq - M;
     const int kv_len = n + Lq;
+    const int nb = p->n_blocks ? p->n_blocks[b] : 1;
     const int g = h / (p->Hq / p->Hkv);
     const uint16_t *qv = p->q + ((row0 + i) * p->Hq + h) * (int64_t)d;
 
     double mx = -INFINITY;
     for (int j = 0; j < kv_len; ++j) {
-        if (!allowed(i, j, n, C, M)) { w[j] = -INFINITY; continue; }
+        if (!allowed(i, j, n, C, M, nb)) { w[j] = -INFINITY; continue; }
         const uint16_t *kp = kv_ptr(p, b, j, 0, g);
         double s = 0.0;
         for (int c = 0; c < d; ++c) s += bf16_to_f64(qv[c]) * bf16_to_f64(kp[c]);
@@ -108,7 +119,7 @@ static fdo_problem make_problem(int Hq, int Hkv, int d, int page_size, int max_p
         const uint16_t *q, const uint16_t *kv, const int32_t *page_table,
         const int32_t *prefix_lens, const int32_t *q_lens, const int32_t *n_mask, double scale)
 {
-    fdo_problem p = { Hq, Hkv, d, page_size, max_pages, q, kv, page_table,
+    fdo_problem p = { Hq, Hkv, d, page_size, max_pages, NULL, q, kv, page_table,
                       prefix_lens, q_lens, n_mask, scale };
     return p;
 }
@@ -150,6 +161,61 @@ void fdo_attn(int B, int Hq, int Hkv, int d, int page_size, int max_pages,
         }
     }
     free(row0);
+}
+
+/* Same with several mask blocks per sequence (the all-hypotheses form of parallel drafting, Eq. 2). */
+void fdo_attn_blocks(int B, int Hq, int Hkv, int d, int page_size, int max_pages,
+        const uint16_t *q, const uint16_t *kv, const int32_t *page_table,
+        const int32_t *prefix_lens, const int32_t *q_lens, const int32_t *n_mask, const int32_t *n_blocks,
+        double scale, double *out)
+{
+    fdo_problem p = make_problem(Hq, Hkv, d, page_size, max_pages, q, kv, page_table,
+                                 prefix_lens, q_lens, n_mask, scale);
+    p.n_blocks = n_blocks;
+    int64_t row0 = 0;
+    int max_kv = 1;
+    for (int b = 0; b < B; ++b)
+        if (prefix_lens[b] + q_lens[b] > max_kv) max_kv = prefix_lens[b] + q_lens[b];
+    for (int b = 0; b < B; ++b) {
+        const int Lq = q_lens[b];
+        #pragma omp parallel
+        {
+            double *w = (double *)malloc(sizeof(double) * (size_t)max_kv);
+            #pragma omp for collapse(2) schedule(dynamic)
+            for (int i = 0; i < Lq; ++i)
+                for (int h = 0; h < Hq; ++h)
+                    attn_row(&p, b, row0, i, h, out + ((row0 + i) * Hq + h) * (int64_t)d, w);
+            free(w);
+        }
+        row0 += Lq;
+    }
+}
+
+/* Branch selection (Sec. 3, "Parallel speculative decoding": once verification has fixed r_acc, the
+ * branch prepared under that hypothesis becomes the next draft).  mask_tokens [sum_b M_b] holds one
+ * proposed token per mask row, sequence-major.  For sequence b with nb blocks of kb tokens the block
+ * of hypothesis r is g = r - (C_b - nb); next_draft [B, max_kb] receives its kb tokens (padded with -1)
+ * and next_len[b] = kb, or next_len[b] = 0 when that hypothesis was not prepared (g < 0), when the
+ * sequence has no mask rows, or when accepted_len[b] < 0. */
+void fdo_select_branch(int B, int max_kb, const int32_t *mask_tokens, const int32_t *q_lens, const int32_t *n_mask,
+        const int32_t *n_blocks, const int32_t *accepted_len, int32_t *next_draft, int32_t *next_len)
+{
+    int64_t m0 = 0;
+    for (int b = 0; b < B; ++b) {
+        const int M = n_mask[b], C = q_lens[b] - M;
+        int nb = n_blocks ? n_blocks[b] : 1;
+        if (nb < 1) nb = 1;
+        for (int u = 0; u < max_kb; ++u) next_draft[(int64_t)b * max_kb + u] = -1;
+        next_len[b] = 0;
+        if (M > 0 && accepted_len[b] >= 0) {
+            const int kb = M / nb, g = accepted_len[b] - (C - nb);
+            if (g >= 0 && g < nb) {
+                for (int u = 0; u < kb; ++u) next_draft[(int64_t)b * max_kb + u] = mask_tokens[m0 + (int64_t)g * kb + u];
+                next_len[b] = kb;
+            }
+        }
+        m0 += M;
+    }
 }
 
 /* A single output row (sampled checks at sizes where the full pass is too slow). */
