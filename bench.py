@@ -187,6 +187,7 @@ class DeviceStep:
         self.pt0, self.pl0 = step.page_table.to(device), step.prefix_lens.to(device)
         self.pt, self.pl = self.pt0.clone(), self.pl0.clone()
         self.ql, self.nm = step.q_lens.to(device), step.n_mask.to(device)
+        self.nb = step.n_blocks.to(device) if step.n_blocks is not None else None
         B = step.batch
         self.acc = torch.empty((B,), dtype=torch.int32, device=device)
         self.bon = torch.empty((B,), dtype=torch.int32, device=device)
@@ -208,8 +209,12 @@ class DeviceStep:
             if time_attn:
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record()
-            fd.fd_attn_draft_verify(self.ctx, st.batch, st.total_q_rows, self.q[l], self.kv[l], st.num_pages, self.pt,
-                                    self.pl, self.ql, self.nm, self.out[l])
+            if self.nb is None:
+                fd.fd_attn_draft_verify(self.ctx, st.batch, st.total_q_rows, self.q[l], self.kv[l], st.num_pages, self.pt,
+                                        self.pl, self.ql, self.nm, self.out[l])
+            else:   # one next-draft branch per hypothesis
+                fd.fd_attn_draft_verify_blocks(self.ctx, st.batch, st.total_q_rows, self.q[l], self.kv[l], st.num_pages,
+                                               self.pt, self.pl, self.ql, self.nm, self.nb, self.out[l])
             if time_attn:
                 e1.record(); self.attn_events.append((e0, e1))
         fd.fd_verify_accept(self.ctx, st.batch, st.total_cand_rows, self.logits, self.drafts, self.ql, self.nm,
@@ -233,6 +238,7 @@ class HostStep:
         self.h_logits, self.h_drafts = pin(ds.logits), pin(ds.drafts)
         self.pt0, self.pl0 = st.page_table.clone(), st.prefix_lens.clone()
         self.h_pt, self.h_pl, self.h_ql, self.h_nm = pin(st.page_table), pin(st.prefix_lens), pin(st.q_lens), pin(st.n_mask)
+        self.h_nb = pin(st.n_blocks) if st.n_blocks is not None else None
         self.h_acc, self.h_bon = pin(ds.acc), pin(ds.bon)
         self.h_freed, self.h_nfreed = pin(ds.freed), pin(ds.n_freed)
         nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
@@ -245,7 +251,7 @@ class HostStep:
         self.h_pt.copy_(self.pt0); self.h_pl.copy_(self.pl0)       # host-side reset of what the commit edited
         fd.fd_step_host(ds.ctx, st.batch, st.total_q_rows, st.total_cand_rows, ds.kv, st.num_pages, self.h_q, self.h_out,
                         self.h_logits, self.h_drafts, self.h_pt, self.h_pl, self.h_ql, self.h_nm, self.h_acc, self.h_bon,
-                        self.h_freed, self.h_nfreed)
+                        self.h_freed, self.h_nfreed, n_blocks_host=self.h_nb)
         ds.torch.cuda.current_stream().synchronize()               # the results are consumed on the host every step
 
 
@@ -299,6 +305,11 @@ def check_against_oracle(ds: DeviceStep, n_rows=6):
     g = torch.Generator().manual_seed(5)
     qc, kvc = ds.q[-1].cpu(), ds.kv[-1].cpu()
     outc = ds.out[-1].float().cpu().numpy()
+    if st.n_blocks is not None:     # several mask blocks: small enough for the full oracle
+        ref = oracle.attn_blocks(qc, kvc, st.page_table, st.prefix_lens, st.q_lens, st.n_mask, st.n_blocks)
+        ok_attn = bool((np.abs(outc - ref) <= 2e-2 + 2e-2 * np.abs(ref)).all())
+        e_acc, e_bon, _ = oracle.accept(ds.logits.cpu(), ds.drafts.cpu(), st.q_lens, st.n_mask)
+        return ok_attn and bool((ds.acc.cpu().numpy() == e_acc).all() and (ds.bon.cpu().numpy() == e_bon).all())
     cu = torch.cumsum(st.q_lens, 0) - st.q_lens
     worst = 0.0
     for _ in range(n_rows):
@@ -400,7 +411,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=4, help="0..4, see workload.WORKLOAD_NAMES")
+    ap.add_argument("--workload", type=int, default=4, help="0..5, see workload.WORKLOAD_NAMES")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count of workload 4")
     ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel")
     ap.add_argument("--ref-heads", type=int, default=8, help="q-heads in the oracle's timed sample")

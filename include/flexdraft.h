@@ -129,6 +129,42 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
                                void* out, void* stream);
 
 /*
+ * The same attention with several mask blocks per sequence: the parallel mode proper, in which the
+ * forward pass that verifies the current draft also prepares one next-draft branch per hypothesis r
+ * ("the first r drafts are accepted", Sec. 3 "Parallel speculative decoding", Eq. 2), each branch
+ * conditioned on the prefix and on those r drafts only.
+ *
+ *   n_blocks   device, [B] int32, or NULL (= fd_attn_draft_verify).  nb_b = n_blocks[b]; 0 and 1 mean one
+ *              block.  For nb_b > 1 the M_b mask rows are nb_b consecutive blocks of M_b / nb_b tokens
+ *              (M_b divisible by nb_b, nb_b <= C_b); block g is the branch of hypothesis
+ *              r = C_b - nb_b + g, so nb_b = C_b prepares every hypothesis r = 0..k_b.
+ *
+ *     A_b(i) for a mask row of block g:  { j < n_b } U { n_b + t : t <= r }  U  { its own block }
+ *
+ * (candidate row 0 is the known bonus token, candidate t the t-th draft); blocks never see each
+ * other; candidate rows are as in fd_attn_draft_verify.  All rows of a sequence still share one
+ * M = 128 tile per kv-head, so G * Lq_b <= 128 bounds the number and size of the branches.
+ * Lengths that break the rules above zero all T rows (FD_DEV_BAD_LENGTHS).
+ */
+fd_status fd_attn_draft_verify_blocks(fd_ctx* ctx, int batch, int total_q_rows,
+                                      const void* q, const void* kv_cache, int num_pages,
+                                      const int32_t* page_table, const int32_t* prefix_lens,
+                                      const int32_t* q_lens, const int32_t* n_mask,
+                                      const int32_t* n_blocks, void* out, void* stream);
+
+/*
+ * Branch selection (Sec. 3: once verification has fixed r_acc, the branch prepared under that
+ * hypothesis is the next draft).  mask_tokens holds one proposed token per mask row, sequence-major
+ * ([sum_b M_b] int32, device).  For each sequence the block g = accepted_len[b] - (C_b - nb_b) is copied to
+ * next_draft[b, 0:kb] (device, [B, max_block_len] int32, padded with -1) and next_len[b] = kb; when that
+ * hypothesis was not prepared (g outside [0, nb_b)), the sequence has no mask rows, or
+ * accepted_len[b] < 0, next_len[b] = 0.  A block longer than max_block_len raises FD_DEV_BAD_LENGTHS.
+ */
+fd_status fd_select_branch(fd_ctx* ctx, int batch, int max_block_len, const int32_t* mask_tokens,
+                           const int32_t* q_lens, const int32_t* n_mask, const int32_t* n_blocks,
+                           const int32_t* accepted_len, int32_t* next_draft, int32_t* next_len, void* stream);
+
+/*
  * Lossless verification at temperature 0 (Sec. 3: draft tokens are accepted up to the
  * first rejection, the token produced there is the bonus token, committed length
  * L_acc = r_acc + 1).  With am[r] = argmax_v logits[r, v] (larger value wins, equal
@@ -199,6 +235,7 @@ fd_status fd_kv_commit(fd_ctx* ctx, int batch, int32_t* page_table, int32_t* pre
  *   logits_host       [R, V] fp32                        draft_tokens_host [R] int32
  *   page_table_host   [B, max_pages_per_seq] int32, in/out (the commit's edits come back)
  *   prefix_lens_host  [B] int32, in/out                  q_lens_host, n_mask_host [B] int32
+ *   n_blocks_host     [B] int32 mask blocks per sequence (see fd_attn_draft_verify_blocks), or NULL
  *   accepted_len_host, bonus_token_host [B] int32, written
  *   freed_pages_host  capacity B * (ceil(max_q_len / P) + 1) int32, written; n_freed_host [1]
  *
@@ -212,6 +249,7 @@ fd_status fd_step_host(fd_ctx* ctx, int batch, int total_q_rows, int total_cand_
                        const float* logits_host, const int32_t* draft_tokens_host,
                        int32_t* page_table_host, int32_t* prefix_lens_host,
                        const int32_t* q_lens_host, const int32_t* n_mask_host,
+                       const int32_t* n_blocks_host,
                        int32_t* accepted_len_host, int32_t* bonus_token_host,
                        int32_t* freed_pages_host, int32_t* n_freed_host, void* stream);
 

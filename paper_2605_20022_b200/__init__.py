@@ -23,7 +23,7 @@ FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch"]
 
 
 class fd_config(ctypes.Structure):
@@ -62,7 +62,9 @@ def load() -> ctypes.CDLL:
         lib.fd_verify_accept_static.argtypes = [ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_host_reserve.argtypes = [vp, ci, ci]
         lib.fd_selftest_wait_timeout.argtypes = [vp, ci, vp]
-        lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 13
+        lib.fd_attn_draft_verify_blocks.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_select_branch.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 14
         lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         lib.fd_attn_path.argtypes = [vp]
         lib.fd_launch_count.argtypes = [vp]
@@ -124,6 +126,21 @@ def fd_attn_draft_verify(ctx, batch, total_q_rows, q, kv_cache, num_pages, page_
     return _check("fd_attn_draft_verify", code, raise_on_error)
 
 
+def fd_attn_draft_verify_blocks(ctx, batch, total_q_rows, q, kv_cache, num_pages, page_table, prefix_lens, q_lens, n_mask,
+                                n_blocks, out, stream=None, raise_on_error=True) -> int:
+    code = load().fd_attn_draft_verify_blocks(ctx, batch, total_q_rows, _ptr(q), _ptr(kv_cache), num_pages,
+                                              _ptr(page_table), _ptr(prefix_lens), _ptr(q_lens), _ptr(n_mask),
+                                              _ptr(n_blocks), _ptr(out), _stream(stream))
+    return _check("fd_attn_draft_verify_blocks", code, raise_on_error)
+
+
+def fd_select_branch(ctx, batch, max_block_len, mask_tokens, q_lens, n_mask, n_blocks, accepted_len, next_draft, next_len,
+                     stream=None, raise_on_error=True) -> int:
+    code = load().fd_select_branch(ctx, batch, max_block_len, _ptr(mask_tokens), _ptr(q_lens), _ptr(n_mask),
+                                   _ptr(n_blocks), _ptr(accepted_len), _ptr(next_draft), _ptr(next_len), _stream(stream))
+    return _check("fd_select_branch", code, raise_on_error)
+
+
 def fd_verify_accept(ctx, batch, total_cand_rows, logits, draft_tokens, q_lens, n_mask, accepted_len, bonus_token,
                      stream=None, raise_on_error=True) -> int:
     code = load().fd_verify_accept(ctx, batch, total_cand_rows, _ptr(logits), _ptr(draft_tokens), _ptr(q_lens),
@@ -154,14 +171,16 @@ def fd_host_reserve(ctx, max_total_q_rows, max_total_cand_rows) -> None:
 
 def fd_step_host(ctx, batch, total_q_rows, total_cand_rows, kv_caches, num_pages, q_host, out_host, logits_host,
                  draft_tokens_host, page_table_host, prefix_lens_host, q_lens_host, n_mask_host, accepted_len_host,
-                 bonus_token_host, freed_pages_host, n_freed_host, stream=None, raise_on_error=True) -> int:
+                 bonus_token_host, freed_pages_host, n_freed_host, stream=None, raise_on_error=True,
+                 n_blocks_host=None) -> int:
     """One whole step from host (CPU, ideally pinned) tensors; `kv_caches` is a list of device tensors, one per
     layer.  `q_host` / `out_host` are [n_layers, T, Hq, d] CPU tensors."""
     n_layers = len(kv_caches)
     arr = (ctypes.c_void_p * n_layers)(*[_ptr(t) for t in kv_caches])
     code = load().fd_step_host(ctx, batch, total_q_rows, total_cand_rows, n_layers, arr, num_pages, _ptr(q_host),
                                _ptr(out_host), _ptr(logits_host), _ptr(draft_tokens_host), _ptr(page_table_host),
-                               _ptr(prefix_lens_host), _ptr(q_lens_host), _ptr(n_mask_host), _ptr(accepted_len_host),
+                               _ptr(prefix_lens_host), _ptr(q_lens_host), _ptr(n_mask_host), _ptr(n_blocks_host),
+                               _ptr(accepted_len_host),
                                _ptr(bonus_token_host), _ptr(freed_pages_host), _ptr(n_freed_host), _stream(stream))
     return _check("fd_step_host", code, raise_on_error)
 

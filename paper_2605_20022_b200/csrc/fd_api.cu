@@ -33,7 +33,7 @@ struct HostStage {
     unsigned char* pool;
     void *q[2], *out[2];
     float* lg;
-    int32_t *drafts, *pt, *pl, *ql, *nm, *acc, *bon, *freed, *nfreed;
+    int32_t *drafts, *pt, *pl, *ql, *nm, *nb, *acc, *bon, *freed, *nfreed;
 };
 
 namespace {
@@ -162,7 +162,7 @@ fd_status fd_host_reserve(fd_ctx* c, int max_total_q_rows, int max_total_cand_ro
     const size_t o_lg = take((size_t)max_total_cand_rows * c->cfg.vocab * 4);
     const size_t o_dr = take((size_t)max_total_cand_rows * 4);
     const size_t o_pt = take((size_t)B * c->cfg.max_pages_per_seq * 4);
-    const size_t o_pl = take(B * 4), o_ql = take(B * 4), o_nm = take(B * 4), o_ac = take(B * 4), o_bo = take(B * 4);
+    const size_t o_pl = take(B * 4), o_ql = take(B * 4), o_nm = take(B * 4), o_nb = take(B * 4), o_ac = take(B * 4), o_bo = take(B * 4);
     const size_t n_fr = (size_t)B * ((c->cfg.max_q_len + 15) / 16 + 1);
     const size_t o_fr = take(n_fr * 4), o_nf = take(4);
     if (cudaMalloc(&h->pool, off) != cudaSuccess) { cudaGetLastError(); delete h; return FD_ERR_WORKSPACE; }
@@ -176,7 +176,8 @@ fd_status fd_host_reserve(fd_ctx* c, int max_total_q_rows, int max_total_cand_ro
     h->lg = reinterpret_cast<float*>(h->pool + o_lg);
     h->drafts = reinterpret_cast<int32_t*>(h->pool + o_dr); h->pt = reinterpret_cast<int32_t*>(h->pool + o_pt);
     h->pl = reinterpret_cast<int32_t*>(h->pool + o_pl); h->ql = reinterpret_cast<int32_t*>(h->pool + o_ql);
-    h->nm = reinterpret_cast<int32_t*>(h->pool + o_nm); h->acc = reinterpret_cast<int32_t*>(h->pool + o_ac);
+    h->nm = reinterpret_cast<int32_t*>(h->pool + o_nm); h->nb = reinterpret_cast<int32_t*>(h->pool + o_nb);
+    h->acc = reinterpret_cast<int32_t*>(h->pool + o_ac);
     h->bon = reinterpret_cast<int32_t*>(h->pool + o_bo); h->freed = reinterpret_cast<int32_t*>(h->pool + o_fr);
     h->nfreed = reinterpret_cast<int32_t*>(h->pool + o_nf);
     c->host = h;
@@ -187,7 +188,7 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
                        const void* const* kv_caches, int num_pages, const void* q_host, void* out_host,
                        const float* logits_host, const int32_t* draft_tokens_host, int32_t* page_table_host,
                        int32_t* prefix_lens_host, const int32_t* q_lens_host, const int32_t* n_mask_host,
-                       int32_t* accepted_len_host, int32_t* bonus_token_host, int32_t* freed_pages_host,
+                       const int32_t* n_blocks_host, int32_t* accepted_len_host, int32_t* bonus_token_host, int32_t* freed_pages_host,
                        int32_t* n_freed_host, void* stream) {
     if (!c || !c->host) return FD_ERR_INVALID_ARG;
     HostStage* h = c->host;
@@ -214,6 +215,7 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
     chk(cudaMemcpyAsync(h->pl, prefix_lens_host, lb, H2D, h->h2d));
     chk(cudaMemcpyAsync(h->ql, q_lens_host, lb, H2D, h->h2d));
     chk(cudaMemcpyAsync(h->nm, n_mask_host, lb, H2D, h->h2d));
+    if (n_blocks_host) chk(cudaMemcpyAsync(h->nb, n_blocks_host, lb, H2D, h->h2d));
     chk(cudaEventRecord(h->meta, h->h2d));
     chk(cudaStreamWaitEvent(s, h->meta, 0));
     fd_status st = FD_OK;
@@ -239,8 +241,8 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         }
         chk(cudaStreamWaitEvent(s, h->q_ready[b], 0));
         if (l >= 2) chk(cudaStreamWaitEvent(s, h->out_copied[b], 0));
-        st = fd_attn_draft_verify(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
-                                  h->out[b], s);
+        st = fd_attn_draft_verify_blocks(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
+                                         n_blocks_host ? h->nb : nullptr, h->out[b], s);
         chk(cudaEventRecord(h->attn_done[b], s));
         chk(cudaStreamWaitEvent(h->d2h, h->attn_done[b], 0));
         chk(cudaMemcpyAsync(static_cast<unsigned char*>(out_host) + (size_t)l * qb, h->out[b], qb, D2H, h->d2h));
@@ -278,6 +280,14 @@ int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
 fd_status fd_attn_draft_verify(fd_ctx* c, int batch, int total_q_rows, const void* q, const void* kv_cache,
                                int num_pages, const int32_t* page_table, const int32_t* prefix_lens,
                                const int32_t* q_lens, const int32_t* n_mask, void* out, void* stream) {
+    return fd_attn_draft_verify_blocks(c, batch, total_q_rows, q, kv_cache, num_pages, page_table, prefix_lens, q_lens,
+                                       n_mask, nullptr, out, stream);
+}
+
+fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, const void* q, const void* kv_cache,
+                                      int num_pages, const int32_t* page_table, const int32_t* prefix_lens,
+                                      const int32_t* q_lens, const int32_t* n_mask, const int32_t* n_blocks,
+                                      void* out, void* stream) {
     if (!c || batch < 0 || total_q_rows < 0 || num_pages < 0) return FD_ERR_INVALID_ARG;
     if (batch > c->cfg.max_batch || (long long)total_q_rows > (long long)batch * c->cfg.max_q_len)
         return FD_ERR_INVALID_ARG;
@@ -297,6 +307,7 @@ fd_status fd_attn_draft_verify(fd_ctx* c, int batch, int total_q_rows, const voi
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.kv = static_cast<const __nv_bfloat16*>(kv_cache);
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.n_mask = n_mask;
+    p.n_blocks = n_blocks;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
 
@@ -350,6 +361,21 @@ fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefi
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.accepted = accepted_len;
     p.freed = freed_pages; p.n_freed = n_freed; p.status = c->status;
     fd::launch_commit(p, s);
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_select_branch(fd_ctx* c, int batch, int max_block_len, const int32_t* mask_tokens, const int32_t* q_lens,
+                           const int32_t* n_mask, const int32_t* n_blocks, const int32_t* accepted_len,
+                           int32_t* next_draft, int32_t* next_len, void* stream) {
+    if (!c || batch < 0 || batch > c->cfg.max_batch || max_block_len < 1) return FD_ERR_INVALID_ARG;
+    if (batch == 0) return FD_OK;
+    if (!q_lens || !n_mask || !accepted_len || !next_draft || !next_len) return FD_ERR_INVALID_ARG;
+    fd::SelectParams p;
+    p.batch = batch; p.max_kb = max_block_len; p.mask_tokens = mask_tokens; p.q_lens = q_lens; p.n_mask = n_mask;
+    p.n_blocks = n_blocks; p.accepted = accepted_len; p.next_draft = next_draft; p.next_len = next_len;
+    p.status = c->status;
+    fd::launch_select_branch(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
         const int n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
         const int kv_len = n + Lq, rows = Lq * p.G, row0 = p.plan.cu_q[b];
         const int i = r / p.G, g = r % p.G;
-        const int limit = (r < rows) ? ((i < Lq - M) ? n + i + 1 : kv_len) : 0;
+        const RowMask rm = row_mask(i, n, Lq, M, p.n_blocks ? p.n_blocks[b] : 1, r < rows);
 
         __syncthreads();  // previous piece is done with qT
         if (r < rows) {
@@ -89,8 +89,14 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
                 }
                 __syncthreads();
                 if (r >= rows) continue;
-                const int nvis = min(min(16, kv_len - pos0), limit - pos0);  // keys of this page the row sees
-                if (nvis <= 0) continue;
+                // keys of this page the row may see (bit k = token k); none -> nothing to do for this row
+                unsigned vis = 0;
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const int j = pos0 + k;
+                    if (j < kv_len && (j < rm.limit || (j >= rm.blk_lo && j < rm.blk_hi))) vis |= 1u << k;
+                }
+                if (vis == 0) continue;
                 float s[16];
 #pragma unroll
                 for (int k = 0; k < 16; ++k) s[k] = 0.f;
@@ -105,7 +111,7 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
                 float pm = -INFINITY;
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    s[k] = (k < nvis) ? s[k] : -INFINITY;  // a select, never a multiply: hidden slots may hold NaN
+                    s[k] = ((vis >> k) & 1u) ? s[k] : -INFINITY;  // a select, never a multiply: hidden slots may hold NaN
                     pm = fmaxf(pm, s[k]);
                 }
                 const float m_new = fmaxf(m, pm);
@@ -115,7 +121,8 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
                 for (int c = 0; c < D; ++c) acc[c] *= alpha;
                 m = m_new;
 #pragma unroll 1
-                for (int k = 0; k < nvis; ++k) {
+                for (int k = 0; k < 16; ++k) {
+                    if (!((vis >> k) & 1u)) continue;
                     const float pj = exp2f(s[k] - m);
                     l += pj;
 #pragma unroll

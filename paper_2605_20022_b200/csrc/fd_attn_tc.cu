@@ -74,7 +74,7 @@ struct Bars {
 };
 
 struct Piece {
-    int b, kvh, tile0, nt, n, Lq, M, kv_len, rows, row0, slot;
+    int b, kvh, tile0, nt, n, Lq, M, nb, kv_len, rows, row0, slot;
     bool complete;
 };
 
@@ -95,6 +95,7 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_
     pc.n = p.prefix_lens[lo];
     pc.Lq = p.q_lens[lo];
     pc.M = p.n_mask[lo];
+    pc.nb = p.n_blocks ? p.n_blocks[lo] : 1;
     pc.kv_len = pc.n + pc.Lq;
     pc.rows = pc.Lq * p.G;
     pc.row0 = p.plan.cu_q[lo];
@@ -344,7 +345,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         if (tid == 0) TRACE(5, 2, w.piece);
         const bool warp_active = (warp & 3) * 32 < pc.rows;
         const int i = r / p.G;
-        const int limit = (r < pc.rows) ? ((i < pc.Lq - pc.M) ? pc.n + i + 1 : pc.kv_len) : 0;
+        const RowMask rm = row_mask(i, pc.n, pc.Lq, pc.M, pc.nb, r < pc.rows);
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         // Warps whose 32 rows are all padding do nothing per tile: warp 0 of the group (always active)
@@ -358,9 +359,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 0, w.g0 + j);
             {
                 const int pos0 = (pc.tile0 + j) * kTileTokens;
-                // tile reaches into the query block (or past kv_len): columns >= lim are invisible
+                // tile reaches into the query block (or past kv_len): the row's mask applies, in tile-local columns
                 const bool masked = pos0 + kTileTokens > pc.n;
-                const int lim = limit - pos0;
+                const int lim = rm.limit - pos0, blo = rm.blk_lo - pos0, bhi = rm.blk_hi - pos0;
                 const uint32_t s_addr = tmem + lane_base + col_s[s];
 
                 // ---- the whole row of S in one round trip: TMEM loads queue behind the MMAs in flight,
@@ -374,7 +375,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     for (int ch = 0; ch < 4; ++ch)
 #pragma unroll
                         for (int k = 0; k < 32; ++k)
-                            if (ch * 32 + k >= lim) sv[ch][k] = 0xff800000u;  // -inf by select: S may be NaN there
+                            if (ch * 32 + k >= lim && (ch * 32 + k < blo || ch * 32 + k >= bhi)) sv[ch][k] = 0xff800000u;  // -inf by select: S may be NaN there
                 }
                 float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll

@@ -50,12 +50,35 @@ struct AttnParams {
     const int32_t* prefix_lens;
     const int32_t* q_lens;
     const int32_t* n_mask;
+    const int32_t* n_blocks;  // [B] mask blocks per sequence, or nullptr (= one block each)
     __nv_bfloat16* out;
     Plan plan;
     PartialView part;
     int n_ctas;       // CTAs of the attention grid (stream-K ranges are cut for this many)
     int* status;
 };
+
+// Hybrid mask of one query row, never materialised: key position j is visible iff
+//     j < limit  ||  (blk_lo <= j && j < blk_hi).
+// Candidate row i: causal (limit = n + i + 1, no block).  Mask row of block g (of nb blocks of M / nb
+// tokens): the branch prepared under the hypothesis "r = C - nb + g drafts accepted" sees the prefix and
+// the candidates 0..r (limit = n + r + 1) and its own block in both directions; with nb = 1 that is
+// every key of the sequence.  Rows that do not exist see nothing.
+struct RowMask {
+    int limit, blk_lo, blk_hi;
+};
+__host__ __device__ inline RowMask row_mask(int i, int n, int Lq, int M, int nb, bool exists) {
+    RowMask rm = {0, 0, 0};
+    if (!exists) return rm;
+    const int C = Lq - M;
+    if (i < C) { rm.limit = n + i + 1; return rm; }
+    if (nb < 1) nb = 1;
+    const int kb = M / nb, g = (i - C) / kb;
+    rm.limit = n + (C - nb + g) + 1;
+    rm.blk_lo = n + C + g * kb;
+    rm.blk_hi = rm.blk_lo + kb;
+    return rm;
+}
 
 // First tile of CTA c when `total` tiles are cut into `n` contiguous ranges.
 __host__ __device__ inline int range_begin(int c, int total, int n) {
@@ -154,6 +177,19 @@ struct AcceptParams {
     int* status;
 };
 void launch_accept(const AcceptParams& p, cudaStream_t s);
+
+struct SelectParams {
+    int batch, max_kb;
+    const int32_t* mask_tokens;
+    const int32_t* q_lens;
+    const int32_t* n_mask;
+    const int32_t* n_blocks;  // may be nullptr
+    const int32_t* accepted;
+    int32_t* next_draft;
+    int32_t* next_len;
+    int* status;
+};
+void launch_select_branch(const SelectParams& p, cudaStream_t s);
 
 struct CommitParams {
     int batch, max_pages, page_size;

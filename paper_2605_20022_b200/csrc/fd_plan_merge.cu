@@ -52,8 +52,11 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
         int q = 0, t = 0;
         if (b < B) {
             const long long n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
-            const bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || Lq * p.G > kMaxRows ||
-                             n + Lq > (long long)p.max_pages * P;
+            const long long nb = p.n_blocks ? p.n_blocks[b] : 1;
+            bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || Lq * p.G > kMaxRows ||
+                       n + Lq > (long long)p.max_pages * P;
+            // several mask blocks: equal sizes, and one hypothesis (a candidate row) per block
+            bad = bad || nb < 0 || (nb > 1 && (M % nb != 0 || nb > Lq - M));
             if (bad) atomicOr(&s_fatal, 1);
             else { q = (int)Lq; t = Lq > 0 ? (int)((n + Lq + kTileTokens - 1) / kTileTokens) : 0; }
             p.plan.seq_ok[b] = 1;

@@ -55,6 +55,7 @@ WORKLOAD_NAMES = [
     "qwen3_8b_b8_parallel_ragged",
     "qwen3_8b_b64_sequential_ragged",
     "qwen3_8b_b16_prefix32768_36layers",
+    "qwen3_8b_b8_all_hypotheses_c4_4x7",
 ]
 
 
@@ -71,6 +72,7 @@ class Step:
     page_table: torch.Tensor          # [B, max_pages_per_seq], -1 = unallocated
     num_pages: int
     spare_pages: torch.Tensor = field(default=None)  # physical ids owned by no sequence
+    n_blocks: Optional[torch.Tensor] = None          # [B] mask blocks per sequence (None = one block each)
 
     @property
     def batch(self) -> int:
@@ -165,6 +167,14 @@ def workload(idx: int, n_layers: Optional[int] = None) -> Step:
         B = 16
         shape = Shape(32, 8, 128, 151936, 36 if n_layers is None else n_layers)
         return make_step(WORKLOAD_NAMES[4], shape, [32768] * B, [32] * B, [16] * B, seed, 0.8)
+    if idx == 5:
+        # beyond the five benchmark configurations: the all-hypotheses form of parallel drafting at the size one
+        # M = 128 tile allows: bonus + 3 drafts, and one 7-token next-draft branch per hypothesis r = 0..3
+        B = 8
+        n = _randint(g, 512, 8192, B)
+        st = make_step(WORKLOAD_NAMES[5], QWEN3_8B, n.tolist(), [32] * B, [28] * B, seed, 0.8)
+        st.n_blocks = torch.full((B,), 4, dtype=torch.int32)
+        return st
     raise ValueError(f"no workload {idx}")
 
 

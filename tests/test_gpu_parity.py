@@ -294,3 +294,61 @@ def test_bounded_wait_times_out_cleanly_and_context_survives():
         got, status = gpu_attn(ctx, step, q, kv)
         assert status == 0
         assert_close(got.numpy(), oracle_attn(step, q, kv), "after timeout")
+
+
+BLOCK_CASES = {
+    # name: (Hq, Hkv, d, prefix_lens, C, M, n_blocks)
+    "all_hypotheses": (32, 8, 128, [700, 130, 2049, 0, 5], [4, 8, 2, 4, 16], [28, 24, 30, 28, 16], [4, 8, 2, 4, 16]),
+    "pruned_and_single": (32, 8, 128, [1000, 77, 300, 4000], [8, 6, 5, 16], [24, 12, 6, 0], [3, 1, 0, 0]),
+    "block_straddles_tiles": (8, 2, 128, [120, 250, 383], [4, 4, 4], [28, 28, 28], [4, 2, 4]),
+    "head_dim64": (16, 4, 64, [90, 513], [4, 8], [12, 24], [4, 8]),
+}
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name", sorted(BLOCK_CASES))
+def test_attention_mask_blocks(name, path):
+    """Several next-draft branches per sequence (one mask block per hypothesis) against the oracle."""
+    Hq, Hkv, d, pl, C, M, nb = BLOCK_CASES[name]
+    step = wl.make_step(name, wl.Shape(Hq, Hkv, d, 1000), pl, [c + m for c, m in zip(C, M)], M,
+                        seed=zlib.crc32(name.encode()) % 10000)
+    q, kv = wl.make_q(step), wl.make_kv(step, poison=float("nan"))
+    n_blocks = torch.tensor(nb, dtype=torch.int32)
+    ref = oracle.attn_blocks(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, n_blocks)
+    with Ctx(step, path) as ctx:
+        dq, dkv = q.cuda(), kv.cuda()
+        out = torch.full_like(dq, float("nan"))
+        fd.fd_attn_draft_verify_blocks(ctx.h, step.batch, step.total_q_rows, dq, dkv, step.num_pages, step.page_table.cuda(),
+                                       step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda(), n_blocks.cuda(), out)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        assert_close(out.float().cpu().numpy(), ref, name)
+        # broken block structure: not divisible / more blocks than hypotheses -> zeros and a status bit
+        for bad in ([3 if m % 3 else 5 for m in M], [c + 1 for c in C]):
+            if all(b_ <= 1 or (m % b_ == 0 and b_ <= c) for b_, m, c in zip(bad, M, C)):
+                continue
+            out.fill_(float("nan"))
+            fd.fd_attn_draft_verify_blocks(ctx.h, step.batch, step.total_q_rows, dq, dkv, step.num_pages, step.page_table.cuda(),
+                                           step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda(),
+                                           torch.tensor(bad, dtype=torch.int32).cuda(), out)
+            assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS and (out == 0).all()
+
+
+def test_select_branch_matches_oracle():
+    g = torch.Generator().manual_seed(4)
+    B = 97
+    C = torch.randint(1, 9, (B,), generator=g)
+    nb = torch.tensor([int(torch.randint(0, int(c) + 1, (1,), generator=g)) for c in C])
+    kb = torch.randint(1, 5, (B,), generator=g)
+    M = torch.where(torch.rand(B, generator=g) < 0.15, torch.zeros_like(kb), kb * nb.clamp(min=1))
+    step = wl.make_step("sel", wl.Shape(32, 8, 128, 1000), [3] * B, (C + M).tolist(), M.tolist(), seed=4)
+    tokens = torch.randint(0, 1000, (int(M.sum()),), generator=g, dtype=torch.int32)
+    acc = torch.tensor([int(torch.randint(-1, int(c), (1,), generator=g)) for c in C], dtype=torch.int32)
+    exp_nd, exp_nl = oracle.select_branch(tokens, step.q_lens, step.n_mask, nb.int(), acc, max_kb=5)
+    with Ctx(step) as ctx:
+        nd = torch.full((B, 5), -9, dtype=torch.int32, device="cuda"); nl = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+        fd.fd_select_branch(ctx.h, B, 5, tokens.cuda(), step.q_lens.cuda(), step.n_mask.cuda(), nb.int().cuda(), acc.cuda(), nd, nl)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        np.testing.assert_array_equal(nd.cpu().numpy(), exp_nd); np.testing.assert_array_equal(nl.cpu().numpy(), exp_nl)
+        fd.fd_select_branch(ctx.h, B, 2, tokens.cuda(), step.q_lens.cuda(), step.n_mask.cuda(), nb.int().cuda(), acc.cuda(),
+                            nd[:, :2].contiguous(), nl)                       # blocks longer than the output rows
+        assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS

@@ -34,6 +34,9 @@ def test_lengths_of_the_five_workloads():
         assert s.shape.page_size == 16
     for s in (s1, s2, s3, s4):
         assert (s.shape.n_q_heads, s.shape.n_kv_heads, s.shape.head_dim, s.shape.vocab) == (32, 8, 128, 151936)
+    s5 = wl.workload(5)
+    assert s5.batch == 8 and (s5.n_blocks == 4).all() and (s5.cand_rows == 4).all() and (s5.n_mask == 28).all()
+    check_tables(s5)
     # same seed -> same lengths
     assert torch.equal(wl.workload(2).prefix_lens, s2.prefix_lens)
 
