@@ -11,6 +11,7 @@ attn(...)        full attention under the hybrid mask (Sec. 4.1), float64 output
 attn_row(...)    one output row of the same definition (sampled checks)
 attn_blocks(...) the same with several mask blocks per sequence (all hypotheses, Eq. 2)
 select_branch(...) pick the prepared next-draft branch of the accepted length
+draft_select(...) draft-side tail: calibrated argmax, confidence, Eq. 5 verify length
 accept(...)      greedy verification: argmax, accepted length, bonus token (Sec. 3)
 commit(...)      KV commit / rollback by page-table truncation
 """
@@ -140,6 +141,22 @@ def accept(logits, draft_tokens, q_lens, n_mask):
     am = np.zeros((max(R, 1),), np.int32)
     _load().fdo_accept(ctypes.c_int(B), ctypes.c_int(V), _p(lg), _p(dt), _p(ql), _p(nm), _p(acc), _p(bon), _p(am))
     return acc, bon, am[:R]
+
+
+def draft_select(logits, bias, n_mask, n_blocks, threshold, max_blocks):
+    """Draft-side tail (Eq. 4 + Eq. 5): returns (tokens [Rm] i32, probs [Rm] f64, cum [Rm] f64, keep_len [B, max_blocks] i32)."""
+    lg = np.ascontiguousarray(logits if isinstance(logits, np.ndarray) else logits.cpu().numpy(), dtype=np.float32)
+    bs = None if bias is None else np.ascontiguousarray(bias if isinstance(bias, np.ndarray) else bias.cpu().numpy(), dtype=np.float32)
+    Rm, V = lg.shape
+    nm = _i32(n_mask)
+    nb = None if n_blocks is None else _i32(n_blocks)
+    B = nm.shape[0]
+    assert int(np.maximum(nm, 0).sum()) == Rm
+    tok = np.zeros((max(Rm, 1),), np.int32); pr = np.zeros((max(Rm, 1),), np.float64); cum = np.zeros((max(Rm, 1),), np.float64)
+    keep = np.zeros((B, max_blocks), np.int32)
+    _load().fdo_draft_select(ctypes.c_int(B), ctypes.c_int(V), ctypes.c_int(max_blocks), _p(lg), None if bs is None else _p(bs), _p(nm),
+                             None if nb is None else _p(nb), ctypes.c_double(threshold), _p(tok), _p(pr), _p(cum), _p(keep))
+    return tok[:Rm], pr[:Rm], cum[:Rm], keep
 
 
 def commit(page_table, prefix_lens, q_lens, accepted_len, page_size=16):

@@ -265,6 +265,60 @@ void fdo_accept(int B, int V, const float *logits, const int32_t *draft_tokens,
     }
 }
 
+/* Draft-side tail of the step (Sec. 4.2, Eq. 4; Sec. 4.3 "Selective verification", Eq. 5).  One row of
+ * draft logits per mask token, sequence-major.  With the calibration bias already evaluated by the caller
+ * (the two-layer MLP of Eq. 4 needs trained weights), the calibrated logits are l~ = l + bias, the drafted
+ * token of a row is argmax l~ (lowest index on ties) and its confidence p = softmax(l~)[token].  Within each
+ * next-draft block (the M_b mask rows of a sequence are nb_b equal blocks) the cumulative confidence of
+ * position i is the product of p over positions 1..i (Eq. 5: the estimate of P(L_acc >= i)); keep_len of
+ * the block is the number of leading positions whose cumulative confidence is still >= threshold, i.e. how
+ * many of its drafts are worth verifying in the next step.
+ *
+ * The sum l + bias is formed in float32, as the kernel forms it, so that the argmax is decided on the same
+ * numbers; everything after that is float64.  tokens [Rm], probs [Rm], cum [Rm], keep_len [B, max_blocks]
+ * (zero where a sequence has fewer blocks). */
+void fdo_draft_select(int B, int V, int max_blocks, const float *logits, const float *bias, const int32_t *n_mask,
+        const int32_t *n_blocks, double threshold, int32_t *tokens, double *probs, double *cum, int32_t *keep_len)
+{
+    int64_t r0 = 0;
+    for (int b = 0; b < B; ++b) {
+        const int M = n_mask[b];
+        int nb = n_blocks ? n_blocks[b] : 1;
+        if (nb < 1) nb = 1;
+        for (int g = 0; g < max_blocks; ++g) keep_len[(int64_t)b * max_blocks + g] = 0;
+        if (M <= 0) continue;
+        const int kb = M / nb;
+        for (int u = 0; u < M; ++u) {
+            const float *lr = logits + (r0 + u) * (int64_t)V;
+            const float *br = bias ? bias + (r0 + u) * (int64_t)V : NULL;
+            int best = 0;
+            float bestv = br ? lr[0] + br[0] : lr[0];
+            for (int v = 1; v < V; ++v) {
+                const float x = br ? lr[v] + br[v] : lr[v];
+                if (x > bestv) { bestv = x; best = v; }
+            }
+            double den = 0.0;
+            for (int v = 0; v < V; ++v) {
+                const float x = br ? lr[v] + br[v] : lr[v];
+                den += exp((double)x - (double)bestv);
+            }
+            tokens[r0 + u] = best;
+            probs[r0 + u] = 1.0 / den;
+        }
+        for (int g = 0; g < nb; ++g) {
+            double c = 1.0;
+            int keep = 0, open = 1;
+            for (int u = 0; u < kb; ++u) {
+                c *= probs[r0 + (int64_t)g * kb + u];
+                cum[r0 + (int64_t)g * kb + u] = c;
+                if (open && c >= threshold) ++keep; else open = 0;
+            }
+            if (g < max_blocks) keep_len[(int64_t)b * max_blocks + g] = keep;
+        }
+        r0 += M;
+    }
+}
+
 /* KV commit / rollback.  In place on page_table [B, max_pages] and prefix_lens [B].
  * Sequences with accepted_len < 0 are left unchanged.  freed_pages is packed in
  * (sequence ascending, logical page ascending) order; returns the number freed. */

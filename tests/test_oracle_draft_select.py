@@ -1,0 +1,79 @@
+"""Pins for the oracle's draft-side tail: calibrated argmax and confidence (Eq. 4), cumulative confidence
+and verify length (Eq. 5)."""
+import numpy as np
+import torch
+
+import oracle
+
+
+def make(B=5, V=300, seed=0, M=(12, 0, 8, 6, 16), nb=(3, 1, 2, 0, 4)):
+    g = torch.Generator().manual_seed(seed)
+    Rm = sum(M)
+    logits = torch.randn((Rm, V), generator=g) * 3
+    bias = torch.randn((Rm, V), generator=g)
+    return logits, bias, np.array(M, np.int32), np.array(nb, np.int32)
+
+
+def test_tokens_and_confidence_against_library_softmax():
+    logits, bias, M, nb = make()
+    tok, pr, cum, keep = oracle.draft_select(logits, bias, M, nb, 0.3, max_blocks=4)
+    x = (logits + bias).float()                                  # float32 sum, as the definition states
+    np.testing.assert_array_equal(tok, x.argmax(dim=1).numpy())
+    ref = torch.softmax(x.double(), dim=1)[torch.arange(x.shape[0]), torch.from_numpy(tok).long()]
+    np.testing.assert_allclose(pr, ref.numpy(), rtol=1e-12)
+    # without a bias the logits themselves decide
+    tok0, pr0, _, _ = oracle.draft_select(logits, None, M, nb, 0.3, max_blocks=4)
+    np.testing.assert_array_equal(tok0, logits.argmax(dim=1).numpy())
+    assert (tok0 != tok).any()                                   # the calibration changes some drafts
+
+
+def test_cumulative_confidence_and_keep_len_against_numpy():
+    logits, bias, M, nb = make(seed=1)
+    for thr in (0.9, 0.2, 1e-3, 0.0, 1.5):
+        tok, pr, cum, keep = oracle.draft_select(logits, bias, M, nb, thr, max_blocks=4)
+        r0 = 0
+        for b in range(len(M)):
+            n_b = max(int(nb[b]), 1)
+            kb = int(M[b]) // n_b if M[b] else 0
+            for g in range(4):
+                if M[b] == 0 or g >= n_b:
+                    assert keep[b, g] == 0
+                    continue
+                p = pr[r0 + g * kb:r0 + (g + 1) * kb]
+                c = np.cumprod(p)
+                np.testing.assert_allclose(cum[r0 + g * kb:r0 + (g + 1) * kb], c, rtol=1e-13)
+                ok = c >= thr
+                assert keep[b, g] == (int(np.argmin(ok)) if not ok.all() else kb)      # leading run only
+            r0 += int(M[b])
+        if thr == 0.0:
+            assert all(keep[b, g] == (M[b] // max(nb[b], 1)) for b in range(len(M)) for g in range(max(nb[b], 1)) if M[b])
+        if thr == 1.5:
+            assert (keep == 0).all()
+
+
+def test_constant_confidence_closed_form():
+    """Every position equally confident with probability p: keep_len = floor(log(thr) / log(p)), capped by the block."""
+    V, kb = 64, 10
+    for peak in (1.0, 3.0, 5.0):
+        logits = torch.zeros((kb, V)); logits[:, 7] = peak
+        p = np.exp(peak) / (np.exp(peak) + V - 1)
+        for thr in (0.5, 0.1, 0.01):
+            tok, pr, cum, keep = oracle.draft_select(logits, None, np.array([kb], np.int32), None, thr, max_blocks=1)
+            np.testing.assert_allclose(pr, p, rtol=1e-12)
+            expect = min(kb, int(np.floor(np.log(thr) / np.log(p) + 1e-12)))
+            assert (tok == 7).all() and keep[0, 0] == expect
+
+
+def test_cumulative_confidence_is_the_independence_estimate_of_eq5():
+    """Eq. 5: if each drafted token is accepted independently with probability p_i, the probability that the
+    accepted length reaches i is the cumulative product the oracle reports."""
+    logits, bias, M, nb = make(B=1, V=40, seed=3, M=(8,), nb=(1,))
+    logits = logits * 0.5 + 2.5 * torch.nn.functional.one_hot(torch.arange(8) * 3, 40)   # confident but not certain drafts
+    tok, pr, cum, keep = oracle.draft_select(logits, None, M, nb, 0.05, max_blocks=1)
+    rng = np.random.default_rng(0)
+    trials = 200000
+    acc = rng.random((trials, 8)) < pr[None, :]
+    run = np.cumprod(acc, axis=1).sum(axis=1)                      # accepted length of each trial
+    for i in range(1, 9):
+        est = (run >= i).mean()
+        assert abs(est - cum[i - 1]) < 4.5 * np.sqrt(cum[i - 1] * (1 - cum[i - 1]) / trials) + 1e-4
