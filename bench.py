@@ -362,6 +362,26 @@ def run_ours(args, step, rank, world, dist):
         ms_graph = timed_region(torch, dist, graph.replay, args.steps, flush)
         del graph
 
+    # rows beyond the step's own: the draft-side tail (calibrated argmax + confidence + Eq. 5 verify length) over the
+    # mask rows of this workload, timed on its own with L2 flushed between calls; parity is covered by the tests
+    draft_tail = None
+    Rm = int(step.n_mask.sum())
+    if Rm > 0 and rank == 0:
+        gl = torch.Generator(device=device).manual_seed(step.seed + 400_000)
+        dl = torch.randn((Rm, step.shape.vocab), generator=gl, device=device)
+        db = torch.randn((Rm, step.shape.vocab), generator=gl, device=device)
+        tok = torch.empty((Rm,), dtype=torch.int32, device=device); pr = torch.empty((Rm,), device=device)
+        keep = torch.empty((step.batch, 32), dtype=torch.int32, device=device)
+        fl = flush if flush is not None else torch.empty((512 << 20,), dtype=torch.uint8, device=device)
+        call = lambda: fd.fd_draft_select(ds.ctx, step.batch, Rm, 32, dl, db, ds.nm, ds.nb, 0.3, tok, pr, keep)
+        for _ in range(3):
+            call()
+        ms_dt = timed_region(torch, None, call, 10, fl) / 10
+        nbytes = 2 * Rm * step.shape.vocab * 4
+        draft_tail = {"us": ms_dt * 1e3, "rows": Rm, "algorithmic_bytes": nbytes, "GB/s": nbytes / ms_dt / 1e6,
+                      "frac_of_measured_peak": nbytes / ms_dt / 1e6 / peak}
+        del dl, db, fl
+
     hs = HostStep(ds)
     for _ in range(2):
         hs.run()
@@ -391,7 +411,7 @@ def run_ours(args, step, rank, world, dist):
                    "l2": "flushed between steps (512 MB write)" if small else "inputs larger than L2 (distinct KV pool per layer)",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU",
                    "parity_vs_oracle_sampled": parity_ok, "device_status": status,
-                   "us_per_step_cuda_graph_replay": us_graph},
+                   "us_per_step_cuda_graph_replay": us_graph, "draft_tail_fd_draft_select": draft_tail},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(step.name) if resolved == "tcgen05" else None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
                      "kernel": "fd_attn_draft_verify (plan launch + split-KV attention launch, merge fused)",

@@ -153,6 +153,33 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* ctx, int batch, int total_q_rows,
                                       const int32_t* n_blocks, void* out, void* stream);
 
 /*
+ * Draft-side tail of the step (Sec. 4.2, Eq. 4; Sec. 4.3 "Selective verification", Eq. 5).  One row of
+ * draft logits per mask token, sequence-major.  Calibrated logits l~ = l + bias (the bias is the output of
+ * the calibration MLP of Eq. 4, evaluated by the caller; NULL = no calibration); the drafted token of a
+ * row is argmax l~ (lowest index on ties, inputs NaN-free), its confidence p = softmax(l~)[token].  Within
+ * every next-draft block (nb_b equal blocks per sequence, as in fd_attn_draft_verify_blocks) the cumulative
+ * confidence of position i is prod_{r <= i} p_r -- Eq. 5's estimate of P(L_acc >= i) -- and keep_len of the
+ * block is the number of leading positions where it is still >= threshold: how many of that branch's
+ * drafts the next step should verify (its candidate rows are then 1 + keep_len).
+ *
+ *   total_mask_rows  Rm; must equal sum_b n_mask[b]
+ *   max_blocks       row length of keep_len; every nb_b must be <= max_blocks
+ *   draft_logits     device, [Rm, V] fp32            bias   device, [Rm, V] fp32, or NULL
+ *   n_mask, n_blocks device, [B] int32 (n_blocks may be NULL)
+ *   threshold        >= 0
+ *   mask_tokens      device, [Rm] int32, written     mask_probs   device, [Rm] fp32, written
+ *   keep_len         device, [B, max_blocks] int32, written (0 where a sequence has fewer blocks)
+ *
+ * Arithmetic: l + bias, the maxima and the confidences in fp32 (the sum of exponentials is accumulated in a
+ * fixed order, so results are run-to-run identical).  Inconsistent lengths: tokens -1, confidences 0,
+ * keep_len 0, FD_DEV_BAD_LENGTHS.
+ */
+fd_status fd_draft_select(fd_ctx* ctx, int batch, int total_mask_rows, int max_blocks,
+                          const float* draft_logits, const float* bias,
+                          const int32_t* n_mask, const int32_t* n_blocks, float threshold,
+                          int32_t* mask_tokens, float* mask_probs, int32_t* keep_len, void* stream);
+
+/*
  * Branch selection (Sec. 3: once verification has fixed r_acc, the branch prepared under that
  * hypothesis is the next draft).  mask_tokens holds one proposed token per mask row, sequence-major
  * ([sum_b M_b] int32, device).  For each sequence the block g = accepted_len[b] - (C_b - nb_b) is copied to

@@ -12,17 +12,6 @@ namespace fd {
 
 constexpr int kVecPerThread = kAcceptChunk / (4 * 256);  // float4 loads in flight per thread
 
-__device__ inline unsigned long long make_key(float v, unsigned idx) {
-    v += 0.0f;  // -0.0 -> +0.0: they compare equal, so the lower index must decide
-    unsigned u = __float_as_uint(v);
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-    return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - idx);
-}
-
-__device__ inline void fold(float& bv, unsigned& bi, float v, unsigned i) {
-    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
-}
-
 __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_per_row) {
     const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
     const float* base = p.logits + (long long)row * p.vocab;

@@ -18,6 +18,10 @@ struct fd_ctx {
     fd::PartialView part;
     unsigned long long* keys;
     unsigned int* ticket;
+    unsigned long long* ds_key;  // draft-select chunk partials [max_rows][chunks]
+    float* ds_sum;
+    unsigned int* ds_ticket;
+    unsigned int* ds_row_ticket;
     int* status;
     int max_rows;      // capacity of keys
     void* tc_state;
@@ -110,6 +114,11 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const size_t o_pl = take(slots * fd::kMaxRows * sizeof(float));
     const size_t o_keys = take((size_t)c->max_rows * sizeof(unsigned long long));
     const size_t o_tick = take(sizeof(unsigned int));
+    const size_t ds_chunks = (size_t)(cfg->vocab + fd::kAcceptChunk - 1) / fd::kAcceptChunk;
+    const size_t o_dsk = take((size_t)c->max_rows * ds_chunks * sizeof(unsigned long long));
+    const size_t o_dss = take((size_t)c->max_rows * ds_chunks * sizeof(float));
+    const size_t o_dst = take(sizeof(unsigned int));
+    const size_t o_dsr = take((size_t)c->max_rows * sizeof(unsigned int));
     const size_t o_stat = take(sizeof(int));
     if (cudaMalloc(&c->pool, off) != cudaSuccess) { cudaGetLastError(); delete c; return FD_ERR_WORKSPACE; }
     if (cudaMemset(c->pool, 0, off) != cudaSuccess) { cudaFree(c->pool); delete c; return FD_ERR_CUDA; }
@@ -124,6 +133,10 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->part.l = reinterpret_cast<float*>(c->pool + o_pl);
     c->keys = reinterpret_cast<unsigned long long*>(c->pool + o_keys);
     c->ticket = reinterpret_cast<unsigned int*>(c->pool + o_tick);
+    c->ds_key = reinterpret_cast<unsigned long long*>(c->pool + o_dsk);
+    c->ds_sum = reinterpret_cast<float*>(c->pool + o_dss);
+    c->ds_ticket = reinterpret_cast<unsigned int*>(c->pool + o_dst);
+    c->ds_row_ticket = reinterpret_cast<unsigned int*>(c->pool + o_dsr);
     c->status = reinterpret_cast<int*>(c->pool + o_stat);
     *out = c;
     return FD_OK;
@@ -361,6 +374,26 @@ fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefi
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.accepted = accepted_len;
     p.freed = freed_pages; p.n_freed = n_freed; p.status = c->status;
     fd::launch_commit(p, s);
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blocks, const float* draft_logits,
+                          const float* bias, const int32_t* n_mask, const int32_t* n_blocks, float threshold,
+                          int32_t* mask_tokens, float* mask_probs, int32_t* keep_len, void* stream) {
+    if (!c || batch < 0 || batch > c->cfg.max_batch || total_mask_rows < 0 || total_mask_rows > c->max_rows || max_blocks < 1)
+        return FD_ERR_INVALID_ARG;
+    if (batch == 0) return total_mask_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
+    if (!n_mask || !keep_len || !(threshold >= 0.f)) return FD_ERR_INVALID_ARG;
+    if (total_mask_rows > 0 && (!draft_logits || !mask_tokens || !mask_probs)) return FD_ERR_INVALID_ARG;
+    const long long ctas = (long long)total_mask_rows * ((c->cfg.vocab + fd::kAcceptChunk - 1) / fd::kAcceptChunk);
+    if (ctas > 0x7fffffffLL) return FD_ERR_UNSUPPORTED;
+    fd::DraftSelectParams p;
+    p.batch = batch; p.total_rows = total_mask_rows; p.vocab = c->cfg.vocab; p.max_blocks = max_blocks;
+    p.logits = draft_logits; p.bias = bias; p.n_mask = n_mask; p.n_blocks = n_blocks; p.threshold = threshold;
+    p.tokens = mask_tokens; p.probs = mask_probs; p.keep_len = keep_len;
+    p.part_key = c->ds_key; p.part_sum = c->ds_sum; p.ticket = c->ds_ticket; p.row_ticket = c->ds_row_ticket; p.status = c->status;
+    fd::launch_draft_select(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }

@@ -164,6 +164,42 @@ void attn_tc_free(void* state);
 void launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);
 void launch_merge(const AttnParams& p, cudaStream_t s);
 
+// (value, index) of a running argmax as one 64-bit key: order-preserving image of the float in the high
+// word, inverted index in the low word, so an unsigned max picks the larger value and, on equal values,
+// the lower index.  A key of 0 means "nothing seen".
+__device__ inline unsigned long long make_key(float v, unsigned idx) {
+    v += 0.0f;  // -0.0 -> +0.0: they compare equal, so the lower index must decide
+    unsigned u = __float_as_uint(v);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - idx);
+}
+__device__ inline float key_value(unsigned long long key) {
+    const unsigned u = (unsigned)(key >> 32);
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+__device__ inline int key_index(unsigned long long key) { return (int)(0xffffffffu - (unsigned)(key & 0xffffffffull)); }
+__device__ inline void fold(float& bv, unsigned& bi, float v, unsigned i) {
+    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+}
+
+struct DraftSelectParams {
+    int batch, total_rows, vocab, max_blocks;
+    const float* logits;
+    const float* bias;        // may be nullptr
+    const int32_t* n_mask;
+    const int32_t* n_blocks;  // may be nullptr
+    float threshold;
+    int32_t* tokens;
+    float* probs;
+    int32_t* keep_len;        // [B, max_blocks]
+    unsigned long long* part_key;  // [rows][chunks] per-chunk (max, argmax)
+    float* part_sum;               // [rows][chunks] per-chunk sum of exp(x - chunk max)
+    unsigned int* ticket;
+    unsigned int* row_ticket;      // [rows] chunks of the row delivered so far (zero between calls)
+    int* status;
+};
+void launch_draft_select(const DraftSelectParams& p, cudaStream_t s);
+
 struct AcceptParams {
     int batch, total_rows, vocab;
     const float* logits;

@@ -352,3 +352,47 @@ def test_select_branch_matches_oracle():
         fd.fd_select_branch(ctx.h, B, 2, tokens.cuda(), step.q_lens.cuda(), step.n_mask.cuda(), nb.int().cuda(), acc.cuda(),
                             nd[:, :2].contiguous(), nl)                       # blocks longer than the output rows
         assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS
+
+
+@pytest.mark.parametrize("V,with_bias", [(151936, True), (151936, False), (4097, True), (1000, True), (37, False), (1, True)])
+def test_draft_select_matches_oracle(V, with_bias):
+    """Draft-side tail (Eq. 4 / Eq. 5): tokens bit-exact, confidences to 1e-4, verify lengths equal wherever the
+    cumulative confidence is not within 1e-3 of the threshold (there the fp32 product may fall on either side)."""
+    g = torch.Generator().manual_seed(V)
+    M = [16, 0, 28, 6, 32, 12, 1]
+    nb = [1, 1, 4, 0, 8, 3, 1]
+    B, Rm = len(M), sum(M)
+    logits = torch.randn((Rm, V), generator=g) * 2
+    if V > 8:                                                   # confident drafts, as a trained drafter gives
+        logits[torch.arange(Rm), torch.randint(0, V, (Rm,), generator=g)] += 9.0 * torch.rand((Rm,), generator=g) + 3.0
+        logits[3, 5] = logits[3].max() + 1; logits[3, 2] = logits[3, 5]          # an exact tie: lowest index wins
+    bias = torch.randn((Rm, V), generator=g) if with_bias else None
+    n_mask, n_blocks = torch.tensor(M, dtype=torch.int32), torch.tensor(nb, dtype=torch.int32)
+    step = wl.make_step("ds", wl.Shape(32, 8, 128, V), [5] * B, [32] * B, M, seed=1)
+    with Ctx(step) as ctx:
+        for thr in (0.5, 0.05):
+            e_tok, e_pr, e_cum, e_keep = oracle.draft_select(logits, bias, n_mask, n_blocks, thr, max_blocks=8)
+            tok = torch.full((Rm,), -9, dtype=torch.int32, device="cuda"); pr = torch.zeros((Rm,), device="cuda")
+            keep = torch.full((B, 8), -9, dtype=torch.int32, device="cuda")
+            fd.fd_draft_select(ctx.h, B, Rm, 8, logits.cuda(), None if bias is None else bias.cuda(), n_mask.cuda(), n_blocks.cuda(),
+                               thr, tok, pr, keep)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            np.testing.assert_array_equal(tok.cpu().numpy(), e_tok)
+            np.testing.assert_allclose(pr.cpu().numpy(), e_pr, rtol=1e-4, atol=1e-30)
+            got = keep.cpu().numpy()
+            r0 = 0
+            for b in range(B):
+                n_b = max(nb[b], 1); kb = M[b] // n_b if M[b] else 0
+                for gk in range(8):
+                    c = e_cum[r0 + gk * kb:r0 + (gk + 1) * kb] if (M[b] and gk < n_b) else np.zeros(0)
+                    if c.size and (np.abs(c - thr) < 1e-3 * thr).any():
+                        continue                                  # too close to call in fp32
+                    assert got[b, gk] == e_keep[b, gk], (b, gk, got[b, gk], e_keep[b, gk])
+                r0 += M[b]
+            keep2 = torch.empty_like(keep); tok2 = torch.empty_like(tok); pr2 = torch.empty_like(pr)
+            fd.fd_draft_select(ctx.h, B, Rm, 8, logits.cuda(), None if bias is None else bias.cuda(), n_mask.cuda(), n_blocks.cuda(),
+                               thr, tok2, pr2, keep2)
+            assert torch.equal(pr, pr2) and torch.equal(tok, tok2) and torch.equal(keep, keep2)      # bitwise repeatable
+        bad = torch.tensor([16, 0, 28, 6, 32, 12, 2], dtype=torch.int32)                             # rows do not add up
+        fd.fd_draft_select(ctx.h, B, Rm, 8, logits.cuda(), None, bad.cuda(), n_blocks.cuda(), 0.5, tok, pr, keep)
+        assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS and (tok == -1).all() and (keep == 0).all()
