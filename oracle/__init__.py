@@ -11,6 +11,7 @@ attn(...)        full attention under the hybrid mask (Sec. 4.1), float64 output
 attn_row(...)    one output row of the same definition (sampled checks)
 attn_blocks(...) the same with several mask blocks per sequence (all hypotheses, Eq. 2)
 select_branch(...) pick the prepared next-draft branch of the accepted length
+kv_append(...)   write the query block's K/V into its pages (append, then attend)
 draft_select(...) draft-side tail: calibrated argmax, confidence, Eq. 5 verify length
 accept(...)      greedy verification: argmax, accepted length, bonus token (Sec. 3)
 commit(...)      KV commit / rollback by page-table truncation
@@ -157,6 +158,19 @@ def draft_select(logits, bias, n_mask, n_blocks, threshold, max_blocks):
     _load().fdo_draft_select(ctypes.c_int(B), ctypes.c_int(V), ctypes.c_int(max_blocks), _p(lg), None if bs is None else _p(bs), _p(nm),
                              None if nb is None else _p(nb), ctypes.c_double(threshold), _p(tok), _p(pr), _p(cum), _p(keep))
     return tok[:Rm], pr[:Rm], cum[:Rm], keep
+
+
+def kv_append(k_new, v_new, kv_cache, page_table, prefix_lens, q_lens):
+    """Returns a copy of kv_cache (uint16 bit pattern, same shape) with the query block's K/V written in."""
+    kb, vb = _bits(k_new), _bits(v_new)
+    kv = _bits(kv_cache).copy()
+    T, Hkv, d = kb.shape
+    P = kv.shape[3]
+    pt, pl, ql = _i32(page_table), _i32(prefix_lens), _i32(q_lens)
+    assert int(ql.sum()) == T and vb.shape == kb.shape
+    _load().fdo_kv_append(ctypes.c_int(pl.shape[0]), ctypes.c_int(Hkv), ctypes.c_int(d), ctypes.c_int(P), ctypes.c_int(pt.shape[1]),
+                          _p(kb), _p(vb), _p(kv), _p(pt), _p(pl), _p(ql))
+    return kv
 
 
 def commit(page_table, prefix_lens, q_lens, accepted_len, page_size=16):

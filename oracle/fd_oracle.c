@@ -319,6 +319,28 @@ void fdo_draft_select(int B, int V, int max_blocks, const float *logits, const f
     }
 }
 
+/* KV append ("append, then attend"): the K/V of the Lq_b query tokens of sequence b (candidates first, then
+ * mask tokens) are written at logical positions n_b .. n_b + Lq_b - 1 of its paged cache, so that the
+ * attention of this step, and after the commit every later step, finds them there (Sec. 4.1 "Inference": the
+ * KV cache built by the target's own forward pass is what later steps reuse).  k_new, v_new [T, Hkv, d] bf16
+ * bits, sequence-major rows; every other byte of the cache is left as it was. */
+void fdo_kv_append(int B, int Hkv, int d, int page_size, int max_pages, const uint16_t *k_new, const uint16_t *v_new,
+        uint16_t *kv, const int32_t *page_table, const int32_t *prefix_lens, const int32_t *q_lens)
+{
+    int64_t row = 0;
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < q_lens[b]; ++i, ++row) {
+            const int j = prefix_lens[b] + i;
+            const int64_t page = page_table[(int64_t)b * max_pages + j / page_size];
+            const int slot = j % page_size;
+            for (int h = 0; h < Hkv; ++h)
+                for (int c = 0; c < d; ++c) {
+                    kv[((((page * 2 + 0) * Hkv + h) * page_size + slot) * (int64_t)d) + c] = k_new[(row * Hkv + h) * (int64_t)d + c];
+                    kv[((((page * 2 + 1) * Hkv + h) * page_size + slot) * (int64_t)d) + c] = v_new[(row * Hkv + h) * (int64_t)d + c];
+                }
+        }
+}
+
 /* KV commit / rollback.  In place on page_table [B, max_pages] and prefix_lens [B].
  * Sequences with accepted_len < 0 are left unchanged.  freed_pages is packed in
  * (sequence ascending, logical page ascending) order; returns the number freed. */
