@@ -129,6 +129,25 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
                                void* out, void* stream);
 
 /*
+ * KV append, the step before the attention ("append, then attend").  The forward pass that verifies the
+ * drafts also produces K/V for the query block; they enter the paged cache at logical positions
+ * n_b .. n_b + Lq_b - 1 (candidates first, then mask tokens), where fd_attn_draft_verify reads them and
+ * where, after fd_kv_commit has kept the accepted part, every later step finds them (Sec. 4.1
+ * "Inference": the KV cache of the clean prefix is reused by all later steps).
+ *
+ *   k_new, v_new   device, [T, Hkv, d] bf16, 16-byte aligned, sequence-major rows
+ *   kv_cache       device, [num_pages, 2, Hkv, P, d] bf16, in/out; only the slots of the block are written
+ *   page_table     device, [B, max_pages_per_seq] int32: pages for positions up to n_b + Lq_b - 1 must be allocated
+ *   prefix_lens, q_lens   device, [B] int32
+ *
+ * A sequence whose rows would pass T or the page table is skipped (FD_DEV_BAD_LENGTHS); a slot whose page
+ * id is outside the pool is skipped (FD_DEV_BAD_PAGE).
+ */
+fd_status fd_kv_append(fd_ctx* ctx, int batch, int total_q_rows, const void* k_new, const void* v_new,
+                       void* kv_cache, int num_pages, const int32_t* page_table,
+                       const int32_t* prefix_lens, const int32_t* q_lens, void* stream);
+
+/*
  * The same attention with several mask blocks per sequence: the parallel mode proper, in which the
  * forward pass that verifies the current draft also prepares one next-draft branch per hypothesis r
  * ("the first r drafts are accepted", Sec. 3 "Parallel speculative decoding", Eq. 2), each branch

@@ -378,6 +378,25 @@ fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefi
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }
 
+fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new, const void* v_new, void* kv_cache,
+                       int num_pages, const int32_t* page_table, const int32_t* prefix_lens, const int32_t* q_lens,
+                       void* stream) {
+    if (!c || batch < 0 || batch > c->cfg.max_batch || total_q_rows < 0 || num_pages < 0) return FD_ERR_INVALID_ARG;
+    if (batch == 0) return total_q_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
+    if (!page_table || !prefix_lens || !q_lens || !kv_cache) return FD_ERR_INVALID_ARG;
+    if (total_q_rows > 0 && (!k_new || !v_new)) return FD_ERR_INVALID_ARG;
+    if (!aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(kv_cache, 16)) return FD_ERR_INVALID_ARG;
+    fd::AppendParams p;
+    p.batch = batch; p.total_rows = total_q_rows; p.num_pages = num_pages; p.Hkv = c->cfg.n_kv_heads; p.d = c->cfg.head_dim;
+    p.max_pages = c->cfg.max_pages_per_seq;
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new); p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    p.kv = static_cast<__nv_bfloat16*>(kv_cache);
+    p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.status = c->status;
+    fd::launch_kv_append(p, static_cast<cudaStream_t>(stream));
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
 fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blocks, const float* draft_logits,
                           const float* bias, const int32_t* n_mask, const int32_t* n_blocks, float threshold,
                           int32_t* mask_tokens, float* mask_probs, int32_t* keep_len, void* stream) {

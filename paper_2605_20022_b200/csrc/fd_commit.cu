@@ -52,6 +52,53 @@ void launch_commit(const CommitParams& p, cudaStream_t s) {
     commit_kernel<<<1, 256, (p.batch + 1) * sizeof(int), s>>>(p);
 }
 
+// KV append: K/V of the query block -> its pages ("append, then attend").  One CTA per sequence; 16-byte copies.
+__global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p) {
+    __shared__ int s_red[8];
+    __shared__ long long s_row0;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    // first query row of this sequence = sum of the lengths before it (block-parallel; negative lengths count as 0)
+    int part = 0;
+    for (int s = tid; s < b; s += blockDim.x) part += max(p.q_lens[s], 0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if ((tid & 31) == 0) s_red[tid >> 5] = part;
+    __syncthreads();
+    if (tid == 0) {
+        long long r = 0;
+        for (int w = 0; w < 8; ++w) r += s_red[w];
+        s_row0 = r;
+    }
+    __syncthreads();
+    const long long row0 = s_row0;
+    const int n = p.prefix_lens[b], Lq = p.q_lens[b];
+    if (Lq <= 0) return;
+    if (n < 0 || row0 + Lq > p.total_rows || (long long)n + Lq > (long long)p.max_pages * 16) {
+        if (tid == 0) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        return;
+    }
+    const int vec_per_head = p.d / 8;                    // 16-byte pieces of one head's row
+    const int per_row = p.Hkv * vec_per_head;
+    for (int e = tid; e < Lq * per_row * 2; e += blockDim.x) {
+        const int which = e / (Lq * per_row), rem = e % (Lq * per_row);
+        const int i = rem / per_row, h = (rem % per_row) / vec_per_head, v = rem % vec_per_head;
+        const int j = n + i;
+        const int page = p.page_table[(long long)b * p.max_pages + (j >> 4)];
+        if ((unsigned)page >= (unsigned)p.num_pages) {   // never form an address from a bad id
+            if (h == 0 && v == 0) atomicOr(p.status, FD_DEV_BAD_PAGE);
+            continue;
+        }
+        const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + ((row0 + i) * p.Hkv + h) * p.d + v * 8;
+        __nv_bfloat16* dst = p.kv + ((((long long)page * 2 + which) * p.Hkv + h) * 16 + (j & 15)) * p.d + v * 8;
+        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    }
+}
+
+void launch_kv_append(const AppendParams& p, cudaStream_t s) {
+    if (p.batch == 0) return;
+    kv_append_kernel<<<p.batch, 256, 0, s>>>(p);
+}
+
 // Branch selection after verification (parallel drafting with one prepared branch per hypothesis):
 // copy the tokens of the block prepared for r = accepted_len drafts accepted.  One CTA.
 __global__ void __launch_bounds__(256) select_branch_kernel(SelectParams p) {

@@ -214,6 +214,18 @@ struct AcceptParams {
 };
 void launch_accept(const AcceptParams& p, cudaStream_t s);
 
+struct AppendParams {
+    int batch, total_rows, num_pages, Hkv, d, max_pages;
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* kv;
+    const int32_t* page_table;
+    const int32_t* prefix_lens;
+    const int32_t* q_lens;
+    int* status;
+};
+void launch_kv_append(const AppendParams& p, cudaStream_t s);
+
 struct SelectParams {
     int batch, max_kb;
     const int32_t* mask_tokens;

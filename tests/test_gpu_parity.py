@@ -396,3 +396,32 @@ def test_draft_select_matches_oracle(V, with_bias):
         bad = torch.tensor([16, 0, 28, 6, 32, 12, 2], dtype=torch.int32)                             # rows do not add up
         fd.fd_draft_select(ctx.h, B, Rm, 8, logits.cuda(), None, bad.cuda(), n_blocks.cuda(), 0.5, tok, pr, keep)
         assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS and (tok == -1).all() and (keep == 0).all()
+
+
+def test_kv_append_matches_oracle_and_feeds_the_attention():
+    """fd_kv_append bit-exact against the oracle (every byte of the pool), then attention over the appended cache."""
+    shape = wl.Shape(32, 8, 128, 1000)
+    step = wl.make_step("append", shape, [0, 15, 16, 700, 2047], [32, 3, 17, 1, 20], [16, 0, 9, 0, 8], seed=33, extra_table_cols=1)
+    kv = wl.make_kv(step, poison=None)
+    g = torch.Generator().manual_seed(3)
+    T = step.total_q_rows
+    k_new = torch.randn((T, 8, 128), generator=g).bfloat16(); v_new = torch.randn((T, 8, 128), generator=g).bfloat16()
+    exp_bits = oracle.kv_append(k_new, v_new, kv, step.page_table, step.prefix_lens, step.q_lens)
+    q = wl.make_q(step)
+    with Ctx(step) as ctx:
+        dkv = kv.cuda()
+        dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
+        fd.fd_kv_append(ctx.h, step.batch, T, k_new.cuda(), v_new.cuda(), dkv, step.num_pages, dpt, dpl, dql)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        got_bits = dkv.cpu().view(torch.int16).numpy().view(np.uint16)
+        np.testing.assert_array_equal(got_bits, exp_bits)
+        out = torch.empty((T, 32, 128), dtype=torch.bfloat16, device="cuda")
+        fd.fd_attn_draft_verify(ctx.h, step.batch, T, q.cuda(), dkv, step.num_pages, dpt, dpl, dql, dnm, out)
+        kv_ref = torch.from_numpy(exp_bits.view(np.int16)).view(torch.bfloat16)
+        assert_close(out.float().cpu().numpy(), oracle.attn(q, kv_ref, step.page_table, step.prefix_lens, step.q_lens, step.n_mask), "append+attend")
+        bad = step.page_table.clone(); bad[2, 1] = -1                       # a page of the block is not allocated
+        dkv2 = kv.cuda()
+        fd.fd_kv_append(ctx.h, step.batch, T, k_new.cuda(), v_new.cuda(), dkv2, step.num_pages, bad.cuda(), dpl, dql)
+        assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_PAGE
+        fd.fd_kv_append(ctx.h, step.batch, T - 1, k_new.cuda(), v_new.cuda(), dkv2, step.num_pages, dpt, dpl, dql)
+        assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS
