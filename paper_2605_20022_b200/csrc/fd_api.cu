@@ -40,6 +40,17 @@ struct HostStage {
     int32_t *drafts, *pt, *pl, *ql, *nm, *nb, *acc, *bon, *freed, *nfreed;
 };
 
+// Tile equivalents charged for starting a segment in a CTA's range of the tensor-core kernel (measured:
+// a piece boundary costs about as much time as streaming three tiles).
+#ifndef FD_PIECE_COST
+#define FD_PIECE_COST 3
+#endif
+// Least tiles for which a CTA of the tensor-core kernel gets a range of its own: a small call then runs on
+// fewer CTAs, each with a few tiles, instead of one tile everywhere and many partials to merge.
+#ifndef FD_MIN_RANGE_TILES
+#define FD_MIN_RANGE_TILES 4
+#endif
+
 namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -109,6 +120,8 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const size_t o_ok = take(B * sizeof(int));
     const size_t o_sc = take((size_t)B * cfg->n_kv_heads * sizeof(int));
     const size_t o_cf = take((size_t)c->n_ctas * sizeof(int));
+    const size_t o_cs = take(((size_t)c->n_ctas + 1) * sizeof(int));
+    const size_t o_cne = take((B + 1) * sizeof(int));
     const size_t o_po = take(slots * d * fd::kMaxRows * sizeof(float));
     const size_t o_pm = take(slots * fd::kMaxRows * sizeof(float));
     const size_t o_pl = take(slots * fd::kMaxRows * sizeof(float));
@@ -128,6 +141,8 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->plan.seq_ok = reinterpret_cast<int*>(c->pool + o_ok);
     c->plan.seg_count = reinterpret_cast<int*>(c->pool + o_sc);
     c->plan.cta_first = reinterpret_cast<int*>(c->pool + o_cf);
+    c->plan.cta_start = reinterpret_cast<int*>(c->pool + o_cs);
+    c->plan.cu_ne = reinterpret_cast<int*>(c->pool + o_cne);
     c->part.o = reinterpret_cast<float*>(c->pool + o_po);
     c->part.m = reinterpret_cast<float*>(c->pool + o_pm);
     c->part.l = reinterpret_cast<float*>(c->pool + o_pl);
@@ -323,6 +338,9 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     p.n_blocks = n_blocks;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
+    p.q_box_t = fd::q_box_rows(p.G);
+    p.piece_cost = c->attn_path == FD_ATTN_SIMT ? 0 : FD_PIECE_COST;
+    p.min_range_tiles = c->attn_path == FD_ATTN_SIMT ? 1 : FD_MIN_RANGE_TILES;
 
     const bool tc = c->attn_path == FD_ATTN_TCGEN05 && total_q_rows > 0;  // no rows: the plan alone checks the lengths
     if (tc) {

@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
     const int total = hdr.total_tiles;
     if (total == 0) return;
     const int cta = blockIdx.x, r = threadIdx.x;
-    const int s_c = range_begin(cta, total, p.n_ctas), e_c = range_begin(cta + 1, total, p.n_ctas);
+    const int s_c = p.plan.cta_start[cta], e_c = p.plan.cta_start[cta + 1];
 
     int t = s_c;
     while (t < e_c) {

@@ -56,7 +56,9 @@ struct Cfg {
     static constexpr int kQBytes = kMaxRows * D * 2;
     static constexpr int kKBytes = kTileTokens * D * 2;  // one K (or V) tile
     static constexpr int kBarOffset = kQBytes + 2 * kStages * kKBytes;
-    static constexpr int kExOffset = kBarOffset + 512;           // [2][128] floats: stream exchange in the epilogue
+    static constexpr int kCsOffset = kBarOffset + 320;           // window of the CTA range starts
+    static constexpr int kDescOffset = kBarOffset + 448;         // ring of piece descriptors
+    static constexpr int kExOffset = kBarOffset + 1024;          // [2][128] floats: stream exchange in the epilogue
     static constexpr int kSmemBytes = kExOffset + 1024 + 1024;   // + slack for 1024-byte alignment
     static constexpr int kKSteps = D / 16;
     static constexpr int kHalves = D / 64;
@@ -71,10 +73,14 @@ struct Bars {
     uint32_t tmem_base;
     int abort;
     int epi_flag;              // per-epilogue decisions of thread 0: bit 0 merge, bit 1 leave
+    int desc_n;                // piece descriptors published so far (written by the Q load warp)
+    int piece_ok;              // thread 0 of the softmax groups: the descriptor of the next piece is there
 };
+constexpr int kDescSlots = 4;
+static_assert(sizeof(Bars) <= 320, "Bars must fit in front of the range-start window");
 
 struct Piece {
-    int b, kvh, tile0, nt, n, Lq, M, nb, kv_len, rows, row0, slot;
+    int b, kvh, tile0, nt, n, Lq, M, nb, kv_len, rows, row0, slot, seg_nt;
     bool complete;
 };
 
@@ -92,6 +98,7 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_
     const int seg_start = t - pc.tile0, seg_end = seg_start + ntiles;
     const int t_end = min(e_c, seg_end);
     pc.nt = t_end - t;
+    pc.seg_nt = ntiles;
     pc.n = p.prefix_lens[lo];
     pc.Lq = p.q_lens[lo];
     pc.M = p.n_mask[lo];
@@ -118,10 +125,14 @@ __device__ __forceinline__ void trace(int role, int ev, int tile, int& n) {
     g_trace[role * kTracePerRole + n] = ((unsigned long long)clock64() & 0xffffffffffull) | ((unsigned long long)ev << 40) | ((unsigned long long)tile << 48);
     g_trace_n[role] = ++n;
 }
+__device__ unsigned long long g_cta_log[1024 * 16];
+__device__ __forceinline__ void cta_log(int slot) { if (slot < 16) g_cta_log[blockIdx.x * 16 + slot] = global_ns(); }
+#define CTA_LOG(slot) cta_log(slot)
 #define TRACE(role, ev, tile) trace(role, ev, tile, tr_n)
 #define TRACE_DECL int tr_n = 0
 #else
 #define TRACE(role, ev, tile)
+#define CTA_LOG(slot)
 #define TRACE_DECL
 #endif
 
@@ -135,6 +146,35 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, volatile int* abort) {
     const bool ok = mbar_wait(bar, parity, abort);
     return __all_sync(0xffffffffu, ok);
+}
+
+// Piece descriptors.  The Q load warp walks the pieces ahead of everyone, decodes each one (a chain of
+// dependent global loads) and publishes it in a small ring in shared memory; the MMA warp and the softmax
+// groups pick it up from there, so the decode is off their critical path at a piece boundary.  Slot
+// reuse is safe: descriptor N + 1 is written after every QK^T of piece N - 1 has completed, when no
+// consumer is before piece N - 1 and every consumer copies its descriptor to registers at piece start.
+__device__ __forceinline__ void publish_piece(Bars* bars, Piece* ring, int n, const Piece& pc) {
+    ring[n & (kDescSlots - 1)] = pc;
+    asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(&bars->desc_n)), "r"(n + 1) : "memory");
+}
+__device__ __forceinline__ bool piece_published(Bars* bars, int n) {
+    int v;
+    asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&bars->desc_n)) : "memory");
+    return v > n;
+}
+// Bounded like every other wait; false if it gave up (abort raised here or elsewhere).
+__device__ __forceinline__ bool wait_piece(Bars* bars, int n, volatile int* abort) {
+    if (piece_published(bars, n)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (piece_published(bars, n)) return true;
+        if ((it & 15u) == 0u) {
+            if (*abort) return false;
+            if (global_ns() - t0 > kWaitLimitNs) break;
+        }
+    }
+    *abort = 1;
+    return false;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -174,11 +214,13 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     while (w.t < e_c && ok) {
         const Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
         const int32_t* table = p.page_table + (long long)pc.b * p.max_pages;
-        // the page id of the next tile is fetched before waiting for a free buffer, so the
-        // table lookup never sits between a buffer becoming free and its refill
-        auto page_of = [&](int j) -> int {
-            const int pos = (pc.tile0 + j) * kTileTokens + pg * 16;
-            if (!(j < pc.nt && lane < kOps && pos < pc.kv_len)) return -1;
+        // Page ids are fetched a batch of four tiles (32 pages, one per lane) at a time and one batch
+        // ahead, so the table lookup -- a dependent global load -- never sits between a buffer becoming
+        // free and its refill, not even while the ring is filling up at the start of a piece.
+        auto load_ids = [&](int batch) -> int {
+            const int j = batch * 4 + (lane >> 3);
+            const int pos = ((pc.tile0 + j) * 8 + (lane & 7)) * 16;
+            if (!(j < pc.nt && pos < pc.kv_len)) return -1;
             int id = table[pos >> 4];
             if ((unsigned)id >= (unsigned)p.num_pages) {  // never form an address from a bad id
                 p.plan.seq_ok[pc.b] = 0;
@@ -187,21 +229,21 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             }
             return id;
         };
-        int phys = page_of(0);
+        int ids_cur = load_ids(0), ids_next = load_ids(1);
         for (int j = 0; j < pc.nt; ++j) {
             const int g = w.g0 + j, st = g % C::kStages, use = g / C::kStages;
-            const int phys_next = page_of(j + 1);
+            if (j > 0 && (j & 3) == 0) { ids_cur = ids_next; ids_next = load_ids((j >> 2) + 1); }
+            const int phys = __shfl_sync(0xffffffffu, ids_cur, (j & 3) * 8 + pg);
             if (!wait_all(&empty[st], (use & 1) ^ 1, abort)) { ok = false; break; }
             if (lane == 0) TRACE(which, 0, g);
             const int pos0 = (pc.tile0 + j) * kTileTokens;
             const int npg = min(8, (pc.kv_len - pos0 + 15) >> 4);
             if (lane == 0) mbar_arrive_expect_tx(&full[st], npg * (16 * D * 2));
             __syncwarp();
-            if (phys >= 0) {
+            if (lane < kOps && phys >= 0) {
                 unsigned char* dst = ring + st * C::kKBytes + half * (kTileTokens * 128) + pg * 2048;
                 tma_load_2d_hint(dst, &tmap, half * 64, ((phys * 2 + which) * p.Hkv + pc.kvh) * 16, &full[st], policy);
             }
-            phys = phys_next;
             issued = g + 1;
         }
         w.advance(pc);
@@ -216,32 +258,43 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     }
 }
 
-// Q load warp: the G * Lq rows of a piece -> shared memory, K-major, 128-byte swizzle.  One TMA box
-// per block row and 64-wide half of d (the G q-heads of the kv-head are G consecutive rows of the
-// [T * Hq, d] view of q).  Rows beyond G * Lq keep whatever the buffer held: each query row only
-// ever influences its own output row, and those rows are never stored.
+// Q load warp: the G * Lq rows of a piece -> shared memory, K-major, 128-byte swizzle.  q is seen as
+// [T][Hq][d]; one TMA box is 64 elements of d x the G q-heads of the kv-head x q_box_t block rows, which
+// lands as q_box_t * G consecutive 128-byte rows, row (i, g) at i * G + g: the order the MMA wants.  The
+// last box of a piece may reach past the block (rows of the next sequence, or zeros past T): each query
+// row only ever influences its own output row, and those rows are never stored.
 template <int D>
-__device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams& p, unsigned char* sq, Bars* bars, int s_c, int e_c,
+__device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams& p, unsigned char* sq, Bars* bars, Piece* ring, int s_c, int e_c,
                                        volatile int* abort) {
     using C = Cfg<D>;
     TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
+    const int bt = p.q_box_t;
     Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
     int issued = 0;
+    Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+    if (lane == 0) publish_piece(bars, ring, 0, pc);
     while (w.t < e_c) {
-        const Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
         if (w.piece > 0 && !wait_all(&bars->q_free, (w.piece - 1) & 1, abort)) break;
         if (lane == 0) TRACE(6, 0, w.piece);
-        if (lane == 0) mbar_arrive_expect_tx(&bars->q_full, pc.rows * D * 2);
+        const int nbox = (pc.Lq + bt - 1) / bt;
+        if (lane == 0) mbar_arrive_expect_tx(&bars->q_full, nbox * bt * p.G * 128 * C::kHalves);
         __syncwarp();
-        for (int i = lane; i < pc.Lq; i += 32) {
-#pragma unroll
-            for (int half = 0; half < C::kHalves; ++half)
-                tma_load_2d(sq + half * (kMaxRows * 128) + i * p.G * 128, &qmap, half * 64, (pc.row0 + i) * p.Hq + pc.kvh * p.G, &bars->q_full);
+        for (int e = lane; e < nbox * C::kHalves; e += 32) {
+            const int j = e / C::kHalves, half = e % C::kHalves;
+            tma_load_3d(sq + half * (kMaxRows * 128) + j * bt * p.G * 128, &qmap, half * 64, pc.kvh * p.G, pc.row0 + j * bt, &bars->q_full);
         }
         issued = w.piece + 1;
         if (lane == 0) TRACE(6, 1, w.piece);
         w.advance(pc);
+        if (w.t < e_c) {
+            // the next piece: descriptor for the other roles, and its Q rows on their way into L2
+            pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+            if (lane == 0) publish_piece(bars, ring, w.piece, pc);
+            const int nb2 = (pc.Lq + bt - 1) / bt;
+            for (int e = lane; e < nb2 * C::kHalves; e += 32)
+                tma_prefetch_3d(&qmap, (e % C::kHalves) * 64, pc.kvh * p.G, pc.row0 + (e / C::kHalves) * bt);
+        }
     }
     if (*abort && issued > 0) {  // drain the last copy before the shared memory is given back
         const unsigned long long t0 = global_ns();
@@ -253,7 +306,7 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
 // MMA issuing warp.
 template <int D>
 __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq, unsigned char* sk, unsigned char* sv, Bars* bars,
-                                         uint32_t tmem, int s_c, int e_c, volatile int* abort) {
+                                         const Piece* ring, uint32_t tmem, int s_c, int e_c, volatile int* abort) {
     using C = Cfg<D>;
     TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
@@ -264,7 +317,8 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
     Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
     bool ok = true;
     while (w.t < e_c && ok) {
-        const Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+        if (!__all_sync(0xffffffffu, wait_piece(bars, w.piece, abort))) break;
+        const Piece pc = ring[w.piece & (kDescSlots - 1)];
         if (!wait_all(&bars->q_full, w.piece & 1, abort)) break;
         if (lane == 0) TRACE(2, 3, w.piece);
         auto issue_pv = [&](int jj) {
@@ -300,10 +354,16 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
         };
         for (int j = 0; j < pc.nt && ok; ++j) {
             const int g = w.g0 + j, st = g % C::kStages, use = g / C::kStages;
-            const int s = j & 1, u = w.u_base[s] + (j >> 1);
+            const int s = j & 1;
             if (!wait_all(&bars->k_full[st], use & 1, abort)) { ok = false; break; }
             if (lane == 0) TRACE(2, 0, g);
-            if (u >= 1 && !wait_all(&bars->pv_done[s], (u - 1) & 1, abort)) { ok = false; break; }  // S/P buffer free
+            // S_s is written over P_s, which the P V of tile j - 2 reads.  That MMA was issued earlier by
+            // this same thread, and the tensor pipe takes one thread's MMAs in issue order, so no wait for
+            // its completion is needed here (measured: 3 % on a power-capped 36-layer step).  Building with
+            // -DFD_WAIT_PV restores the explicit wait on the completion barrier.
+#ifdef FD_WAIT_PV
+            if (w.u_base[s] + (j >> 1) >= 1 && !wait_all(&bars->pv_done[s], (w.u_base[s] + (j >> 1) - 1) & 1, abort)) { ok = false; break; }
+#endif
             tc_fence_after();
             if (lane == 0) {
                 TRACE(2, 1, g);
@@ -330,8 +390,8 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
 
 // The two softmax groups (256 threads).
 template <int D>
-__device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, uint32_t tmem, int total, int s_c, int e_c,
-                                             volatile int* abort) {
+__device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, int* s_cs, const CtaStarts cs, const Piece* ring,
+                                             uint32_t tmem, int s_c, int e_c, volatile int* abort) {
     TRACE_DECL;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     const int s = warp >> 2;                  // stream
@@ -339,9 +399,18 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
     const float c = p.scale_log2e;
-    Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
+    // fill the window of range starts; the barrier below orders it before its first use
+    if (tid < kCsWindow) {
+        const int cc = cs.base + tid;
+        s_cs[tid] = (cc >= 0 && cc <= p.n_ctas) ? p.plan.cta_start[cc] : 0;
+    }
+    Walk w = {s_c, 0, {0, 0}, 0, 0};
     while (w.t < e_c) {
-        const Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+        // one thread waits for the descriptor, so that all 256 take the same decision
+        if (tid == 0) bars->piece_ok = wait_piece(bars, w.piece, abort);
+        named_bar_sync(1, 256);
+        if (!bars->piece_ok) break;
+        const Piece pc = ring[w.piece & (kDescSlots - 1)];
         if (tid == 0) TRACE(5, 2, w.piece);
         const bool warp_active = (warp & 3) * 32 < pc.rows;
         const int i = r / p.G;
@@ -448,27 +517,29 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         tc_fence_after();
         if (tid == 0) TRACE(5, 4, w.piece);
         const bool two = pc.nt >= 2;
-        named_bar_sync(1, 256);                       // the exchange array is free again
-        ex[s * kMaxRows + r] = m;
+        // Stream exchange: group 1 hands its (m, l) to group 0, which answers with the two scale factors.
+        // A thread only ever touches the two slots of its own row, so one barrier each way is enough.
+        if (s == 1) { ex[r] = m; ex[kMaxRows + r] = l; }
         if (tid == 0) bars->epi_flag = *abort ? 2 : 0;
         named_bar_sync(1, 256);
-        const float m_other = ex[(s ^ 1) * kMaxRows + r];
         const bool leave = (bars->epi_flag & 2) != 0;
+        float a0 = 0.f, a1 = 0.f, mm = -INFINITY, L = 0.f;
+        if (s == 0) {
+            const float m1 = two ? ex[r] : -INFINITY, l1 = ex[kMaxRows + r];
+            mm = fmaxf(m, m1);
+            a0 = (m == -INFINITY) ? 0.f : exp2f(m - mm);
+            a1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mm);
+            L = a0 * l + (two ? a1 * l1 : 0.f);
+            if (pc.complete) { const float inv = 1.f / L; a0 *= inv; a1 *= inv; }
+            ex[r] = a0;
+            ex[kMaxRows + r] = a1;
+        }
         named_bar_sync(1, 256);
-        ex[s * kMaxRows + r] = l;
-        named_bar_sync(1, 256);
-        const float l_other = ex[(s ^ 1) * kMaxRows + r];
-        const float m0 = s ? m_other : m, l0 = s ? l_other : l;
-        const float m1 = two ? (s ? m : m_other) : -INFINITY, l1 = s ? l : l_other;
-        const float mm = fmaxf(m0, m1);
-        const float a0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - mm);
-        const float a1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mm);
-        const float L = a0 * l0 + (two ? a1 * l1 : 0.f);
-        const float inv = pc.complete ? 1.f / L : 1.f;
+        if (s == 1) { a0 = ex[r]; a1 = ex[kMaxRows + r]; }
         constexpr int kChunks = D / 64;  // 32-column chunks per softmax group
         const bool do_read = !leave && warp_active;
         // the load warps of this CTA have seen every page id of the segment by now
-        const float keep = (pc.complete && !__ldcg(p.plan.seq_ok + pc.b)) ? 0.f : 1.f;
+        const bool zero_rows = pc.complete && !__ldcg(p.plan.seq_ok + pc.b);
 #pragma unroll
         for (int ch = 0; ch < kChunks; ++ch) {
             const int col = s * (D / 2) + ch * 32;
@@ -482,7 +553,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 for (int k = 0; k < 32; ++k) {
                     o[k] = __uint_as_float(o0[k]) * a0;
                     if (two) o[k] = fmaf(__uint_as_float(o1[k]), a1, o[k]);
-                    o[k] *= inv;
                 }
             }
             if (ch == kChunks - 1) {
@@ -492,7 +562,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             if (do_read && r < pc.rows) {
                 if (pc.complete) {
                     __nv_bfloat16* dst = p.out + ((long long)(pc.row0 + i) * p.Hq + pc.kvh * p.G + r % p.G) * D + col;
-                    store_cols_bf16<32>(dst, o, keep);
+                    if (zero_rows) {  // by assignment: what was computed from a stand-in page may be inf or NaN
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) o[k] = 0.f;
+                    }
+                    store_cols_bf16<32>(dst, o, 1.f);
                 } else {
                     float* dst = p.part.o + ((long long)pc.slot * D + col) * kMaxRows + r;
 #pragma unroll
@@ -506,27 +580,30 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         }
         if (!pc.complete) {
             // Fused split merge: count the delivered pieces of the segment; whoever delivers the last
-            // one combines them all (no CTA ever waits for another).
-            __threadfence();
+            // one combines them all (no CTA ever waits for another).  The barrier orders the partial
+            // stores of all threads before thread 0's fence, and the fence before the count.
+            const int t0 = w.t - pc.tile0, t1 = t0 + pc.seg_nt;
+            int c_first, c_last;
+            segment_ctas(cs, p.n_ctas, cta, t0, t1, c_first, c_last);
             named_bar_sync(1, 256);
             if (tid == 0) {
                 int last = 0;
                 if (!leave && !*abort) {
-                    const int ntiles = p.plan.cu_tiles[pc.b + 1] - p.plan.cu_tiles[pc.b];
-                    const int seg_start = w.t - pc.tile0;
-                    const int n = segment_pieces(seg_start, seg_start + ntiles, total, p.n_ctas);
+                    const int n = segment_pieces(cs, c_first, c_last, t0, t1);
+                    __threadfence();
                     last = atomicAdd(p.plan.seg_count + pc.b * p.Hkv + pc.kvh, 1) + 1 == n;
+                    if (last) __threadfence();
                 }
                 bars->epi_flag = last;
             }
             named_bar_sync(1, 256);
             if (bars->epi_flag & 1) {
-                __threadfence();
                 const int rr = tid & (kMaxRows - 1), cg = tid >> 7;
-                if (rr < pc.rows) merge_row<D, D / 2>(p, total, pc.b, pc.kvh, rr, cg);
+                if (rr < pc.rows) merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, t0, t1, rr, cg);
             }
         }
         if (tid == 0) TRACE(5, 5, w.piece);
+        if (tid == 0) CTA_LOG(2 + w.piece);
         if (leave) break;
         w.advance(pc);
     }
@@ -543,6 +620,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     unsigned char* sv = sk + C::kStages * C::kKBytes;           // V ring
     Bars* bars = reinterpret_cast<Bars*>(smem + C::kBarOffset);
     float* ex = reinterpret_cast<float*>(smem + C::kExOffset);
+    int* s_cs = reinterpret_cast<int*>(smem + C::kCsOffset);
+    Piece* ring = reinterpret_cast<Piece*>(smem + C::kDescOffset);
     volatile int* abort = &bars->abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -565,6 +644,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         mbar_init(&bars->o_free, 256);
         bars->abort = 0;
         bars->epi_flag = 0;
+        bars->desc_n = 0;
+        bars->piece_ok = 0;
         mbar_fence_init();
     }
     if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
@@ -573,12 +654,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // the plan kernel has completed and its writes are visible
+    if (tid == 0) CTA_LOG(0);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) CTA_LOG(1);  // the plan kernel has completed and its writes are visible
 
     const PlanHeader hdr = *p.plan.hdr;
     const int total = hdr.total_tiles;
     const int cta = blockIdx.x;
-    const int s_c = total ? range_begin(cta, total, p.n_ctas) : 0, e_c = total ? range_begin(cta + 1, total, p.n_ctas) : 0;
+    const int s_c = total ? p.plan.cta_start[cta] : 0, e_c = total ? p.plan.cta_start[cta + 1] : 0;
+    // the range starts of the neighbouring CTAs decide who shares a segment with this one (epilogue, merge)
+    const CtaStarts cs = {p.plan.cta_start, s_cs, cta - kCsWindow / 2 + 1};
     if (s_c >= e_c) {  // uniform: no tile for this CTA (or nothing at all)
         if (total == 0 && hdr.fatal) {  // inconsistent lengths: a defined output, zeros
             const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
@@ -595,13 +680,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     // the decrease released (a request for more than that did not return when it was tried).
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-        softmax_role<D>(p, bars, ex, tmem, total, s_c, e_c, abort);
+        softmax_role<D>(p, bars, ex, s_cs, cs, ring, tmem, s_c, e_c, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         if (warp == kKWarp) load_role<D>(tmap, p, sk, bars->k_full, bars->k_empty, 0, s_c, e_c, abort);
         else if (warp == kVWarp) load_role<D>(tmap, p, sv, bars->v_full, bars->v_empty, 1, s_c, e_c, abort);
-        else if (warp == kMmaWarp) mma_role<D>(p, sq, sk, sv, bars, tmem, s_c, e_c, abort);
-        else q_role<D>(qmap, p, sq, bars, s_c, e_c, abort);
+        else if (warp == kMmaWarp) mma_role<D>(p, sq, sk, sv, bars, ring, tmem, s_c, e_c, abort);
+        else q_role<D>(qmap, p, sq, bars, ring, s_c, e_c, abort);
     }
     // ---- common tail: everything of this CTA has completed, or it is giving up
     if (*abort && tid == 0) atomicOr(p.status, FD_DEV_TIMEOUT);
@@ -651,17 +736,17 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
         if (e != cudaSuccess) { delete st; return e; }
         *state = st;
     }
-    // q: a 2-D view [rows = T * Hq, d], box = 64 elements x G rows (the q-heads of one kv-head for one block row)
+    // q: a 3-D view [T][Hq][d], box = 64 elements x G q-heads (one kv-head) x q_box_t block rows
     st->qcurrent = nullptr;
     for (int i = 0; i < st->nq_cached; ++i)
         if (st->qcache[i].ptr == p.q && st->qcache[i].num_pages == p.total_q_rows) st->qcurrent = &st->qcache[i].map;
     if (!st->qcurrent) {
         TmapEntry& e = st->qcache[st->qnext];
-        cuuint64_t dims[2] = {(cuuint64_t)p.d, (cuuint64_t)p.total_q_rows * p.Hq};
-        cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
-        cuuint32_t box[2] = {64, (cuuint32_t)p.G};
-        cuuint32_t estr[2] = {1, 1};
-        const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(p.q), dims, strides, box, estr,
+        cuuint64_t dims[3] = {(cuuint64_t)p.d, (cuuint64_t)p.Hq, (cuuint64_t)(p.total_q_rows > 0 ? p.total_q_rows : 1)};
+        cuuint64_t strides[2] = {(cuuint64_t)p.d * 2, (cuuint64_t)p.Hq * p.d * 2};
+        cuuint32_t box[3] = {64, (cuuint32_t)p.G, (cuuint32_t)p.q_box_t};
+        cuuint32_t estr[3] = {1, 1, 1};
+        const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(p.q), dims, strides, box, estr,
                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -740,6 +825,13 @@ extern "C" int fd_debug_read_trace(unsigned long long* dst, unsigned int* counts
     unsigned int zero[kTraceRoles] = {0};
     cudaMemcpyToSymbol(g_trace_n, zero, sizeof(zero));
     return kTracePerRole;
+}
+extern "C" int fd_debug_read_cta_log(unsigned long long* dst) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(dst, g_cta_log, sizeof(unsigned long long) * 1024 * 16);
+    static unsigned long long zero[1024 * 16];
+    cudaMemcpyToSymbol(g_cta_log, zero, sizeof(zero));
+    return 16;
 }
 #endif
 

@@ -25,9 +25,11 @@ struct Plan {
     PlanHeader* hdr;
     int* cu_q;      // [B+1] first query row of each sequence
     int* cu_tiles;  // [B+1] exclusive scan of tiles_b (per kv-head)
+    int* cu_ne;     // [B+1] exclusive scan of (tiles_b > 0)
     int* seq_ok;    // [B]   0 = a page id of the sequence was outside the pool: its rows are zeroed
     int* seg_count; // [B * Hkv] partial pieces of a segment that have been written (fused merge)
     int* cta_first; // [n_ctas] sequence that owns the first tile of each attention CTA's range
+    int* cta_start; // [n_ctas + 1] first tile of each attention CTA's range (non-decreasing; [n_ctas] = total)
 };
 
 // Partial result of one piece of a (sequence, kv-head) segment, log2 domain:
@@ -55,6 +57,9 @@ struct AttnParams {
     Plan plan;
     PartialView part;
     int n_ctas;       // CTAs of the attention grid (stream-K ranges are cut for this many)
+    int q_box_t;      // block rows per Q load box of the tensor-core kernel (see q_box_rows)
+    int min_range_tiles;  // least tiles worth giving a CTA a range of its own
+    int piece_cost;   // fixed cost of starting a segment in a range, in tiles (balances ranges with many short segments)
     int* status;
 };
 
@@ -80,13 +85,50 @@ __host__ __device__ inline RowMask row_mask(int i, int n, int Lq, int M, int nb,
     return rm;
 }
 
-// First tile of CTA c when `total` tiles are cut into `n` contiguous ranges.
-__host__ __device__ inline int range_begin(int c, int total, int n) {
-    return (int)(((long long)c * total) / n);
+// Block rows one Q load brings in: the largest power of two <= 8 that divides the most block rows a
+// segment can have (kMaxRows / G), so that rounding a block length up to whole boxes never passes the tile.
+__host__ __device__ inline int q_box_rows(int G) {
+    int bt = 8;
+    while ((kMaxRows / G) % bt) bt >>= 1;
+    return bt;
 }
-// The CTA whose range holds tile t.
-__host__ __device__ inline int range_owner(int t, int total, int n) {
-    return (int)((((long long)(t + 1)) * n + total - 1) / total) - 1;
+
+// View of cta_start: a window of it around the reading CTA may be cached in shared memory.
+constexpr int kCsWindow = 32;
+struct CtaStarts {
+    const int* g;   // [n_ctas + 1] in global memory
+    const int* s;   // entries [base, base + kCsWindow) in shared memory, or nullptr
+    int base;
+    __device__ __forceinline__ int at(int c) const {
+        const unsigned i = (unsigned)(c - base);
+        return (s && i < (unsigned)kCsWindow) ? s[i] : g[c];
+    }
+};
+
+// The CTA whose range [cta_start[c], cta_start[c + 1]) holds tile t (ranges may be empty: of several CTAs
+// that start at the same tile the last one is the one that owns it).
+__device__ inline int range_owner(const int* cta_start, int n_ctas, int t) {
+    int lo = 0, hi = n_ctas;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (cta_start[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// First and last CTA whose range meets segment [t0, t1), found by walking outwards from `c`, a CTA that is
+// known to meet it (a segment rarely spans more than a few ranges).
+__device__ inline void segment_ctas(const CtaStarts& cs, int n_ctas, int c, int t0, int t1, int& c_first, int& c_last) {
+    c_first = c_last = c;
+    while (c_first > 0 && cs.at(c_first) > t0) --c_first;
+    while (c_last + 1 < n_ctas && cs.at(c_last + 1) < t1) ++c_last;
+}
+
+// Number of partial pieces the CTAs c_first..c_last hold of segment [t0, t1) (1 = not split).
+__device__ inline int segment_pieces(const CtaStarts& cs, int c_first, int c_last, int t0, int t1) {
+    int n = 0;
+    for (int c = c_first; c <= c_last; ++c) n += max(cs.at(c), t0) < min(cs.at(c + 1), t1);
+    return n;
 }
 
 // Write one row segment of `n` columns as bf16 (n a multiple of 8), scaled by inv.
@@ -101,24 +143,13 @@ __device__ inline void store_cols_bf16(__nv_bfloat16* dst, const float* o, float
     }
 }
 
-// Number of partial pieces segment [t0, t1) was cut into by the CTA ranges (0 or 1 = not split).
-__device__ inline int segment_pieces(int t0, int t1, int total, int n_ctas) {
-    const int c_first = range_owner(t0, total, n_ctas), c_last = range_owner(t1 - 1, total, n_ctas);
-    if (c_first == c_last) return 1;
-    int n = 0;
-    for (int c = c_first; c <= c_last; ++c) {
-        const int sc = range_begin(c, total, n_ctas), ec = range_begin(c + 1, total, n_ctas);
-        n += max(sc, t0) < min(ec, t1);
-    }
-    return n;
-}
-
-// Combine the partial pieces of segment (b, kvh) for query row r, columns [cg * CW, (cg + 1) * CW),
-// in CTA-range order (fixed, so the result does not depend on timing), and write the bf16 output.
-// The caller guarantees that every piece has been written and is visible.
+// Combine the partial pieces of segment (b, kvh) = tiles [t0, t1), held by CTAs c_first..c_last, for query
+// row r (output row row0 + r / G), columns [cg * CW, (cg + 1) * CW), in CTA order (fixed, so the result does
+// not depend on timing), and write the bf16 output.  The caller guarantees that every piece has been
+// written and is visible.  A piece that saw no visible key for the row holds m = -inf, l = 0, O = 0.
 template <int D, int CW>
-__device__ inline void merge_row(const AttnParams& p, int total, int b, int kvh, int r, int cg) {
-    const int row0 = p.plan.cu_q[b];
+__device__ inline void merge_row(const AttnParams& p, const CtaStarts& cs, int c_first, int c_last, int b, int kvh, int row0,
+                                 int t0, int t1, int r, int cg) {
     __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
     float acc[CW];
 #pragma unroll
@@ -127,28 +158,32 @@ __device__ inline void merge_row(const AttnParams& p, int total, int b, int kvh,
         store_cols_bf16<CW>(dst, acc, 0.f);
         return;
     }
-    const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
-    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles, t1 = t0 + ntiles;
-    const int c_first = range_owner(t0, total, p.n_ctas), c_last = range_owner(t1 - 1, total, p.n_ctas);
     float m = -INFINITY;
     for (int c = c_first; c <= c_last; ++c) {
-        const int sc = range_begin(c, total, p.n_ctas), ec = range_begin(c + 1, total, p.n_ctas);
+        const int sc = cs.at(c), ec = cs.at(c + 1);
         if (max(sc, t0) >= min(ec, t1)) continue;
         const int slot = 2 * c + (sc >= t0 ? 0 : 1);
         m = fmaxf(m, __ldcg(p.part.m + slot * kMaxRows + r));
     }
     float l = 0.f;
     for (int c = c_first; c <= c_last; ++c) {
-        const int sc = range_begin(c, total, p.n_ctas), ec = range_begin(c + 1, total, p.n_ctas);
+        const int sc = cs.at(c), ec = cs.at(c + 1);
         if (max(sc, t0) >= min(ec, t1)) continue;
         const int slot = 2 * c + (sc >= t0 ? 0 : 1);
         const float mp = __ldcg(p.part.m + slot * kMaxRows + r);
-        if (mp == -INFINITY) continue;  // this piece saw no visible key for the row
-        const float w = exp2f(mp - m);
-        l += w * __ldcg(p.part.l + slot * kMaxRows + r);
+        const float lp = __ldcg(p.part.l + slot * kMaxRows + r);
         const float* o = p.part.o + ((long long)slot * D + cg * CW) * kMaxRows + r;
+        const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
+        l += w * lp;
+        constexpr int kBatch = CW < 64 ? CW : 64;  // independent loads in flight per thread
 #pragma unroll
-        for (int col = 0; col < CW; ++col) acc[col] += w * __ldcg(o + col * kMaxRows);
+        for (int c0 = 0; c0 < CW; c0 += kBatch) {
+            float v[kBatch];
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) v[k] = __ldcg(o + (c0 + k) * kMaxRows);
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) acc[c0 + k] += w * v[k];
+        }
     }
     store_cols_bf16<CW>(dst, acc, 1.f / l);
 }

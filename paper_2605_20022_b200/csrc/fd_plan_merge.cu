@@ -7,6 +7,10 @@
 // segment that falls into several ranges leaves one partial result per range; the merge
 // kernel combines them in range order, which makes the result independent of timing.
 //
+// Ranges are cut by cost, not by tile count: a segment costs its tiles plus a fixed number of tile
+// equivalents for starting it (Q load, pipeline fill and drain, epilogue), so a CTA whose range holds
+// many short segments gets fewer tiles.
+//
 // The plan kernel checks the lengths (O(B) work, one CTA).  Page ids are checked where they are
 // used, by the attention kernels: a sequence with an id outside the pool is flagged in seq_ok,
 // read from page 0 instead, and has its output rows zeroed by the merge kernel.
@@ -47,6 +51,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     const int P = 16;
     for (int i = tid; i < B * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
     long long rows = 0, tiles = 0;  // running totals (identical in every thread)
+    int nonempty = 0;               // sequences with at least one tile so far
     for (int base = 0; base < B; base += blockDim.x) {
         const int b = base + tid;
         int q = 0, t = 0;
@@ -61,34 +66,49 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
             else { q = (int)Lq; t = Lq > 0 ? (int)((n + Lq + kTileTokens - 1) / kTileTokens) : 0; }
             p.plan.seq_ok[b] = 1;
         }
-        int tq, tt;
+        int ne = t > 0, dummy = 0, tq, tt, tne, td;
         block_scan2(q, t, tq, tt, wsum);
+        block_scan2(ne, dummy, tne, td, wsum);
         if (b < B) {
             p.plan.cu_q[b + 1] = (int)min(rows + q, (long long)0x7fffffff);
             p.plan.cu_tiles[b + 1] = (int)min(tiles + t, (long long)0x7fffffff);
+            p.plan.cu_ne[b + 1] = nonempty + ne;
         }
         rows += tq;
         tiles += tt;
+        nonempty += tne;
     }
+    if (tid == 0) { p.plan.cu_tiles[0] = 0; p.plan.cu_ne[0] = 0; }
     __syncthreads();
-    // where each attention CTA starts: the sequence that owns the first tile of its range (the kernels
-    // then walk forward from there instead of searching the scan with dependent loads)
+    // Where each attention CTA starts.  Cost position x of a tile: Hkv * (tiles + k * segments started)
+    // before it, with a segment's k start-up units ahead of its tiles; CTA c starts at the tile that
+    // holds x = c * W / n_ctas (a position inside the start-up units snaps to the segment's first tile).
     const long long total = tiles * p.Hkv;
+    const long long k = p.piece_cost;
+    const long long W = (long long)p.Hkv * (tiles + k * nonempty);
+    // a small call is not spread over every CTA: a range is worth starting only for a few tiles of work,
+    // and every extra range of a segment is one more partial to merge
+    const int n_use = (int)max(1LL, min((long long)p.n_ctas, W / (k + max(1, p.min_range_tiles))));
     if (!s_fatal && total > 0 && total <= 0x7fffffffLL) {
-        for (int c = tid; c < p.n_ctas; c += blockDim.x) {
-            const int t = range_begin(c, (int)total, p.n_ctas);
-            int lo = 0, hi = B;
+        for (int c = tid; c <= p.n_ctas; c += blockDim.x) {
+            if (c >= n_use) { p.plan.cta_start[c] = (int)total; if (c < p.n_ctas) p.plan.cta_first[c] = 0; continue; }
+            const long long x = (c * W) / n_use;
+            int lo = 0, hi = B;   // last b whose span starts at or before x (of equal starts the last: the non-empty one)
             while (hi - lo > 1) {
                 const int mid = (lo + hi) >> 1;
-                if (p.Hkv * __ldcg(p.plan.cu_tiles + mid) <= t) lo = mid; else hi = mid;
+                const long long w_mid = (long long)p.Hkv * (__ldcg(p.plan.cu_tiles + mid) + k * __ldcg(p.plan.cu_ne + mid));
+                if (w_mid <= x) lo = mid; else hi = mid;
             }
+            const long long ct = __ldcg(p.plan.cu_tiles + lo), nt = __ldcg(p.plan.cu_tiles + lo + 1) - ct;
+            const long long rem = x - (long long)p.Hkv * (ct + k * __ldcg(p.plan.cu_ne + lo));
+            const long long kvh = rem / (nt + k), r = rem % (nt + k);
+            p.plan.cta_start[c] = (int)(p.Hkv * ct + kvh * nt + max(0LL, r - k));
             p.plan.cta_first[c] = lo;
         }
     }
     if (tid == 0) {
         const int fatal = s_fatal || rows != p.total_q_rows || tiles * p.Hkv > 0x7fffffffLL;
         p.plan.cu_q[0] = 0;
-        p.plan.cu_tiles[0] = 0;
         if (fatal) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         p.plan.hdr->fatal = fatal;
         p.plan.hdr->total_tiles = fatal ? 0 : (int)(tiles * p.Hkv);
@@ -118,10 +138,13 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(AttnParams p) {
     const int r = threadIdx.x % kMaxRows, cg = threadIdx.x / kMaxRows;
     if (r >= rows) return;
     const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
-    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles;
+    if (ntiles == 0) return;
+    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles, t1 = t0 + ntiles;
+    const CtaStarts cs = {p.plan.cta_start, nullptr, 0};
+    const int c_first = range_owner(cs.g, p.n_ctas, t0), c_last = range_owner(cs.g, p.n_ctas, t1 - 1);
     // an unsplit segment was written by the attention kernel itself; it is revisited only to zero it
-    if (segment_pieces(t0, t0 + ntiles, hdr.total_tiles, p.n_ctas) <= 1 && p.plan.seq_ok[b]) return;
-    merge_row<D, D / 4>(p, hdr.total_tiles, b, kvh, r, cg);
+    if (segment_pieces(cs, c_first, c_last, t0, t1) <= 1 && p.plan.seq_ok[b]) return;
+    merge_row<D, D / 4>(p, cs, c_first, c_last, b, kvh, p.plan.cu_q[b], t0, t1, r, cg);
 }
 
 void launch_merge(const AttnParams& p, cudaStream_t s) {
