@@ -205,6 +205,8 @@ class DeviceStep:
         """One step on the current stream; the commit works on copies restored every step."""
         fd, torch, st = self.fd, self.torch, self.step
         self.pt.copy_(self.pt0); self.pl.copy_(self.pl0)
+        if self.L > 1:   # every layer of the step has the same lengths: one work list serves them all
+            fd.fd_plan_pin(self.ctx, st.batch, st.total_q_rows, self.pl, self.ql, self.nm, self.nb)
         for l in range(self.L):
             if time_attn:
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
@@ -217,6 +219,8 @@ class DeviceStep:
                                                self.pt, self.pl, self.ql, self.nm, self.nb, self.out[l])
             if time_attn:
                 e1.record(); self.attn_events.append((e0, e1))
+        if self.L > 1:
+            fd.fd_plan_unpin(self.ctx)   # the commit below changes prefix_lens
         fd.fd_verify_accept(self.ctx, st.batch, st.total_cand_rows, self.logits, self.drafts, self.ql, self.nm,
                             self.acc, self.bon)
         fd.fd_kv_commit(self.ctx, st.batch, self.pt, self.pl, self.ql, self.acc, self.freed, self.n_freed)

@@ -129,6 +129,21 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
                                void* out, void* stream);
 
 /*
+ * Optional: pin the work list of a step.  The attention call derives a work list (which CTA streams which
+ * KV tiles) from the lengths alone; it is the same for every layer of a step.  fd_plan_pin computes it once;
+ * until fd_plan_unpin, every fd_attn_draft_verify[_blocks] call with the same batch, total_q_rows and the
+ * same four length pointers reuses it instead of recomputing it (a call with anything else recomputes and
+ * drops the pin).  The caller must not change the contents of the length arrays while the pin holds
+ * (fd_kv_commit does: unpin before the next step), and must unpin after a FD_DEV_TIMEOUT status.
+ * The paper does not describe a work list; this follows from "all layers of a step share the lengths".
+ *
+ *   prefix_lens, q_lens, n_mask   device, [B] int32;  n_blocks   device, [B] int32 or NULL
+ */
+fd_status fd_plan_pin(fd_ctx* ctx, int batch, int total_q_rows, const int32_t* prefix_lens, const int32_t* q_lens,
+                      const int32_t* n_mask, const int32_t* n_blocks, void* stream);
+fd_status fd_plan_unpin(fd_ctx* ctx);
+
+/*
  * KV append, the step before the attention ("append, then attend").  The forward pass that verifies the
  * drafts also produces K/V for the query block; they enter the paged cache at logical positions
  * n_b .. n_b + Lq_b - 1 (candidates first, then mask tokens), where fd_attn_draft_verify reads them and

@@ -23,7 +23,7 @@ FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin"]
 
 
 class fd_config(ctypes.Structure):
@@ -64,6 +64,8 @@ def load() -> ctypes.CDLL:
         lib.fd_selftest_wait_timeout.argtypes = [vp, ci, vp]
         lib.fd_attn_draft_verify_blocks.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_select_branch.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.fd_plan_pin.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp]
+        lib.fd_plan_unpin.argtypes = [vp]
         lib.fd_kv_append.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp]
         lib.fd_draft_select.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
         lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 14
@@ -134,6 +136,15 @@ def fd_attn_draft_verify_blocks(ctx, batch, total_q_rows, q, kv_cache, num_pages
                                               _ptr(page_table), _ptr(prefix_lens), _ptr(q_lens), _ptr(n_mask),
                                               _ptr(n_blocks), _ptr(out), _stream(stream))
     return _check("fd_attn_draft_verify_blocks", code, raise_on_error)
+
+
+def fd_plan_pin(ctx, batch, total_q_rows, prefix_lens, q_lens, n_mask, n_blocks=None, stream=None, raise_on_error=True) -> int:
+    code = load().fd_plan_pin(ctx, batch, total_q_rows, _ptr(prefix_lens), _ptr(q_lens), _ptr(n_mask), _ptr(n_blocks), _stream(stream))
+    return _check("fd_plan_pin", code, raise_on_error)
+
+
+def fd_plan_unpin(ctx, raise_on_error=True) -> int:
+    return _check("fd_plan_unpin", load().fd_plan_unpin(ctx), raise_on_error)
 
 
 def fd_kv_append(ctx, batch, total_q_rows, k_new, v_new, kv_cache, num_pages, page_table, prefix_lens, q_lens, stream=None,

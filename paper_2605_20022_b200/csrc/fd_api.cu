@@ -26,6 +26,10 @@ struct fd_ctx {
     int max_rows;      // capacity of keys
     void* tc_state;
     long long launches;
+    // a pinned plan: the work list of one step, reused by every attention call with these lengths
+    bool pinned;
+    int pin_batch, pin_rows;
+    const int32_t *pin_pl, *pin_ql, *pin_nm, *pin_nb;
     struct HostStage* host;  // staging for fd_step_host, nullptr until fd_host_reserve
 };
 
@@ -41,14 +45,14 @@ struct HostStage {
 };
 
 // Tile equivalents charged for starting a segment in a CTA's range of the tensor-core kernel (measured:
-// a piece boundary costs about as much time as streaming three tiles).
+// ranges balance best when a segment start is charged about five tiles).
 #ifndef FD_PIECE_COST
-#define FD_PIECE_COST 3
+#define FD_PIECE_COST 5
 #endif
 // Least tiles for which a CTA of the tensor-core kernel gets a range of its own: a small call then runs on
 // fewer CTAs, each with a few tiles, instead of one tile everywhere and many partials to merge.
 #ifndef FD_MIN_RANGE_TILES
-#define FD_MIN_RANGE_TILES 4
+#define FD_MIN_RANGE_TILES 2
 #endif
 
 namespace {
@@ -58,6 +62,23 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 }  // namespace
+
+// The part of the attention parameters that the plan kernel needs (lengths and geometry).
+static fd::AttnParams attn_params(fd_ctx* c, int batch, int total_q_rows, const int32_t* prefix_lens, const int32_t* q_lens,
+                                  const int32_t* n_mask, const int32_t* n_blocks) {
+    fd::AttnParams p = {};
+    p.batch = batch; p.total_q_rows = total_q_rows;
+    p.Hq = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.Hq / p.Hkv; p.d = c->cfg.head_dim;
+    p.max_pages = c->cfg.max_pages_per_seq; p.max_q_len = c->cfg.max_q_len;
+    p.scale_log2e = c->scale_log2e;
+    p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.n_mask = n_mask; p.n_blocks = n_blocks;
+    p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
+    p.q_box_t = fd::q_box_rows(p.G);
+    p.piece_cost = c->attn_path == FD_ATTN_SIMT ? 0 : FD_PIECE_COST;
+    p.min_range_tiles = c->attn_path == FD_ATTN_SIMT ? 1 : FD_MIN_RANGE_TILES;
+    return p;
+}
+
 
 extern "C" {
 
@@ -94,6 +115,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->launches = 0;
     c->tc_state = nullptr;
     c->host = nullptr;
+    c->pinned = false;
     if (cudaGetDevice(&c->device) != cudaSuccess ||
         cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
         delete c;
@@ -269,6 +291,10 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         }
         chk(cudaStreamWaitEvent(s, h->q_ready[b], 0));
         if (l >= 2) chk(cudaStreamWaitEvent(s, h->out_copied[b], 0));
+        if (l == 0 && n_layers > 1) {  // one work list for all layers of the step
+            st = fd_plan_pin(c, batch, total_q_rows, h->pl, h->ql, h->nm, n_blocks_host ? h->nb : nullptr, s);
+            if (st != FD_OK) return st;
+        }
         st = fd_attn_draft_verify_blocks(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
                                          n_blocks_host ? h->nb : nullptr, h->out[b], s);
         chk(cudaEventRecord(h->attn_done[b], s));
@@ -276,6 +302,7 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         chk(cudaMemcpyAsync(static_cast<unsigned char*>(out_host) + (size_t)l * qb, h->out[b], qb, D2H, h->d2h));
         chk(cudaEventRecord(h->out_copied[b], h->d2h));
     }
+    c->pinned = false;  // the commit below changes the lengths
     if (st != FD_OK) return st;
     if (n_layers < 2 && total_cand_rows > 0) {
         chk(cudaMemcpyAsync(h->lg, logits_host, (size_t)total_cand_rows * c->cfg.vocab * 4, H2D, h->h2d));
@@ -327,37 +354,55 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     if ((long long)num_pages * 2 * c->cfg.n_kv_heads * 16 > 0x7fffffffLL) return FD_ERR_UNSUPPORTED;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    fd::AttnParams p;
-    p.batch = batch; p.total_q_rows = total_q_rows; p.num_pages = num_pages;
-    p.Hq = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.Hq / p.Hkv; p.d = c->cfg.head_dim;
-    p.max_pages = c->cfg.max_pages_per_seq; p.max_q_len = c->cfg.max_q_len;
-    p.scale_log2e = c->scale_log2e;
+    fd::AttnParams p = attn_params(c, batch, total_q_rows, prefix_lens, q_lens, n_mask, n_blocks);
+    p.num_pages = num_pages;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.kv = static_cast<const __nv_bfloat16*>(kv_cache);
-    p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.n_mask = n_mask;
-    p.n_blocks = n_blocks;
+    p.page_table = page_table;
     p.out = static_cast<__nv_bfloat16*>(out);
-    p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
-    p.q_box_t = fd::q_box_rows(p.G);
-    p.piece_cost = c->attn_path == FD_ATTN_SIMT ? 0 : FD_PIECE_COST;
-    p.min_range_tiles = c->attn_path == FD_ATTN_SIMT ? 1 : FD_MIN_RANGE_TILES;
 
     const bool tc = c->attn_path == FD_ATTN_TCGEN05 && total_q_rows > 0;  // no rows: the plan alone checks the lengths
     if (tc) {
         if (fd::attn_tc_prepare(&c->tc_state, p) != cudaSuccess) { cudaGetLastError(); return FD_ERR_CUDA; }
     }
-    fd::launch_plan(p, s);
-    if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
+    // a pinned plan serves this call if it was made for exactly these lengths; anything else replaces it
+    const bool reuse = c->pinned && batch == c->pin_batch && total_q_rows == c->pin_rows && prefix_lens == c->pin_pl &&
+                       q_lens == c->pin_ql && n_mask == c->pin_nm && n_blocks == c->pin_nb;
+    if (!reuse) {
+        c->pinned = false;
+        fd::launch_plan(p, s);
         c->launches += 1;
+    }
+    if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
     } else if (tc) {
         fd::launch_attn_tc(c->tc_state, p, s);  // merges split segments in its own epilogue
-        c->launches += 2;
+        c->launches += 1;
     } else {
         fd::launch_attn_simt(p, s);
         fd::launch_merge(p, s);
-        c->launches += 3;
+        c->launches += 2;
     }
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_plan_pin(fd_ctx* c, int batch, int total_q_rows, const int32_t* prefix_lens, const int32_t* q_lens,
+                      const int32_t* n_mask, const int32_t* n_blocks, void* stream) {
+    if (!c || batch <= 0 || total_q_rows < 0) return FD_ERR_INVALID_ARG;
+    if (batch > c->cfg.max_batch || (long long)total_q_rows > (long long)batch * c->cfg.max_q_len) return FD_ERR_INVALID_ARG;
+    if (!prefix_lens || !q_lens || !n_mask) return FD_ERR_INVALID_ARG;
+    const fd::AttnParams p = attn_params(c, batch, total_q_rows, prefix_lens, q_lens, n_mask, n_blocks);
+    fd::launch_plan(p, static_cast<cudaStream_t>(stream));
+    c->launches += 1;
+    c->pinned = true;
+    c->pin_batch = batch; c->pin_rows = total_q_rows;
+    c->pin_pl = prefix_lens; c->pin_ql = q_lens; c->pin_nm = n_mask; c->pin_nb = n_blocks;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_plan_unpin(fd_ctx* c) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    c->pinned = false;
+    return FD_OK;
 }
 
 fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const float* logits,

@@ -143,9 +143,9 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
                 const int slot = 2 * cta + (t == s_c ? 0 : 1);
                 p.part.m[slot * kMaxRows + r] = m;
                 p.part.l[slot * kMaxRows + r] = l;
-                float* o = p.part.o + (long long)slot * D * kMaxRows + r;
+                float4* o = partial_o4(p.part, D, slot, 0, r);
 #pragma unroll
-                for (int c = 0; c < D; ++c) o[c * kMaxRows] = acc[c];
+                for (int c = 0; c < D; c += 4) o[(c >> 2) * kMaxRows] = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
             }
         }
         t = t_end;

@@ -536,6 +536,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         }
         named_bar_sync(1, 256);
         if (s == 1) { a0 = ex[r]; a1 = ex[kMaxRows + r]; }
+        if (tid == 0) TRACE(5, 6, w.piece);
         constexpr int kChunks = D / 64;  // 32-column chunks per softmax group
         const bool do_read = !leave && warp_active;
         // the load warps of this CTA have seen every page id of the segment by now
@@ -549,6 +550,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 tmem_ld32(tmem + lane_base + col_o[0] + col, o0);
                 if (two) tmem_ld32(tmem + lane_base + col_o[1] + col, o1);
                 tc_wait_ld();
+                if (tid == 0) TRACE(5, 11 + 2 * ch, w.piece);
 #pragma unroll
                 for (int k = 0; k < 32; ++k) {
                     o[k] = __uint_as_float(o0[k]) * a0;
@@ -568,11 +570,12 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     }
                     store_cols_bf16<32>(dst, o, 1.f);
                 } else {
-                    float* dst = p.part.o + ((long long)pc.slot * D + col) * kMaxRows + r;
+                    float4* dst = partial_o4(p.part, D, pc.slot, col, r);
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) dst[k * kMaxRows] = o[k];
+                    for (int k = 0; k < 32; k += 4) dst[(k >> 2) * kMaxRows] = make_float4(o[k], o[k + 1], o[k + 2], o[k + 3]);
                 }
             }
+            if (tid == 0) TRACE(5, 12 + 2 * ch, w.piece);
         }
         if (do_read && r < pc.rows && !pc.complete && s == 0) {
             p.part.m[pc.slot * kMaxRows + r] = mm;
@@ -585,14 +588,22 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             const int t0 = w.t - pc.tile0, t1 = t0 + pc.seg_nt;
             int c_first, c_last;
             segment_ctas(cs, p.n_ctas, cta, t0, t1, c_first, c_last);
+            if (tid == 0) TRACE(5, 7, w.piece);
             named_bar_sync(1, 256);
             if (tid == 0) {
                 int last = 0;
                 if (!leave && !*abort) {
                     const int n = segment_pieces(cs, c_first, c_last, t0, t1);
+                    TRACE(5, 8, w.piece);
                     __threadfence();
-                    last = atomicAdd(p.plan.seg_count + pc.b * p.Hkv + pc.kvh, 1) + 1 == n;
-                    if (last) __threadfence();
+                    TRACE(5, 9, w.piece);
+                    int* count = p.plan.seg_count + pc.b * p.Hkv + pc.kvh;
+                    last = atomicAdd(count, 1) + 1 == n;
+                    if (last) {
+                        *count = 0;  // everyone has been counted: ready for the next call that uses this plan
+                        __threadfence();
+                    }
+                    TRACE(5, 10, w.piece);
                 }
                 bars->epi_flag = last;
             }
@@ -654,6 +665,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
+    // a dependent launch behind this one (the next layer's call, when the plan is pinned) may bring its
+    // CTAs in as ours retire and do its own set-up; it waits for this grid to complete before reading anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) CTA_LOG(0);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) CTA_LOG(1);  // the plan kernel has completed and its writes are visible

@@ -34,13 +34,20 @@ struct Plan {
 
 // Partial result of one piece of a (sequence, kv-head) segment, log2 domain:
 //   m[r] = max_j s2[r][j],  l[r] = sum_j exp2(s2[r][j] - m[r]),  O[r][c] = sum_j exp2(s2 - m) V[j][c]
-// with s2 = scale * log2(e) * <q, k>.  Stored column-major (o[c * kMaxRows + r]) so that a
-// thread-per-row kernel reads and writes it coalesced.
+// with s2 = scale * log2(e) * <q, k>.  O is stored in groups of four columns, rows interleaved
+// (o[(c / 4) * kMaxRows + r][c % 4]), so that a thread-per-row kernel moves it with 16-byte
+// accesses that are contiguous across the warp.
 struct PartialView {
-    float* o;  // [slots][d][kMaxRows]
+    float* o;  // [slots][d / 4][kMaxRows][4]
     float* m;  // [slots][kMaxRows]
     float* l;  // [slots][kMaxRows]
 };
+
+// Where row r of partial `slot` keeps columns [col, col + 4) (col a multiple of 4); the next four columns
+// are kMaxRows float4 further on.
+__device__ __forceinline__ float4* partial_o4(const PartialView& part, int d, int slot, int col, int r) {
+    return reinterpret_cast<float4*>(part.o) + ((long long)slot * (d / 4) + (col >> 2)) * kMaxRows + r;
+}
 
 struct AttnParams {
     int batch, total_q_rows, num_pages;
@@ -172,17 +179,18 @@ __device__ inline void merge_row(const AttnParams& p, const CtaStarts& cs, int c
         const int slot = 2 * c + (sc >= t0 ? 0 : 1);
         const float mp = __ldcg(p.part.m + slot * kMaxRows + r);
         const float lp = __ldcg(p.part.l + slot * kMaxRows + r);
-        const float* o = p.part.o + ((long long)slot * D + cg * CW) * kMaxRows + r;
+        const float4* o = partial_o4(p.part, D, slot, cg * CW, r);
         const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
         l += w * lp;
-        constexpr int kBatch = CW < 64 ? CW : 64;  // independent loads in flight per thread
+        float4 v[CW / 4];  // independent 16-byte loads, all in flight together
 #pragma unroll
-        for (int c0 = 0; c0 < CW; c0 += kBatch) {
-            float v[kBatch];
+        for (int k = 0; k < CW / 4; ++k) v[k] = __ldcg(o + k * kMaxRows);
 #pragma unroll
-            for (int k = 0; k < kBatch; ++k) v[k] = __ldcg(o + (c0 + k) * kMaxRows);
-#pragma unroll
-            for (int k = 0; k < kBatch; ++k) acc[c0 + k] += w * v[k];
+        for (int k = 0; k < CW / 4; ++k) {
+            acc[4 * k] += w * v[k].x;
+            acc[4 * k + 1] += w * v[k].y;
+            acc[4 * k + 2] += w * v[k].z;
+            acc[4 * k + 3] += w * v[k].w;
         }
     }
     store_cols_bf16<CW>(dst, acc, 1.f / l);

@@ -43,6 +43,9 @@ __device__ inline void block_scan2(int& a, int& b, int& ta, int& tb, int (*wsum)
 __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     __shared__ int s_fatal;
     __shared__ int wsum[8][2];
+    // copies of the two scans the range search needs, so that its dependent probes are not global loads
+    constexpr int kCache = 1024;
+    __shared__ int s_ct[kCache + 1], s_ne[kCache + 1];
     // let the attention kernel behind us start its set-up now; it waits for our completion before it reads the plan
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int B = p.batch, tid = threadIdx.x;
@@ -73,13 +76,17 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
             p.plan.cu_q[b + 1] = (int)min(rows + q, (long long)0x7fffffff);
             p.plan.cu_tiles[b + 1] = (int)min(tiles + t, (long long)0x7fffffff);
             p.plan.cu_ne[b + 1] = nonempty + ne;
+            if (b < kCache) { s_ct[b + 1] = (int)min(tiles + t, (long long)0x7fffffff); s_ne[b + 1] = nonempty + ne; }
         }
         rows += tq;
         tiles += tt;
         nonempty += tne;
     }
-    if (tid == 0) { p.plan.cu_tiles[0] = 0; p.plan.cu_ne[0] = 0; }
+    if (tid == 0) { p.plan.cu_tiles[0] = 0; p.plan.cu_ne[0] = 0; s_ct[0] = 0; s_ne[0] = 0; }
     __syncthreads();
+    const bool cached = B <= kCache;
+    auto ct_at = [&](int b) -> long long { return cached ? s_ct[b] : __ldcg(p.plan.cu_tiles + b); };
+    auto ne_at = [&](int b) -> long long { return cached ? s_ne[b] : __ldcg(p.plan.cu_ne + b); };
     // Where each attention CTA starts.  Cost position x of a tile: Hkv * (tiles + k * segments started)
     // before it, with a segment's k start-up units ahead of its tiles; CTA c starts at the tile that
     // holds x = c * W / n_ctas (a position inside the start-up units snaps to the segment's first tile).
@@ -96,11 +103,11 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
             int lo = 0, hi = B;   // last b whose span starts at or before x (of equal starts the last: the non-empty one)
             while (hi - lo > 1) {
                 const int mid = (lo + hi) >> 1;
-                const long long w_mid = (long long)p.Hkv * (__ldcg(p.plan.cu_tiles + mid) + k * __ldcg(p.plan.cu_ne + mid));
+                const long long w_mid = (long long)p.Hkv * (ct_at(mid) + k * ne_at(mid));
                 if (w_mid <= x) lo = mid; else hi = mid;
             }
-            const long long ct = __ldcg(p.plan.cu_tiles + lo), nt = __ldcg(p.plan.cu_tiles + lo + 1) - ct;
-            const long long rem = x - (long long)p.Hkv * (ct + k * __ldcg(p.plan.cu_ne + lo));
+            const long long ct = ct_at(lo), nt = ct_at(lo + 1) - ct;
+            const long long rem = x - (long long)p.Hkv * (ct + k * ne_at(lo));
             const long long kvh = rem / (nt + k), r = rem % (nt + k);
             p.plan.cta_start[c] = (int)(p.Hkv * ct + kvh * nt + max(0LL, r - k));
             p.plan.cta_first[c] = lo;

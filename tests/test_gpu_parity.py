@@ -425,3 +425,29 @@ def test_kv_append_matches_oracle_and_feeds_the_attention():
         assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_PAGE
         fd.fd_kv_append(ctx.h, step.batch, T - 1, k_new.cuda(), v_new.cuda(), dkv2, step.num_pages, dpt, dpl, dql)
         assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS
+
+
+def test_pinned_plan_serves_every_layer_and_is_dropped_on_other_lengths():
+    """fd_plan_pin: several attention calls reuse one work list; a call with other lengths recomputes it."""
+    step = wl.workload(2)
+    step2 = wl.make_step("other", step.shape, [300, 500], [20, 7], [16, 0], seed=77)
+    wide = torch.full((2, step.max_pages_per_seq), -1, dtype=torch.int32)   # the context fixes the table width
+    wide[:, :step2.max_pages_per_seq] = step2.page_table
+    step2.page_table = wide
+    with Ctx(step) as ctx:
+        dev = {k: getattr(step, k).cuda() for k in ("page_table", "prefix_lens", "q_lens", "n_mask")}
+        fd.fd_plan_pin(ctx.h, step.batch, step.total_q_rows, dev["prefix_lens"], dev["q_lens"], dev["n_mask"])
+        before = fd.fd_launch_count(ctx.h)
+        for layer in range(3):
+            q, kv = wl.make_q(step, layer), wl.make_kv(step, layer)
+            out = torch.empty(q.shape, dtype=torch.bfloat16, device="cuda")
+            fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, q.cuda(), kv.cuda(), step.num_pages, dev["page_table"],
+                                    dev["prefix_lens"], dev["q_lens"], dev["n_mask"], out)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            assert_close(out.float().cpu().numpy(), oracle_attn(step, q, kv), f"pinned layer {layer}")
+        assert fd.fd_launch_count(ctx.h) - before == 3          # one kernel per call: no plan launches
+        q2, kv2 = wl.make_q(step2), wl.make_kv(step2)
+        got, status = gpu_attn(ctx, step2, q2, kv2)             # other lengths: the pin is dropped, a new plan is made
+        assert status == 0
+        assert_close(got.numpy(), oracle_attn(step2, q2, kv2), "after the pin")
+        fd.fd_plan_unpin(ctx.h)
