@@ -13,6 +13,7 @@ attn_blocks(...) the same with several mask blocks per sequence (all hypotheses,
 select_branch(...) pick the prepared next-draft branch of the accepted length
 kv_append(...)   write the query block's K/V into its pages (append, then attend)
 draft_select(...) draft-side tail: calibrated argmax, confidence, Eq. 5 verify length
+accept_stochastic(...) verification by speculative sampling at temperature > 0 (Sec. 3)
 accept(...)      greedy verification: argmax, accepted length, bonus token (Sec. 3)
 commit(...)      KV commit / rollback by page-table truncation
 """
@@ -142,6 +143,27 @@ def accept(logits, draft_tokens, q_lens, n_mask):
     am = np.zeros((max(R, 1),), np.int32)
     _load().fdo_accept(ctypes.c_int(B), ctypes.c_int(V), _p(lg), _p(dt), _p(ql), _p(nm), _p(acc), _p(bon), _p(am))
     return acc, bon, am[:R]
+
+
+def accept_stochastic(logits, draft_logits, draft_tokens, q_lens, n_mask, temperature, u_accept, u_bonus, want_weights=False):
+    """Speculative sampling (Sec. 3).  Returns (accepted_len [B], bonus_token [B], ratio [R] f64[, weights [B,V] f64])."""
+    lg = np.ascontiguousarray(logits if isinstance(logits, np.ndarray) else logits.cpu().numpy(), dtype=np.float32)
+    dl = None if draft_logits is None else np.ascontiguousarray(
+        draft_logits if isinstance(draft_logits, np.ndarray) else draft_logits.cpu().numpy(), dtype=np.float32)
+    R, V = lg.shape
+    dt, ql, nm = _i32(draft_tokens), _i32(q_lens), _i32(n_mask)
+    ua = np.ascontiguousarray(u_accept if isinstance(u_accept, np.ndarray) else u_accept.cpu().numpy(), dtype=np.float32)
+    ub = np.ascontiguousarray(u_bonus if isinstance(u_bonus, np.ndarray) else u_bonus.cpu().numpy(), dtype=np.float32)
+    B = ql.shape[0]
+    assert int(np.maximum(ql - nm, 0).sum()) == R and dt.shape[0] == R and ua.shape[0] == R and ub.shape[0] == B
+    assert dl is None or dl.shape == lg.shape
+    acc = np.zeros((B,), np.int32); bon = np.zeros((B,), np.int32)
+    ratio = np.zeros((max(R, 1),), np.float64)
+    w = np.zeros((B, V), np.float64) if want_weights else None
+    _load().fdo_accept_stochastic(ctypes.c_int(B), ctypes.c_int(V), _p(lg), None if dl is None else _p(dl), _p(dt), _p(ql), _p(nm),
+                                  ctypes.c_double(temperature), _p(ua), _p(ub), _p(acc), _p(bon), _p(ratio),
+                                  None if w is None else _p(w))
+    return (acc, bon, ratio[:R], w) if want_weights else (acc, bon, ratio[:R])
 
 
 def draft_select(logits, bias, n_mask, n_blocks, threshold, max_blocks):

@@ -16,6 +16,9 @@
  *   - fdo_accept: greedy (temperature 0) reading of the verification rule of
  *     Sec. 3: a draft is accepted while it equals the target argmax, the token at
  *     the first mismatch is the bonus token, committed length = accepted + 1.
+ *   - fdo_accept_stochastic: the same rule at temperature > 0, i.e. speculative
+ *     sampling as Sec. 3 states it (accept by the ratio of target and drafter
+ *     probabilities, bonus from the residual distribution).
  *   - fdo_commit: KV commit / rollback.  The paper only implies it (the clean KV
  *     cache "can be reused across all decoding steps", mask tokens are invisible
  *     to clean tokens); the reading implemented is: keep bonus + accepted drafts,
@@ -263,6 +266,81 @@ void fdo_accept(int B, int V, const float *logits, const int32_t *draft_tokens,
         free(am);
         r0 += C;
     }
+}
+
+/* Verification by speculative sampling (Sec. 3: a draft is accepted "according to the ratio between" the
+ * target distribution p and the drafter distribution q, and at the first rejected position a new token is
+ * drawn "from the residual target distribution"; committed length = accepted + 1.  The rule itself is the
+ * published speculative-sampling algorithm the paper cites).  Rows and draft_tokens as in fdo_accept.
+ *
+ *   p_j = softmax(logits[r0 + j] / T)              target distribution after candidate row j
+ *   q_j = softmax(draft_logits[r0 + j] / T)        distribution draft j + 1 was proposed from, or, with
+ *                                                  draft_logits == NULL, all mass on the proposed token
+ *   for j = 0 .. k-1, x = draft_tokens[r0 + j + 1]:
+ *       accept x  iff  u_accept[r0 + j] < min(1, p_j(x) / q_j(x));  the first rejection ends the loop
+ *   rejected at j:   bonus ~ max(0, p_j - q_j) normalised      all k accepted:   bonus ~ p_k
+ *
+ * Random numbers are inputs: u_accept [R] (the entry of a sequence's last row is unused) and u_bonus [B], all
+ * in [0, 1).  A token is drawn from weights w by inverting the cumulative sum in index order: the first y
+ * with w[0] + .. + w[y] > u * sum(w).  ratio [R] (optional) receives p_j(x) / q_j(x) for every tested draft
+ * (-1 elsewhere) and weights [B, V] (optional) the unnormalised weights the bonus token was drawn from, so
+ * that a test can tell a wrong decision from one that sits on a rounding boundary. */
+void fdo_accept_stochastic(int B, int V, const float *logits, const float *draft_logits, const int32_t *draft_tokens,
+        const int32_t *q_lens, const int32_t *n_mask, double temperature, const float *u_accept,
+        const float *u_bonus, int32_t *accepted_len, int32_t *bonus_token, double *ratio, double *weights)
+{
+    double *p = (double *)malloc(sizeof(double) * (size_t)V);
+    double *q = (double *)malloc(sizeof(double) * (size_t)V);
+    int64_t r0 = 0;
+    for (int b = 0; b < B; ++b) {
+        const int C = q_lens[b] - n_mask[b];
+        if (C <= 0) { accepted_len[b] = -1; bonus_token[b] = -1; continue; }
+        const int k = C - 1;
+        int a = 0, rejected = 0;
+        for (int j = 0; j <= k; ++j) {
+            /* p_j, and q_j where there is a draft to test */
+            const float *row = logits + (r0 + j) * (int64_t)V;
+            double mx = row[0];
+            for (int v = 1; v < V; ++v) if (row[v] > mx) mx = row[v];
+            double z = 0.0;
+            for (int v = 0; v < V; ++v) { p[v] = exp(((double)row[v] - mx) / temperature); z += p[v]; }
+            for (int v = 0; v < V; ++v) p[v] /= z;
+            if (ratio) ratio[r0 + j] = -1.0;
+            if (j == k) break;               /* every draft accepted: the bonus comes from p_k */
+            const int x = draft_tokens[r0 + j + 1];
+            if (draft_logits) {
+                const float *dr = draft_logits + (r0 + j) * (int64_t)V;
+                double dm = dr[0];
+                for (int v = 1; v < V; ++v) if (dr[v] > dm) dm = dr[v];
+                double dz = 0.0;
+                for (int v = 0; v < V; ++v) { q[v] = exp(((double)dr[v] - dm) / temperature); dz += q[v]; }
+                for (int v = 0; v < V; ++v) q[v] /= dz;
+            } else {
+                for (int v = 0; v < V; ++v) q[v] = 0.0;
+                q[x] = 1.0;
+            }
+            const double rho = p[x] / q[x];
+            if (ratio) ratio[r0 + j] = rho;
+            if ((double)u_accept[r0 + j] < (rho < 1.0 ? rho : 1.0)) { ++a; continue; }
+            rejected = 1;
+            for (int v = 0; v < V; ++v) { const double w = p[v] - q[v]; p[v] = w > 0.0 ? w : 0.0; }
+            break;
+        }
+        (void)rejected;
+        /* p now holds the weights of the bonus token: the residual, or p_k */
+        double total = 0.0;
+        for (int v = 0; v < V; ++v) total += p[v];
+        const double target = (double)u_bonus[b] * total;
+        double cum = 0.0;
+        int tok = V - 1;
+        for (int v = 0; v < V; ++v) { cum += p[v]; if (cum > target) { tok = v; break; } }
+        accepted_len[b] = a;
+        bonus_token[b] = tok;
+        if (weights) memcpy(weights + (int64_t)b * V, p, sizeof(double) * (size_t)V);
+        r0 += C;
+    }
+    free(p);
+    free(q);
 }
 
 /* Draft-side tail of the step (Sec. 4.2, Eq. 4; Sec. 4.3 "Selective verification", Eq. 5).  One row of
