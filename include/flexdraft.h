@@ -253,6 +253,31 @@ fd_status fd_verify_accept(fd_ctx* ctx, int batch, int total_cand_rows,
                            int32_t* accepted_len, int32_t* bonus_token, void* stream);
 
 /*
+ * Verification at temperature > 0 by speculative sampling (Sec. 3: a draft is accepted according to the
+ * ratio between the target distribution p and the drafter distribution q; at the first rejected position
+ * the bonus token is drawn from the residual target distribution; committed length = accepted + 1).
+ * Rows and draft_tokens as in fd_verify_accept.  With p_j = softmax(logits[row j] / T) and q_j =
+ * softmax(draft_logits[row j] / T), draft j + 1 = x is accepted iff u_accept[row j] < min(1, p_j(x) / q_j(x));
+ * rejected at j: bonus ~ max(0, p_j - q_j) normalised; all k accepted: bonus ~ p_k.  A token is drawn from
+ * weights w by inverting their cumulative sum in index order at u_bonus[b] * sum(w).
+ *
+ *   logits        device, [R, V] fp32: target logits of the candidate rows
+ *   draft_logits  device, [R, V] fp32 or NULL: row r holds the (calibrated) draft logits the token fed at row
+ *                 r + 1 was proposed from; NULL = the drafter put all its mass on the proposed token
+ *   temperature   > 0
+ *   u_accept      device, [R] fp32 in [0, 1): one uniform per candidate row (a sequence's last row: unused)
+ *   u_bonus       device, [B] fp32 in [0, 1)
+ *   accepted_len, bonus_token   device, [B] int32, out; -1 for a sequence without candidate rows
+ *
+ * Probabilities are formed in fp32; a decision whose two sides differ by less than fp32 rounding may fall
+ * either way.  Lengths that do not add up to R raise FD_DEV_BAD_LENGTHS.
+ */
+fd_status fd_verify_accept_sample(fd_ctx* ctx, int batch, int total_cand_rows, const float* logits,
+                                  const float* draft_logits, const int32_t* draft_tokens, const int32_t* q_lens,
+                                  const int32_t* n_mask, float temperature, const float* u_accept,
+                                  const float* u_bonus, int32_t* accepted_len, int32_t* bonus_token, void* stream);
+
+/*
  * KV commit / rollback.  The paper implies it (the clean-prefix KV cache is reused by
  * every later step, Sec. 4.1 "Inference" and Sec. 4.3 "Decoupled execution"; mask tokens
  * are invisible to clean tokens) without spelling it out; the reading implemented: the

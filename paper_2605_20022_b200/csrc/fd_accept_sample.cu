@@ -1,0 +1,325 @@
+// Verification by speculative sampling (temperature > 0): accept each draft with probability
+// min(1, p(x) / q(x)), draw the bonus token from the residual max(0, p - q) at the first rejection, or from
+// p after the last draft when everything was accepted.  p = softmax(target logits / T), q = softmax(draft
+// logits / T), or all mass on the proposed token when no draft logits are given.  The uniforms are inputs.
+//
+// Two sweeps, both made of 4096-logit chunks:
+//   stats   one CTA per (candidate row, chunk): chunk maximum and sum exp((x - max) / T) of the target row
+//           and of the draft row.  The CTA that delivers a row's last chunk folds them into the row's
+//           (max, Z); the CTA that finishes last of all runs the accept test of every sequence -- it needs
+//           p(x) and q(x) of single tokens only -- and notes which row each bonus token is drawn from.
+//   sample  one CTA per (sequence, chunk): sum of the chunk's weights w(y) (p, p without x, or the clipped
+//           difference).  The CTA that delivers a sequence's last chunk inverts the cumulative sum in index
+//           order: it finds the chunk in which u * total is crossed, recomputes that chunk and finds the token.
+// Every reduction has a fixed order, so results do not depend on timing.
+#include "fd_internal.cuh"
+
+namespace fd {
+
+namespace {
+
+constexpr int kVec = kAcceptChunk / (4 * 256);  // float4 per thread and chunk
+
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Loads this thread's 4 * kVec logits of chunk [c0, c0 + n) of `row_ptr`; -inf past the end.
+__device__ __forceinline__ void load_chunk(const float* base, int n, int tid, float (&x)[4 * kVec]) {
+    const bool vec = (reinterpret_cast<uintptr_t>(base) & 15) == 0;
+#pragma unroll
+    for (int k = 0; k < kVec; ++k) {
+        const int e = 4 * (tid + k * 256);
+        if (vec && e + 3 < n) {
+            const float4 a = __ldcs(reinterpret_cast<const float4*>(base + e));
+            x[4 * k] = a.x; x[4 * k + 1] = a.y; x[4 * k + 2] = a.z; x[4 * k + 3] = a.w;
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) x[4 * k + q] = (e + q < n) ? base[e + q] : -INFINITY;
+        }
+    }
+}
+
+// Block-wide maximum / sum over 256 threads in a fixed order; every thread gets the result.
+__device__ __forceinline__ float block_max(float v, float* sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = sh[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) r = fmaxf(r, sh[w]);
+    return r;
+}
+__device__ __forceinline__ float block_sum(float v, float* sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) r += sh[w];
+    return r;
+}
+
+// (max, sum exp((x - max) * kt)) of this CTA's chunk.
+__device__ __forceinline__ float2 chunk_stats(const float (&x)[4 * kVec], float kt, float* sh) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < 4 * kVec; ++k) m = fmaxf(m, x[k]);
+    m = block_max(m, sh);
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4 * kVec; ++k) s += ex2f((x[k] - m) * kt);  // -inf padding adds 0
+    s = block_sum(s, sh);
+    return make_float2(m, s);
+}
+
+__global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunks) {
+    __shared__ float sh[8];
+    __shared__ bool row_last, last;
+    const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks, tid = threadIdx.x;
+    const int c0 = chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
+    const long long off = (long long)row * p.vocab + c0;
+    float x[4 * kVec];
+    load_chunk(p.logits + off, n, tid, x);
+    const float2 tp = chunk_stats(x, p.kt, sh);
+    float2 dp = make_float2(0.f, 1.f);
+    if (p.draft_logits) {
+        load_chunk(p.draft_logits + off, n, tid, x);
+        dp = chunk_stats(x, p.kt, sh);
+    }
+    if (tid == 0) {
+        p.part[((long long)row * chunks + chunk) * 2] = tp;
+        p.part[((long long)row * chunks + chunk) * 2 + 1] = dp;
+        __threadfence();
+        row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks - 1;
+    }
+    __syncthreads();
+    if (row_last && tid < 64) {  // warp 0: target row, warp 1: draft row
+        __threadfence();
+        const int which = tid >> 5;
+        // the partials of a row are interleaved (target, draft): view one of them with stride 2
+        const float2* part = p.part + (long long)row * chunks * 2 + which;
+        float m = -INFINITY;
+        for (int c = (tid & 31); c < chunks; c += 32) m = fmaxf(m, __ldcg(&part[2 * c].x));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float z = 0.f;
+        for (int c = (tid & 31); c < chunks; c += 32) {
+            const float2 v = __ldcg(part + 2 * c);
+            z += v.y * ex2f((v.x - m) * p.kt);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+        if ((tid & 31) == 0) {
+            p.row_stat[2 * row + which] = make_float2(m, z);
+            if (which == 0) p.row_ticket[row] = 0u;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+
+    // ---- one CTA.  First the accept test of every row against the draft fed at the next row, all rows in
+    //      parallel (each test reads single logits that no cache holds); a sequence's last row has no draft
+    //      to test and its flag is never looked at.
+    for (int r = tid; r < p.total_rows; r += blockDim.x) {
+        bool okf = false;
+        const int xt = r + 1 < p.total_rows ? p.drafts[r + 1] : -1;
+        if ((unsigned)xt < (unsigned)p.vocab) {  // anything else is not a token and cannot be accepted
+            const float2 ts = __ldcg(p.row_stat + 2 * r);
+            const float px = ex2f((p.logits[(long long)r * p.vocab + xt] - ts.x) * p.kt) / ts.y;
+            float qx = 1.f;
+            if (p.draft_logits) {
+                const float2 ds = __ldcg(p.row_stat + 2 * r + 1);
+                qx = ex2f((p.draft_logits[(long long)r * p.vocab + xt] - ds.x) * p.kt) / ds.y;
+            }
+            okf = p.u_accept[r] * qx < px;  // u < min(1, p / q), with u < 1
+        }
+        p.flags[r] = okf ? 1 : 0;
+    }
+    // ---- then a thread per sequence: first candidate row by a scan, accepted length = leading passes
+    __shared__ int carry, wcnt[8], s_bad;
+    if (tid == 0) { carry = 0; s_bad = 0; }
+    __syncthreads();
+    for (int base = 0; base < p.batch; base += blockDim.x) {
+        const int b = base + tid;
+        int C = 0;
+        if (b < p.batch) {
+            C = p.q_lens[b] - p.n_mask[b];
+            if (C < 0 || p.n_mask[b] < 0) { atomicOr(&s_bad, 1); C = 0; }
+        }
+        int inc = C;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, inc, o);
+            if ((tid & 31) >= o) inc += u;
+        }
+        if ((tid & 31) == 31) wcnt[tid >> 5] = inc;
+        __syncthreads();
+        long long offr = carry;
+        for (int w = 0; w < (tid >> 5); ++w) offr += wcnt[w];
+        const long long r0 = offr + inc - C;
+        if (b < p.batch) {
+            int a = -1, srow = -1, mode = 0, xs = -1;
+            if (C > 0 && r0 + C <= p.total_rows) {
+                const int k = C - 1;
+                a = 0;
+                while (a < k && p.flags[r0 + a]) ++a;
+                if (a < k) xs = p.drafts[r0 + a + 1];
+                srow = (int)(r0 + a);
+                mode = (a == k) ? 0 : (p.draft_logits ? 1 : 2);
+                if (mode == 2 && (unsigned)xs >= (unsigned)p.vocab) mode = 0;  // nothing to take out of p
+            }
+            p.accepted[b] = a;
+            if (a < 0) p.bonus[b] = -1;
+            p.seq_info[b] = make_int4(srow, mode, xs, 0);
+        }
+        __syncthreads();
+        if (tid == blockDim.x - 1) carry = (int)min(offr + inc, (long long)0x7fffffff);
+        __syncthreads();
+    }
+    if (tid == 0) {
+        if (s_bad || carry != p.total_rows) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        *p.ticket = 0u;
+    }
+}
+
+// Weight of token y in the distribution the bonus token is drawn from.
+__device__ __forceinline__ float weight(float lt, float ld, int y, int mode, int xs, float2 ts, float2 ds, float kt) {
+    const float pv = ex2f((lt - ts.x) * kt) / ts.y;
+    if (mode == 0) return pv;
+    if (mode == 2) return y == xs ? 0.f : pv;
+    return fmaxf(pv - ex2f((ld - ds.x) * kt) / ds.y, 0.f);
+}
+
+__global__ void __launch_bounds__(256) sv_sample_kernel(SampleParams p, int chunks) {
+    __shared__ float sh[8];
+    __shared__ bool seq_last;
+    __shared__ int s_chunk;
+    __shared__ float s_before;
+    const int b = blockIdx.x / chunks, chunk = blockIdx.x % chunks, tid = threadIdx.x;
+    const int4 info = p.seq_info[b];
+    const int row = info.x, mode = info.y, xs = info.z;
+    if (row < 0) return;  // uniform: no candidate rows, outputs already written
+    const float2 ts = p.row_stat[2 * row], ds = p.row_stat[2 * row + 1];
+    {
+        const int c0 = chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
+        const long long off = (long long)row * p.vocab + c0;
+        float x[4 * kVec], d[4 * kVec];
+        load_chunk(p.logits + off, n, tid, x);
+        if (mode == 1) load_chunk(p.draft_logits + off, n, tid, d);
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < kVec; ++k)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int e = 4 * (tid + k * 256) + q;
+                if (e < n) s += weight(x[4 * k + q], mode == 1 ? d[4 * k + q] : 0.f, c0 + e, mode, xs, ts, ds, p.kt);
+            }
+        s = block_sum(s, sh);
+        if (tid == 0) {
+            p.chunk_w[(long long)b * chunks + chunk] = s;
+            __threadfence();
+            seq_last = atomicAdd(p.seq_ticket + b, 1u) == (unsigned)chunks - 1;
+        }
+    }
+    __syncthreads();
+    if (!seq_last) return;
+    __threadfence();
+    // ---- the chunk in which the cumulative weight passes u * total (one thread: a few dozen chunks)
+    if (tid == 0) {
+        const float* cw = p.chunk_w + (long long)b * chunks;
+        float total = 0.f;
+        for (int c = 0; c < chunks; ++c) total += __ldcg(cw + c);
+        const float target = p.u_bonus[b] * total;
+        float cum = 0.f, before = 0.f;
+        int pick = -1, last_pos = 0;
+        for (int c = 0; c < chunks; ++c) {
+            const float wc = __ldcg(cw + c);
+            if (wc > 0.f) last_pos = c;
+            if (cum + wc > target) { pick = c; before = cum; break; }
+            cum += wc;
+        }
+        if (pick < 0) {  // rounding left the target at or past the total: the last chunk with any weight
+            pick = last_pos;
+            before = 0.f;
+            for (int c = 0; c < pick; ++c) before += __ldcg(cw + c);
+        }
+        s_chunk = pick;
+        s_before = target - before;  // what is left to cross inside the chunk
+        p.seq_ticket[b] = 0u;
+    }
+    __syncthreads();
+    // ---- inside the chunk: thread t owns 16 consecutive tokens; exclusive scan of the thread sums, in order
+    const int c0 = s_chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
+    const float rest = s_before;
+    const long long off = (long long)row * p.vocab + c0;
+    constexpr int kPer = kAcceptChunk / 256;
+    float w[kPer];
+    float mine = 0.f;
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        const int e = tid * kPer + k;
+        w[k] = 0.f;
+        if (e < n) w[k] = weight(p.logits[off + e], mode == 1 ? p.draft_logits[off + e] : 0.f, c0 + e, mode, xs, ts, ds, p.kt);
+        mine += w[k];
+    }
+    __shared__ float wsum[8];
+    __shared__ int s_tok, s_lastpos;
+    float inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float u = __shfl_up_sync(0xffffffffu, inc, o);
+        if ((tid & 31) >= o) inc += u;
+    }
+    if (tid == 0) { s_tok = 0x7fffffff; s_lastpos = -1; }
+    if ((tid & 31) == 31) wsum[tid >> 5] = inc;
+    __syncthreads();
+    float excl = inc - mine;
+    for (int wv = 0; wv < (tid >> 5); ++wv) excl += wsum[wv];
+    // first token whose inclusive cumulative weight exceeds `rest`
+    float cum = excl;
+    int found = 0x7fffffff, lastpos = -1;
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        if (w[k] > 0.f) lastpos = c0 + tid * kPer + k;
+        cum += w[k];
+        if (found == 0x7fffffff && w[k] > 0.f && cum > rest) found = c0 + tid * kPer + k;
+    }
+    if (found != 0x7fffffff) atomicMin(&s_tok, found);
+    if (lastpos >= 0) atomicMax(&s_lastpos, lastpos);
+    __syncthreads();
+    if (tid == 0) p.bonus[b] = s_tok != 0x7fffffff ? s_tok : max(s_lastpos, 0);
+}
+
+__global__ void sv_empty_kernel(SampleParams p) {
+    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) {
+        if (p.q_lens[b] - p.n_mask[b] != 0) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        p.accepted[b] = -1;
+        p.bonus[b] = -1;
+    }
+}
+
+}  // namespace
+
+int launch_accept_sample(const SampleParams& p, cudaStream_t s) {
+    if (p.batch == 0) return 0;
+    if (p.total_rows == 0) { sv_empty_kernel<<<1, 256, 0, s>>>(p); return 1; }
+    const int chunks = (p.vocab + kAcceptChunk - 1) / kAcceptChunk;
+    sv_stats_kernel<<<p.total_rows * chunks, 256, 0, s>>>(p, chunks);
+    sv_sample_kernel<<<p.batch * chunks, 256, 0, s>>>(p, chunks);
+    return 2;
+}
+
+}  // namespace fd

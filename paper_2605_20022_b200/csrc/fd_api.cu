@@ -22,6 +22,12 @@ struct fd_ctx {
     float* ds_sum;
     unsigned int* ds_ticket;
     unsigned int* ds_row_ticket;
+    float2* sv_part;             // speculative-sampling scratch
+    float2* sv_row;
+    unsigned int *sv_row_ticket, *sv_ticket, *sv_seq_ticket;
+    int4* sv_seq;
+    float* sv_chunk_w;
+    unsigned char* sv_flags;
     int* status;
     int max_rows;      // capacity of keys
     void* tc_state;
@@ -154,6 +160,14 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const size_t o_dss = take((size_t)c->max_rows * ds_chunks * sizeof(float));
     const size_t o_dst = take(sizeof(unsigned int));
     const size_t o_dsr = take((size_t)c->max_rows * sizeof(unsigned int));
+    const size_t o_svp = take((size_t)c->max_rows * ds_chunks * 2 * sizeof(float2));
+    const size_t o_svr = take((size_t)c->max_rows * 2 * sizeof(float2));
+    const size_t o_svrt = take((size_t)c->max_rows * sizeof(unsigned int));
+    const size_t o_svt = take(sizeof(unsigned int));
+    const size_t o_svst = take((size_t)B * sizeof(unsigned int));
+    const size_t o_svs = take((size_t)B * sizeof(int4));
+    const size_t o_svw = take((size_t)B * ds_chunks * sizeof(float));
+    const size_t o_svf = take((size_t)c->max_rows);
     const size_t o_stat = take(sizeof(int));
     if (cudaMalloc(&c->pool, off) != cudaSuccess) { cudaGetLastError(); delete c; return FD_ERR_WORKSPACE; }
     if (cudaMemset(c->pool, 0, off) != cudaSuccess) { cudaFree(c->pool); delete c; return FD_ERR_CUDA; }
@@ -174,6 +188,14 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->ds_sum = reinterpret_cast<float*>(c->pool + o_dss);
     c->ds_ticket = reinterpret_cast<unsigned int*>(c->pool + o_dst);
     c->ds_row_ticket = reinterpret_cast<unsigned int*>(c->pool + o_dsr);
+    c->sv_part = reinterpret_cast<float2*>(c->pool + o_svp);
+    c->sv_row = reinterpret_cast<float2*>(c->pool + o_svr);
+    c->sv_row_ticket = reinterpret_cast<unsigned int*>(c->pool + o_svrt);
+    c->sv_ticket = reinterpret_cast<unsigned int*>(c->pool + o_svt);
+    c->sv_seq_ticket = reinterpret_cast<unsigned int*>(c->pool + o_svst);
+    c->sv_seq = reinterpret_cast<int4*>(c->pool + o_svs);
+    c->sv_chunk_w = reinterpret_cast<float*>(c->pool + o_svw);
+    c->sv_flags = c->pool + o_svf;
     c->status = reinterpret_cast<int*>(c->pool + o_stat);
     *out = c;
     return FD_OK;
@@ -423,6 +445,30 @@ fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const floa
     p.keys = c->keys; p.ticket = c->ticket; p.status = c->status;
     fd::launch_accept(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, const float* logits, const float* draft_logits,
+                                  const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask, float temperature,
+                                  const float* u_accept, const float* u_bonus, int32_t* accepted_len, int32_t* bonus_token,
+                                  void* stream) {
+    if (!c || batch < 0 || total_cand_rows < 0 || !(temperature > 0.f)) return FD_ERR_INVALID_ARG;
+    if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
+    if (batch == 0) return total_cand_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
+    if (!q_lens || !n_mask || !accepted_len || !bonus_token || !u_bonus) return FD_ERR_INVALID_ARG;
+    if (total_cand_rows > 0 && (!logits || !draft_tokens || !u_accept)) return FD_ERR_INVALID_ARG;
+    if (!aligned(logits, 4) || !aligned(draft_logits, 4)) return FD_ERR_INVALID_ARG;
+    const long long chunks = (c->cfg.vocab + fd::kAcceptChunk - 1) / fd::kAcceptChunk;
+    if ((long long)total_cand_rows * chunks > 0x7fffffffLL) return FD_ERR_UNSUPPORTED;
+    fd::SampleParams p;
+    p.batch = batch; p.total_rows = total_cand_rows; p.vocab = c->cfg.vocab;
+    p.kt = 1.4426950408889634f / temperature;
+    p.logits = logits; p.draft_logits = draft_logits; p.drafts = draft_tokens; p.q_lens = q_lens; p.n_mask = n_mask;
+    p.u_accept = u_accept; p.u_bonus = u_bonus; p.accepted = accepted_len; p.bonus = bonus_token;
+    p.part = c->sv_part; p.row_stat = c->sv_row; p.row_ticket = c->sv_row_ticket; p.ticket = c->sv_ticket;
+    p.seq_info = c->sv_seq; p.chunk_w = c->sv_chunk_w; p.seq_ticket = c->sv_seq_ticket; p.flags = c->sv_flags;
+    p.status = c->status;
+    c->launches += fd::launch_accept_sample(p, static_cast<cudaStream_t>(stream));
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }
 

@@ -257,6 +257,30 @@ struct AcceptParams {
 };
 void launch_accept(const AcceptParams& p, cudaStream_t s);
 
+struct SampleParams {
+    int batch, total_rows, vocab;
+    float kt;                      // log2(e) / temperature
+    const float* logits;
+    const float* draft_logits;     // may be nullptr: all mass on the proposed token
+    const int32_t* drafts;
+    const int32_t* q_lens;
+    const int32_t* n_mask;
+    const float* u_accept;
+    const float* u_bonus;
+    int32_t* accepted;
+    int32_t* bonus;
+    float2* part;                  // [rows][chunks][2] chunk (max, sum) of the target and of the draft row
+    float2* row_stat;              // [rows][2] row (max, Z)
+    unsigned int* row_ticket;      // [rows], zero between calls
+    unsigned int* ticket;          // [1], zero between calls
+    int4* seq_info;                // [B] (row the bonus is drawn from, mode, rejected token, -)
+    float* chunk_w;                // [B][chunks] weight sums
+    unsigned int* seq_ticket;      // [B], zero between calls
+    unsigned char* flags;          // [rows] accept test passed
+    int* status;
+};
+int launch_accept_sample(const SampleParams& p, cudaStream_t s);  // returns the number of kernels launched
+
 struct AppendParams {
     int batch, total_rows, num_pages, Hkv, d, max_pages;
     const __nv_bfloat16* k_new;

@@ -451,3 +451,79 @@ def test_pinned_plan_serves_every_layer_and_is_dropped_on_other_lengths():
         assert status == 0
         assert_close(got.numpy(), oracle_attn(step2, q2, kv2), "after the pin")
         fd.fd_plan_unpin(ctx.h)
+
+
+def _stochastic_case(seed, V, B, T, with_q, max_c=8):
+    rng = np.random.default_rng(seed)
+    C = rng.integers(0, max_c + 1, size=B); C[0] = max_c; C[-1] = 1
+    M = rng.integers(0, 4, size=B)
+    R = int(C.sum())
+    logits = (rng.normal(size=(R, V)) * 2.0).astype(np.float32)
+    dlog = (logits + rng.normal(size=(R, V)).astype(np.float32) * 0.7).astype(np.float32)
+    drafts = rng.integers(0, V, size=R).astype(np.int32)
+    for r in range(R - 1):                                   # proposals drawn from q (or its argmax): mostly accepted
+        z = (dlog[r].astype(np.float64) - dlog[r].max()) / T
+        if with_q:
+            pr = np.exp(z); pr /= pr.sum()
+            drafts[r + 1] = rng.choice(V, p=pr)
+        else:
+            drafts[r + 1] = int(np.argmax(logits[r])) if rng.random() < 0.7 else int(rng.integers(0, V))
+    ua = rng.random(R, dtype=np.float32); ub = rng.random(B, dtype=np.float32)
+    return (C + M).astype(np.int32), M.astype(np.int32), logits, (dlog if with_q else None), drafts, ua, ub
+
+
+@pytest.mark.parametrize("V,B,T,with_q", [(1000, 33, 1.0, True), (5000, 16, 0.6, True), (5000, 16, 0.3, False),
+                                         (151936, 6, 0.6, True), (151936, 6, 1.0, False)])
+def test_stochastic_verification_matches_oracle(V, B, T, with_q):
+    """fd_verify_accept_sample against the speculative-sampling oracle on the same uniforms.  A decision is compared
+    exactly unless the oracle shows that it sits on a rounding boundary (the kernel forms probabilities in fp32)."""
+    ql, nm, logits, dlog, drafts, ua, ub = _stochastic_case(1234 + V + B, V, B, T, with_q)
+    R = logits.shape[0]
+    acc_ref, bon_ref, ratio, w = oracle.accept_stochastic(logits, dlog, drafts, ql, nm, T, ua, ub, want_weights=True)
+    h = fd.fd_create(32, 8, 128, V, B, 16, 8)
+    try:
+        t = lambda a: torch.from_numpy(a).cuda()
+        acc = torch.full((B,), -7, dtype=torch.int32, device="cuda"); bon = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        for _ in range(2):                                   # twice: the scratch counters must come back to zero
+            fd.fd_verify_accept_sample(h, B, R, t(logits), None if dlog is None else t(dlog), t(drafts), t(ql), t(nm), T, t(ua), t(ub),
+                                       acc, bon)
+            assert fd.fd_last_device_status(h) == 0
+        acc, bon = acc.cpu().numpy(), bon.cpu().numpy()
+    finally:
+        fd.fd_destroy(h)
+    C = ql - nm
+    r0, boundary = 0, 0
+    for b in range(B):
+        if C[b] == 0:
+            assert acc[b] == -1 and bon[b] == -1
+            continue
+        tested = np.arange(r0, r0 + C[b] - 1)
+        near = np.abs(ua[tested] - np.minimum(1.0, ratio[tested])) < 2e-5 + 1e-4 * ratio[tested]
+        if acc[b] != acc_ref[b]:                             # allowed only where the test they part at is a near-tie
+            d = min(int(acc[b]), int(acc_ref[b]))
+            assert 0 <= d < len(tested) and near[d], (b, acc[b], acc_ref[b])
+            boundary += 1
+        else:
+            cdf = np.cumsum(w[b]); tot = cdf[-1]
+            tk = int(bon[b])
+            assert 0 <= tk < V
+            if tk != bon_ref[b]:
+                lo = (cdf[tk - 1] if tk > 0 else 0.0) / tot; hi = cdf[tk] / tot
+                assert w[b][tk] > 0 and lo - 1e-5 <= float(ub[b]) <= hi + 1e-5, (b, tk, bon_ref[b], lo, hi, ub[b])
+                boundary += 1
+        r0 += C[b]
+    assert boundary <= max(1, B // 10), boundary
+
+
+def test_stochastic_verification_errors():
+    h = fd.fd_create(32, 8, 128, 1000, 4, 16, 8)
+    try:
+        z = torch.zeros((8, 1000), dtype=torch.float32, device="cuda"); i4 = torch.zeros((8,), dtype=torch.int32, device="cuda")
+        u = torch.zeros((8,), dtype=torch.float32, device="cuda")
+        assert fd.fd_verify_accept_sample(h, 2, 4, z, None, i4, i4, i4, 0.0, u, u, i4, i4, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        assert fd.fd_verify_accept_sample(h, 2, 4, None, None, i4, i4, i4, 1.0, u, u, i4, i4, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        ql = torch.tensor([3, 2], dtype=torch.int32, device="cuda"); nm = torch.zeros((2,), dtype=torch.int32, device="cuda")
+        fd.fd_verify_accept_sample(h, 2, 4, z, None, i4, ql, nm, 1.0, u, u, i4[:2], i4[2:4])      # 5 rows claimed, 4 given
+        assert fd.fd_last_device_status(h) == fd.FD_DEV_BAD_LENGTHS
+    finally:
+        fd.fd_destroy(h)
