@@ -435,7 +435,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=4, help="0..5, see workload.WORKLOAD_NAMES")
+    ap.add_argument("--workload", type=int, default=4, help="0..6, see workload.WORKLOAD_NAMES")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count of workload 4")
     ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel")
     ap.add_argument("--ref-heads", type=int, default=8, help="q-heads in the oracle's timed sample")

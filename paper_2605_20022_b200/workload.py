@@ -56,6 +56,7 @@ WORKLOAD_NAMES = [
     "qwen3_8b_b64_sequential_ragged",
     "qwen3_8b_b16_prefix32768_36layers",
     "qwen3_8b_b8_all_hypotheses_c4_4x7",
+    "qwen3_8b_b64_sequential_draft_pass",
 ]
 
 
@@ -144,7 +145,7 @@ def make_step(name: str, shape: Shape, prefix_lens: Sequence[int], q_lens: Seque
 
 
 def workload(idx: int, n_layers: Optional[int] = None) -> Step:
-    """The benchmark workload ``idx`` (0..4)."""
+    """The benchmark workload ``idx`` (0..4), or one of the two extra ones (5, 6)."""
     seed = BASE_SEED + 1000 * (idx + 1)
     g = _cpu_gen(seed)
     if idx == 0:
@@ -175,6 +176,13 @@ def workload(idx: int, n_layers: Optional[int] = None) -> Step:
         st = make_step(WORKLOAD_NAMES[5], QWEN3_8B, n.tolist(), [32] * B, [28] * B, seed, 0.8)
         st.n_blocks = torch.full((B,), 4, dtype=torch.int32)
         return st
+    if idx == 6:
+        # beyond the five benchmark configurations: the draft pass of sequential mode on its own -- the resolved
+        # bonus token and 16 mask tokens against the committed KV of the batch-64 workload (one candidate row,
+        # so the accept call that follows only turns that row's argmax into the next bonus token)
+        B = 64
+        n = _randint(g, 1024, 4096, B)
+        return make_step(WORKLOAD_NAMES[6], QWEN3_8B, n.tolist(), [17] * B, [16] * B, seed, 0.75)
     raise ValueError(f"no workload {idx}")
 
 

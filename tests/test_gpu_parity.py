@@ -21,7 +21,7 @@ def oracle_attn(step, q, kv):
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 6])
 def test_attention_workloads(idx, path):
     step = wl.workload(idx)
     q, kv = wl.make_q(step), wl.make_kv(step)

@@ -37,6 +37,10 @@ def test_lengths_of_the_five_workloads():
     s5 = wl.workload(5)
     assert s5.batch == 8 and (s5.n_blocks == 4).all() and (s5.cand_rows == 4).all() and (s5.n_mask == 28).all()
     check_tables(s5)
+    s6 = wl.workload(6)
+    assert s6.batch == 64 and (s6.cand_rows == 1).all() and (s6.n_mask == 16).all()
+    assert (s6.prefix_lens >= 1024).all() and (s6.prefix_lens <= 4096).all()
+    check_tables(s6)
     # same seed -> same lengths
     assert torch.equal(wl.workload(2).prefix_lens, s2.prefix_lens)
 
