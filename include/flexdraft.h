@@ -135,6 +135,8 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * same four length pointers reuses it instead of recomputing it (a call with anything else recomputes and
  * drops the pin).  The caller must not change the contents of the length arrays while the pin holds
  * (fd_kv_commit does: unpin before the next step), and must unpin after a FD_DEV_TIMEOUT status.
+ * A sequence flagged for a page id outside the pool (FD_DEV_BAD_PAGE) stays flagged, and its rows zero,
+ * for every call served by the same pin.
  * The paper does not describe a work list; this follows from "all layers of a step share the lengths".
  *
  *   prefix_lens, q_lens, n_mask   device, [B] int32;  n_blocks   device, [B] int32 or NULL
