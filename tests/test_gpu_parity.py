@@ -224,6 +224,8 @@ def test_long_context_full_size_sampled(path):
     dpt, dpl, dql, dnm = (t.cuda() for t in (step.page_table, step.prefix_lens, step.q_lens, step.n_mask))
     g = torch.Generator().manual_seed(1)
     with Ctx(step, path) as ctx:
+        # as the benchmark does for a multi-layer step: one work list, pinned, for every layer
+        fd.fd_plan_pin(ctx.h, step.batch, step.total_q_rows, dpl, dql, dnm)
         for layer in range(2):
             q = wl.make_q(step, layer, device="cuda")
             kv = wl.make_kv(step, layer, device="cuda")
