@@ -541,10 +541,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         const bool do_read = !leave && warp_active;
         // the load warps of this CTA have seen every page id of the segment by now
         const bool zero_rows = pc.complete && !__ldcg(p.plan.seq_ok + pc.b);
+        float o[kChunks][32];  // this thread's row, its group's half of the columns
 #pragma unroll
         for (int ch = 0; ch < kChunks; ++ch) {
             const int col = s * (D / 2) + ch * 32;
-            float o[32];
             if (do_read) {
                 uint32_t o0[32], o1[32];
                 tmem_ld32(tmem + lane_base + col_o[0] + col, o0);
@@ -553,9 +553,12 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 if (tid == 0) TRACE(5, 11 + 2 * ch, w.piece);
 #pragma unroll
                 for (int k = 0; k < 32; ++k) {
-                    o[k] = __uint_as_float(o0[k]) * a0;
-                    if (two) o[k] = fmaf(__uint_as_float(o1[k]), a1, o[k]);
+                    o[ch][k] = __uint_as_float(o0[k]) * a0;
+                    if (two) o[ch][k] = fmaf(__uint_as_float(o1[k]), a1, o[ch][k]);
                 }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) o[ch][k] = 0.f;
             }
             if (ch == kChunks - 1) {
                 tc_fence_before();
@@ -566,13 +569,13 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     __nv_bfloat16* dst = p.out + ((long long)(pc.row0 + i) * p.Hq + pc.kvh * p.G + r % p.G) * D + col;
                     if (zero_rows) {  // by assignment: what was computed from a stand-in page may be inf or NaN
 #pragma unroll
-                        for (int k = 0; k < 32; ++k) o[k] = 0.f;
+                        for (int k = 0; k < 32; ++k) o[ch][k] = 0.f;
                     }
-                    store_cols_bf16<32>(dst, o, 1.f);
+                    store_cols_bf16<32>(dst, o[ch], 1.f);
                 } else {
                     float4* dst = partial_o4(p.part, D, pc.slot, col, r);
 #pragma unroll
-                    for (int k = 0; k < 32; k += 4) dst[(k >> 2) * kMaxRows] = make_float4(o[k], o[k + 1], o[k + 2], o[k + 3]);
+                    for (int k = 0; k < 32; k += 4) dst[(k >> 2) * kMaxRows] = make_float4(o[ch][k], o[ch][k + 1], o[ch][k + 2], o[ch][k + 3]);
                 }
             }
             if (tid == 0) TRACE(5, 12 + 2 * ch, w.piece);
@@ -610,7 +613,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             named_bar_sync(1, 256);
             if (bars->epi_flag & 1) {
                 const int rr = tid & (kMaxRows - 1), cg = tid >> 7;
-                if (rr < pc.rows) merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, t0, t1, rr, cg);
+                // rr == r and cg == s: the columns a thread merges are the ones it has just produced
+                if (rr < pc.rows) merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, t0, t1, rr, cg, &o[0][0], cta);
             }
         }
         if (tid == 0) TRACE(5, 5, w.piece);

@@ -154,9 +154,11 @@ __device__ inline void store_cols_bf16(__nv_bfloat16* dst, const float* o, float
 // row r (output row row0 + r / G), columns [cg * CW, (cg + 1) * CW), in CTA order (fixed, so the result does
 // not depend on timing), and write the bf16 output.  The caller guarantees that every piece has been
 // written and is visible.  A piece that saw no visible key for the row holds m = -inf, l = 0, O = 0.
+// `own` (or nullptr): the O values of CTA own_cta's piece for exactly this row and these columns, still in
+// the caller's registers -- the same numbers it stored, so using them instead of loading changes nothing.
 template <int D, int CW>
 __device__ inline void merge_row(const AttnParams& p, const CtaStarts& cs, int c_first, int c_last, int b, int kvh, int row0,
-                                 int t0, int t1, int r, int cg) {
+                                 int t0, int t1, int r, int cg, const float* own = nullptr, int own_cta = -1) {
     __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
     float acc[CW];
 #pragma unroll
@@ -182,6 +184,11 @@ __device__ inline void merge_row(const AttnParams& p, const CtaStarts& cs, int c
         const float4* o = partial_o4(p.part, D, slot, cg * CW, r);
         const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
         l += w * lp;
+        if (own && c == own_cta) {
+#pragma unroll
+            for (int k = 0; k < CW; ++k) acc[k] += w * own[k];
+            continue;
+        }
         float4 v[CW / 4];  // independent 16-byte loads, all in flight together
 #pragma unroll
         for (int k = 0; k < CW / 4; ++k) v[k] = __ldcg(o + k * kMaxRows);
