@@ -386,6 +386,25 @@ def run_ours(args, step, rank, world, dist):
                       "frac_of_measured_peak": nbytes / ms_dt / 1e6 / peak}
         del dl, db, fl
 
+    # and the verification at temperature > 0 (speculative sampling) over the same candidate rows, with a drafter
+    # distribution: two sweeps of the target and draft logits for the row statistics, one per sequence for the draw
+    sample_row = None
+    if step.total_cand_rows > 0 and rank == 0:
+        R, V = step.total_cand_rows, step.shape.vocab
+        gl = torch.Generator(device=device).manual_seed(step.seed + 500_000)
+        dlg = ds.logits + 0.7 * torch.randn((R, V), generator=gl, device=device)
+        ua = torch.rand((R,), generator=gl, device=device); ub = torch.rand((step.batch,), generator=gl, device=device)
+        acc2 = torch.empty_like(ds.acc); bon2 = torch.empty_like(ds.bon)
+        fl = flush if flush is not None else torch.empty((512 << 20,), dtype=torch.uint8, device=device)
+        call = lambda: fd.fd_verify_accept_sample(ds.ctx, step.batch, R, ds.logits, dlg, ds.drafts, ds.ql, ds.nm, 0.6, ua, ub, acc2, bon2)
+        for _ in range(3):
+            call()
+        ms_sv = timed_region(torch, None, call, 10, fl) / 10
+        nbytes = 2 * (R + step.batch) * V * 4
+        sample_row = {"us": ms_sv * 1e3, "rows": R, "temperature": 0.6, "algorithmic_bytes": nbytes, "GB/s": nbytes / ms_sv / 1e6,
+                      "frac_of_measured_peak": nbytes / ms_sv / 1e6 / peak}
+        del dlg, fl
+
     hs = HostStep(ds)
     for _ in range(2):
         hs.run()
@@ -415,7 +434,8 @@ def run_ours(args, step, rank, world, dist):
                    "l2": "flushed between steps (512 MB write)" if small else "inputs larger than L2 (distinct KV pool per layer)",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU",
                    "parity_vs_oracle_sampled": parity_ok, "device_status": status,
-                   "us_per_step_cuda_graph_replay": us_graph, "draft_tail_fd_draft_select": draft_tail},
+                   "us_per_step_cuda_graph_replay": us_graph, "draft_tail_fd_draft_select": draft_tail,
+                   "sampling_fd_verify_accept_sample": sample_row},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(step.name) if resolved == "tcgen05" else None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
                      "kernel": "fd_attn_draft_verify (plan launch + split-KV attention launch, merge fused)",

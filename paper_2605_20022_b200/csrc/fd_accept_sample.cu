@@ -42,18 +42,7 @@ __device__ __forceinline__ void load_chunk(const float* base, int n, int tid, fl
     }
 }
 
-// Block-wide maximum / sum over 256 threads in a fixed order; every thread gets the result.
-__device__ __forceinline__ float block_max(float v, float* sh) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-    __syncthreads();
-    float r = sh[0];
-#pragma unroll
-    for (int w = 1; w < 8; ++w) r = fmaxf(r, sh[w]);
-    return r;
-}
+// Block-wide sum over 256 threads in a fixed order; every thread gets the result.
 __device__ __forceinline__ float block_sum(float v, float* sh) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -66,36 +55,49 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
     return r;
 }
 
-// (max, sum exp((x - max) * kt)) of this CTA's chunk.
-__device__ __forceinline__ float2 chunk_stats(const float (&x)[4 * kVec], float kt, float* sh) {
+// (max, sum exp((x - max) * kt)) of this CTA's chunk: every warp reduces its own share to (max, sum) with
+// shuffles, thread 0 folds the eight pairs in warp order -- one barrier, fixed order.  `sh` holds 8 float2.
+__device__ __forceinline__ void warp_stats(const float (&x)[4 * kVec], float kt, float2* sh) {
     float m = -INFINITY;
 #pragma unroll
     for (int k = 0; k < 4 * kVec; ++k) m = fmaxf(m, x[k]);
-    m = block_max(m, sh);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float s = 0.f;
+    if (m > -INFINITY) {  // a warp whose share lies wholly past the end of the row has nothing
+#pragma unroll
+        for (int k = 0; k < 4 * kVec; ++k) s += ex2f((x[k] - m) * kt);  // -inf padding adds 0
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = make_float2(m, s);
+}
+__device__ __forceinline__ float2 fold_stats(const float2* sh, float kt) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = fmaxf(m, sh[w].x);
     float s = 0.f;
 #pragma unroll
-    for (int k = 0; k < 4 * kVec; ++k) s += ex2f((x[k] - m) * kt);  // -inf padding adds 0
-    s = block_sum(s, sh);
+    for (int w = 0; w < 8; ++w)
+        if (sh[w].x > -INFINITY) s += sh[w].y * ex2f((sh[w].x - m) * kt);
     return make_float2(m, s);
 }
 
 __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunks) {
-    __shared__ float sh[8];
+    __shared__ float2 sh_t[8], sh_d[8];
     __shared__ bool row_last, last;
     const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks, tid = threadIdx.x;
     const int c0 = chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
     const long long off = (long long)row * p.vocab + c0;
-    float x[4 * kVec];
-    load_chunk(p.logits + off, n, tid, x);
-    const float2 tp = chunk_stats(x, p.kt, sh);
-    float2 dp = make_float2(0.f, 1.f);
-    if (p.draft_logits) {
-        load_chunk(p.draft_logits + off, n, tid, x);
-        dp = chunk_stats(x, p.kt, sh);
-    }
+    float x[4 * kVec], d[4 * kVec];
+    load_chunk(p.logits + off, n, tid, x);                        // both rows' loads are in flight together
+    if (p.draft_logits) load_chunk(p.draft_logits + off, n, tid, d);
+    warp_stats(x, p.kt, sh_t);
+    if (p.draft_logits) warp_stats(d, p.kt, sh_d);
+    __syncthreads();
     if (tid == 0) {
-        p.part[((long long)row * chunks + chunk) * 2] = tp;
-        p.part[((long long)row * chunks + chunk) * 2 + 1] = dp;
+        p.part[((long long)row * chunks + chunk) * 2] = fold_stats(sh_t, p.kt);
+        p.part[((long long)row * chunks + chunk) * 2 + 1] = p.draft_logits ? fold_stats(sh_d, p.kt) : make_float2(0.f, 1.f);
         __threadfence();
         row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks - 1;
     }

@@ -56,30 +56,32 @@ __global__ void __launch_bounds__(256) draft_select_kernel(DraftSelectParams p, 
         const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
         key = other > key ? other : key;
     }
+    // every warp: its maximum (as a key) and the sum of exp(x - that maximum); thread 0 folds the eight
+    // pairs in warp order -- one barrier for the whole chunk
     __shared__ unsigned long long wkey[8];
     __shared__ float wsum[8];
     __shared__ bool last;
-    if ((tid & 31) == 0) wkey[tid >> 5] = key;
-    __syncthreads();
-    key = wkey[0];
-#pragma unroll
-    for (int w = 1; w < 8; ++w) key = wkey[w] > key ? wkey[w] : key;
-    const float m = key_value(key);  // chunk maximum (a chunk is never empty)
+    const float mw = key ? key_value(key) : 0.f;  // a warp wholly past the end of the row has key 0 and adds nothing
     float s = 0.f;
 #pragma unroll
     for (int k = 0; k < kDsVec; ++k)
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-            if (4 * (tid + k * 256) + q < n) s += exp_neg(x[4 * k + q] - m);
+            if (4 * (tid + k * 256) + q < n) s += exp_neg(x[4 * k + q] - mw);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if ((tid & 31) == 0) wsum[tid >> 5] = s;
+    if ((tid & 31) == 0) { wkey[tid >> 5] = key; wsum[tid >> 5] = s; }
     __syncthreads();
     __shared__ bool row_last;
     if (tid == 0) {
+        key = wkey[0];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) key = wkey[w] > key ? wkey[w] : key;
+        const float m = key_value(key);  // chunk maximum (a chunk is never empty)
         float t = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) t += wsum[w];
+        for (int w = 0; w < 8; ++w)
+            if (wkey[w]) t += wsum[w] * exp_neg(key_value(wkey[w]) - m);
         p.part_key[(long long)row * chunks_per_row + chunk] = key;
         p.part_sum[(long long)row * chunks_per_row + chunk] = t;
         __threadfence();
