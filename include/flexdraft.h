@@ -146,6 +146,19 @@ fd_status fd_plan_pin(fd_ctx* ctx, int batch, int total_q_rows, const int32_t* p
 fd_status fd_plan_unpin(fd_ctx* ctx);
 
 /*
+ * Host-side view of the work split, for schedulers and tests: how fd_attn_draft_verify cuts the 128-token KV
+ * tiles of a call (numbered sequence-major, then kv-head, then position) into n_ranges contiguous ranges, one
+ * per CTA of the tensor-core kernel.  Ranges have equal cost, a segment (sequence, kv-head) counting its tiles
+ * plus a fixed start-up charge; a small call leaves the last ranges empty.  Runs on the CPU, touches no GPU.
+ * The paper does not describe a work split; this is this library's own.
+ *
+ *   prefix_lens, q_lens   HOST, [B] int32 (a sequence has ceil((n_b + Lq_b) / 128) tiles per kv-head, none if Lq_b = 0)
+ *   range_start           HOST, [n_ranges + 1] int32, out: first tile of every range; [n_ranges] = all tiles
+ */
+fd_status fd_plan_ranges_host(int batch, int n_kv_heads, const int32_t* prefix_lens, const int32_t* q_lens,
+                              int n_ranges, int32_t* range_start);
+
+/*
  * KV append, the step before the attention ("append, then attend").  The forward pass that verifies the
  * drafts also produces K/V for the query block; they enter the paged cache at logical positions
  * n_b .. n_b + Lq_b - 1 (candidates first, then mask tokens), where fd_attn_draft_verify reads them and

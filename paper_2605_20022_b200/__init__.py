@@ -23,7 +23,7 @@ FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_verify_accept_sample"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_verify_accept_sample", "fd_plan_ranges_host"]
 
 
 class fd_config(ctypes.Structure):
@@ -65,6 +65,7 @@ def load() -> ctypes.CDLL:
         lib.fd_attn_draft_verify_blocks.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_select_branch.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.fd_verify_accept_sample.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
+        lib.fd_plan_ranges_host.argtypes = [ci, ci, vp, vp, ci, vp]
         lib.fd_plan_pin.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp]
         lib.fd_plan_unpin.argtypes = [vp]
         lib.fd_kv_append.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp]
@@ -145,6 +146,16 @@ def fd_verify_accept_sample(ctx, batch, total_cand_rows, logits, draft_logits, d
                                           _ptr(q_lens), _ptr(n_mask), float(temperature), _ptr(u_accept), _ptr(u_bonus),
                                           _ptr(accepted_len), _ptr(bonus_token), _stream(stream))
     return _check("fd_verify_accept_sample", code, raise_on_error)
+
+
+def fd_plan_ranges_host(prefix_lens, q_lens, n_kv_heads: int, n_ranges: int):
+    """Host-only: the first tile of each of the n_ranges ranges (+ the total), as a list of ints."""
+    import numpy as np
+    pl = np.ascontiguousarray(np.asarray(prefix_lens), dtype=np.int32); ql = np.ascontiguousarray(np.asarray(q_lens), dtype=np.int32)
+    out = np.zeros((n_ranges + 1,), np.int32)
+    code = load().fd_plan_ranges_host(int(pl.shape[0]), n_kv_heads, pl.ctypes.data, ql.ctypes.data, n_ranges, out.ctypes.data)
+    _check("fd_plan_ranges_host", code, True)
+    return out.tolist()
 
 
 def fd_plan_pin(ctx, batch, total_q_rows, prefix_lens, q_lens, n_mask, n_blocks=None, stream=None, raise_on_error=True) -> int:

@@ -1,6 +1,7 @@
 // C ABI of libflexdraft: context, argument checks, launch sequencing.
 #include <math.h>
 #include <algorithm>
+#include <vector>
 #include <new>
 
 #include "fd_internal.cuh"
@@ -419,6 +420,36 @@ fd_status fd_plan_pin(fd_ctx* c, int batch, int total_q_rows, const int32_t* pre
     c->pin_batch = batch; c->pin_rows = total_q_rows;
     c->pin_pl = prefix_lens; c->pin_ql = q_lens; c->pin_nm = n_mask; c->pin_nb = n_blocks;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
+}
+
+namespace {
+struct ScanAt {  // read access to a host scan, callable from the host-and-device range cutter
+    const long long* a;
+    __host__ __device__ long long operator()(int b) const { return a[b]; }
+};
+}  // namespace
+
+fd_status fd_plan_ranges_host(int batch, int n_kv_heads, const int32_t* prefix_lens, const int32_t* q_lens, int n_ranges,
+                              int32_t* range_start) {
+    if (batch <= 0 || n_kv_heads <= 0 || n_ranges <= 0 || !prefix_lens || !q_lens || !range_start) return FD_ERR_INVALID_ARG;
+    std::vector<long long> ct(batch + 1, 0), ne(batch + 1, 0);
+    for (int b = 0; b < batch; ++b) {
+        if (prefix_lens[b] < 0 || q_lens[b] < 0) return FD_ERR_INVALID_ARG;
+        const long long t = q_lens[b] > 0 ? ((long long)prefix_lens[b] + q_lens[b] + fd::kTileTokens - 1) / fd::kTileTokens : 0;
+        ct[b + 1] = ct[b] + t;
+        ne[b + 1] = ne[b] + (t > 0);
+    }
+    const long long total = ct[batch] * n_kv_heads, k = FD_PIECE_COST;
+    if (total > 0x7fffffffLL) return FD_ERR_UNSUPPORTED;
+    const long long W = (long long)n_kv_heads * (ct[batch] + k * ne[batch]);
+    const int n_use = fd::ranges_in_use(W, k, FD_MIN_RANGE_TILES, n_ranges);
+    for (int c = 0; c <= n_ranges; ++c) {
+        int first;
+        range_start[c] = (c >= n_use || total == 0)
+                             ? (int)total
+                             : fd::range_cut(c, n_use, W, batch, n_kv_heads, k, ScanAt{ct.data()}, ScanAt{ne.data()}, &first);
+    }
+    return FD_OK;
 }
 
 fd_status fd_plan_unpin(fd_ctx* c) {

@@ -100,6 +100,35 @@ __host__ __device__ inline int q_box_rows(int G) {
     return bt;
 }
 
+// Range cutting (host and device).  Cost position x of a tile: Hkv * (tiles + k * segments started) before
+// it, with a segment's k start-up units ahead of its tiles.  A call worth W units is spread over
+//     n_use = clamp(W / (k + min_range_tiles), 1, n_ranges)
+// ranges; range c starts at the tile that holds x = c * W / n_use (a position inside the start-up units
+// snaps to the segment's first tile).  ct_at(b) / ne_at(b): exclusive scans over the sequences of tiles
+// per kv-head and of "has tiles".  Returns the first tile of range c; *first_seq = the sequence it lies in.
+__host__ __device__ inline int ranges_in_use(long long W, long long k, int min_range_tiles, int n_ranges) {
+    const long long per = k + (min_range_tiles > 1 ? min_range_tiles : 1);
+    long long n = W / per;
+    if (n > n_ranges) n = n_ranges;
+    return (int)(n < 1 ? 1 : n);
+}
+template <class CtAt, class NeAt>
+__host__ __device__ inline int range_cut(int c, int n_use, long long W, int B, int Hkv, long long k, CtAt ct_at, NeAt ne_at,
+                                         int* first_seq) {
+    const long long x = ((long long)c * W) / n_use;
+    int lo = 0, hi = B;  // last b whose span starts at or before x (of equal starts the last: the non-empty one)
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        const long long w_mid = (long long)Hkv * ((long long)ct_at(mid) + k * (long long)ne_at(mid));
+        if (w_mid <= x) lo = mid; else hi = mid;
+    }
+    const long long ct = ct_at(lo), nt = (long long)ct_at(lo + 1) - ct;
+    const long long rem = x - (long long)Hkv * (ct + k * (long long)ne_at(lo));
+    const long long kvh = rem / (nt + k), r = rem % (nt + k);
+    *first_seq = lo;
+    return (int)(Hkv * ct + kvh * nt + (r > k ? r - k : 0));
+}
+
 // View of cta_start: a window of it around the reading CTA may be cached in shared memory.
 constexpr int kCsWindow = 32;
 struct CtaStarts {

@@ -87,29 +87,17 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     const bool cached = B <= kCache;
     auto ct_at = [&](int b) -> long long { return cached ? s_ct[b] : __ldcg(p.plan.cu_tiles + b); };
     auto ne_at = [&](int b) -> long long { return cached ? s_ne[b] : __ldcg(p.plan.cu_ne + b); };
-    // Where each attention CTA starts.  Cost position x of a tile: Hkv * (tiles + k * segments started)
-    // before it, with a segment's k start-up units ahead of its tiles; CTA c starts at the tile that
-    // holds x = c * W / n_ctas (a position inside the start-up units snaps to the segment's first tile).
+    // Where each attention CTA starts (range_cut): a small call is not spread over every CTA -- a range is
+    // worth starting only for a few tiles of work, and every extra range of a segment is one more partial to merge.
     const long long total = tiles * p.Hkv;
     const long long k = p.piece_cost;
     const long long W = (long long)p.Hkv * (tiles + k * nonempty);
-    // a small call is not spread over every CTA: a range is worth starting only for a few tiles of work,
-    // and every extra range of a segment is one more partial to merge
-    const int n_use = (int)max(1LL, min((long long)p.n_ctas, W / (k + max(1, p.min_range_tiles))));
+    const int n_use = ranges_in_use(W, k, p.min_range_tiles, p.n_ctas);
     if (!s_fatal && total > 0 && total <= 0x7fffffffLL) {
         for (int c = tid; c <= p.n_ctas; c += blockDim.x) {
             if (c >= n_use) { p.plan.cta_start[c] = (int)total; if (c < p.n_ctas) p.plan.cta_first[c] = 0; continue; }
-            const long long x = (c * W) / n_use;
-            int lo = 0, hi = B;   // last b whose span starts at or before x (of equal starts the last: the non-empty one)
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                const long long w_mid = (long long)p.Hkv * (ct_at(mid) + k * ne_at(mid));
-                if (w_mid <= x) lo = mid; else hi = mid;
-            }
-            const long long ct = ct_at(lo), nt = ct_at(lo + 1) - ct;
-            const long long rem = x - (long long)p.Hkv * (ct + k * ne_at(lo));
-            const long long kvh = rem / (nt + k), r = rem % (nt + k);
-            p.plan.cta_start[c] = (int)(p.Hkv * ct + kvh * nt + max(0LL, r - k));
+            int lo;
+            p.plan.cta_start[c] = range_cut(c, n_use, W, B, p.Hkv, k, ct_at, ne_at, &lo);
             p.plan.cta_first[c] = lo;
         }
     }
