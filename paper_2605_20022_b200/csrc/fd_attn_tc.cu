@@ -2,8 +2,8 @@
 // tcgen05 MMAs with accumulators in tensor memory, softmax in registers.
 //
 // Work decomposition.  The plan kernel numbers all 128-token KV tiles of the call
-// (sequence-major, then kv-head, then position) and each of the n_ctas persistent CTAs takes
-// one contiguous range, so every SM streams the same number of KV bytes.  A range is walked
+// (sequence-major, then kv-head, then position) and cuts them into one contiguous range per
+// persistent CTA, of equal cost (tiles plus a start-up charge per segment).  A range is walked
 // piece by piece, a piece being its intersection with one (sequence b, kv-head) segment.
 //
 // One piece.  The G * Lq_b <= 128 query rows that share the kv-head (row r = block row
@@ -28,9 +28,10 @@
 //
 // Pieces are pipelined as well: every role walks the CTA's pieces on its own and meets the others only
 // through mbarriers.  The load warps run ahead through the K / V rings; a fourth helper warp brings
-// the next piece's Q tile in (cp.async) as soon as the last QK^T of the current piece has completed;
-// the MMA warp starts the next piece while the softmax groups are still in the epilogue of the
-// current one (the first P V of a piece waits until the epilogue has read O).
+// the next piece's Q tile in (TMA) as soon as the last QK^T of the current piece has completed, has
+// the piece after that prefetched into L2, and publishes every piece's descriptor for the MMA warp and
+// the softmax groups; the MMA warp starts the next piece while the softmax groups are still in the
+// epilogue of the current one (the first P V of a piece waits until the epilogue has read O).
 //
 // Every wait is bounded.  A wait that runs out raises a CTA-wide abort flag: all roles leave
 // their loops, in-flight TMA copies are drained, TMEM is released and FD_DEV_TIMEOUT is set.
