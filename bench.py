@@ -62,7 +62,7 @@ def measured_peaks():
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,clocks.mem,power.draw")
 
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
@@ -82,7 +82,7 @@ class ClockSampler:
         time.sleep(0.15)
         self.proc.terminate()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, mem, power, reasons = [], [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
@@ -95,8 +95,13 @@ class ClockSampler:
             for name, v in zip(names, f[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
+            try:
+                mem.append(float(f[6])); power.append(float(f[7]))
+            except (IndexError, ValueError):
+                pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "mem_mhz": statistics.median(mem) if mem else None,
+                "power_w": statistics.median(power) if power else None}
 
 
 # ----------------------------------------------------------------------------------------------
