@@ -529,3 +529,84 @@ def test_stochastic_verification_errors():
         assert fd.fd_last_device_status(h) == fd.FD_DEV_BAD_LENGTHS
     finally:
         fd.fd_destroy(h)
+
+
+def test_multi_step_decode_loop_append_attend_accept_commit():
+    """Twelve decode steps of a toy target through the C ABI -- KV append, attention, greedy accept, commit with
+    rollback, pages handed back and reused -- against the same loop run on the oracle; both must stay in lockstep
+    (bit-exact lengths, tokens and page tables; attention within tolerance; the cache bit-exact) and commit exactly
+    the greedy sequence of the toy target."""
+    V, B, k, M, steps, P, W = 50, 3, 5, 4, 12, 16, 16
+    Hq, Hkv, d = 8, 2, 128
+    rng = np.random.default_rng(21)
+    table = rng.standard_normal((V, V)).astype(np.float32)
+    nxt = np.argmax(table, axis=1)
+    g = torch.Generator().manual_seed(5)
+    emb_k = torch.randn((V + 1, Hkv, d), generator=g).bfloat16(); emb_v = torch.randn((V + 1, Hkv, d), generator=g).bfloat16()
+    num_pages = 64
+    kv_ref = torch.zeros((num_pages, 2, Hkv, P, d), dtype=torch.bfloat16)          # oracle side cache
+    kv_gpu = kv_ref.clone().cuda()
+    pt = np.full((B, W), -1, np.int32); pl = np.zeros((B,), np.int32)
+    free = list(range(num_pages - 1, -1, -1))
+    bonus = [3, 11, 29]
+    committed = [[] for _ in range(B)]
+    h = fd.fd_create(Hq, Hkv, d, V, B, 16, W)
+    try:
+        for step_i in range(steps):
+            fed_all, ql, nm = [], [], []
+            for b in range(B):
+                drafts, prev = [], bonus[b]
+                for _ in range(k if b != 1 else 2):                                  # ragged: sequence 1 drafts less
+                    t = int(nxt[prev]) if rng.random() < 0.7 else int(rng.integers(V))
+                    drafts.append(t); prev = t
+                fed = [bonus[b]] + drafts
+                m_b = M if b != 2 else 0                                             # sequence 2 runs without mask tokens
+                need = -(-(int(pl[b]) + len(fed) + m_b) // P)
+                for pg in range(need):
+                    if pt[b, pg] < 0:
+                        pt[b, pg] = free.pop()
+                fed_all.append(fed); ql.append(len(fed) + m_b); nm.append(m_b)
+            ql_a, nm_a = np.array(ql, np.int32), np.array(nm, np.int32)
+            tok_rows = [t for b in range(B) for t in fed_all[b] + [V] * nm[b]]      # mask token = extra embedding row V
+            k_new, v_new = emb_k[tok_rows], emb_v[tok_rows]
+            T = len(tok_rows)
+            q = torch.randn((T, Hq, d), generator=g).bfloat16()
+            cand_tok = np.array([t for b in range(B) for t in fed_all[b]], np.int32)
+            logits = table[cand_tok]
+            # oracle side
+            bits = oracle.kv_append(k_new, v_new, kv_ref, pt, pl, ql_a)
+            kv_ref = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+            ref_out = oracle.attn(q, kv_ref, pt, pl, ql_a, nm_a)
+            acc_r, bon_r, _ = oracle.accept(logits, cand_tok, ql_a, nm_a)
+            pt_r, pl_r, freed_r = oracle.commit(pt, pl, ql_a, acc_r)
+            # GPU side
+            t32 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+            dpt, dpl, dql, dnm = t32(pt), t32(pl), t32(ql_a), t32(nm_a)
+            fd.fd_kv_append(h, B, T, k_new.cuda(), v_new.cuda(), kv_gpu, num_pages, dpt, dpl, dql)
+            out = torch.empty((T, Hq, d), dtype=torch.bfloat16, device="cuda")
+            fd.fd_attn_draft_verify(h, B, T, q.cuda(), kv_gpu, num_pages, dpt, dpl, dql, dnm, out)
+            acc = torch.empty((B,), dtype=torch.int32, device="cuda"); bon = torch.empty_like(acc)
+            fd.fd_verify_accept(h, B, len(cand_tok), t32(logits), t32(cand_tok), dql, dnm, acc, bon)
+            freed = torch.full((B * W,), -7, dtype=torch.int32, device="cuda"); nf = torch.zeros((1,), dtype=torch.int32, device="cuda")
+            fd.fd_kv_commit(h, B, dpt, dpl, dql, acc, freed, nf)
+            assert fd.fd_last_device_status(h) == 0
+            assert torch.equal(kv_gpu.cpu().view(torch.int16), kv_ref.view(torch.int16)), f"cache, step {step_i}"
+            assert_close(out.float().cpu().numpy(), ref_out, f"attention, step {step_i}")
+            np.testing.assert_array_equal(acc.cpu().numpy(), acc_r); np.testing.assert_array_equal(bon.cpu().numpy(), bon_r)
+            np.testing.assert_array_equal(dpt.cpu().numpy(), pt_r); np.testing.assert_array_equal(dpl.cpu().numpy(), pl_r)
+            n = int(nf.item())
+            np.testing.assert_array_equal(freed.cpu().numpy()[:n], freed_r)
+            for b in range(B):
+                committed[b] += fed_all[b][:int(acc_r[b]) + 1]
+                bonus[b] = int(bon_r[b])
+            free += freed_r.tolist()[::-1]
+            pt, pl = pt_r, pl_r
+            assert [len(c) for c in committed] == pl.tolist()
+    finally:
+        fd.fd_destroy(h)
+    for b, start in enumerate([3, 11, 29]):                                          # lossless: plain greedy decoding
+        greedy = [start]
+        for _ in range(len(committed[b])):
+            greedy.append(int(nxt[greedy[-1]]))
+        assert committed[b] == greedy[:len(committed[b])] and bonus[b] == greedy[len(committed[b])]
+    assert sorted(free + pt[pt >= 0].tolist()) == list(range(num_pages))
