@@ -610,3 +610,36 @@ def test_multi_step_decode_loop_append_attend_accept_commit():
             greedy.append(int(nxt[greedy[-1]]))
         assert committed[b] == greedy[:len(committed[b])] and bonus[b] == greedy[len(committed[b])]
     assert sorted(free + pt[pt >= 0].tolist()) == list(range(num_pages))
+
+
+def test_stochastic_verification_is_lossless_on_the_gpu():
+    """The defining property, measured on the kernel itself: whatever the drafter proposes, the token committed at
+    the first position is distributed as the target distribution p_0 (98 304 draws, small vocabulary)."""
+    rng = np.random.default_rng(8)
+    V, B, calls, T = 11, 4096, 24, 0.8
+    lp = (rng.normal(size=(2, V)) * 1.5).astype(np.float32)
+    ld = (lp + rng.normal(size=(2, V))).astype(np.float32)
+    sm = lambda x: np.exp((x.astype(np.float64) - x.max()) / T) / np.exp((x.astype(np.float64) - x.max()) / T).sum()
+    p0, q0 = sm(lp[0]), sm(ld[0])
+    logits = torch.from_numpy(np.tile(lp, (B, 1))).cuda(); dlog = torch.from_numpy(np.tile(ld, (B, 1))).cuda()
+    ql = torch.full((B,), 2, dtype=torch.int32, device="cuda"); nm = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    acc = torch.empty((B,), dtype=torch.int32, device="cuda"); bon = torch.empty_like(acc)
+    counts = np.zeros((V,), np.int64); accepted = 0
+    h = fd.fd_create(32, 8, 128, V, B, 16, 8)
+    try:
+        for _ in range(calls):
+            x = rng.choice(V, size=B, p=q0).astype(np.int32)
+            drafts = np.zeros((2 * B,), np.int32); drafts[1::2] = x
+            ua = torch.from_numpy(rng.random(2 * B, dtype=np.float32)).cuda(); ub = torch.from_numpy(rng.random(B, dtype=np.float32)).cuda()
+            fd.fd_verify_accept_sample(h, B, 2 * B, logits, dlog, torch.from_numpy(drafts).cuda(), ql, nm, T, ua, ub, acc, bon)
+            a, bo = acc.cpu().numpy(), bon.cpu().numpy()
+            assert set(np.unique(a)) <= {0, 1}
+            counts += np.bincount(np.where(a == 1, x, bo), minlength=V)
+            accepted += int((a == 1).sum())
+        assert fd.fd_last_device_status(h) == 0
+    finally:
+        fd.fd_destroy(h)
+    n = B * calls
+    freq = counts / n
+    assert np.all(np.abs(freq - p0) < 4.5 * np.sqrt(p0 * (1 - p0) / n) + 1e-9), (freq, p0)
+    assert abs(accepted / n - np.minimum(p0, q0).sum()) < 5e-3
