@@ -143,6 +143,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Warp-uniform bounded wait.
 __device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, volatile int* abort) {
     const bool ok = mbar_wait(bar, parity, abort);
@@ -447,15 +453,15 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                         for (int k = 0; k < 32; ++k)
                             if (ch * 32 + k >= lim && (ch * 32 + k < blo || ch * 32 + k >= bhi)) sv[ch][k] = 0xff800000u;  // -inf by select: S may be NaN there
                 }
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // three-input max: 64 instructions per row
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch)
 #pragma unroll
-                    for (int k = 0; k < 32; k += 4) {
-                        mx[0] = fmaxf(mx[0], __uint_as_float(sv[ch][k]));
-                        mx[1] = fmaxf(mx[1], __uint_as_float(sv[ch][k + 1]));
-                        mx[2] = fmaxf(mx[2], __uint_as_float(sv[ch][k + 2]));
-                        mx[3] = fmaxf(mx[3], __uint_as_float(sv[ch][k + 3]));
+                    for (int k = 0; k < 32; k += 8) {
+                        mx[0] = max3(mx[0], __uint_as_float(sv[ch][k]), __uint_as_float(sv[ch][k + 1]));
+                        mx[1] = max3(mx[1], __uint_as_float(sv[ch][k + 2]), __uint_as_float(sv[ch][k + 3]));
+                        mx[2] = max3(mx[2], __uint_as_float(sv[ch][k + 4]), __uint_as_float(sv[ch][k + 5]));
+                        mx[3] = max3(mx[3], __uint_as_float(sv[ch][k + 6]), __uint_as_float(sv[ch][k + 7]));
                     }
                 const float m_new = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c);
                 if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 1, w.g0 + j);
