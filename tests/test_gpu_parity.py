@@ -50,6 +50,13 @@ EDGE = {
                             [min(1 + (5 * b) % 24, (3 * b) % 17) for b in range(150)]),
     # one CTA range holds the tail of a long segment, whole short ones and the head of another long one
     "long_short_long": (32, 8, 128, [9000, 100, 37, 260, 12000, 5], [32, 4, 17, 32, 32, 9], [16, 0, 1, 16, 16, 0]),
+    # group sizes that are not powers of two: the Q load boxes are 2, 1 and 1 block rows high
+    "gqa3_up_to_32_rows": (6, 2, 128, [300, 1, 2500], [32, 31, 7], [16, 3, 0]),
+    "gqa5_up_to_25_rows": (5, 1, 64, [700, 64], [25, 24], [9, 24]),
+    "gqa6_up_to_21_rows": (12, 2, 128, [129, 4000, 0], [21, 20, 2], [5, 0, 1]),
+    # a call small enough to leave most CTAs without a range, and one that fills exactly one tile
+    "few_ranges": (8, 2, 128, [100, 40], [8, 3], [4, 0]),
+    "exactly_one_tile": (4, 1, 128, [120], [8], [2]),
 }
 
 
