@@ -9,9 +9,11 @@
 // One piece.  The G * Lq_b <= 128 query rows that share the kv-head (row r = block row
 // r / G of q-head kvh * G + r % G) form the M = 128 operand of every MMA, so each KV tile is
 // read from HBM once for all of them.  Per tile j of the piece:
-//     producer warps: one for K, one for V; 16 lanes issue one 2 KB TMA box each (8 pages x two
-//                     64-wide halves of d) into a 128B-swizzled buffer of a 3-deep ring per
-//                     operand; a K buffer is released by the QK^T commit, a V buffer by P V;
+//     producer warps: one for K, one for V; 8 lanes issue one TMA box each -- a whole page of the
+//                     kv-head, both 64-wide halves of d (4 KB: the TMA unit's cost is mostly per
+//                     box, measured 20.9 B/clk per SM with 2 KB boxes, 28.9 with 4 KB) -- into a
+//                     128B-swizzled buffer [8-token group][half][8 rows][128 B] of a 3-deep ring
+//                     per operand; a K buffer is released by the QK^T commit, a V buffer by P V;
 //     MMA warp      : S_s = Q K^T (tcgen05.mma, A and B from shared memory, S in TMEM), and
 //                     after the softmax O_s += P_s V (A = P from TMEM, B = V MN-major);
 //     softmax group : 128 threads, one query row each: tcgen05.ld the row of S, hybrid mask
@@ -63,6 +65,10 @@ struct Cfg {
     static constexpr int kSmemBytes = kExOffset + 1024 + 1024;   // + slack for 1024-byte alignment
     static constexpr int kKSteps = D / 16;
     static constexpr int kHalves = D / 64;
+    // A K or V tile in shared memory: [8-token group][half of d][8 rows][128 B] -- what one TMA box per page
+    // (two groups) lands; for either half the 16 groups lie kGroupBytes apart, the stride the MMA descriptors name.
+    static constexpr int kGroupBytes = kHalves * 1024;
+    static constexpr int kPageBytes = 2 * kGroupBytes;
 };
 
 struct Bars {
@@ -210,8 +216,8 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     using C = Cfg<D>;
     TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
-    constexpr int kOps = 8 * C::kHalves;
-    const int pg = lane / C::kHalves, half = lane % C::kHalves;
+    constexpr int kOps = 8;  // pages of a tile: one box each
+    const int pg = lane;
     int issued = 0;
     // the KV stream is read once: let it leave L2 first, so that Q, the split partials and the page
     // table (all re-read) stay resident next to a stream many times the size of the cache
@@ -248,8 +254,8 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             if (lane == 0) mbar_arrive_expect_tx(&full[st], npg * (16 * D * 2));
             __syncwarp();
             if (lane < kOps && phys >= 0) {
-                unsigned char* dst = ring + st * C::kKBytes + half * (kTileTokens * 128) + pg * 2048;
-                tma_load_2d_hint(dst, &tmap, half * 64, ((phys * 2 + which) * p.Hkv + pc.kvh) * 16, &full[st], policy);
+                unsigned char* dst = ring + st * C::kKBytes + pg * C::kPageBytes;
+                tma_load_4d_hint(dst, &tmap, 0, 0, 0, ((phys * 2 + which) * p.Hkv + pc.kvh) * 2, &full[st], policy);
             }
             issued = g + 1;
         }
@@ -338,7 +344,8 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
                 const int nbad = kTileTokens - valid;
                 for (int e = lane; e < nbad * 8 * C::kHalves; e += 32) {
                     const int r = valid + e / (8 * C::kHalves), wd = e % (8 * C::kHalves);
-                    *reinterpret_cast<uint4*>(vt + (wd >> 3) * (kTileTokens * 128) + r * 128 + ((wd & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(vt + (r >> 3) * C::kGroupBytes + (wd >> 3) * 1024 + (r & 7) * 128 + ((wd & 7) << 4)) =
+                        make_uint4(0, 0, 0, 0);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -352,8 +359,9 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
                 const uint32_t v_addr = smem_u32(vt);
 #pragma unroll
                 for (int kk = 0; kk < kTileTokens / 16; ++kk)
+                    // one page per K step: its two 8-token groups lie kGroupBytes apart, the two halves of d 1 KB apart
                     umma_ts(tmem + col_o[s], tmem + col_s[s] + kk * 8,
-                            make_smem_desc(v_addr + kk * 2048, kTileTokens * 128, 1024), idesc_pv, jj >= 2 || kk > 0);
+                            make_smem_desc(v_addr + kk * C::kPageBytes, 1024, C::kGroupBytes), idesc_pv, jj >= 2 || kk > 0);
                 umma_commit(&bars->v_empty[st]);
                 umma_commit(&bars->pv_done[s]);
             }
@@ -377,8 +385,9 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
                 const uint32_t k_addr = smem_u32(sk + st * C::kKBytes);
 #pragma unroll
                 for (int kk = 0; kk < C::kKSteps; ++kk) {
-                    const uint32_t off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
-                    umma_ss(tmem + col_s[s], make_smem_desc(q_addr + off, 16, 1024), make_smem_desc(k_addr + off, 16, 1024),
+                    const uint32_t q_off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
+                    const uint32_t k_off = (kk >> 2) * 1024 + (kk & 3) * 32;
+                    umma_ss(tmem + col_s[s], make_smem_desc(q_addr + q_off, 16, 1024), make_smem_desc(k_addr + k_off, 16, C::kGroupBytes),
                             idesc_qk, kk > 0);
                 }
                 umma_commit(&bars->k_empty[st]);
@@ -743,8 +752,8 @@ bool attn_tc_supported(int d, int G, int max_q_len) {
     return (d == 64 || d == 128) && G * max_q_len <= kMaxRows;
 }
 
-// Looks up (or encodes) the tensor map of this KV pool: a 2-D view [rows = pages*2*Hkv*16, d]
-// with a 16-row x 64-element box and 128-byte swizzle.
+// Looks up (or encodes) the tensor map of this KV pool: a 4-D view [groups of 8 rows][d / 64 halves][8 rows][64]
+// with a box of one page of one kv-head (two groups, both halves) and 128-byte swizzle.
 cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
     TcState* st = static_cast<TcState*>(*state);
     if (!st) {
@@ -784,11 +793,13 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
     for (int i = 0; i < st->n_cached; ++i)
         if (st->cache[i].ptr == p.kv && st->cache[i].num_pages == p.num_pages) { st->current = &st->cache[i].map; return cudaSuccess; }
     TmapEntry& e = st->cache[st->next];
-    cuuint64_t dims[2] = {(cuuint64_t)p.d, (cuuint64_t)p.num_pages * 2 * p.Hkv * 16};
-    cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
-    cuuint32_t box[2] = {64, 16};
-    cuuint32_t estr[2] = {1, 1};
-    const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(p.kv), dims, strides, box, estr,
+    // 64 elements x 8 rows x the 64-wide halves of d x groups of 8 rows: a box of two groups is one page of one
+    // kv-head and lands as [group][half][8 rows][128 B]
+    cuuint64_t dims[4] = {64, 8, (cuuint64_t)p.d / 64, (cuuint64_t)p.num_pages * 2 * p.Hkv * 2};
+    cuuint64_t strides[3] = {(cuuint64_t)p.d * 2, 128, (cuuint64_t)p.d * 2 * 8};
+    cuuint32_t box[4] = {64, 8, (cuuint32_t)p.d / 64, 2};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(p.kv), dims, strides, box, estr,
                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
