@@ -102,7 +102,8 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
         row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks - 1;
     }
     __syncthreads();
-    if (row_last && tid < 64) {  // warp 0: target row, warp 1: draft row
+    if (!row_last) return;  // only the CTA that completes a row goes on: one fence + count per chunk, not two
+    if (tid < 64) {  // warp 0: target row, warp 1: draft row
         __threadfence();
         const int which = tid >> 5;
         // the partials of a row are interleaved (target, draft): view one of them with stride 2
@@ -124,9 +125,9 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
         }
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid == 0) {  // rows completed so far: whoever completes the last row finishes the call
         __threadfence();
-        last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+        last = atomicAdd(p.ticket, 1u) == (unsigned)p.total_rows - 1;
     }
     __syncthreads();
     if (!last) return;

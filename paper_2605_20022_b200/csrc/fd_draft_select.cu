@@ -19,7 +19,7 @@ __device__ __forceinline__ float exp_neg(float x) {
     return y;
 }
 
-__global__ void __launch_bounds__(256) draft_select_kernel(DraftSelectParams p, int chunks_per_row) {
+__global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams p, int chunks_per_row) {
     const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
     const long long rbase = (long long)row * p.vocab;
     const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
@@ -88,7 +88,8 @@ __global__ void __launch_bounds__(256) draft_select_kernel(DraftSelectParams p, 
         row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks_per_row - 1;
     }
     __syncthreads();
-    if (row_last && tid < 32) {
+    if (!row_last) return;  // only the CTA that completes a row goes on: one fence + count per chunk, not two
+    if (tid < 32) {
         // the CTA that delivers the last chunk of a row finishes the row: lanes over chunks, maximum by an
         // exact reduction, sum of the rescaled chunk sums by a fixed shuffle tree (deterministic)
         __threadfence();
@@ -113,9 +114,9 @@ __global__ void __launch_bounds__(256) draft_select_kernel(DraftSelectParams p, 
         }
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid == 0) {  // rows completed so far: whoever completes the last row finishes the call
         __threadfence();
-        last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+        last = atomicAdd(p.ticket, 1u) == (unsigned)p.total_rows - 1;
     }
     __syncthreads();
     if (!last) return;
