@@ -196,10 +196,11 @@ class DeviceStep:
         B = step.batch
         self.acc = torch.empty((B,), dtype=torch.int32, device=device)
         self.bon = torch.empty((B,), dtype=torch.int32, device=device)
-        self.freed = torch.empty((B * 4,), dtype=torch.int32, device=device)
+        self.max_q_len = max(min(128 // (s.n_q_heads // s.n_kv_heads), 32), int(step.q_lens.max()))
+        self.freed = torch.empty((B * ((self.max_q_len + 15) // 16 + 1),), dtype=torch.int32, device=device)
         self.n_freed = torch.empty((1,), dtype=torch.int32, device=device)
         G = s.n_q_heads // s.n_kv_heads
-        self.ctx = fd.fd_create(s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab, B, min(128 // G, 32),
+        self.ctx = fd.fd_create(s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab, B, self.max_q_len,
                                 step.max_pages_per_seq, s.page_size, 0.0, attn_path)
         self.attn_events = []
 
@@ -496,7 +497,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=4, help="0..6, see workload.WORKLOAD_NAMES")
+    ap.add_argument("--workload", type=int, default=4, help="0..7, see workload.WORKLOAD_NAMES")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count of workload 4")
     ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel")
     ap.add_argument("--ref-heads", type=int, default=8, help="q-heads in the oracle's timed sample")

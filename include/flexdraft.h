@@ -78,7 +78,9 @@ typedef struct {
     int page_size;            /* P: 16 */
     int vocab;                /* V >= 1 */
     int max_batch;            /* largest B of any call; at most 4096 */
-    int max_q_len;            /* largest Lq_b; G * max_q_len <= 128 */
+    int max_q_len;            /* largest Lq_b, <= 4096.  Up to 128 / G block rows share one 128-row MMA tile; a
+                                 longer query block is processed as several such row blocks, each streaming
+                                 the sequence's KV on its own (the O(N^2) regime of preparing every hypothesis) */
     int max_pages_per_seq;    /* row length of page_table */
     float softmax_scale;      /* 0 selects 1/sqrt(d) */
     int attn_path;            /* FD_ATTN_* */

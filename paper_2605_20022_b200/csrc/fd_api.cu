@@ -31,6 +31,7 @@ struct fd_ctx {
     unsigned char* sv_flags;
     int* status;
     int max_rows;      // capacity of keys
+    int max_rb;        // capacity of the row-block arrays of the plan
     void* tc_state;
     long long launches;
     // a pinned plan: the work list of one step, reused by every attention call with these lengths
@@ -77,6 +78,9 @@ static fd::AttnParams attn_params(fd_ctx* c, int batch, int total_q_rows, const 
     p.batch = batch; p.total_q_rows = total_q_rows;
     p.Hq = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.Hq / p.Hkv; p.d = c->cfg.head_dim;
     p.max_pages = c->cfg.max_pages_per_seq; p.max_q_len = c->cfg.max_q_len;
+    p.rb_rows = fd::kMaxRows / p.G;
+    p.rb_per_seq = (p.max_q_len + p.rb_rows - 1) / p.rb_rows;
+    p.max_rb = c->max_rb;
     p.scale_log2e = c->scale_log2e;
     p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.n_mask = n_mask; p.n_blocks = n_blocks;
     p.plan = c->plan; p.part = c->part; p.n_ctas = c->n_ctas; p.status = c->status;
@@ -113,7 +117,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     if (cfg->attn_path < FD_ATTN_AUTO || cfg->attn_path > FD_ATTN_TCGEN05) return FD_ERR_INVALID_ARG;
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
     if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return FD_ERR_UNSUPPORTED;
-    if ((long long)G * cfg->max_q_len > fd::kMaxRows) return FD_ERR_UNSUPPORTED;
+    if (G > fd::kMaxRows || cfg->max_q_len > 4096) return FD_ERR_UNSUPPORTED;  // at least one block row per 128-row tile
     if ((long long)cfg->max_pages_per_seq * 16 > 0x3fffffffLL || cfg->max_batch > 4096) return FD_ERR_UNSUPPORTED;
 
     fd_ctx* c = new (std::nothrow) fd_ctx();
@@ -143,14 +147,19 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->max_rows = (int)std::min<long long>((long long)B * cfg->max_q_len, 0x7fffffffLL);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    // a query block longer than 128 / G rows is handled as several row blocks: size their arrays for the worst case
+    const int rb_rows = fd::kMaxRows / G;
+    c->max_rb = (int)std::min<long long>((long long)B * ((cfg->max_q_len + rb_rows - 1) / rb_rows), 0x7fffffffLL / 64);
+    const size_t NR = (size_t)c->max_rb;
     const size_t o_hdr = take(sizeof(fd::PlanHeader));
-    const size_t o_cuq = take((B + 1) * sizeof(int));
-    const size_t o_cut = take((B + 1) * sizeof(int));
+    const size_t o_rb = take(NR * sizeof(fd::RowBlock));
+    const size_t o_cuq = take((NR + 1) * sizeof(int));
+    const size_t o_cut = take((NR + 1) * sizeof(int));
     const size_t o_ok = take(B * sizeof(int));
-    const size_t o_sc = take((size_t)B * cfg->n_kv_heads * sizeof(int));
+    const size_t o_sc = take(NR * cfg->n_kv_heads * sizeof(int));
     const size_t o_cf = take((size_t)c->n_ctas * sizeof(int));
     const size_t o_cs = take(((size_t)c->n_ctas + 1) * sizeof(int));
-    const size_t o_cne = take((B + 1) * sizeof(int));
+    const size_t o_cne = take((NR + 1) * sizeof(int));
     const size_t o_po = take(slots * d * fd::kMaxRows * sizeof(float));
     const size_t o_pm = take(slots * fd::kMaxRows * sizeof(float));
     const size_t o_pl = take(slots * fd::kMaxRows * sizeof(float));
@@ -173,6 +182,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     if (cudaMalloc(&c->pool, off) != cudaSuccess) { cudaGetLastError(); delete c; return FD_ERR_WORKSPACE; }
     if (cudaMemset(c->pool, 0, off) != cudaSuccess) { cudaFree(c->pool); delete c; return FD_ERR_CUDA; }
     c->plan.hdr = reinterpret_cast<fd::PlanHeader*>(c->pool + o_hdr);
+    c->plan.rb = reinterpret_cast<fd::RowBlock*>(c->pool + o_rb);
     c->plan.cu_q = reinterpret_cast<int*>(c->pool + o_cuq);
     c->plan.cu_tiles = reinterpret_cast<int*>(c->pool + o_cut);
     c->plan.seq_ok = reinterpret_cast<int*>(c->pool + o_ok);

@@ -36,22 +36,24 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
 
     int t = s_c;
     while (t < e_c) {
-        // sequence that owns tile t: last b with Hkv * cu_tiles[b] <= t
-        int lo = 0, hi = p.batch;
+        // row block that owns tile t: last v with Hkv * cu_tiles[v] <= t
+        int lo = 0, hi = hdr.n_rb;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if (p.Hkv * p.plan.cu_tiles[mid] <= t) lo = mid; else hi = mid;
         }
-        const int b = lo;
-        const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
-        const int rem = t - p.Hkv * p.plan.cu_tiles[b];
+        const int v = lo;
+        const RowBlock rb = p.plan.rb[v];
+        const int b = rb.b;
+        const int ntiles = p.plan.cu_tiles[v + 1] - p.plan.cu_tiles[v];
+        const int rem = t - p.Hkv * p.plan.cu_tiles[v];
         const int kvh = rem / ntiles, tile0 = rem % ntiles;
         const int seg_start = t - tile0, seg_end = seg_start + ntiles;
         const int t_end = min(e_c, seg_end);
-        const int n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
-        const int kv_len = n + Lq, rows = Lq * p.G, row0 = p.plan.cu_q[b];
+        const int n = rb.n, Lq = rb.Lq, M = rb.M;
+        const int kv_len = n + Lq, rows = min(p.rb_rows, Lq - rb.i0) * p.G, row0 = p.plan.cu_q[v];
         const int i = r / p.G, g = r % p.G;
-        const RowMask rm = row_mask(i, n, Lq, M, p.n_blocks ? p.n_blocks[b] : 1, r < rows);
+        const RowMask rm = row_mask(rb.i0 + i, n, Lq, M, rb.nb, r < rows);
 
         __syncthreads();  // previous piece is done with qT
         if (r < rows) {

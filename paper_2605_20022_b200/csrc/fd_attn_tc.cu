@@ -87,17 +87,17 @@ constexpr int kDescSlots = 4;
 static_assert(sizeof(Bars) <= 320, "Bars must fit in front of the range-start window");
 
 struct Piece {
-    int b, kvh, tile0, nt, n, Lq, M, nb, kv_len, rows, row0, slot, seg_nt;
+    int v, b, kvh, tile0, nt, n, Lq, M, nb, i0, Lv, kv_len, rows, row0, slot, seg_nt;  // v: row block; Lv: its block rows
     bool complete;
 };
 
-// Piece that starts at tile t.  `b_hint` is a sequence at or before the one that owns t (pieces are
-// walked in order, so the previous piece's sequence will do): a short forward walk replaces a search.
-__device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_c, int e_c, int cta, int b_hint) {
+// Piece that starts at tile t.  `hint` is a row block at or before the one that owns t (pieces are walked in
+// order, so the previous piece's row block will do): a short forward walk replaces a search.
+__device__ __forceinline__ Piece decode_piece(const AttnParams& p, int n_rb, int t, int s_c, int e_c, int cta, int hint) {
     Piece pc;
-    int lo = b_hint;
-    while (lo + 1 < p.batch && p.Hkv * p.plan.cu_tiles[lo + 1] <= t) ++lo;
-    pc.b = lo;
+    int lo = hint;
+    while (lo + 1 < n_rb && p.Hkv * p.plan.cu_tiles[lo + 1] <= t) ++lo;
+    pc.v = lo;
     const int ntiles = p.plan.cu_tiles[lo + 1] - p.plan.cu_tiles[lo];
     const int rem = t - p.Hkv * p.plan.cu_tiles[lo];
     pc.kvh = rem / ntiles;
@@ -106,12 +106,17 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int t, int s_
     const int t_end = min(e_c, seg_end);
     pc.nt = t_end - t;
     pc.seg_nt = ntiles;
-    pc.n = p.prefix_lens[lo];
-    pc.Lq = p.q_lens[lo];
-    pc.M = p.n_mask[lo];
-    pc.nb = p.n_blocks ? p.n_blocks[lo] : 1;
+    const int4* rbp = reinterpret_cast<const int4*>(p.plan.rb + lo);
+    const int4 r0 = rbp[0], r1 = rbp[1];  // (b, i0, n, Lq), (M, nb, -, -)
+    pc.b = r0.x;
+    pc.i0 = r0.y;
+    pc.n = r0.z;
+    pc.Lq = r0.w;
+    pc.M = r1.x;
+    pc.nb = r1.y;
+    pc.Lv = min(p.rb_rows, pc.Lq - pc.i0);
     pc.kv_len = pc.n + pc.Lq;
-    pc.rows = pc.Lq * p.G;
+    pc.rows = pc.Lv * p.G;
     pc.row0 = p.plan.cu_q[lo];
     pc.complete = (t == seg_start) && (t_end == seg_end);
     pc.slot = 2 * cta + (t == s_c ? 0 : 1);
@@ -200,7 +205,7 @@ __device__ __forceinline__ bool wait_piece(Bars* bars, int n, volatile int* abor
 struct Walk {
     int t, g0, u_base[2], piece, b;
     __device__ __forceinline__ void advance(const Piece& pc) {
-        b = pc.b;
+        b = pc.v;  // the row block: the next piece's walk starts from it
         g0 += pc.nt;
         u_base[0] += (pc.nt + 1) >> 1;
         u_base[1] += pc.nt >> 1;
@@ -211,7 +216,7 @@ struct Walk {
 
 // K (which = 0) or V (which = 1) load warp.
 template <int D>
-__device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnParams& p, unsigned char* ring, uint64_t* full,
+__device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnParams& p, int n_rb, unsigned char* ring, uint64_t* full,
                                           uint64_t* empty, int which, int s_c, int e_c, volatile int* abort) {
     using C = Cfg<D>;
     TRACE_DECL;
@@ -225,7 +230,7 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
     bool ok = true;
     while (w.t < e_c && ok) {
-        const Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+        const Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
         const int32_t* table = p.page_table + (long long)pc.b * p.max_pages;
         // Page ids are fetched a batch of four tiles (32 pages, one per lane) at a time and one batch
         // ahead, so the table lookup -- a dependent global load -- never sits between a buffer becoming
@@ -277,20 +282,20 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
 // last box of a piece may reach past the block (rows of the next sequence, or zeros past T): each query
 // row only ever influences its own output row, and those rows are never stored.
 template <int D>
-__device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams& p, unsigned char* sq, Bars* bars, Piece* ring, int s_c, int e_c,
-                                       volatile int* abort) {
+__device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams& p, int n_rb, unsigned char* sq, Bars* bars, Piece* ring,
+                                       int s_c, int e_c, volatile int* abort) {
     using C = Cfg<D>;
     TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     const int bt = p.q_box_t;
     Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
     int issued = 0;
-    Piece pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+    Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
     if (lane == 0) publish_piece(bars, ring, 0, pc);
     while (w.t < e_c) {
         if (w.piece > 0 && !wait_all(&bars->q_free, (w.piece - 1) & 1, abort)) break;
         if (lane == 0) TRACE(6, 0, w.piece);
-        const int nbox = (pc.Lq + bt - 1) / bt;
+        const int nbox = (pc.Lv + bt - 1) / bt;
         if (lane == 0) mbar_arrive_expect_tx(&bars->q_full, nbox * bt * p.G * 128 * C::kHalves);
         __syncwarp();
         for (int e = lane; e < nbox * C::kHalves; e += 32) {
@@ -302,9 +307,9 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
         w.advance(pc);
         if (w.t < e_c) {
             // the next piece: descriptor for the other roles, and its Q rows on their way into L2
-            pc = decode_piece(p, w.t, s_c, e_c, cta, w.b);
+            pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
             if (lane == 0) publish_piece(bars, ring, w.piece, pc);
-            const int nb2 = (pc.Lq + bt - 1) / bt;
+            const int nb2 = (pc.Lv + bt - 1) / bt;
             for (int e = lane; e < nb2 * C::kHalves; e += 32)
                 tma_prefetch_3d(&qmap, (e % C::kHalves) * 64, pc.kvh * p.G, pc.row0 + (e / C::kHalves) * bt);
         }
@@ -430,7 +435,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         if (tid == 0) TRACE(5, 2, w.piece);
         const bool warp_active = (warp & 3) * 32 < pc.rows;
         const int i = r / p.G;
-        const RowMask rm = row_mask(i, pc.n, pc.Lq, pc.M, pc.nb, r < pc.rows);
+        const RowMask rm = row_mask(pc.i0 + i, pc.n, pc.Lq, pc.M, pc.nb, r < pc.rows);
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         // Warps whose 32 rows are all padding do nothing per tile: warp 0 of the group (always active)
@@ -616,7 +621,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     TRACE(5, 8, w.piece);
                     __threadfence();
                     TRACE(5, 9, w.piece);
-                    int* count = p.plan.seg_count + pc.b * p.Hkv + pc.kvh;
+                    int* count = p.plan.seg_count + pc.v * p.Hkv + pc.kvh;
                     last = atomicAdd(count, 1) + 1 == n;
                     if (last) {
                         *count = 0;  // everyone has been counted: ready for the next call that uses this plan
@@ -717,10 +722,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         softmax_role<D>(p, bars, ex, s_cs, cs, ring, tmem, s_c, e_c, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-        if (warp == kKWarp) load_role<D>(tmap, p, sk, bars->k_full, bars->k_empty, 0, s_c, e_c, abort);
-        else if (warp == kVWarp) load_role<D>(tmap, p, sv, bars->v_full, bars->v_empty, 1, s_c, e_c, abort);
+        if (warp == kKWarp) load_role<D>(tmap, p, hdr.n_rb, sk, bars->k_full, bars->k_empty, 0, s_c, e_c, abort);
+        else if (warp == kVWarp) load_role<D>(tmap, p, hdr.n_rb, sv, bars->v_full, bars->v_empty, 1, s_c, e_c, abort);
         else if (warp == kMmaWarp) mma_role<D>(p, sq, sk, sv, bars, ring, tmem, s_c, e_c, abort);
-        else q_role<D>(qmap, p, sq, bars, ring, s_c, e_c, abort);
+        else q_role<D>(qmap, p, hdr.n_rb, sq, bars, ring, s_c, e_c, abort);
     }
     // ---- common tail: everything of this CTA has completed, or it is giving up
     if (*abort && tid == 0) atomicOr(p.status, FD_DEV_TIMEOUT);
@@ -749,7 +754,8 @@ struct TcState {
 }  // namespace
 
 bool attn_tc_supported(int d, int G, int max_q_len) {
-    return (d == 64 || d == 128) && G * max_q_len <= kMaxRows;
+    (void)max_q_len;  // any length: a long query block is cut into row blocks of kMaxRows / G block rows
+    return (d == 64 || d == 128) && G <= kMaxRows;
 }
 
 // Looks up (or encodes) the tensor map of this KV pool: a 4-D view [groups of 8 rows][d / 64 halves][8 rows][64]

@@ -15,20 +15,32 @@ constexpr int kAcceptChunk = 4096; // logits per CTA of the vocab sweep (smaller
 
 // Written by the plan kernel, read by the attention and merge kernels.
 struct PlanHeader {
-    int total_tiles;   // Hkv * sum_b tiles_b
+    int total_tiles;   // Hkv * sum over row blocks of their tiles
     int fatal;         // lengths inconsistent: nothing is computed, out is zeroed
+    int n_rb;          // row blocks of the call
+    int pad;
+};
+
+// A row block: up to rb_rows consecutive block rows of one sequence -- as many as fit the 128-row MMA tile
+// together with their G q-heads.  A sequence whose query block is longer is handled as several row blocks,
+// each streaming the sequence's KV on its own.  Everything the attention kernels index "per sequence" (scans,
+// segments, piece counters) is per row block.
+struct RowBlock {
+    int b, i0;         // sequence, first block row
+    int n, Lq, M, nb;  // the sequence's prefix length, query block length, mask tokens, mask blocks
     int pad[2];
 };
 
 // Device-side view of the plan arrays (all live in the context's scratch memory).
 struct Plan {
     PlanHeader* hdr;
-    int* cu_q;      // [B+1] first query row of each sequence
-    int* cu_tiles;  // [B+1] exclusive scan of tiles_b (per kv-head)
-    int* cu_ne;     // [B+1] exclusive scan of (tiles_b > 0)
+    RowBlock* rb;   // [n_rb] row blocks, sequence-major
+    int* cu_q;      // [n_rb+1] first query row of each row block
+    int* cu_tiles;  // [n_rb+1] exclusive scan of the row blocks' tiles (per kv-head)
+    int* cu_ne;     // [n_rb+1] exclusive scan of (tiles > 0)
     int* seq_ok;    // [B]   0 = a page id of the sequence was outside the pool: its rows are zeroed
-    int* seg_count; // [B * Hkv] partial pieces of a segment that have been written (fused merge)
-    int* cta_first; // [n_ctas] sequence that owns the first tile of each attention CTA's range
+    int* seg_count; // [n_rb * Hkv] partial pieces of a segment that have been written (fused merge)
+    int* cta_first; // [n_ctas] row block that owns the first tile of each attention CTA's range
     int* cta_start; // [n_ctas + 1] first tile of each attention CTA's range (non-decreasing; [n_ctas] = total)
 };
 
@@ -63,6 +75,9 @@ struct AttnParams {
     __nv_bfloat16* out;
     Plan plan;
     PartialView part;
+    int rb_rows;      // block rows per row block: kMaxRows / G
+    int rb_per_seq;   // most row blocks a sequence can have: ceil(max_q_len / rb_rows)
+    int max_rb;       // capacity of the row-block arrays
     int n_ctas;       // CTAs of the attention grid (stream-K ranges are cut for this many)
     int q_box_t;      // block rows per Q load box of the tensor-core kernel (see q_box_rows)
     int min_range_tiles;  // least tiles worth giving a CTA a range of its own

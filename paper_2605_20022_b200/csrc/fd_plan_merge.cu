@@ -14,6 +14,8 @@
 // The plan kernel checks the lengths (O(B) work, one CTA).  Page ids are checked where they are
 // used, by the attention kernels: a sequence with an id outside the pool is flagged in seq_ok,
 // read from page 0 instead, and has its output rows zeroed by the merge kernel.
+#include <algorithm>
+
 #include "fd_internal.cuh"
 
 namespace fd {
@@ -52,31 +54,55 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     if (tid == 0) s_fatal = 0;
     __syncthreads();
     const int P = 16;
-    for (int i = tid; i < B * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
-    long long rows = 0, tiles = 0;  // running totals (identical in every thread)
-    int nonempty = 0;               // sequences with at least one tile so far
+    // ---- pass 1, over sequences: check the lengths, cut every query block into row blocks
+    int n_rb = 0;  // running total (identical in every thread)
     for (int base = 0; base < B; base += blockDim.x) {
         const int b = base + tid;
-        int q = 0, t = 0;
+        int cnt = 0, dummy = 0, tc, td;
+        long long n = 0, Lq = 0, M = 0, nb = 1;
         if (b < B) {
-            const long long n = p.prefix_lens[b], Lq = p.q_lens[b], M = p.n_mask[b];
-            const long long nb = p.n_blocks ? p.n_blocks[b] : 1;
-            bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || Lq * p.G > kMaxRows ||
-                       n + Lq > (long long)p.max_pages * P;
+            n = p.prefix_lens[b]; Lq = p.q_lens[b]; M = p.n_mask[b];
+            nb = p.n_blocks ? p.n_blocks[b] : 1;
+            bool bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || n + Lq > (long long)p.max_pages * P;
             // several mask blocks: equal sizes, and one hypothesis (a candidate row) per block
             bad = bad || nb < 0 || (nb > 1 && (M % nb != 0 || nb > Lq - M));
-            if (bad) atomicOr(&s_fatal, 1);
-            else { q = (int)Lq; t = Lq > 0 ? (int)((n + Lq + kTileTokens - 1) / kTileTokens) : 0; }
+            if (bad) { atomicOr(&s_fatal, 1); Lq = 0; }
+            cnt = Lq > 0 ? (int)((Lq + p.rb_rows - 1) / p.rb_rows) : 1;  // an empty sequence keeps one (empty) row block
             p.plan.seq_ok[b] = 1;
+        }
+        const int mine = cnt;
+        block_scan2(cnt, dummy, tc, td, wsum);
+        if (b < B) {
+            const int v0 = n_rb + cnt - mine;
+            for (int j = 0; j < mine && v0 + j < p.max_rb; ++j) {
+                RowBlock rb = {b, j * p.rb_rows, (int)n, (int)Lq, (int)M, (int)nb, {0, 0}};
+                p.plan.rb[v0 + j] = rb;
+            }
+        }
+        n_rb += tc;
+    }
+    if (n_rb > p.max_rb) { if (tid == 0) atomicOr(&s_fatal, 1); n_rb = p.max_rb; }
+    __syncthreads();
+    for (int i = tid; i < n_rb * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
+    // ---- pass 2, over row blocks: the scans the attention kernels index by
+    long long rows = 0, tiles = 0;  // running totals (identical in every thread)
+    int nonempty = 0;               // row blocks with at least one tile so far
+    for (int base = 0; base < n_rb; base += blockDim.x) {
+        const int v = base + tid;
+        int q = 0, t = 0;
+        if (v < n_rb) {
+            const RowBlock rb = p.plan.rb[v];
+            q = max(0, min(p.rb_rows, rb.Lq - rb.i0));
+            t = q > 0 ? (int)(((long long)rb.n + rb.Lq + kTileTokens - 1) / kTileTokens) : 0;
         }
         int ne = t > 0, dummy = 0, tq, tt, tne, td;
         block_scan2(q, t, tq, tt, wsum);
         block_scan2(ne, dummy, tne, td, wsum);
-        if (b < B) {
-            p.plan.cu_q[b + 1] = (int)min(rows + q, (long long)0x7fffffff);
-            p.plan.cu_tiles[b + 1] = (int)min(tiles + t, (long long)0x7fffffff);
-            p.plan.cu_ne[b + 1] = nonempty + ne;
-            if (b < kCache) { s_ct[b + 1] = (int)min(tiles + t, (long long)0x7fffffff); s_ne[b + 1] = nonempty + ne; }
+        if (v < n_rb) {
+            p.plan.cu_q[v + 1] = (int)min(rows + q, (long long)0x7fffffff);
+            p.plan.cu_tiles[v + 1] = (int)min(tiles + t, (long long)0x7fffffff);
+            p.plan.cu_ne[v + 1] = nonempty + ne;
+            if (v < kCache) { s_ct[v + 1] = (int)min(tiles + t, (long long)0x7fffffff); s_ne[v + 1] = nonempty + ne; }
         }
         rows += tq;
         tiles += tt;
@@ -84,7 +110,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     }
     if (tid == 0) { p.plan.cu_tiles[0] = 0; p.plan.cu_ne[0] = 0; s_ct[0] = 0; s_ne[0] = 0; }
     __syncthreads();
-    const bool cached = B <= kCache;
+    const bool cached = n_rb <= kCache;
     auto ct_at = [&](int b) -> long long { return cached ? s_ct[b] : __ldcg(p.plan.cu_tiles + b); };
     auto ne_at = [&](int b) -> long long { return cached ? s_ne[b] : __ldcg(p.plan.cu_ne + b); };
     // Where each attention CTA starts (range_cut): a small call is not spread over every CTA -- a range is
@@ -97,7 +123,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
         for (int c = tid; c <= p.n_ctas; c += blockDim.x) {
             if (c >= n_use) { p.plan.cta_start[c] = (int)total; if (c < p.n_ctas) p.plan.cta_first[c] = 0; continue; }
             int lo;
-            p.plan.cta_start[c] = range_cut(c, n_use, W, B, p.Hkv, k, ct_at, ne_at, &lo);
+            p.plan.cta_start[c] = range_cut(c, n_use, W, n_rb, p.Hkv, k, ct_at, ne_at, &lo);
             p.plan.cta_first[c] = lo;
         }
     }
@@ -107,6 +133,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
         if (fatal) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         p.plan.hdr->fatal = fatal;
         p.plan.hdr->total_tiles = fatal ? 0 : (int)(tiles * p.Hkv);
+        p.plan.hdr->n_rb = n_rb;
     }
 }
 
@@ -128,22 +155,25 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(AttnParams p) {
             o[i] = make_uint4(0, 0, 0, 0);
         return;
     }
-    const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
-    const int rows = (p.plan.cu_q[b + 1] - p.plan.cu_q[b]) * p.G;
+    const int v = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    if (v >= hdr.n_rb) return;
+    const int rows = (p.plan.cu_q[v + 1] - p.plan.cu_q[v]) * p.G;
     const int r = threadIdx.x % kMaxRows, cg = threadIdx.x / kMaxRows;
     if (r >= rows) return;
-    const int ntiles = p.plan.cu_tiles[b + 1] - p.plan.cu_tiles[b];
+    const int ntiles = p.plan.cu_tiles[v + 1] - p.plan.cu_tiles[v];
     if (ntiles == 0) return;
-    const int t0 = p.Hkv * p.plan.cu_tiles[b] + kvh * ntiles, t1 = t0 + ntiles;
+    const int b = p.plan.rb[v].b;
+    const int t0 = p.Hkv * p.plan.cu_tiles[v] + kvh * ntiles, t1 = t0 + ntiles;
     const CtaStarts cs = {p.plan.cta_start, nullptr, 0};
     const int c_first = range_owner(cs.g, p.n_ctas, t0), c_last = range_owner(cs.g, p.n_ctas, t1 - 1);
     // an unsplit segment was written by the attention kernel itself; it is revisited only to zero it
     if (segment_pieces(cs, c_first, c_last, t0, t1) <= 1 && p.plan.seq_ok[b]) return;
-    merge_row<D, D / 4>(p, cs, c_first, c_last, b, kvh, p.plan.cu_q[b], t0, t1, r, cg);
+    merge_row<D, D / 4>(p, cs, c_first, c_last, b, kvh, p.plan.cu_q[v], t0, t1, r, cg);
 }
 
 void launch_merge(const AttnParams& p, cudaStream_t s) {
-    const int grid = p.batch * p.Hkv;
+    // the number of row blocks is known on the device only: surplus CTAs leave at once
+    const int grid = (int)std::min<long long>((long long)p.batch * p.rb_per_seq, p.max_rb) * p.Hkv;
     if (grid == 0) return;
     if (p.d == 64) merge_kernel<64><<<grid, kMergeThreads, 0, s>>>(p);
     else merge_kernel<128><<<grid, kMergeThreads, 0, s>>>(p);

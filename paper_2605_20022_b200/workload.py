@@ -57,6 +57,7 @@ WORKLOAD_NAMES = [
     "qwen3_8b_b16_prefix32768_36layers",
     "qwen3_8b_b8_all_hypotheses_c4_4x7",
     "qwen3_8b_b64_sequential_draft_pass",
+    "qwen3_8b_b4_all_17_hypotheses_k16",
 ]
 
 
@@ -145,7 +146,7 @@ def make_step(name: str, shape: Shape, prefix_lens: Sequence[int], q_lens: Seque
 
 
 def workload(idx: int, n_layers: Optional[int] = None) -> Step:
-    """The benchmark workload ``idx`` (0..4), or one of the two extra ones (5, 6)."""
+    """The benchmark workload ``idx`` (0..4), or one of the extra ones (5, 6, 7)."""
     seed = BASE_SEED + 1000 * (idx + 1)
     g = _cpu_gen(seed)
     if idx == 0:
@@ -183,6 +184,15 @@ def workload(idx: int, n_layers: Optional[int] = None) -> Step:
         B = 64
         n = _randint(g, 1024, 4096, B)
         return make_step(WORKLOAD_NAMES[6], QWEN3_8B, n.tolist(), [17] * B, [16] * B, seed, 0.75)
+    if idx == 7:
+        # beyond the five benchmark configurations: the paper's parallel mode in full -- bonus + 16 drafts, and one
+        # 16-token next-draft branch for every hypothesis r = 0..16 (Eq. 2): 289 query rows per sequence, which the
+        # kernels process as ten row blocks of 32 block rows, each streaming the sequence's KV
+        B = 4
+        n = _randint(g, 512, 8192, B)
+        st = make_step(WORKLOAD_NAMES[7], QWEN3_8B, n.tolist(), [289] * B, [272] * B, seed, 0.8)
+        st.n_blocks = torch.full((B,), 17, dtype=torch.int32)
+        return st
     raise ValueError(f"no workload {idx}")
 
 

@@ -124,7 +124,7 @@ def test_host_detected_errors_launch_nothing():
     with pytest.raises(fd.FlexDraftError):
         fd.fd_create(32, 8, 96, 1000, 1, 32, 8)             # head_dim 96
     with pytest.raises(fd.FlexDraftError):
-        fd.fd_create(32, 8, 128, 1000, 1, 33, 8)            # G * max_q_len > 128
+        fd.fd_create(32, 8, 128, 1000, 1, 4097, 8)          # max_q_len beyond the supported 4096
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
@@ -311,6 +311,10 @@ BLOCK_CASES = {
     "pruned_and_single": (32, 8, 128, [1000, 77, 300, 4000], [8, 6, 5, 16], [24, 12, 6, 0], [3, 1, 0, 0]),
     "block_straddles_tiles": (8, 2, 128, [120, 250, 383], [4, 4, 4], [28, 28, 28], [4, 2, 4]),
     "head_dim64": (16, 4, 64, [90, 513], [4, 8], [12, 24], [4, 8]),
+    # query blocks longer than one 128-row tile holds (128 / G block rows): several row blocks per sequence.
+    # First sequence = the paper's full parallel mode: bonus + 16 drafts and one 16-token branch per hypothesis.
+    "long_blocks_all_17_hypotheses": (32, 8, 128, [300, 1000, 50, 700, 0], [17, 32, 16, 36, 40], [272, 8, 16, 64, 0], [17, 1, 1, 4, 0]),
+    "long_blocks_gqa8_head_dim64": (16, 2, 64, [200, 31], [9, 20], [36, 30], [9, 2]),
 }
 
 
@@ -324,7 +328,7 @@ def test_attention_mask_blocks(name, path):
     q, kv = wl.make_q(step), wl.make_kv(step, poison=float("nan"))
     n_blocks = torch.tensor(nb, dtype=torch.int32)
     ref = oracle.attn_blocks(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, n_blocks)
-    with Ctx(step, path) as ctx:
+    with Ctx(step, path, max_q_len=max(int(step.q_lens.max()), 1)) as ctx:
         dq, dkv = q.cuda(), kv.cuda()
         out = torch.full_like(dq, float("nan"))
         fd.fd_attn_draft_verify_blocks(ctx.h, step.batch, step.total_q_rows, dq, dkv, step.num_pages, step.page_table.cuda(),

@@ -41,6 +41,9 @@ def test_lengths_of_the_five_workloads():
     assert s6.batch == 64 and (s6.cand_rows == 1).all() and (s6.n_mask == 16).all()
     assert (s6.prefix_lens >= 1024).all() and (s6.prefix_lens <= 4096).all()
     check_tables(s6)
+    s7 = wl.workload(7)
+    assert s7.batch == 4 and (s7.cand_rows == 17).all() and (s7.n_mask == 272).all() and (s7.n_blocks == 17).all()
+    check_tables(s7)
     # same seed -> same lengths
     assert torch.equal(wl.workload(2).prefix_lens, s2.prefix_lens)
 
