@@ -3,53 +3,60 @@
 
 namespace fd {
 
+// How many pages sequence b gives back, or -1 if its entry is inconsistent (left unchanged), 0 if it takes no part.
+__device__ __forceinline__ int pages_released(const CommitParams& p, int b, int& a, int& n, int& Lq) {
+    const int P = p.page_size;
+    a = p.accepted[b]; Lq = p.q_lens[b]; n = p.prefix_lens[b];
+    if (a < 0) return 0;
+    if (a >= Lq || Lq < 0 || n < 0 || (long long)n + Lq > (long long)p.max_pages * P) return -1;
+    return (n + Lq + P - 1) / P - (n + a + 1 + P - 1) / P;
+}
+
 __global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
-    extern __shared__ int s_off[];  // [B+1] exclusive scan of pages freed per sequence
+    __shared__ int wsum[8], carry;
     const int tid = threadIdx.x, P = p.page_size;
-    for (int b = tid; b < p.batch; b += blockDim.x) {
-        const int a = p.accepted[b], Lq = p.q_lens[b], n = p.prefix_lens[b];
-        int cnt = 0;
-        if (a >= 0) {
-            if (a >= Lq || Lq < 0 || n < 0 || (long long)n + Lq > (long long)p.max_pages * P) {
-                atomicOr(p.status, FD_DEV_BAD_ACCEPT);
-                cnt = -1;  // marks "leave unchanged"
-            } else {
-                cnt = (n + Lq + P - 1) / P - (n + a + 1 + P - 1) / P;
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    // sequences in chunks of 256: block scan of the pages each gives back -> its place in the freed list
+    for (int base = 0; base < p.batch; base += blockDim.x) {
+        const int b = base + tid;
+        int a = -1, n = 0, Lq = 0, cnt = 0;
+        if (b < p.batch) {
+            cnt = pages_released(p, b, a, n, Lq);
+            if (cnt < 0) atomicOr(p.status, FD_DEV_BAD_ACCEPT);
+        }
+        const int mine = max(cnt, 0);
+        int inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, inc, o);
+            if ((tid & 31) >= o) inc += u;
+        }
+        if ((tid & 31) == 31) wsum[tid >> 5] = inc;
+        __syncthreads();
+        int off = carry;
+        for (int w = 0; w < (tid >> 5); ++w) off += wsum[w];
+        off += inc - mine;
+        if (b < p.batch && a >= 0 && cnt >= 0) {
+            const int new_len = n + a + 1;
+            const int keep = (new_len + P - 1) / P;
+            int32_t* row = p.page_table + (long long)b * p.max_pages;
+            for (int k = 0; k < cnt; ++k) {
+                p.freed[off + k] = row[keep + k];
+                row[keep + k] = -1;
             }
+            p.prefix_lens[b] = new_len;
         }
-        s_off[b + 1] = cnt;
+        __syncthreads();
+        if (tid == blockDim.x - 1) carry = off + mine;
+        __syncthreads();
     }
-    __syncthreads();
-    if (tid == 0) {
-        int run = 0;
-        s_off[0] = 0;
-        for (int b = 0; b < p.batch; ++b) {
-            const int cnt = s_off[b + 1];
-            s_off[b + 1] = (cnt < 0) ? -(run + 1) : run + cnt;  // negative = skip, still carries the offset
-            run += max(cnt, 0);
-        }
-        *p.n_freed = run;
-    }
-    __syncthreads();
-    for (int b = tid; b < p.batch; b += blockDim.x) {
-        const int a = p.accepted[b];
-        if (a < 0 || s_off[b + 1] < 0) continue;
-        int prev = s_off[b];
-        if (prev < 0) prev = -prev - 1;
-        const int n = p.prefix_lens[b], new_len = n + a + 1;
-        const int keep = (new_len + P - 1) / P, old_pages = (n + p.q_lens[b] + P - 1) / P;
-        int32_t* row = p.page_table + (long long)b * p.max_pages;
-        for (int pg = keep; pg < old_pages; ++pg) {
-            p.freed[prev + (pg - keep)] = row[pg];
-            row[pg] = -1;
-        }
-        p.prefix_lens[b] = new_len;
-    }
+    if (tid == 0) *p.n_freed = carry;
 }
 
 void launch_commit(const CommitParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
-    commit_kernel<<<1, 256, (p.batch + 1) * sizeof(int), s>>>(p);
+    commit_kernel<<<1, 256, 0, s>>>(p);
 }
 
 // KV append: K/V of the query block -> its pages ("append, then attend").  One CTA per sequence; 16-byte copies.
