@@ -57,6 +57,8 @@ EDGE = {
     # a call small enough to leave most CTAs without a range, and one that fills exactly one tile
     "few_ranges": (8, 2, 128, [100, 40], [8, 3], [4, 0]),
     "exactly_one_tile": (4, 1, 128, [120], [8], [2]),
+    # more row blocks than the plan kernel keeps in shared memory (its range search then probes global memory)
+    "batch_1500": (8, 2, 128, [(11 * b) % 37 for b in range(1500)], [1 + b % 3 for b in range(1500)], [b % 2 for b in range(1500)]),
 }
 
 
