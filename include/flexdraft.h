@@ -138,7 +138,9 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * drops the pin).  The caller must not change the contents of the length arrays while the pin holds
  * (fd_kv_commit does: unpin before the next step), and must unpin after a FD_DEV_TIMEOUT status.
  * A sequence flagged for a page id outside the pool (FD_DEV_BAD_PAGE) stays flagged, and its rows zero,
- * for every call served by the same pin.
+ * for every call served by the same pin.  The calls served by a pin must be ordered after fd_plan_pin (the
+ * same stream, or streams the caller has ordered) and must not overlap one another: they share the context's
+ * scratch memory, as all attention calls on one context do.
  * The paper does not describe a work list; this follows from "all layers of a step share the lengths".
  *
  *   prefix_lens, q_lens, n_mask   device, [B] int32;  n_blocks   device, [B] int32 or NULL
