@@ -10,8 +10,12 @@
  *
  * against that sequence's paged KV cache under the hybrid mask, followed, once per
  * step, by lossless verification of the drafts and by the commit / rollback of the KV
- * positions written for this block.  This library exports exactly those three
- * operations.  Everything runs in hand-written CUDA kernels; there is no CPU fallback.
+ * positions written for this block.  This library exports those three operations
+ * (fd_attn_draft_verify, fd_verify_accept, fd_kv_commit) and the steps next to them: the
+ * all-hypotheses form of the attention and the branch selection (Eq. 2), the draft-side
+ * tail (Eq. 4, Eq. 5), verification by sampling at temperature > 0 (Sec. 3), the KV
+ * append, and a whole step from host buffers.  Everything runs in hand-written CUDA
+ * kernels; there is no CPU fallback.
  *
  * Conventions (all entry points)
  *   - "device pointer": memory on the GPU that is current when fd_create() ran, owned
