@@ -199,8 +199,9 @@ fd_status fd_kv_append(fd_ctx* ctx, int batch, int total_q_rows, const void* k_n
  *     A_b(i) for a mask row of block g:  { j < n_b } U { n_b + t : t <= r }  U  { its own block }
  *
  * (candidate row 0 is the known bonus token, candidate t the t-th draft); blocks never see each
- * other; candidate rows are as in fd_attn_draft_verify.  All rows of a sequence still share one
- * M = 128 tile per kv-head, so G * Lq_b <= 128 bounds the number and size of the branches.
+ * other; candidate rows are as in fd_attn_draft_verify.  A query block may be as long as max_q_len
+ * (the paper's full form, bonus + 16 drafts and 17 branches of 16 tokens, is 289 rows): 128 / G block
+ * rows share one MMA tile per kv-head, a longer block is processed in several such row blocks.
  * Lengths that break the rules above zero all T rows (FD_DEV_BAD_LENGTHS).
  */
 fd_status fd_attn_draft_verify_blocks(fd_ctx* ctx, int batch, int total_q_rows,

@@ -1,12 +1,14 @@
 // Tensor-core split-KV attention under the hybrid mask for sm_100a: TMA-staged KV pages,
 // tcgen05 MMAs with accumulators in tensor memory, softmax in registers.
 //
-// Work decomposition.  The plan kernel numbers all 128-token KV tiles of the call
-// (sequence-major, then kv-head, then position) and cuts them into one contiguous range per
-// persistent CTA, of equal cost (tiles plus a start-up charge per segment).  A range is walked
-// piece by piece, a piece being its intersection with one (sequence b, kv-head) segment.
+// Work decomposition.  The plan kernel cuts every sequence's query block into row blocks (as many
+// block rows as fit a 128-row tile with their G q-heads; one per sequence unless the block is long),
+// numbers all 128-token KV tiles of the call (row block, then kv-head, then position) and cuts them
+// into one contiguous range per persistent CTA, of equal cost (tiles plus a start-up charge per
+// segment).  A range is walked piece by piece, a piece being its intersection with one
+// (row block, kv-head) segment.
 //
-// One piece.  The G * Lq_b <= 128 query rows that share the kv-head (row r = block row
+// One piece.  The at most 128 query rows of a row block that share the kv-head (row r = block row
 // r / G of q-head kvh * G + r % G) form the M = 128 operand of every MMA, so each KV tile is
 // read from HBM once for all of them.  Per tile j of the piece:
 //     producer warps: one for K, one for V; 8 lanes issue one TMA box each -- a whole page of the

@@ -10,7 +10,7 @@
 namespace fd {
 
 constexpr int kTileTokens = 128;   // KV tokens per work tile (8 pages of 16)
-constexpr int kMaxRows = 128;      // query rows sharing one kv-head: G * Lq <= 128
+constexpr int kMaxRows = 128;      // query rows of one MMA tile: a row block has kMaxRows / G block rows
 constexpr int kAcceptChunk = 4096; // logits per CTA of the vocab sweep (smaller chunks measured faster: shorter CTA tails)
 
 // Written by the plan kernel, read by the attention and merge kernels.
