@@ -54,7 +54,25 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     if (tid == 0) s_fatal = 0;
     __syncthreads();
     const int P = 16;
+    long long rows = 0, tiles = 0;  // running totals over row blocks (identical in every thread)
+    int nonempty = 0;               // row blocks with at least one tile so far
+    // one 256-wide step of the scans the attention kernels index by: row block v has q block rows and t tiles
+    auto scan_step = [&](int v, bool live, int q, int t) {
+        int ne = t > 0, dummy = 0, tq, tt, tne, td;
+        block_scan2(q, t, tq, tt, wsum);
+        block_scan2(ne, dummy, tne, td, wsum);
+        if (live) {
+            p.plan.cu_q[v + 1] = (int)min(rows + q, (long long)0x7fffffff);
+            p.plan.cu_tiles[v + 1] = (int)min(tiles + t, (long long)0x7fffffff);
+            p.plan.cu_ne[v + 1] = nonempty + ne;
+            if (v < kCache) { s_ct[v + 1] = (int)min(tiles + t, (long long)0x7fffffff); s_ne[v + 1] = nonempty + ne; }
+        }
+        rows += tq;
+        tiles += tt;
+        nonempty += tne;
+    };
     // ---- pass 1, over sequences: check the lengths, cut every query block into row blocks
+    const bool one_each = p.rb_per_seq == 1;  // no block is longer than a row block: sequence b is row block b, one pass
     int n_rb = 0;  // running total (identical in every thread)
     for (int base = 0; base < B; base += blockDim.x) {
         const int b = base + tid;
@@ -70,6 +88,15 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
             cnt = Lq > 0 ? (int)((Lq + p.rb_rows - 1) / p.rb_rows) : 1;  // an empty sequence keeps one (empty) row block
             p.plan.seq_ok[b] = 1;
         }
+        if (one_each) {
+            if (b < B) {
+                RowBlock rb = {b, 0, (int)n, (int)Lq, (int)M, (int)nb, {0, 0}};
+                p.plan.rb[b] = rb;
+            }
+            scan_step(b, b < B, (int)Lq, Lq > 0 ? (int)((n + Lq + kTileTokens - 1) / kTileTokens) : 0);
+            n_rb = B;
+            continue;
+        }
         const int mine = cnt;
         block_scan2(cnt, dummy, tc, td, wsum);
         if (b < B) {
@@ -84,10 +111,8 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     if (n_rb > p.max_rb) { if (tid == 0) atomicOr(&s_fatal, 1); n_rb = p.max_rb; }
     __syncthreads();
     for (int i = tid; i < n_rb * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
-    // ---- pass 2, over row blocks: the scans the attention kernels index by
-    long long rows = 0, tiles = 0;  // running totals (identical in every thread)
-    int nonempty = 0;               // row blocks with at least one tile so far
-    for (int base = 0; base < n_rb; base += blockDim.x) {
+    // ---- pass 2, over row blocks (only where some block was cut)
+    for (int base = 0; base < n_rb && !one_each; base += blockDim.x) {
         const int v = base + tid;
         int q = 0, t = 0;
         if (v < n_rb) {
@@ -95,18 +120,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
             q = max(0, min(p.rb_rows, rb.Lq - rb.i0));
             t = q > 0 ? (int)(((long long)rb.n + rb.Lq + kTileTokens - 1) / kTileTokens) : 0;
         }
-        int ne = t > 0, dummy = 0, tq, tt, tne, td;
-        block_scan2(q, t, tq, tt, wsum);
-        block_scan2(ne, dummy, tne, td, wsum);
-        if (v < n_rb) {
-            p.plan.cu_q[v + 1] = (int)min(rows + q, (long long)0x7fffffff);
-            p.plan.cu_tiles[v + 1] = (int)min(tiles + t, (long long)0x7fffffff);
-            p.plan.cu_ne[v + 1] = nonempty + ne;
-            if (v < kCache) { s_ct[v + 1] = (int)min(tiles + t, (long long)0x7fffffff); s_ne[v + 1] = nonempty + ne; }
-        }
-        rows += tq;
-        tiles += tt;
-        nonempty += tne;
+        scan_step(v, v < n_rb, q, t);
     }
     if (tid == 0) { p.plan.cu_tiles[0] = 0; p.plan.cu_ne[0] = 0; s_ct[0] = 0; s_ne[0] = 0; }
     __syncthreads();
