@@ -198,12 +198,13 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
     }
 }
 
-// Weight of token y in the distribution the bonus token is drawn from.
+// Weight of token y in the distribution the bonus token is drawn from.  ts / ds: (row maximum, 1 / Z) of the target
+// and of the draft row.
 __device__ __forceinline__ float weight(float lt, float ld, int y, int mode, int xs, float2 ts, float2 ds, float kt) {
-    const float pv = ex2f((lt - ts.x) * kt) / ts.y;
+    const float pv = ex2f((lt - ts.x) * kt) * ts.y;
     if (mode == 0) return pv;
     if (mode == 2) return y == xs ? 0.f : pv;
-    return fmaxf(pv - ex2f((ld - ds.x) * kt) / ds.y, 0.f);
+    return fmaxf(pv - ex2f((ld - ds.x) * kt) * ds.y, 0.f);
 }
 
 __global__ void __launch_bounds__(256) sv_sample_kernel(SampleParams p, int chunks) {
@@ -215,7 +216,9 @@ __global__ void __launch_bounds__(256) sv_sample_kernel(SampleParams p, int chun
     const int4 info = p.seq_info[b];
     const int row = info.x, mode = info.y, xs = info.z;
     if (row < 0) return;  // uniform: no candidate rows, outputs already written
-    const float2 ts = p.row_stat[2 * row], ds = p.row_stat[2 * row + 1];
+    float2 ts = p.row_stat[2 * row], ds = p.row_stat[2 * row + 1];
+    ts.y = 1.f / ts.y;  // the weights multiply by 1 / Z
+    ds.y = 1.f / ds.y;
     {
         const int c0 = chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
         const long long off = (long long)row * p.vocab + c0;
@@ -240,28 +243,52 @@ __global__ void __launch_bounds__(256) sv_sample_kernel(SampleParams p, int chun
     __syncthreads();
     if (!seq_last) return;
     __threadfence();
-    // ---- the chunk in which the cumulative weight passes u * total (one thread: a few dozen chunks)
-    if (tid == 0) {
+    // ---- the chunk in which the cumulative weight passes u * total: warp 0, a lane per chunk (32 at a time), the
+    //      running sums by a shuffle scan in chunk order, so that the loads of a group are one round trip
+    if (tid < 32) {
         const float* cw = p.chunk_w + (long long)b * chunks;
-        float total = 0.f;
-        for (int c = 0; c < chunks; ++c) total += __ldcg(cw + c);
+        float total = 0.f;  // identical in every lane
+        for (int base = 0; base < chunks; base += 32) {
+            float v = base + tid < chunks ? __ldcg(cw + base + tid) : 0.f;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float u = __shfl_up_sync(0xffffffffu, v, o);
+                if (tid >= o) v += u;
+            }
+            total += __shfl_sync(0xffffffffu, v, 31);
+        }
         const float target = p.u_bonus[b] * total;
-        float cum = 0.f, before = 0.f;
         int pick = -1, last_pos = 0;
-        for (int c = 0; c < chunks; ++c) {
-            const float wc = __ldcg(cw + c);
-            if (wc > 0.f) last_pos = c;
-            if (cum + wc > target) { pick = c; before = cum; break; }
-            cum += wc;
+        float before = 0.f, carry = 0.f, last_before = 0.f;
+        for (int base = 0; base < chunks && pick < 0; base += 32) {
+            const float wc = base + tid < chunks ? __ldcg(cw + base + tid) : 0.f;
+            float inc = wc;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float u = __shfl_up_sync(0xffffffffu, inc, o);
+                if (tid >= o) inc += u;
+            }
+            const float cum_before = carry + inc - wc;           // weight of the chunks before this lane's
+            const unsigned hit = __ballot_sync(0xffffffffu, wc > 0.f && cum_before + wc > target);
+            const unsigned pos = __ballot_sync(0xffffffffu, wc > 0.f);
+            if (pos) {
+                const int lp = 31 - __clz(pos);
+                last_pos = base + lp;
+                last_before = __shfl_sync(0xffffffffu, cum_before, lp);
+            }
+            if (hit) {
+                const int first = __ffs(hit) - 1;
+                pick = base + first;
+                before = __shfl_sync(0xffffffffu, cum_before, first);
+            }
+            carry += __shfl_sync(0xffffffffu, inc, 31);
         }
-        if (pick < 0) {  // rounding left the target at or past the total: the last chunk with any weight
-            pick = last_pos;
-            before = 0.f;
-            for (int c = 0; c < pick; ++c) before += __ldcg(cw + c);
+        if (pick < 0) { pick = last_pos; before = last_before; }  // rounding left the target at or past the total
+        if (tid == 0) {
+            s_chunk = pick;
+            s_before = target - before;  // what is left to cross inside the chunk
+            p.seq_ticket[b] = 0u;
         }
-        s_chunk = pick;
-        s_before = target - before;  // what is left to cross inside the chunk
-        p.seq_ticket[b] = 0u;
     }
     __syncthreads();
     // ---- inside the chunk: thread t owns 16 consecutive tokens; exclusive scan of the thread sums, in order
