@@ -18,13 +18,15 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_
     const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
     const int tid = threadIdx.x;
 
+    // A thread meets its elements in index order (head, body, tail), so "greater wins" keeps the lowest index of
+    // equal values; a thread whose elements are all -inf falls back to the first one it owns.
     float bv = -INFINITY;
-    unsigned bi = 0xffffffffu;
+    unsigned bi = 0xffffffffu, first = 0xffffffffu;
     // scalar head up to the first 16-byte boundary, float4 body, scalar tail
     const int mis = (int)((reinterpret_cast<uintptr_t>(base + c0) >> 2) & 3);
     const int head = min(c1 - c0, (4 - mis) & 3);
     const int nvec = (c1 - c0 - head) >> 2;
-    if (tid < head) fold(bv, bi, base[c0 + tid], c0 + tid);
+    if (tid < head) { first = c0 + tid; const float v0 = base[c0 + tid]; if (v0 > bv) { bv = v0; bi = c0 + tid; } }
     const float4* vp = reinterpret_cast<const float4*>(base + c0 + head);
     float4 v[kVecPerThread];
 #pragma unroll
@@ -32,18 +34,22 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_
         const int e = tid + k * 256;
         v[k] = (e < nvec) ? __ldcs(vp + e) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
+    if (first == 0xffffffffu && tid < nvec) first = c0 + head + 4 * tid;
 #pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
+    for (int k = 0; k < kVecPerThread; ++k) {  // padding is -inf and never wins
         const unsigned i0 = c0 + head + 4 * (tid + k * 256);
-        if (tid + k * 256 < nvec) {
-            fold(bv, bi, v[k].x, i0);
-            fold(bv, bi, v[k].y, i0 + 1);
-            fold(bv, bi, v[k].z, i0 + 2);
-            fold(bv, bi, v[k].w, i0 + 3);
-        }
+        if (v[k].x > bv) { bv = v[k].x; bi = i0; }
+        if (v[k].y > bv) { bv = v[k].y; bi = i0 + 1; }
+        if (v[k].z > bv) { bv = v[k].z; bi = i0 + 2; }
+        if (v[k].w > bv) { bv = v[k].w; bi = i0 + 3; }
     }
     const int tail0 = c0 + head + 4 * nvec;
-    if (tail0 + tid < c1) fold(bv, bi, base[tail0 + tid], tail0 + tid);
+    if (tail0 + tid < c1) {
+        if (first == 0xffffffffu) first = tail0 + tid;
+        const float vt = base[tail0 + tid];
+        if (vt > bv) { bv = vt; bi = tail0 + tid; }
+    }
+    if (bi == 0xffffffffu) bi = first;
 
     unsigned long long key = (bi == 0xffffffffu) ? 0ull : make_key(bv, bi);
 #pragma unroll

@@ -41,15 +41,16 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
             for (int q = 0; q < 4; ++q) x[4 * k + q] = (e + q < n) ? (bs ? lg[e + q] + bs[e + q] : lg[e + q]) : -INFINITY;
         }
     }
+    // a thread meets its elements in index order, so "greater wins" keeps the lowest index of equal values;
+    // padding (-inf) never wins, and a thread whose real elements are all -inf falls back to its first one
     float bv = -INFINITY;
     unsigned bi = 0xffffffffu;
 #pragma unroll
     for (int k = 0; k < kDsVec; ++k)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int e = 4 * (tid + k * 256) + q;
-            if (e < n) fold(bv, bi, x[4 * k + q], (unsigned)(c0 + e));
-        }
+        for (int q = 0; q < 4; ++q)
+            if (x[4 * k + q] > bv) { bv = x[4 * k + q]; bi = (unsigned)(c0 + 4 * (tid + k * 256) + q); }
+    if (bi == 0xffffffffu && 4 * tid < n) bi = (unsigned)(c0 + 4 * tid);
     unsigned long long key = (bi == 0xffffffffu) ? 0ull : make_key(bv, bi);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
     for (int k = 0; k < kDsVec; ++k)
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-            if (4 * (tid + k * 256) + q < n) s += exp_neg(x[4 * k + q] - mw);
+            s += exp_neg(x[4 * k + q] - mw);  // padding is -inf and adds 0
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if ((tid & 31) == 0) { wkey[tid >> 5] = key; wsum[tid >> 5] = s; }
@@ -164,9 +165,16 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
                 const int kb = M / nb;
                 const float* pr = p.probs + m0[b] + g * kb;  // written by other CTAs: read through L2
                 float c = 1.f;
-                for (int u = 0; u < kb; ++u) {
-                    c *= __ldcg(pr + u);
-                    if (c >= p.threshold) ++keep; else break;
+                bool open = true;
+                for (int u0 = 0; u0 < kb && open; u0 += 8) {  // eight confidences per round trip, then the product in order
+                    float v[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) v[k] = u0 + k < kb ? __ldcg(pr + u0 + k) : 0.f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        c *= v[k];
+                        if (open && u0 + k < kb && c >= p.threshold) ++keep; else open = false;
+                    }
                 }
             }
         }
