@@ -91,8 +91,8 @@ typedef struct {
 } fd_config;
 
 /* Create a context on the current CUDA device.  Allocates all scratch memory: about 20 MB for
- * the attention (split partials, work list) plus, for the vocabulary sweeps, 36 bytes per
- * (row, 4096-logit chunk) with max_batch * max_q_len rows -- 3 MB at batch 64, 32 rows and a
+ * the attention (split partials, work list) plus, for the vocabulary sweeps, about 30 bytes per
+ * (row, 4096-logit chunk) with max_batch * max_q_len rows -- 2 MB at batch 64, 32 rows and a
  * 152k vocabulary; size max_batch and max_q_len for the job.  *ctx is NULL on failure
  * (FD_ERR_WORKSPACE if the device has no room). */
 fd_status fd_create(fd_ctx** ctx, const fd_config* cfg);
