@@ -177,7 +177,7 @@ def run_reference(args, step):
 class DeviceStep:
     """All tensors of one workload resident on the device + the fd context."""
 
-    def __init__(self, step, device, attn_path=0):
+    def __init__(self, step, device, attn_path=0, n_slots=1):
         import torch
         import paper_2605_20022_b200 as fd
         from paper_2605_20022_b200 import workload as wl
@@ -190,7 +190,11 @@ class DeviceStep:
         logits, drafts, self.target = wl.make_logits(step, device)
         self.logits, self.drafts = logits, drafts.to(device)
         self.pt0, self.pl0 = step.page_table.to(device), step.prefix_lens.to(device)
-        self.pt, self.pl = self.pt0.clone(), self.pl0.clone()
+        # the commit rewrites the page table and the prefix lengths: every step of a timed region gets a copy of its own,
+        # restored outside the timed region (restore()), so that the timed step holds the method's kernels only
+        self.slots = [(self.pt0.clone(), self.pl0.clone()) for _ in range(max(1, n_slots))]
+        self.cur = 0
+        self.pt, self.pl = self.slots[0]
         self.ql, self.nm = step.q_lens.to(device), step.n_mask.to(device)
         self.nb = step.n_blocks.to(device) if step.n_blocks is not None else None
         B = step.batch
@@ -207,10 +211,22 @@ class DeviceStep:
     def close(self):
         self.fd.fd_destroy(self.ctx)
 
-    def run(self, time_attn=False):
-        """One step on the current stream; the commit works on copies restored every step."""
+    def restore(self):
+        """Fresh page table and prefix lengths in every slot (not part of a step)."""
+        for pt, pl in self.slots:
+            pt.copy_(self.pt0); pl.copy_(self.pl0)
+        self.cur = 0
+
+    def run(self, time_attn=False, restore_inline=False):
+        """One step on the current stream, on the next restored copy of the page table and lengths.  With
+        restore_inline the copy is refreshed inside the step (a replayed CUDA graph has no other way)."""
         fd, torch, st = self.fd, self.torch, self.step
-        self.pt.copy_(self.pt0); self.pl.copy_(self.pl0)
+        if restore_inline:
+            self.pt, self.pl = self.slots[0]
+            self.pt.copy_(self.pt0); self.pl.copy_(self.pl0)
+        else:
+            self.pt, self.pl = self.slots[self.cur % len(self.slots)]
+            self.cur += 1
         if self.L > 1:   # every layer of the step has the same lengths: one work list serves them all
             fd.fd_plan_pin(self.ctx, st.batch, st.total_q_rows, self.pl, self.ql, self.nm, self.nb)
         for l in range(self.L):
@@ -265,9 +281,12 @@ class HostStep:
         ds.torch.cuda.current_stream().synchronize()               # the results are consumed on the host every step
 
 
-def timed_region(torch, dist, fn, steps, flush=None):
-    """barrier + synchronize, `steps` x fn() between two CUDA events, synchronize + barrier."""
+def timed_region(torch, dist, fn, steps, flush=None, prepare=None):
+    """barrier + synchronize, `steps` x fn() between two CUDA events, synchronize + barrier.  `prepare` (input
+    restoration) runs outside the timed events."""
     from paper_2605_20022_b200 import replicas
+    if prepare is not None:
+        prepare()
     replicas.barrier(dist)
     torch.cuda.synchronize()
     if flush is None:
@@ -297,10 +316,10 @@ def capture_step_graph(torch, ds):
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
-        ds.run()
+        ds.run(restore_inline=True)
         side.synchronize()
         with torch.cuda.graph(g, stream=side):
-            ds.run()
+            ds.run(restore_inline=True)
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     return g
@@ -311,7 +330,7 @@ def check_against_oracle(ds: DeviceStep, n_rows=6):
     import numpy as np
     import oracle
     torch, st = ds.torch, ds.step
-    ds.run(); torch.cuda.synchronize()
+    ds.restore(); ds.run(); torch.cuda.synchronize()
     g = torch.Generator().manual_seed(5)
     qc, kvc = ds.q[-1].cpu(), ds.kv[-1].cpu()
     outc = ds.out[-1].float().cpu().numpy()
@@ -344,11 +363,12 @@ def run_ours(args, step, rank, world, dist):
     torch.cuda.set_device(dev_index)
     device = torch.device("cuda", dev_index)
     peak, peak_src = measured_peaks()
-    ds = DeviceStep(step, device, args.attn_path)
+    ds = DeviceStep(step, device, args.attn_path, n_slots=max(args.steps, args.warmup, 5) + 1)
     resolved = {1: "simt", 2: "tcgen05"}[fd.fd_attn_path(ds.ctx)]
     small = step.attn_bytes() * step.shape.n_layers < 4 * 126e6      # fits (mostly) in the 126 MB L2
     flush = torch.empty((512 << 20,), dtype=torch.uint8, device=device) if small else None
 
+    ds.restore()
     for _ in range(args.warmup):
         ds.run()
     parity_ok = check_against_oracle(ds) if rank == 0 else True
@@ -358,7 +378,7 @@ def run_ours(args, step, rank, world, dist):
     sampler.start()
     launches0 = fd.fd_launch_count(ds.ctx)
     ds.attn_events = []
-    ms = timed_region(torch, dist, lambda: ds.run(time_attn=True), args.steps, flush)
+    ms = timed_region(torch, dist, lambda: ds.run(time_attn=True), args.steps, flush, prepare=ds.restore)
     launches = fd.fd_launch_count(ds.ctx) - launches0
     clocks = sampler.stop()
     attn_ms = [a.elapsed_time(b) for a, b in ds.attn_events]
@@ -387,7 +407,8 @@ def run_ours(args, step, rank, world, dist):
         oc = torch.empty_like(qc[0])
 
         def split_step():
-            ds.pt.copy_(ds.pt0); ds.pl.copy_(ds.pl0)
+            ds.pt, ds.pl = ds.slots[ds.cur % len(ds.slots)]
+            ds.cur += 1
             fd.fd_plan_pin(ds.ctx, step.batch, Tc, ds.pl, cand, zero)
             for l in range(ds.L - n_last):
                 fd.fd_attn_draft_verify(ds.ctx, step.batch, Tc, qc[l], ds.kv[l], step.num_pages, ds.pt, ds.pl, cand, zero, oc)
@@ -399,10 +420,11 @@ def run_ours(args, step, rank, world, dist):
             fd.fd_verify_accept(ds.ctx, step.batch, step.total_cand_rows, ds.logits, ds.drafts, ds.ql, ds.nm, ds.acc, ds.bon)
             fd.fd_kv_commit(ds.ctx, step.batch, ds.pt, ds.pl, ds.ql, ds.acc, ds.freed, ds.n_freed)
 
+        ds.restore()
         for _ in range(2):
             split_step()
         n_split = max(2, min(args.steps, 5))
-        ms_split = timed_region(torch, None, split_step, n_split) / n_split
+        ms_split = timed_region(torch, None, split_step, n_split, prepare=ds.restore) / n_split
         layer_split = {"us_per_step": ms_split * 1e3, "steps": n_split, "layers_without_mask_rows": ds.L - n_last,
                        "layers_with_mask_rows": n_last, "device_status": fd.fd_last_device_status(ds.ctx)}
         del qc, oc
@@ -473,6 +495,8 @@ def run_ours(args, step, rank, world, dist):
                    "cand_rows": step.total_cand_rows, "vocab": step.shape.vocab,
                    "attn_path": resolved,
                    "l2": "flushed between steps (512 MB write)" if small else "inputs larger than L2 (distinct KV pool per layer)",
+                   "timed_step": "plan + attention x layers + accept + commit; the page table and lengths the commit rewrites are "
+                                 "restored outside the timed region (a copy per step); the CUDA-graph replay restores them inside",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU",
                    "parity_vs_oracle_sampled": parity_ok, "device_status": status,
                    "us_per_step_cuda_graph_replay": us_graph, "draft_tail_fd_draft_select": draft_tail,
