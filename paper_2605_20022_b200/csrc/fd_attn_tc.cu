@@ -717,13 +717,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         return;
     }
     // Warp-specialised register budgets: the softmax groups keep a whole 128-column row of S in registers.
-    // 8 x 32 x 216 + 4 x 32 x 72 = 384 x 168, what the launch allocated: the increase is served by what
-    // the decrease released (a request for more than that did not return when it was tried).
+    // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168, what the launch allocated: the increase is served exactly by what
+    // the decrease released (a request for more than that does not return).
     if (warp < 8) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         softmax_role<D>(p, bars, ex, s_cs, cs, ring, tmem, s_c, e_c, abort);
     } else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         if (warp == kKWarp) load_role<D>(tmap, p, hdr.n_rb, sk, bars->k_full, bars->k_empty, 0, s_c, e_c, abort);
         else if (warp == kVWarp) load_role<D>(tmap, p, hdr.n_rb, sv, bars->v_full, bars->v_empty, 1, s_c, e_c, abort);
         else if (warp == kMmaWarp) mma_role<D>(p, sq, sk, sv, bars, ring, tmem, s_c, e_c, abort);
