@@ -529,6 +529,11 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: bring up the N replicas ourselves, one rank per GPU
+        from paper_2605_20022_b200 import replicas
+        sys.exit(replicas.launch_replicas(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
+
     from paper_2605_20022_b200 import workload as wl
     step = wl.workload(args.workload, n_layers=args.layers)
     rank, world = int(os.environ.get("RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))

@@ -142,8 +142,10 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * KV tiles) from the lengths alone; it is the same for every layer of a step.  fd_plan_pin computes it once;
  * until fd_plan_unpin, every fd_attn_draft_verify[_blocks] call with the same batch, total_q_rows and the
  * same four length pointers reuses it instead of recomputing it (a call with anything else recomputes and
- * drops the pin).  The caller must not change the contents of the length arrays while the pin holds
- * (fd_kv_commit does: unpin before the next step), and must unpin after a FD_DEV_TIMEOUT status.
+ * drops the pin).  The caller must not change the contents of the length arrays while the pin holds, and
+ * must unpin after a FD_DEV_TIMEOUT status.  fd_kv_commit rewrites prefix_lens and therefore drops the pin
+ * itself: the first attention call of the next step plans afresh (or is preceded by a new fd_plan_pin).
+ * fd_kv_append leaves the lengths alone and keeps the pin.
  * A sequence flagged for a page id outside the pool (FD_DEV_BAD_PAGE) stays flagged, and its rows zero,
  * for every call served by the same pin.  The calls served by a pin must be ordered after fd_plan_pin (the
  * same stream, or streams the caller has ordered) and must not overlap one another: they share the context's

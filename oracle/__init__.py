@@ -166,8 +166,9 @@ def accept_stochastic(logits, draft_logits, draft_tokens, q_lens, n_mask, temper
     return (acc, bon, ratio[:R], w) if want_weights else (acc, bon, ratio[:R])
 
 
-def draft_select(logits, bias, n_mask, n_blocks, threshold, max_blocks):
-    """Draft-side tail (Eq. 4 + Eq. 5): returns (tokens [Rm] i32, probs [Rm] f64, cum [Rm] f64, keep_len [B, max_blocks] i32)."""
+def draft_select(logits, bias, n_mask, n_blocks, threshold, max_blocks, want_gap=False):
+    """Draft-side tail (Eq. 4 + Eq. 5): returns (tokens [Rm] i32, probs [Rm] f64, cum [Rm] f64, keep_len [B, max_blocks] i32),
+    and with want_gap also the margin [Rm] f64 by which each row's winning calibrated logit beats the best other one."""
     lg = np.ascontiguousarray(logits if isinstance(logits, np.ndarray) else logits.cpu().numpy(), dtype=np.float32)
     bs = None if bias is None else np.ascontiguousarray(bias if isinstance(bias, np.ndarray) else bias.cpu().numpy(), dtype=np.float32)
     Rm, V = lg.shape
@@ -176,9 +177,12 @@ def draft_select(logits, bias, n_mask, n_blocks, threshold, max_blocks):
     B = nm.shape[0]
     assert int(np.maximum(nm, 0).sum()) == Rm
     tok = np.zeros((max(Rm, 1),), np.int32); pr = np.zeros((max(Rm, 1),), np.float64); cum = np.zeros((max(Rm, 1),), np.float64)
+    gap = np.zeros((max(Rm, 1),), np.float64)
     keep = np.zeros((B, max_blocks), np.int32)
     _load().fdo_draft_select(ctypes.c_int(B), ctypes.c_int(V), ctypes.c_int(max_blocks), _p(lg), None if bs is None else _p(bs), _p(nm),
-                             None if nb is None else _p(nb), ctypes.c_double(threshold), _p(tok), _p(pr), _p(cum), _p(keep))
+                             None if nb is None else _p(nb), ctypes.c_double(threshold), _p(tok), _p(pr), _p(cum), _p(keep), _p(gap))
+    if want_gap:
+        return tok[:Rm], pr[:Rm], cum[:Rm], keep, gap[:Rm]
     return tok[:Rm], pr[:Rm], cum[:Rm], keep
 
 

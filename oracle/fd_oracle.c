@@ -268,23 +268,28 @@ void fdo_accept(int B, int V, const float *logits, const int32_t *draft_tokens,
     }
 }
 
-/* Verification by speculative sampling (Sec. 3: a draft is accepted "according to the ratio between" the
- * target distribution p and the drafter distribution q, and at the first rejected position a new token is
- * drawn "from the residual target distribution"; committed length = accepted + 1.  The rule itself is the
- * published speculative-sampling algorithm the paper cites).  Rows and draft_tokens as in fdo_accept.
+/* Verification by speculative sampling (Sec. 3).  Each draft is kept or dropped by comparing the target
+ * distribution p with the drafter distribution q at the drafted token; where the first draft is dropped, a
+ * replacement is drawn from what is left of p once q has been taken out; committed length = accepted + 1.
+ * The rule itself is the published speculative-sampling algorithm that Sec. 3 refers to.  Rows and
+ * draft_tokens as in fdo_accept.
  *
  *   p_j = softmax(logits[r0 + j] / T)              target distribution after candidate row j
  *   q_j = softmax(draft_logits[r0 + j] / T)        distribution draft j + 1 was proposed from, or, with
  *                                                  draft_logits == NULL, all mass on the proposed token
  *   for j = 0 .. k-1, x = draft_tokens[r0 + j + 1]:
- *       accept x  iff  u_accept[r0 + j] < min(1, p_j(x) / q_j(x));  the first rejection ends the loop
+ *       accept x  iff  u_accept[r0 + j] * q_j(x) < p_j(x)      (for q_j(x) > 0 this is u < min(1, p/q), since
+ *                                                  u < 1; written as a product it is also defined for a token
+ *                                                  the drafter gives no mass: accepted iff p_j(x) > 0; a token
+ *                                                  with p = q = 0 is rejected);  the first rejection ends the loop
  *   rejected at j:   bonus ~ max(0, p_j - q_j) normalised      all k accepted:   bonus ~ p_k
  *
  * Random numbers are inputs: u_accept [R] (the entry of a sequence's last row is unused) and u_bonus [B], all
  * in [0, 1).  A token is drawn from weights w by inverting the cumulative sum in index order: the first y
  * with w[0] + .. + w[y] > u * sum(w).  ratio [R] (optional) receives p_j(x) / q_j(x) for every tested draft
- * (-1 elsewhere) and weights [B, V] (optional) the unnormalised weights the bonus token was drawn from, so
- * that a test can tell a wrong decision from one that sits on a rounding boundary. */
+ * (-1 elsewhere; +inf or NaN where q_j(x) = 0) and weights [B, V] (optional) the unnormalised weights the
+ * bonus token was drawn from, so that a test can tell a wrong decision from one that sits on a rounding
+ * boundary. */
 void fdo_accept_stochastic(int B, int V, const float *logits, const float *draft_logits, const int32_t *draft_tokens,
         const int32_t *q_lens, const int32_t *n_mask, double temperature, const float *u_accept,
         const float *u_bonus, int32_t *accepted_len, int32_t *bonus_token, double *ratio, double *weights)
@@ -321,7 +326,7 @@ void fdo_accept_stochastic(int B, int V, const float *logits, const float *draft
             }
             const double rho = p[x] / q[x];
             if (ratio) ratio[r0 + j] = rho;
-            if ((double)u_accept[r0 + j] < (rho < 1.0 ? rho : 1.0)) { ++a; continue; }
+            if ((double)u_accept[r0 + j] * q[x] < p[x]) { ++a; continue; }
             rejected = 1;
             for (int v = 0; v < V; ++v) { const double w = p[v] - q[v]; p[v] = w > 0.0 ? w : 0.0; }
             break;
@@ -352,11 +357,14 @@ void fdo_accept_stochastic(int B, int V, const float *logits, const float *draft
  * the block is the number of leading positions whose cumulative confidence is still >= threshold, i.e. how
  * many of its drafts are worth verifying in the next step.
  *
- * The sum l + bias is formed in float32, as the kernel forms it, so that the argmax is decided on the same
- * numbers; everything after that is float64.  tokens [Rm], probs [Rm], cum [Rm], keep_len [B, max_blocks]
- * (zero where a sequence has fewer blocks). */
+ * Eq. 4 defines the sum, not a precision: everything here is float64 (the float32 inputs convert exactly).
+ * tokens [Rm], probs [Rm], cum [Rm], keep_len [B, max_blocks] (zero where a sequence has fewer blocks).
+ * gap [Rm] (optional) receives the margin by which the winning calibrated logit beats the best other one
+ * (0 on an exact tie, +inf when V = 1), so that a test can tell a wrong argmax from one that a
+ * lower-precision sum may legitimately decide the other way. */
 void fdo_draft_select(int B, int V, int max_blocks, const float *logits, const float *bias, const int32_t *n_mask,
-        const int32_t *n_blocks, double threshold, int32_t *tokens, double *probs, double *cum, int32_t *keep_len)
+        const int32_t *n_blocks, double threshold, int32_t *tokens, double *probs, double *cum, int32_t *keep_len,
+        double *gap)
 {
     int64_t r0 = 0;
     for (int b = 0; b < B; ++b) {
@@ -370,18 +378,20 @@ void fdo_draft_select(int B, int V, int max_blocks, const float *logits, const f
             const float *lr = logits + (r0 + u) * (int64_t)V;
             const float *br = bias ? bias + (r0 + u) * (int64_t)V : NULL;
             int best = 0;
-            float bestv = br ? lr[0] + br[0] : lr[0];
+            double bestv = br ? (double)lr[0] + (double)br[0] : (double)lr[0];
             for (int v = 1; v < V; ++v) {
-                const float x = br ? lr[v] + br[v] : lr[v];
+                const double x = br ? (double)lr[v] + (double)br[v] : (double)lr[v];
                 if (x > bestv) { bestv = x; best = v; }
             }
-            double den = 0.0;
+            double den = 0.0, second = -INFINITY;
             for (int v = 0; v < V; ++v) {
-                const float x = br ? lr[v] + br[v] : lr[v];
-                den += exp((double)x - (double)bestv);
+                const double x = br ? (double)lr[v] + (double)br[v] : (double)lr[v];
+                den += exp(x - bestv);
+                if (v != best && x > second) second = x;
             }
             tokens[r0 + u] = best;
             probs[r0 + u] = 1.0 / den;
+            if (gap) gap[r0 + u] = bestv - second;
         }
         for (int g = 0; g < nb; ++g) {
             double c = 1.0;

@@ -192,8 +192,17 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
         if (tid == blockDim.x - 1) carry = (int)min(offr + inc, (long long)0x7fffffff);
         __syncthreads();
     }
+    // lengths that do not add up: a defined output, -1 everywhere, and nothing for the draw kernel to do
+    const bool bad = s_bad || carry != p.total_rows;  // final after the loop's last barrier
+    if (bad) {
+        for (int b = tid; b < p.batch; b += blockDim.x) {
+            p.accepted[b] = -1;
+            p.bonus[b] = -1;
+            p.seq_info[b] = make_int4(-1, 0, -1, 0);
+        }
+    }
     if (tid == 0) {
-        if (s_bad || carry != p.total_rows) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        if (bad) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         *p.ticket = 0u;
     }
 }

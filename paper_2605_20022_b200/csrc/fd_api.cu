@@ -324,19 +324,30 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         }
         chk(cudaStreamWaitEvent(s, h->q_ready[b], 0));
         if (l >= 2) chk(cudaStreamWaitEvent(s, h->out_copied[b], 0));
-        if (l == 0 && n_layers > 1) {  // one work list for all layers of the step
+        if (l == 0 && n_layers > 1)  // one work list for all layers of the step
             st = fd_plan_pin(c, batch, total_q_rows, h->pl, h->ql, h->nm, n_blocks_host ? h->nb : nullptr, s);
-            if (st != FD_OK) return st;
-        }
-        st = fd_attn_draft_verify_blocks(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
-                                         n_blocks_host ? h->nb : nullptr, h->out[b], s);
+        if (st == FD_OK)
+            st = fd_attn_draft_verify_blocks(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
+                                             n_blocks_host ? h->nb : nullptr, h->out[b], s);
+        // on an error the events of this layer are still recorded, so that nothing queued on the copy streams
+        // waits for an event that never comes
         chk(cudaEventRecord(h->attn_done[b], s));
         chk(cudaStreamWaitEvent(h->d2h, h->attn_done[b], 0));
         chk(cudaMemcpyAsync(static_cast<unsigned char*>(out_host) + (size_t)l * qb, h->out[b], qb, D2H, h->d2h));
         chk(cudaEventRecord(h->out_copied[b], h->d2h));
     }
     c->pinned = false;  // the commit below changes the lengths
-    if (st != FD_OK) return st;
+    // A failed call leaves the three streams consistent: whatever was queued on the copy streams is joined back
+    // into `stream` before the error is returned, so no stream is left waiting and the staging may be reused.
+    auto fail = [&](fd_status code) {
+        cudaEventRecord(h->fin, h->h2d);
+        cudaStreamWaitEvent(s, h->fin, 0);
+        cudaEventRecord(h->done, h->d2h);
+        cudaStreamWaitEvent(s, h->done, 0);
+        cudaGetLastError();
+        return code;
+    };
+    if (st != FD_OK) return fail(st);
     if (n_layers < 2 && total_cand_rows > 0) {
         chk(cudaMemcpyAsync(h->lg, logits_host, (size_t)total_cand_rows * c->cfg.vocab * 4, H2D, h->h2d));
         chk(cudaMemcpyAsync(h->drafts, draft_tokens_host, (size_t)total_cand_rows * 4, H2D, h->h2d));
@@ -344,9 +355,9 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
     }
     if (total_cand_rows > 0) chk(cudaStreamWaitEvent(s, h->logits, 0));
     st = fd_verify_accept(c, batch, total_cand_rows, h->lg, h->drafts, h->ql, h->nm, h->acc, h->bon, s);
-    if (st != FD_OK) return st;
+    if (st != FD_OK) return fail(st);
     st = fd_kv_commit(c, batch, h->pt, h->pl, h->ql, h->acc, h->freed, h->nfreed, s);
-    if (st != FD_OK) return st;
+    if (st != FD_OK) return fail(st);
     chk(cudaEventRecord(h->done, s));
     chk(cudaStreamWaitEvent(h->d2h, h->done, 0));
     chk(cudaMemcpyAsync(accepted_len_host, h->acc, lb, D2H, h->d2h));
@@ -357,7 +368,7 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
     chk(cudaMemcpyAsync(n_freed_host, h->nfreed, 4, D2H, h->d2h));
     chk(cudaEventRecord(h->fin, h->d2h));
     chk(cudaStreamWaitEvent(s, h->fin, 0));  // `stream` is complete only when every result is on the host
-    if (!ok) { cudaGetLastError(); return FD_ERR_CUDA; }
+    if (!ok) return fail(FD_ERR_CUDA);
     return FD_OK;
 }
 
@@ -523,6 +534,7 @@ fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefi
     p.batch = batch; p.max_pages = c->cfg.max_pages_per_seq; p.page_size = c->cfg.page_size;
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.accepted = accepted_len;
     p.freed = freed_pages; p.n_freed = n_freed; p.status = c->status;
+    c->pinned = false;  // the commit rewrites prefix_lens: a work list made for the old lengths must not be reused
     fd::launch_commit(p, s);
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;

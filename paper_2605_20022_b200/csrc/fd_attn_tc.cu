@@ -42,6 +42,8 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <vector>
+
 #include "fd_internal.cuh"
 #include "fd_sm100.cuh"
 
@@ -54,6 +56,11 @@ namespace {
 constexpr int kThreads = 384;  // warps 0-3 softmax group 0, 4-7 softmax group 1, 8 K loads, 9 V loads, 10 MMA, 11 Q loads
 constexpr int kKWarp = 8, kVWarp = 9, kMmaWarp = 10;  // warp 11 loads Q
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+// How Q K^T(j) is kept from overwriting P(j - 2) before the P V that reads it has completed (see mma_role).
+#ifndef FD_QK_MODE
+#define FD_QK_MODE 1
+#endif
 
 template <int D>
 struct Cfg {
@@ -125,30 +132,6 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int n_rb, int
     return pc;
 }
 
-#ifdef FD_TRACE
-// Debug build only: per-role timestamps of CTA 0 for pipeline analysis.  Each role's tracing thread
-// owns a region and a private counter, so an event costs one clock read and one store.
-constexpr int kTraceRoles = 7, kTracePerRole = 4096;
-__device__ unsigned long long g_trace[kTraceRoles * kTracePerRole];
-__device__ unsigned int g_trace_n[kTraceRoles];
-__device__ __forceinline__ void trace(int role, int ev, int tile, int& n) {
-#ifndef FD_TRACE_CTA
-#define FD_TRACE_CTA 0
-#endif
-    if (blockIdx.x != FD_TRACE_CTA || n >= kTracePerRole) return;
-    g_trace[role * kTracePerRole + n] = ((unsigned long long)clock64() & 0xffffffffffull) | ((unsigned long long)ev << 40) | ((unsigned long long)tile << 48);
-    g_trace_n[role] = ++n;
-}
-__device__ unsigned long long g_cta_log[1024 * 16];
-__device__ __forceinline__ void cta_log(int slot) { if (slot < 16) g_cta_log[blockIdx.x * 16 + slot] = global_ns(); }
-#define CTA_LOG(slot) cta_log(slot)
-#define TRACE(role, ev, tile) trace(role, ev, tile, tr_n)
-#define TRACE_DECL int tr_n = 0
-#else
-#define TRACE(role, ev, tile)
-#define CTA_LOG(slot)
-#define TRACE_DECL
-#endif
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -221,7 +204,6 @@ template <int D>
 __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnParams& p, int n_rb, unsigned char* ring, uint64_t* full,
                                           uint64_t* empty, int which, int s_c, int e_c, volatile int* abort) {
     using C = Cfg<D>;
-    TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     constexpr int kOps = 8;  // pages of a tile: one box each
     const int pg = lane;
@@ -255,7 +237,6 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             if (j > 0 && (j & 3) == 0) { ids_cur = ids_next; ids_next = load_ids((j >> 2) + 1); }
             const int phys = __shfl_sync(0xffffffffu, ids_cur, (j & 3) * 8 + pg);
             if (!wait_all(&empty[st], (use & 1) ^ 1, abort)) { ok = false; break; }
-            if (lane == 0) TRACE(which, 0, g);
             const int pos0 = (pc.tile0 + j) * kTileTokens;
             const int npg = min(8, (pc.kv_len - pos0 + 15) >> 4);
             if (lane == 0) mbar_arrive_expect_tx(&full[st], npg * (16 * D * 2));
@@ -287,7 +268,6 @@ template <int D>
 __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams& p, int n_rb, unsigned char* sq, Bars* bars, Piece* ring,
                                        int s_c, int e_c, volatile int* abort) {
     using C = Cfg<D>;
-    TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     const int bt = p.q_box_t;
     Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
@@ -296,7 +276,6 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
     if (lane == 0) publish_piece(bars, ring, 0, pc);
     while (w.t < e_c) {
         if (w.piece > 0 && !wait_all(&bars->q_free, (w.piece - 1) & 1, abort)) break;
-        if (lane == 0) TRACE(6, 0, w.piece);
         const int nbox = (pc.Lv + bt - 1) / bt;
         if (lane == 0) mbar_arrive_expect_tx(&bars->q_full, nbox * bt * p.G * 128 * C::kHalves);
         __syncwarp();
@@ -305,7 +284,6 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
             tma_load_3d(sq + half * (kMaxRows * 128) + j * bt * p.G * 128, &qmap, half * 64, pc.kvh * p.G, pc.row0 + j * bt, &bars->q_full);
         }
         issued = w.piece + 1;
-        if (lane == 0) TRACE(6, 1, w.piece);
         w.advance(pc);
         if (w.t < e_c) {
             // the next piece: descriptor for the other roles, and its Q rows on their way into L2
@@ -328,9 +306,9 @@ template <int D>
 __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq, unsigned char* sk, unsigned char* sv, Bars* bars,
                                          const Piece* ring, uint32_t tmem, int s_c, int e_c, volatile int* abort) {
     using C = Cfg<D>;
-    TRACE_DECL;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
+    constexpr uint32_t idesc_qk_half = make_idesc_bf16(128, kTileTokens / 2, false);
     constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
     const uint32_t q_addr = smem_u32(sq);
@@ -340,7 +318,6 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
         if (!__all_sync(0xffffffffu, wait_piece(bars, w.piece, abort))) break;
         const Piece pc = ring[w.piece & (kDescSlots - 1)];
         if (!wait_all(&bars->q_full, w.piece & 1, abort)) break;
-        if (lane == 0) TRACE(2, 3, w.piece);
         auto issue_pv = [&](int jj) {
             const int gg = w.g0 + jj, s = jj & 1, st = gg % C::kStages, u = w.u_base[s] + (jj >> 1);
             if (!wait_all(&bars->v_full[st], (gg / C::kStages) & 1, abort)) { ok = false; return; }
@@ -362,7 +339,6 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
             if (!wait_all(&bars->p_full[s], u & 1, abort)) { ok = false; return; }
             tc_fence_after();
             if (lane == 0) {
-                TRACE(2, 2, gg);
                 const uint32_t v_addr = smem_u32(vt);
 #pragma unroll
                 for (int kk = 0; kk < kTileTokens / 16; ++kk)
@@ -378,24 +354,38 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
             const int g = w.g0 + j, st = g % C::kStages, use = g / C::kStages;
             const int s = j & 1;
             if (!wait_all(&bars->k_full[st], use & 1, abort)) { ok = false; break; }
-            if (lane == 0) TRACE(2, 0, g);
-            // S_s is written over P_s, which the P V of tile j - 2 reads.  That MMA was issued earlier by
-            // this same thread, and the tensor pipe takes one thread's MMAs in issue order, so no wait for
-            // its completion is needed here (measured: 3 % on a power-capped 36-layer step).  Building with
-            // -DFD_WAIT_PV restores the explicit wait on the completion barrier.
-#ifdef FD_WAIT_PV
-            if (w.u_base[s] + (j >> 1) >= 1 && !wait_all(&bars->pv_done[s], (w.u_base[s] + (j >> 1) - 1) & 1, abort)) { ok = false; break; }
-#endif
+            // S_s is written over P_s (its first 64 columns), which the P V of tile j - 2 of this stream reads, and
+            // nothing orders two MMAs with different accumulators but the completion of the first: Q K^T waits for
+            // that P V's completion barrier (FD_QK_MODE 1, the default).  Measured alternatives, kept for
+            // measurements only: 2 = Q K^T as two N = 64 halves, the tokens 64..127 (columns the P V does not read)
+            // ahead of the wait (11 % slower: the half-width MMAs cost more than the wait); 0 = no wait, relying on
+            // one thread's MMAs executing in issue order (5 % faster than the default, not a documented guarantee).
+            [[maybe_unused]] const int u_prev = w.u_base[s] + (j >> 1) - 1;  // the stream's previous tile, over all pieces
             tc_fence_after();
+            const uint32_t k_addr = smem_u32(sk + st * C::kKBytes);
+#if FD_QK_MODE == 2
             if (lane == 0) {
-                TRACE(2, 1, g);
-                const uint32_t k_addr = smem_u32(sk + st * C::kKBytes);
+#pragma unroll
+                for (int kk = 0; kk < C::kKSteps; ++kk) {
+                    const uint32_t q_off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
+                    const uint32_t k_off = (kk >> 2) * 1024 + (kk & 3) * 32 + 8 * C::kGroupBytes;
+                    umma_ss(tmem + col_s[s] + 64, make_smem_desc(q_addr + q_off, 16, 1024), make_smem_desc(k_addr + k_off, 16, C::kGroupBytes),
+                            idesc_qk_half, kk > 0);
+                }
+            }
+            __syncwarp();
+#endif
+#if FD_QK_MODE != 0
+            if (u_prev >= 0 && !wait_all(&bars->pv_done[s], u_prev & 1, abort)) { ok = false; break; }
+            tc_fence_after();
+#endif
+            if (lane == 0) {
 #pragma unroll
                 for (int kk = 0; kk < C::kKSteps; ++kk) {
                     const uint32_t q_off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
                     const uint32_t k_off = (kk >> 2) * 1024 + (kk & 3) * 32;
                     umma_ss(tmem + col_s[s], make_smem_desc(q_addr + q_off, 16, 1024), make_smem_desc(k_addr + k_off, 16, C::kGroupBytes),
-                            idesc_qk, kk > 0);
+                            FD_QK_MODE == 2 ? idesc_qk_half : idesc_qk, kk > 0);
                 }
                 umma_commit(&bars->k_empty[st]);
                 umma_commit(&bars->s_full[s]);
@@ -415,7 +405,6 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
 template <int D>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, int* s_cs, const CtaStarts cs, const Piece* ring,
                                              uint32_t tmem, int s_c, int e_c, volatile int* abort) {
-    TRACE_DECL;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     const int s = warp >> 2;                  // stream
     const int r = (warp & 3) * 32 + lane;     // query row == TMEM lane
@@ -434,7 +423,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         named_bar_sync(1, 256);
         if (!bars->piece_ok) break;
         const Piece pc = ring[w.piece & (kDescSlots - 1)];
-        if (tid == 0) TRACE(5, 2, w.piece);
         const bool warp_active = (warp & 3) * 32 < pc.rows;
         const int i = r / p.G;
         const RowMask rm = row_mask(pc.i0 + i, pc.n, pc.Lq, pc.M, pc.nb, r < pc.rows);
@@ -448,7 +436,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             const int u = w.u_base[s] + (j >> 1);
             if (!wait_all(&bars->s_full[s], u & 1, abort)) { ok = false; break; }
             tc_fence_after();
-            if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 0, w.g0 + j);
             {
                 const int pos0 = (pc.tile0 + j) * kTileTokens;
                 // tile reaches into the query block (or past kv_len): the row's mask applies, in tile-local columns
@@ -480,7 +467,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                         mx[3] = max3(mx[3], __uint_as_float(sv[ch][k + 6]), __uint_as_float(sv[ch][k + 7]));
                     }
                 const float m_new = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c);
-                if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 1, w.g0 + j);
                 float alpha = 1.f;
                 if (j < 2 || m == -INFINITY) {
                     m = m_new;  // nothing accumulated yet (O is overwritten, or exactly zero)
@@ -529,7 +515,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             tc_fence_before();
             mbar_arrive(&bars->p_full[s]);
             if ((warp & 3) == 0 && lane == 0 && n_idle_threads) mbar_arrive_cnt(&bars->p_full[s], n_idle_threads);
-            if ((warp & 3) == 0 && lane == 0) TRACE(3 + s, 2, w.g0 + j);
         }
 
         // ---- epilogue: merge the two streams, then final rows, or a partial plus -- if this CTA is the
@@ -538,7 +523,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         //      uniform (leave, merge) are taken by thread 0 alone and published through shared memory.
         if (warp_active) ok = ok && wait_all(&bars->all_done, w.piece & 1, abort);
         tc_fence_after();
-        if (tid == 0) TRACE(5, 4, w.piece);
         const bool two = pc.nt >= 2;
         // Stream exchange: group 1 hands its (m, l) to group 0, which answers with the two scale factors.
         // A thread only ever touches the two slots of its own row, so one barrier each way is enough.
@@ -559,7 +543,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         }
         named_bar_sync(1, 256);
         if (s == 1) { a0 = ex[r]; a1 = ex[kMaxRows + r]; }
-        if (tid == 0) TRACE(5, 6, w.piece);
         constexpr int kChunks = D / 64;  // 32-column chunks per softmax group
         const bool do_read = !leave && warp_active;
         // the load warps of this CTA have seen every page id of the segment by now
@@ -573,7 +556,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 tmem_ld32(tmem + lane_base + col_o[0] + col, o0);
                 if (two) tmem_ld32(tmem + lane_base + col_o[1] + col, o1);
                 tc_wait_ld();
-                if (tid == 0) TRACE(5, 11 + 2 * ch, w.piece);
 #pragma unroll
                 for (int k = 0; k < 32; ++k) {
                     o[ch][k] = __uint_as_float(o0[k]) * a0;
@@ -601,7 +583,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     for (int k = 0; k < 32; k += 4) dst[(k >> 2) * kMaxRows] = make_float4(o[ch][k], o[ch][k + 1], o[ch][k + 2], o[ch][k + 3]);
                 }
             }
-            if (tid == 0) TRACE(5, 12 + 2 * ch, w.piece);
         }
         if (do_read && r < pc.rows && !pc.complete && s == 0) {
             p.part.m[pc.slot * kMaxRows + r] = mm;
@@ -614,22 +595,18 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             const int t0 = w.t - pc.tile0, t1 = t0 + pc.seg_nt;
             int c_first, c_last;
             segment_ctas(cs, p.n_ctas, cta, t0, t1, c_first, c_last);
-            if (tid == 0) TRACE(5, 7, w.piece);
             named_bar_sync(1, 256);
             if (tid == 0) {
                 int last = 0;
                 if (!leave && !*abort) {
                     const int n = segment_pieces(cs, c_first, c_last, t0, t1);
-                    TRACE(5, 8, w.piece);
                     __threadfence();
-                    TRACE(5, 9, w.piece);
                     int* count = p.plan.seg_count + pc.v * p.Hkv + pc.kvh;
                     last = atomicAdd(count, 1) + 1 == n;
                     if (last) {
                         *count = 0;  // everyone has been counted: ready for the next call that uses this plan
                         __threadfence();
                     }
-                    TRACE(5, 10, w.piece);
                 }
                 bars->epi_flag = last;
             }
@@ -640,8 +617,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 if (rr < pc.rows) merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, t0, t1, rr, cg, &o[0][0], cta);
             }
         }
-        if (tid == 0) TRACE(5, 5, w.piece);
-        if (tid == 0) CTA_LOG(2 + w.piece);
         if (leave) break;
         w.advance(pc);
     }
@@ -695,9 +670,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     // a dependent launch behind this one (the next layer's call, when the plan is pinned) may bring its
     // CTAs in as ours retire and do its own set-up; it waits for this grid to complete before reading anything
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid == 0) CTA_LOG(0);
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (tid == 0) CTA_LOG(1);  // the plan kernel has completed and its writes are visible
 
     const PlanHeader hdr = *p.plan.hdr;
     const int total = hdr.total_tiles;
@@ -738,16 +711,37 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 
 struct TmapEntry {
     const void* ptr;
-    int num_pages;  // KV pool: pages; q: rows
+    int n;  // KV pool: pages; q: rows
     CUtensorMap map;
+};
+
+// Tensor maps already encoded, keyed by (pointer, extent).  A model calls the attention once per layer with that
+// layer's pool and q buffer, in the same order every step: the entry after the last hit is tried first, then the
+// whole list; the list grows with the number of distinct operands (one per layer) and is recycled round-robin
+// only past kMaxEntries.
+struct TmapCache {
+    static constexpr size_t kMaxEntries = 4096;
+    std::vector<TmapEntry> e;
+    size_t last = 0, victim = 0;
+    const CUtensorMap* find(const void* ptr, int n) {
+        const size_t cnt = e.size();
+        for (size_t k = 0; k < cnt; ++k) {
+            const size_t i = (last + 1 + k) % cnt;
+            if (e[i].ptr == ptr && e[i].n == n) { last = i; return &e[i].map; }
+        }
+        return nullptr;
+    }
+    TmapEntry& slot() {
+        if (e.size() < kMaxEntries) { e.emplace_back(); last = e.size() - 1; return e.back(); }
+        last = victim;
+        victim = (victim + 1) % kMaxEntries;
+        return e[last];
+    }
 };
 
 struct TcState {
     PFN_cuTensorMapEncodeTiled_v12000 encode;
-    TmapEntry cache[64];
-    int n_cached, next;
-    TmapEntry qcache[64];
-    int nq_cached, qnext;
+    TmapCache kv, q;
     int d, hkv;
     const CUtensorMap* current;
     const CUtensorMap* qcurrent;
@@ -766,8 +760,6 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
     TcState* st = static_cast<TcState*>(*state);
     if (!st) {
         st = new TcState();
-        st->n_cached = st->next = 0;
-        st->nq_cached = st->qnext = 0;
         st->encode = nullptr;
         cudaDriverEntryPointQueryResult qres;
         cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", reinterpret_cast<void**>(&st->encode), cudaEnableDefault, &qres);
@@ -779,43 +771,41 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
         *state = st;
     }
     // q: a 3-D view [T][Hq][d], box = 64 elements x G q-heads (one kv-head) x q_box_t block rows
-    st->qcurrent = nullptr;
-    for (int i = 0; i < st->nq_cached; ++i)
-        if (st->qcache[i].ptr == p.q && st->qcache[i].num_pages == p.total_q_rows) st->qcurrent = &st->qcache[i].map;
+    st->qcurrent = st->q.find(p.q, p.total_q_rows);
     if (!st->qcurrent) {
-        TmapEntry& e = st->qcache[st->qnext];
+        CUtensorMap map;
         cuuint64_t dims[3] = {(cuuint64_t)p.d, (cuuint64_t)p.Hq, (cuuint64_t)(p.total_q_rows > 0 ? p.total_q_rows : 1)};
         cuuint64_t strides[2] = {(cuuint64_t)p.d * 2, (cuuint64_t)p.Hq * p.d * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)p.G, (cuuint32_t)p.q_box_t};
         cuuint32_t estr[3] = {1, 1, 1};
-        const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(p.q), dims, strides, box, estr,
+        const CUresult r = st->encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(p.q), dims, strides, box, estr,
                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        TmapEntry& e = st->q.slot();
         e.ptr = p.q;
-        e.num_pages = p.total_q_rows;
+        e.n = p.total_q_rows;
+        e.map = map;
         st->qcurrent = &e.map;
-        st->qnext = (st->qnext + 1) % 64;
-        if (st->nq_cached < 64) ++st->nq_cached;
     }
-    for (int i = 0; i < st->n_cached; ++i)
-        if (st->cache[i].ptr == p.kv && st->cache[i].num_pages == p.num_pages) { st->current = &st->cache[i].map; return cudaSuccess; }
-    TmapEntry& e = st->cache[st->next];
+    st->current = st->kv.find(p.kv, p.num_pages);
+    if (st->current) return cudaSuccess;
     // 64 elements x 8 rows x the 64-wide halves of d x groups of 8 rows: a box of two groups is one page of one
     // kv-head and lands as [group][half][8 rows][128 B]
+    CUtensorMap map;
     cuuint64_t dims[4] = {64, 8, (cuuint64_t)p.d / 64, (cuuint64_t)p.num_pages * 2 * p.Hkv * 2};
     cuuint64_t strides[3] = {(cuuint64_t)p.d * 2, 128, (cuuint64_t)p.d * 2 * 8};
     cuuint32_t box[4] = {64, 8, (cuuint32_t)p.d / 64, 2};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    const CUresult r = st->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(p.kv), dims, strides, box, estr,
+    const CUresult r = st->encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(p.kv), dims, strides, box, estr,
                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    TmapEntry& e = st->kv.slot();
     e.ptr = p.kv;
-    e.num_pages = p.num_pages;
+    e.n = p.num_pages;
+    e.map = map;
     st->current = &e.map;
-    st->next = (st->next + 1) % 64;
-    if (st->n_cached < 64) ++st->n_cached;
     return cudaSuccess;
 }
 
@@ -859,24 +849,5 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
 void launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s) {
     wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, limit_ns);
 }
-
-#ifdef FD_TRACE
-// dst: [roles][per_role] packed events; counts: [roles].  Resets the counters.
-extern "C" int fd_debug_read_trace(unsigned long long* dst, unsigned int* counts) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(counts, g_trace_n, sizeof(unsigned int) * kTraceRoles);
-    cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * kTraceRoles * kTracePerRole);
-    unsigned int zero[kTraceRoles] = {0};
-    cudaMemcpyToSymbol(g_trace_n, zero, sizeof(zero));
-    return kTracePerRole;
-}
-extern "C" int fd_debug_read_cta_log(unsigned long long* dst) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(dst, g_cta_log, sizeof(unsigned long long) * 1024 * 16);
-    static unsigned long long zero[1024 * 16];
-    cudaMemcpyToSymbol(g_cta_log, zero, sizeof(zero));
-    return 16;
-}
-#endif
 
 }  // namespace fd

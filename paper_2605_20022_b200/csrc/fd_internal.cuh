@@ -272,9 +272,6 @@ __device__ inline float key_value(unsigned long long key) {
     return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
 }
 __device__ inline int key_index(unsigned long long key) { return (int)(0xffffffffu - (unsigned)(key & 0xffffffffull)); }
-__device__ inline void fold(float& bv, unsigned& bi, float v, unsigned i) {
-    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
-}
 
 struct DraftSelectParams {
     int batch, total_rows, vocab, max_blocks;

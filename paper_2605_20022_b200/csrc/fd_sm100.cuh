@@ -78,14 +78,7 @@ __device__ __forceinline__ void named_bar_sync(int id, int threads) {
 }
 
 // ---------------------------------------------------------------- TMA (no multicast anywhere)
-// 2-D tiled load: box lands at `dst` (128B-swizzled by the tensor map), completion on `bar`.
-__device__ __forceinline__ void tma_load_2d(void* dst, const void* tmap, int c0, int c1, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
-        : "memory");
-}
-// 3-D tiled load (coordinates innermost first).
+// 3-D tiled load (coordinates innermost first): the box lands at `dst`, swizzled as the tensor map says; completion on `bar`.
 __device__ __forceinline__ void tma_load_3d(void* dst, const void* tmap, int c0, int c1, int c2, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
@@ -102,13 +95,6 @@ __device__ __forceinline__ void tma_load_4d_hint(void* dst, const void* tmap, in
 // Bring the box of a 3-D tiled load into L2 only (no destination, no completion to wait for).
 __device__ __forceinline__ void tma_prefetch_3d(const void* tmap, int c0, int c1, int c2) {
     asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];" ::"l"(tmap), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-// Same, with an L2 eviction policy (see make_policy_evict_first): for data that is read exactly once.
-__device__ __forceinline__ void tma_load_2d_hint(void* dst, const void* tmap, int c0, int c1, uint64_t* bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(smem_u32(dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy)
-        : "memory");
 }
 __device__ __forceinline__ uint64_t make_policy_evict_first() {
     uint64_t pol;

@@ -47,5 +47,19 @@ def whole_job_us_per_step(ms_total: float, steps: int, world: int) -> float:
     return ms_total * 1e3 / (steps * world)
 
 
-def scaling_label() -> str:
-    return "weak"           # per-GPU work is fixed as N grows
+def free_port() -> int:
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def launch_replicas(n: int, script: str, argv: Sequence[str]) -> int:
+    """Run `script argv` as `n` ranks on this node (one process per GPU) under torch.distributed.run and return
+    its exit code.  Used when the benchmark is started as a plain process with --gpus N > 1 and no rank
+    environment; the ranks then find RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* in their environment as usual."""
+    import subprocess
+    import sys
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), script, *argv]
+    return subprocess.run(cmd).returncode

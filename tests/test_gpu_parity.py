@@ -224,14 +224,25 @@ def test_commit_random_and_degenerate():
         np.testing.assert_array_equal(freed, efreed)
 
 
+_LONG_REF = {}   # layer -> oracle output of the whole layer, computed once and shared by both attention paths
+
+
+def _long_context_reference(step, layer):
+    if layer not in _LONG_REF:
+        q, kv = wl.make_q(step, layer, device="cuda").cpu(), wl.make_kv(step, layer, device="cuda").cpu()
+        _LONG_REF[layer] = oracle_attn(step, q, kv)
+    return _LONG_REF[layer]
+
+
 @pytest.mark.parametrize("path", PATHS)
-def test_long_context_full_size_sampled(path):
-    """Workload 5 at its full per-layer size (16 x 32 800 tokens, 2.15 GB of KV per layer, two
-    layers with distinct pools), in the launch configuration the benchmark times; the oracle
-    computes sampled output rows one by one."""
+def test_long_context_full_size_every_element(path):
+    """Workload 5 at its full per-layer size (16 x 32 800 tokens, 2.15 GB of KV per layer, two layers with
+    distinct pools), in the launch configuration the benchmark times (one pinned work list for all layers).
+    Every output element of both layers is compared with the oracle.  At this length an output element is an
+    average over 32 800 values and has a standard deviation near 0.009, so beside the elementwise bound every
+    (row, head) vector must also agree to 2 % of its own length -- a lost tile or a wrong split weight shows there."""
     step = wl.workload(4, n_layers=2)
     dpt, dpl, dql, dnm = (t.cuda() for t in (step.page_table, step.prefix_lens, step.q_lens, step.n_mask))
-    g = torch.Generator().manual_seed(1)
     with Ctx(step, path) as ctx:
         # as the benchmark does for a multi-layer step: one work list, pinned, for every layer
         fd.fd_plan_pin(ctx.h, step.batch, step.total_q_rows, dpl, dql, dnm)
@@ -247,14 +258,13 @@ def test_long_context_full_size_sampled(path):
                     fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, q, kv, step.num_pages, dpt, dpl, dql, dnm, again)
                     assert torch.equal(out, again), "two runs on the same inputs differ bitwise"
                 del again
-            qc, kvc, outc = q.cpu(), kv.cpu(), out.float().cpu().numpy()
-            assert np.isfinite(outc).all()
-            for _ in range(24):
-                b = int(torch.randint(0, 16, (1,), generator=g)); i = int(torch.randint(0, 32, (1,), generator=g))
-                h = int(torch.randint(0, 32, (1,), generator=g))
-                ref = oracle.attn_row(qc, kvc, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, b, i, h)
-                assert_close(outc[b * 32 + i, h], ref, f"layer {layer} b {b} row {i} head {h}")
+            outc = out.float().cpu().numpy()
             del q, kv, out
+            assert np.isfinite(outc).all()
+            ref = _long_context_reference(step, layer)
+            assert_close(outc, ref, f"layer {layer}")
+            rel = np.linalg.norm(outc - ref, axis=-1) / np.linalg.norm(ref, axis=-1)
+            assert rel.max() <= 2e-2, f"layer {layer}: worst (row, head) vector off by {rel.max():.3e} of its length"
 
 
 def test_host_buffer_step_matches_oracle():
@@ -377,8 +387,10 @@ def test_select_branch_matches_oracle():
 
 @pytest.mark.parametrize("V,with_bias", [(151936, True), (151936, False), (4097, True), (1000, True), (37, False), (1, True)])
 def test_draft_select_matches_oracle(V, with_bias):
-    """Draft-side tail (Eq. 4 / Eq. 5): tokens bit-exact, confidences to 1e-4, verify lengths equal wherever the
-    cumulative confidence is not within 1e-3 of the threshold (there the fp32 product may fall on either side)."""
+    """Draft-side tail (Eq. 4 / Eq. 5) against the float64 oracle: tokens equal except where the oracle's margin
+    between the two largest calibrated logits is below what a float32 sum can resolve (counted, bounded), confidences
+    to 1e-4, verify lengths equal wherever the cumulative confidence is not within 1e-3 of the threshold (there the
+    fp32 product may fall on either side)."""
     g = torch.Generator().manual_seed(V)
     M = [16, 0, 28, 6, 32, 12, 1]
     nb = [1, 1, 4, 0, 8, 3, 1]
@@ -392,21 +404,29 @@ def test_draft_select_matches_oracle(V, with_bias):
     step = wl.make_step("ds", wl.Shape(32, 8, 128, V), [5] * B, [32] * B, M, seed=1)
     with Ctx(step) as ctx:
         for thr in (0.5, 0.05):
-            e_tok, e_pr, e_cum, e_keep = oracle.draft_select(logits, bias, n_mask, n_blocks, thr, max_blocks=8)
+            e_tok, e_pr, e_cum, e_keep, e_gap = oracle.draft_select(logits, bias, n_mask, n_blocks, thr, max_blocks=8, want_gap=True)
             tok = torch.full((Rm,), -9, dtype=torch.int32, device="cuda"); pr = torch.zeros((Rm,), device="cuda")
             keep = torch.full((B, 8), -9, dtype=torch.int32, device="cuda")
             fd.fd_draft_select(ctx.h, B, Rm, 8, logits.cuda(), None if bias is None else bias.cuda(), n_mask.cuda(), n_blocks.cuda(),
                                thr, tok, pr, keep)
             assert fd.fd_last_device_status(ctx.h) == 0
-            np.testing.assert_array_equal(tok.cpu().numpy(), e_tok)
-            np.testing.assert_allclose(pr.cpu().numpy(), e_pr, rtol=1e-4, atol=1e-30)
+            # a float32 sum l + bias carries half an ulp of the sum per operand pair: two calibrated logits closer than
+            # that may be ordered either way (or tie, lowest index first); anything wider must agree
+            x_abs = float((logits.abs() + (bias.abs() if bias is not None else 0)).max())
+            near = e_gap <= 2 * np.spacing(np.float32(x_abs))
+            g_tok = tok.cpu().numpy()
+            differ = g_tok != e_tok
+            assert not (differ & ~near).any(), np.nonzero(differ & ~near)
+            assert differ.sum() <= max(1, Rm // 20)
+            same = ~differ
+            np.testing.assert_allclose(pr.cpu().numpy()[same], e_pr[same], rtol=1e-4, atol=1e-30)
             got = keep.cpu().numpy()
             r0 = 0
             for b in range(B):
                 n_b = max(nb[b], 1); kb = M[b] // n_b if M[b] else 0
                 for gk in range(8):
                     c = e_cum[r0 + gk * kb:r0 + (gk + 1) * kb] if (M[b] and gk < n_b) else np.zeros(0)
-                    if c.size and (np.abs(c - thr) < 1e-3 * thr).any():
+                    if c.size and ((np.abs(c - thr) < 1e-3 * thr).any() or differ[r0 + gk * kb:r0 + (gk + 1) * kb].any()):
                         continue                                  # too close to call in fp32
                     assert got[b, gk] == e_keep[b, gk], (b, gk, got[b, gk], e_keep[b, gk])
                 r0 += M[b]
@@ -472,6 +492,40 @@ def test_pinned_plan_serves_every_layer_and_is_dropped_on_other_lengths():
         assert status == 0
         assert_close(got.numpy(), oracle_attn(step2, q2, kv2), "after the pin")
         fd.fd_plan_unpin(ctx.h)
+
+
+def test_commit_drops_the_pinned_plan():
+    """pin, attend, accept-less commit, attend again on the same length arrays without pinning again: the commit has
+    rewritten prefix_lens in place, so the second call must plan for the new lengths, not reuse the old work list."""
+    shape = wl.Shape(32, 8, 128, 1000)
+    step = wl.make_step("pin_commit", shape, [700, 200, 3000], [20, 8, 32], [4, 4, 16], seed=41, extra_table_cols=3)
+    q, kv = wl.make_q(step), wl.make_kv(step, poison=None)           # every page holds data: pages get reassigned below
+    with Ctx(step) as ctx:
+        dq, dkv = q.cuda(), kv.cuda()
+        dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
+        out = torch.empty_like(dq)
+        fd.fd_plan_pin(ctx.h, step.batch, step.total_q_rows, dpl, dql, dnm)
+        fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, dq, dkv, step.num_pages, dpt, dpl, dql, dnm, out)
+        assert_close(out.float().cpu().numpy(), oracle_attn(step, q, kv), "pinned")
+        acc = torch.tensor([15, 0, 7], dtype=torch.int32)
+        freed = torch.empty((64,), dtype=torch.int32, device="cuda"); nf = torch.zeros((1,), dtype=torch.int32, device="cuda")
+        fd.fd_kv_commit(ctx.h, step.batch, dpt, dpl, dql, acc.cuda(), freed, nf)
+        ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, acc)
+        np.testing.assert_array_equal(dpl.cpu().numpy(), epl)
+        # the host hands pages back for the next block (same device arrays, new contents)
+        pool = efreed.tolist() + step.spare_pages.tolist()
+        npt = ept.copy()
+        for b in range(step.batch):
+            for pg in range(-(-(int(epl[b]) + int(step.q_lens[b])) // 16)):
+                if npt[b, pg] < 0:
+                    npt[b, pg] = pool.pop()
+        dpt.copy_(torch.from_numpy(npt))
+        before = fd.fd_launch_count(ctx.h)
+        fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, dq, dkv, step.num_pages, dpt, dpl, dql, dnm, out)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        assert fd.fd_launch_count(ctx.h) - before >= 1
+        ref = oracle.attn(q, kv, npt, epl, step.q_lens, step.n_mask)
+        assert_close(out.float().cpu().numpy(), ref, "after the commit")
 
 
 def _stochastic_case(seed, V, B, T, with_q, max_c=8):
@@ -544,8 +598,13 @@ def test_stochastic_verification_errors():
         assert fd.fd_verify_accept_sample(h, 2, 4, z, None, i4, i4, i4, 0.0, u, u, i4, i4, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
         assert fd.fd_verify_accept_sample(h, 2, 4, None, None, i4, i4, i4, 1.0, u, u, i4, i4, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
         ql = torch.tensor([3, 2], dtype=torch.int32, device="cuda"); nm = torch.zeros((2,), dtype=torch.int32, device="cuda")
-        fd.fd_verify_accept_sample(h, 2, 4, z, None, i4, ql, nm, 1.0, u, u, i4[:2], i4[2:4])      # 5 rows claimed, 4 given
+        acc = torch.full((2,), 7, dtype=torch.int32, device="cuda"); bon = torch.full((2,), 7, dtype=torch.int32, device="cuda")
+        fd.fd_verify_accept_sample(h, 2, 4, z, None, i4, ql, nm, 1.0, u, u, acc, bon)             # 5 rows claimed, 4 given
         assert fd.fd_last_device_status(h) == fd.FD_DEV_BAD_LENGTHS
+        assert (acc == -1).all() and (bon == -1).all()           # the convention of every call: -1 for all sequences
+        ql = torch.tensor([3, 1], dtype=torch.int32, device="cuda")
+        fd.fd_verify_accept_sample(h, 2, 4, z, None, i4, ql, nm, 1.0, u, u, acc, bon)             # the context still works
+        assert fd.fd_last_device_status(h) == 0 and (acc >= 0).all() and (bon >= 0).all()
     finally:
         fd.fd_destroy(h)
 

@@ -130,3 +130,20 @@ def test_sequences_without_candidate_rows():
     acc, bon, _ = oracle.accept_stochastic(np.zeros((0, 5), np.float32), None, np.zeros((0,), np.int32), np.array([4], np.int32),
                                           np.array([4], np.int32), 1.0, np.zeros((0,), np.float32), np.zeros((1,), np.float32))
     assert acc[0] == -1 and bon[0] == -1
+
+
+def test_draft_token_without_drafter_mass():
+    """A draft the drafter itself gives probability 0 (Sec. 3's ratio p/q has no value there): the product form of
+    the test, u q(x) < p(x), accepts it exactly when the target gives it mass, and rejects it when neither does."""
+    V, T = 6, 1.0
+    lp = np.zeros((3, 2, V), np.float32); ld = np.zeros((3, 2, V), np.float32)
+    ld[:, 0, 2] = -np.inf                             # q_0(2) = 0 in every sequence
+    lp[1, 0, 2] = -np.inf                             # sequence 1: p_0(2) = 0 as well
+    lp[2, 0, :] = -np.inf; lp[2, 0, 2] = 0.0          # sequence 2: p_0 is a point mass on token 2
+    drafts = np.zeros((6,), np.int32); drafts[1::2] = 2
+    ql = np.full((3,), 2, np.int32); nm = np.zeros((3,), np.int32)
+    for u in (0.0, 0.5, 0.999):
+        ua = np.full((6,), u, np.float32); ub = np.full((3,), 0.3, np.float32)
+        acc, bon, ratio = oracle.accept_stochastic(lp.reshape(6, V), ld.reshape(6, V), drafts, ql, nm, T, ua, ub)
+        assert acc.tolist() == [1, 0, 1]
+        assert bon[1] != 2                            # the residual of sequence 1 has no mass on the rejected token

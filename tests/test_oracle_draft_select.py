@@ -16,15 +16,29 @@ def make(B=5, V=300, seed=0, M=(12, 0, 8, 6, 16), nb=(3, 1, 2, 0, 4)):
 
 def test_tokens_and_confidence_against_library_softmax():
     logits, bias, M, nb = make()
-    tok, pr, cum, keep = oracle.draft_select(logits, bias, M, nb, 0.3, max_blocks=4)
-    x = (logits + bias).float()                                  # float32 sum, as the definition states
+    tok, pr, cum, keep, gap = oracle.draft_select(logits, bias, M, nb, 0.3, max_blocks=4, want_gap=True)
+    x = logits.double() + bias.double()                          # Eq. 4's sum, exact in float64 for float32 inputs
     np.testing.assert_array_equal(tok, x.argmax(dim=1).numpy())
-    ref = torch.softmax(x.double(), dim=1)[torch.arange(x.shape[0]), torch.from_numpy(tok).long()]
+    ref = torch.softmax(x, dim=1)[torch.arange(x.shape[0]), torch.from_numpy(tok).long()]
     np.testing.assert_allclose(pr, ref.numpy(), rtol=1e-12)
+    top2 = torch.topk(x, 2, dim=1).values
+    np.testing.assert_allclose(gap, (top2[:, 0] - top2[:, 1]).numpy(), rtol=0, atol=0)
     # without a bias the logits themselves decide
     tok0, pr0, _, _ = oracle.draft_select(logits, None, M, nb, 0.3, max_blocks=4)
     np.testing.assert_array_equal(tok0, logits.argmax(dim=1).numpy())
     assert (tok0 != tok).any()                                   # the calibration changes some drafts
+
+
+def test_sum_is_not_rounded_to_float32():
+    """Two calibrated logits that a float32 sum makes equal (lower index would win) but whose exact sums differ."""
+    V = 8
+    logits = np.zeros((1, V), np.float32); bias = np.zeros((1, V), np.float32)
+    logits[0, 2] = 1.0; bias[0, 2] = 2.0 ** -26                 # 1 + 2^-26 rounds to 1 in float32
+    logits[0, 5] = 1.0; bias[0, 5] = 2.0 ** -25                 # so does 1 + 2^-25, the larger exact sum
+    assert np.float32(logits[0, 2] + bias[0, 2]) == np.float32(logits[0, 5] + bias[0, 5])
+    tok, pr, cum, keep, gap = oracle.draft_select(logits, bias, np.array([1], np.int32), None, 0.5, max_blocks=1, want_gap=True)
+    assert tok[0] == 5
+    assert 0 < gap[0] < 1e-7
 
 
 def test_cumulative_confidence_and_keep_len_against_numpy():

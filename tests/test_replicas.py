@@ -58,3 +58,16 @@ def test_reference_arm_under_two_ranks_prints_once():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["higher_is_better"] is False
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["vs_baseline"] is None and line["value"] > 0 and line["unit"] == "us/step"
+
+
+def test_plain_process_with_gpus_2_starts_two_ranks_itself():
+    """`python bench.py --gpus 2` without a rank environment re-launches itself as two ranks (one per GPU on a GPU
+    box); shown here on CPU with the reference arm: one JSON line comes back, from rank 0, with n_gpus = 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--workload", "0", "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
