@@ -72,8 +72,24 @@ enum {
 enum {
     FD_ATTN_AUTO = 0,         /* tensor-core kernel when the shape allows it, else the SIMT kernel */
     FD_ATTN_SIMT = 1,         /* CUDA-core split-KV kernel (any supported shape) */
-    FD_ATTN_TCGEN05 = 2       /* tcgen05 / TMEM / TMA split-KV kernel (head_dim 64 or 128) */
+    FD_ATTN_TCGEN05 = 2,      /* tcgen05 / TMEM / TMA split-KV kernel (head_dim 64 or 128); how it finds its work is
+                                 chosen per call, see FD_TC_* */
+    FD_ATTN_TCGEN05_PLANNED = 3,      /* the same kernel, always on the plan kernel's work list (FD_TC_PLANNED) */
+    FD_ATTN_TCGEN05_SELF_PLANNED = 4  /* the same kernel, planning for itself wherever the call is small enough
+                                         (FD_TC_SELF_PLANNED), never one cluster per segment */
 };
+
+/* How a call of the tensor-core attention kernel found its work (fd_attn_last_mode).  All three give the same
+ * result to within rounding order; the choice is about fixed cost.
+ *   FD_TC_PLANNED       a one-CTA plan kernel (or fd_plan_pin, once per step) cuts all KV tiles of the call into
+ *                       one range per SM ("stream-K"); ranges that share a (sequence, kv-head) segment leave
+ *                       partial results in scratch memory and the last to arrive merges them.
+ *   FD_TC_SELF_PLANNED  at most 24 sequences with query blocks of at most 128 / G rows: every CTA makes the same
+ *                       cut itself in its prologue; one launch, nothing to wait for.
+ *   FD_TC_CLUSTER       at most 18 segments (batch 1-2 at 8 kv-heads, the paper's parallel-mode operating point):
+ *                       one thread-block cluster of up to 16 CTAs per segment splits its tiles evenly and merges
+ *                       through distributed shared memory; one launch, no scratch memory, no counters. */
+enum { FD_TC_PLANNED = 0, FD_TC_SELF_PLANNED = 1, FD_TC_CLUSTER = 2 };
 
 typedef struct {
     int n_q_heads;            /* Hq */
@@ -141,13 +157,14 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * Optional: pin the work list of a step.  The attention call derives a work list (which CTA streams which
  * KV tiles) from the lengths alone; it is the same for every layer of a step.  fd_plan_pin computes it once;
  * until fd_plan_unpin, every fd_attn_draft_verify[_blocks] call with the same batch, total_q_rows and the
- * same four length pointers reuses it instead of recomputing it (a call with anything else recomputes and
- * drops the pin).  The caller must not change the contents of the length arrays while the pin holds, and
- * must unpin after a FD_DEV_TIMEOUT status.  fd_kv_commit rewrites prefix_lens and therefore drops the pin
+ * same four length pointers reuses it instead of recomputing it (a call with anything else that needs the plan
+ * kernel recomputes and drops the pin; calls that plan for themselves, FD_TC_SELF_PLANNED and FD_TC_CLUSTER,
+ * leave it alone).  The caller must not change the contents of the length arrays while the pin holds, and
+ * must unpin after a FD_DEV_TIMEOUT status (fd_last_device_status does so
+ * itself when it reports that bit).  fd_kv_commit rewrites prefix_lens and therefore drops the pin
  * itself: the first attention call of the next step plans afresh (or is preceded by a new fd_plan_pin).
  * fd_kv_append leaves the lengths alone and keeps the pin.
- * A sequence flagged for a page id outside the pool (FD_DEV_BAD_PAGE) stays flagged, and its rows zero,
- * for every call served by the same pin.  The calls served by a pin must be ordered after fd_plan_pin (the
+ * The calls served by a pin must be ordered after fd_plan_pin (the
  * same stream, or streams the caller has ordered) and must not overlap one another: they share the context's
  * scratch memory, as all attention calls on one context do.
  * The paper does not describe a work list; this follows from "all layers of a step share the lengths".
@@ -419,6 +436,9 @@ fd_status fd_selftest_wait_timeout(fd_ctx* ctx, int limit_ms, void* stream);
 
 /* Which attention kernel the context resolved to: FD_ATTN_SIMT or FD_ATTN_TCGEN05. */
 int fd_attn_path(const fd_ctx* ctx);
+
+/* FD_TC_* of the context's most recent tensor-core attention call, -1 before the first one. */
+int fd_attn_last_mode(const fd_ctx* ctx);
 
 /* Number of CUDA kernels this library has launched through `ctx` since fd_create. */
 int64_t fd_launch_count(const fd_ctx* ctx);

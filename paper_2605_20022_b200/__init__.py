@@ -20,9 +20,11 @@ FD_ERR_STATIC_LIMIT = 6
 FD_STATIC_MAX_ROWS, FD_STATIC_MAX_BATCH = 4096, 4096
 FD_DEV_BAD_LENGTHS, FD_DEV_BAD_PAGE, FD_DEV_TIMEOUT, FD_DEV_BAD_ACCEPT = 1, 2, 4, 8
 FD_ATTN_AUTO, FD_ATTN_SIMT, FD_ATTN_TCGEN05 = 0, 1, 2
+FD_ATTN_TCGEN05_PLANNED, FD_ATTN_TCGEN05_SELF_PLANNED = 3, 4
+FD_TC_PLANNED, FD_TC_SELF_PLANNED, FD_TC_CLUSTER = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
-           "fd_last_device_status", "fd_attn_path", "fd_launch_count", "fd_status_string",
+           "fd_last_device_status", "fd_attn_path", "fd_attn_last_mode", "fd_launch_count", "fd_status_string",
            "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_verify_accept_sample", "fd_plan_ranges_host"]
 
 
@@ -73,6 +75,7 @@ def load() -> ctypes.CDLL:
         lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 14
         lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         lib.fd_attn_path.argtypes = [vp]
+        lib.fd_attn_last_mode.argtypes = [vp]
         lib.fd_launch_count.argtypes = [vp]
         lib.fd_launch_count.restype = ctypes.c_int64
         lib.fd_status_string.argtypes = [ci]
@@ -245,6 +248,10 @@ def fd_last_device_status(ctx, stream=None) -> int:
 
 def fd_attn_path(ctx) -> int:
     return load().fd_attn_path(ctx)
+
+
+def fd_attn_last_mode(ctx) -> int:
+    return load().fd_attn_last_mode(ctx)
 
 
 def fd_launch_count(ctx) -> int:

@@ -11,7 +11,10 @@ struct fd_ctx {
     int device;
     int n_sms;
     int n_ctas;        // attention grid
-    int attn_path;     // resolved FD_ATTN_*
+    int attn_path;     // resolved FD_ATTN_SIMT or FD_ATTN_TCGEN05
+    int tc_choice;     // FD_ATTN_TCGEN05 (per call), FD_ATTN_TCGEN05_PLANNED or FD_ATTN_TCGEN05_SELF_PLANNED
+    int last_mode;     // FD_TC_* of the last tensor-core call
+    int epoch;         // number of the last attention call (never 0 once a call was made)
     float scale_log2e;
     // scratch (device)
     unsigned char* pool;
@@ -114,7 +117,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
         cfg->max_q_len <= 0 || cfg->max_pages_per_seq <= 0 || cfg->softmax_scale < 0.f)
         return FD_ERR_INVALID_ARG;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FD_ERR_INVALID_ARG;
-    if (cfg->attn_path < FD_ATTN_AUTO || cfg->attn_path > FD_ATTN_TCGEN05) return FD_ERR_INVALID_ARG;
+    if (cfg->attn_path < FD_ATTN_AUTO || cfg->attn_path > FD_ATTN_TCGEN05_SELF_PLANNED) return FD_ERR_INVALID_ARG;
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
     if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return FD_ERR_UNSUPPORTED;
     if (G > fd::kMaxRows || cfg->max_q_len > 4096) return FD_ERR_UNSUPPORTED;  // at least one block row per 128-row tile
@@ -136,7 +139,10 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->scale_log2e = scale * 1.4426950408889634f;
 
     const bool tc_ok = fd::attn_tc_supported(cfg->head_dim, G, cfg->max_q_len);
-    if (cfg->attn_path == FD_ATTN_TCGEN05 && !tc_ok) { delete c; return FD_ERR_UNSUPPORTED; }
+    if (cfg->attn_path >= FD_ATTN_TCGEN05 && !tc_ok) { delete c; return FD_ERR_UNSUPPORTED; }
+    c->tc_choice = cfg->attn_path >= FD_ATTN_TCGEN05 ? cfg->attn_path : FD_ATTN_TCGEN05;
+    c->last_mode = -1;
+    c->epoch = 0;
     c->attn_path = (cfg->attn_path == FD_ATTN_SIMT || !tc_ok) ? FD_ATTN_SIMT : FD_ATTN_TCGEN05;
     // SIMT kernel: two 74 KB CTAs fit an SM; tensor-core kernel: one persistent CTA per SM
     c->n_ctas = c->attn_path == FD_ATTN_SIMT ? 2 * c->n_sms : c->n_sms;
@@ -185,7 +191,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->plan.rb = reinterpret_cast<fd::RowBlock*>(c->pool + o_rb);
     c->plan.cu_q = reinterpret_cast<int*>(c->pool + o_cuq);
     c->plan.cu_tiles = reinterpret_cast<int*>(c->pool + o_cut);
-    c->plan.seq_ok = reinterpret_cast<int*>(c->pool + o_ok);
+    c->plan.seq_bad = reinterpret_cast<int*>(c->pool + o_ok);
     c->plan.seg_count = reinterpret_cast<int*>(c->pool + o_sc);
     c->plan.cta_first = reinterpret_cast<int*>(c->pool + o_cf);
     c->plan.cta_start = reinterpret_cast<int*>(c->pool + o_cs);
@@ -374,6 +380,8 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
 
 int fd_attn_path(const fd_ctx* c) { return c ? c->attn_path : -1; }
 
+int fd_attn_last_mode(const fd_ctx* c) { return c ? c->last_mode : -1; }
+
 int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
 
 fd_status fd_attn_draft_verify(fd_ctx* c, int batch, int total_q_rows, const void* q, const void* kv_cache,
@@ -409,18 +417,31 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     if (tc) {
         if (fd::attn_tc_prepare(&c->tc_state, p) != cudaSuccess) { cudaGetLastError(); return FD_ERR_CUDA; }
     }
+    c->epoch = c->epoch == 0x7fffffff ? 1 : c->epoch + 1;
+    p.epoch = c->epoch;
     // a pinned plan serves this call if it was made for exactly these lengths; anything else replaces it
     const bool reuse = c->pinned && batch == c->pin_batch && total_q_rows == c->pin_rows && prefix_lens == c->pin_pl &&
                        q_lens == c->pin_ql && n_mask == c->pin_nm && n_blocks == c->pin_nb;
-    if (!reuse) {
+    // How the tensor-core kernel finds its work.  A call of few segments runs one cluster per segment; a call of
+    // few sequences plans for itself (unless a pinned plan is there to use); everything else uses the plan kernel.
+    int mode = fd::kTcPlanned;
+    if (tc && p.rb_per_seq == 1 && c->tc_choice != FD_ATTN_TCGEN05_PLANNED) {
+        const int n_seg = batch * p.Hkv;
+        const int cl = (c->tc_choice == FD_ATTN_TCGEN05 && batch <= fd::kSelfPlanMaxRb && n_seg <= fd::kClusterMaxSegments)
+                           ? fd::attn_tc_cluster_size(c->tc_state, n_seg, c->n_sms) : 0;
+        if (cl >= 2) { mode = fd::kTcCluster; p.cluster = cl; }
+        else if (batch <= fd::kSelfPlanMaxRb && !reuse) mode = fd::kTcSelfPlanned;
+    }
+    if (mode == fd::kTcPlanned && !reuse) {
         c->pinned = false;
         fd::launch_plan(p, s);
         c->launches += 1;
     }
     if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
     } else if (tc) {
-        fd::launch_attn_tc(c->tc_state, p, s);  // merges split segments in its own epilogue
+        fd::launch_attn_tc(c->tc_state, p, mode, s);  // merges split segments in its own epilogue
         c->launches += 1;
+        c->last_mode = mode;
     } else {
         fd::launch_attn_simt(p, s);
         fd::launch_merge(p, s);
@@ -607,6 +628,11 @@ fd_status fd_last_device_status(fd_ctx* c, int32_t* code, void* stream) {
     if (cudaMemcpyAsync(code, c->status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return FD_ERR_CUDA;
     if (cudaMemsetAsync(c->status, 0, sizeof(int), s) != cudaSuccess) return FD_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return FD_ERR_CUDA;
+    if (*code & FD_DEV_TIMEOUT) {
+        // a call that gave up may have left pieces counted on segments nobody merged: start the next call clean
+        c->pinned = false;
+        if (cudaMemsetAsync(c->plan.seg_count, 0, (size_t)c->max_rb * c->cfg.n_kv_heads * sizeof(int), s) != cudaSuccess) return FD_ERR_CUDA;
+    }
     return FD_OK;
 }
 

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kMaxRows) attn_simt_kernel(AttnParams p) {
                 if (pos0 >= kv_len) break;
                 int phys = p.page_table[(long long)b * p.max_pages + pos0 / 16];
                 if ((unsigned)phys >= (unsigned)p.num_pages) {  // never form an address from a bad id
-                    if (r == 0) { p.plan.seq_ok[b] = 0; atomicOr(p.status, FD_DEV_BAD_PAGE); }
+                    if (r == 0) flag_sequence(p, b);
                     phys = 0;
                 }
                 const __nv_bfloat16* kp = p.kv + (((long long)phys * 2 + 0) * p.Hkv + kvh) * 16 * D;

@@ -62,16 +62,26 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units
 #define FD_QK_MODE 1
 #endif
 
-template <int D>
+template <int D, int MODE>
 struct Cfg {
-    static constexpr int kStages = (D == 128) ? 3 : 6;   // buffers in the K ring, and again in the V ring
+    static constexpr int kFullStages = (D == 128) ? 3 : 6;
+    // buffers in the K ring, and again in the V ring.  With one cluster per segment a CTA has few tiles and gives a
+    // third of the ring space to the partial results its peers send it (see the epilogue of softmax_role).
+    static constexpr int kStages = MODE == kTcCluster ? ((D == 128) ? 2 : 5) : kFullStages;
     static constexpr int kQBytes = kMaxRows * D * 2;
     static constexpr int kKBytes = kTileTokens * D * 2;  // one K (or V) tile
-    static constexpr int kBarOffset = kQBytes + 2 * kStages * kKBytes;
+    static constexpr int kRecvOffset = kQBytes + 2 * kStages * kKBytes;        // kTcCluster: (m, l) pairs, then rows of O, from the peers
+    static constexpr int kRecvBytes = 2 * (kFullStages - kStages) * kKBytes;
+    static constexpr int kRecvMlBytes = kMaxRows * 8;                           // [cluster size][rows per CTA] float2
+    static constexpr int kBarOffset = kQBytes + 2 * kFullStages * kKBytes;
     static constexpr int kCsOffset = kBarOffset + 320;           // window of the CTA range starts
     static constexpr int kDescOffset = kBarOffset + 448;         // ring of piece descriptors
+    static constexpr int kScanOffset = kBarOffset + 720;         // SelfScans: the scans of a call that plans for itself
     static constexpr int kExOffset = kBarOffset + 1024;          // [2][128] floats: stream exchange in the epilogue
-    static constexpr int kSmemBytes = kExOffset + 1024 + 1024;   // + slack for 1024-byte alignment
+    static constexpr int kRbOffset = kBarOffset + 2048;          // row blocks of a call that plans for itself
+    static constexpr int kSmemBytes = kBarOffset + 3072;         // the dynamic shared memory is declared 1024-byte aligned
+    // what a CTA receives: (m, l) of every peer, and O rows of every peer but itself, for its 128 / cluster-size rows
+    static_assert(MODE != kTcCluster || kRecvMlBytes + (kMaxRows * D * 4) / 2 <= kRecvBytes, "receive area too small for a cluster of 2");
     static constexpr int kKSteps = D / 16;
     static constexpr int kHalves = D / 64;
     // A K or V tile in shared memory: [8-token group][half of d][8 rows][128 B] -- what one TMA box per page
@@ -91,8 +101,22 @@ struct Bars {
     int epi_flag;              // per-epilogue decisions of thread 0: bit 0 merge, bit 1 leave
     int desc_n;                // piece descriptors published so far (written by the Q load warp)
     int piece_ok;              // thread 0 of the softmax groups: the descriptor of the next piece is there
+    int first;                 // a call that plans for itself: the row block that owns the first tile of this CTA's range
 };
 constexpr int kDescSlots = 4;
+
+// The plan of a call that plans for itself (at most kSelfPlanMaxRb sequences, one row block each), in shared memory.
+struct SelfScans {
+    int cu_q[kSelfPlanMaxRb + 1], cu_tiles[kSelfPlanMaxRb + 1], cu_ne[kSelfPlanMaxRb + 1];
+    int fatal;
+};
+static_assert(sizeof(SelfScans) <= 304, "SelfScans must fit between the descriptor ring and the exchange buffer");
+static_assert(sizeof(RowBlock) * kSelfPlanMaxRb <= 1024, "row blocks of a self-planned call must fit their slot");
+
+// The tiles [s_c, e_c) a CTA works on and the row block that owns the first of them.
+struct Range {
+    int s_c, e_c, first;
+};
 static_assert(sizeof(Bars) <= 320, "Bars must fit in front of the range-start window");
 
 struct Piece {
@@ -103,6 +127,7 @@ struct Piece {
 // Piece that starts at tile t.  `hint` is a row block at or before the one that owns t (pieces are walked in
 // order, so the previous piece's row block will do): a short forward walk replaces a search.
 __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int n_rb, int t, int s_c, int e_c, int cta, int hint) {
+    // p.plan may point into shared memory (a call that plans for itself): plain loads either way
     Piece pc;
     int lo = hint;
     while (lo + 1 < n_rb && p.Hkv * p.plan.cu_tiles[lo + 1] <= t) ++lo;
@@ -127,7 +152,8 @@ __device__ __forceinline__ Piece decode_piece(const AttnParams& p, int n_rb, int
     pc.kv_len = pc.n + pc.Lq;
     pc.rows = pc.Lv * p.G;
     pc.row0 = p.plan.cu_q[lo];
-    pc.complete = (t == seg_start) && (t_end == seg_end);
+    // with one cluster per segment every piece goes through the cluster merge, a piece that holds all tiles too
+    pc.complete = (t == seg_start) && (t_end == seg_end) && p.cluster == 0;
     pc.slot = 2 * cta + (t == s_c ? 0 : 1);
     return pc;
 }
@@ -200,10 +226,10 @@ struct Walk {
 };
 
 // K (which = 0) or V (which = 1) load warp.
-template <int D>
+template <int D, int MODE>
 __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnParams& p, int n_rb, unsigned char* ring, uint64_t* full,
-                                          uint64_t* empty, int which, int s_c, int e_c, volatile int* abort) {
-    using C = Cfg<D>;
+                                          uint64_t* empty, int which, const Range rg, volatile int* abort) {
+    using C = Cfg<D, MODE>;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     constexpr int kOps = 8;  // pages of a tile: one box each
     const int pg = lane;
@@ -211,7 +237,8 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     // the KV stream is read once: let it leave L2 first, so that Q, the split partials and the page
     // table (all re-read) stay resident next to a stream many times the size of the cache
     const uint64_t policy = make_policy_evict_first();
-    Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
+    const int s_c = rg.s_c, e_c = rg.e_c;
+    Walk w = {s_c, 0, {0, 0}, 0, rg.first};
     bool ok = true;
     while (w.t < e_c && ok) {
         const Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
@@ -225,8 +252,7 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             if (!(j < pc.nt && pos < pc.kv_len)) return -1;
             int id = table[pos >> 4];
             if ((unsigned)id >= (unsigned)p.num_pages) {  // never form an address from a bad id
-                p.plan.seq_ok[pc.b] = 0;
-                atomicOr(p.status, FD_DEV_BAD_PAGE);
+                flag_sequence(p, pc.b);
                 id = 0;
             }
             return id;
@@ -264,13 +290,14 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
 // lands as q_box_t * G consecutive 128-byte rows, row (i, g) at i * G + g: the order the MMA wants.  The
 // last box of a piece may reach past the block (rows of the next sequence, or zeros past T): each query
 // row only ever influences its own output row, and those rows are never stored.
-template <int D>
+template <int D, int MODE>
 __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams& p, int n_rb, unsigned char* sq, Bars* bars, Piece* ring,
-                                       int s_c, int e_c, volatile int* abort) {
-    using C = Cfg<D>;
+                                       const Range rg, volatile int* abort) {
+    using C = Cfg<D, MODE>;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     const int bt = p.q_box_t;
-    Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
+    const int s_c = rg.s_c, e_c = rg.e_c;
+    Walk w = {s_c, 0, {0, 0}, 0, rg.first};
     int issued = 0;
     Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
     if (lane == 0) publish_piece(bars, ring, 0, pc);
@@ -302,17 +329,18 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
 }
 
 // MMA issuing warp.
-template <int D>
+template <int D, int MODE>
 __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq, unsigned char* sk, unsigned char* sv, Bars* bars,
-                                         const Piece* ring, uint32_t tmem, int s_c, int e_c, volatile int* abort) {
-    using C = Cfg<D>;
-    const int lane = threadIdx.x & 31, cta = blockIdx.x;
+                                         const Piece* ring, uint32_t tmem, const Range rg, volatile int* abort) {
+    using C = Cfg<D, MODE>;
+    const int lane = threadIdx.x & 31;
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
     constexpr uint32_t idesc_qk_half = make_idesc_bf16(128, kTileTokens / 2, false);
     constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
     const uint32_t q_addr = smem_u32(sq);
-    Walk w = {s_c, 0, {0, 0}, 0, p.plan.cta_first[cta]};
+    const int s_c = rg.s_c, e_c = rg.e_c;
+    Walk w = {s_c, 0, {0, 0}, 0, rg.first};
     bool ok = true;
     while (w.t < e_c && ok) {
         if (!__all_sync(0xffffffffu, wait_piece(bars, w.piece, abort))) break;
@@ -401,21 +429,119 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
     }
 }
 
-// The two softmax groups (256 threads).
+// ---------------------------------------------------------------------------------------------
+// One cluster per segment (kTcCluster).  The CTAs of a cluster split the segment's tiles evenly.  Query row r of the
+// segment is owned by CTA r / share of the cluster (share = 128 / cluster size): every CTA sends the unnormalised
+// partial result of the rows it does not own -- O in fp32 and (m, l) -- straight into the owner's shared memory
+// (st.shared::cluster: stores need no round trip), keeps the rows it owns in registers, and after ONE cluster
+// barrier each owner combines what it received with its own part, in rank order (fixed, so the result does not
+// depend on timing), and writes the bf16 rows.  After the barrier nobody touches a peer's memory again, so a CTA
+// may leave as soon as its own rows are written.  No global scratch, no counters, no waiting on flags.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {  // every thread of every CTA of the cluster
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t peer_addr(uint32_t saddr, uint32_t rank) {  // the same offset in CTA `rank` of the cluster
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_peer_v4(uint32_t addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_peer_v2(uint32_t addr, float2 v) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v.x), "f"(v.y) : "memory");
+}
+__device__ __forceinline__ float2 lds_v2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 lds_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+constexpr int kMaxCluster = 16;
+
+// The receive area of a CTA: (m, l) of source CTA c for owned row rl at ml[c * share + rl]; the O row of source c
+// (c != own rank; slot = c, less one past the own rank) as D / 4 16-byte words, word w at position w ^ (rl & 31):
+// the thread-per-row stores of the senders and of the owner's reads then both spread over all banks.
 template <int D>
+struct Recv {
+    uint32_t base;  // shared-memory address (the same offset in every CTA of the cluster)
+    int share;
+    __device__ __forceinline__ uint32_t ml(int c, int rl) const { return base + (uint32_t)(c * share + rl) * 8; }
+    __device__ __forceinline__ uint32_t o(int slot, int rl, int word) const {
+        return base + kMaxRows * 8 + (uint32_t)((slot * share + rl) * (D / 4) + (word ^ (rl & (D / 4 - 1)))) * 16;
+    }
+};
+
+// Owner side, after the cluster barrier: thread (row r, half s of the columns) combines the C parts of its row.
+// `own`: this CTA's own part of the row, the thread's D / 2 columns (nullptr: it had no tiles).
+template <int D>
+__device__ __forceinline__ void cluster_reduce_row(const AttnParams& p, const Recv<D> rv, int rank, int r, int s, const float* own, int b,
+                                                   int kvh, int row0) {
+    const int C = p.cluster, rl = r % rv.share;
+    float m = -INFINITY;
+    for (int c = 0; c < C; ++c) m = fmaxf(m, lds_v2(rv.ml(c, rl)).x);
+    float acc[D / 2];
+#pragma unroll
+    for (int k = 0; k < D / 2; ++k) acc[k] = 0.f;
+    float l = 0.f;
+    for (int c = 0; c < C; ++c) {
+        const float2 ml = lds_v2(rv.ml(c, rl));
+        if (ml.x == -INFINITY) continue;  // that CTA saw no visible key for the row: it sent no O
+        const float w = exp2f(ml.x - m);
+        l += w * ml.y;
+        if (c == rank) {
+            if (own) {
+#pragma unroll
+                for (int k = 0; k < D / 2; ++k) acc[k] += w * own[k];
+            }
+        } else {
+            const int slot = c < rank ? c : c - 1;
+#pragma unroll
+            for (int k = 0; k < D / 8; ++k) {
+                const float4 v = lds_v4(rv.o(slot, rl, s * (D / 8) + k));
+                acc[4 * k] += w * v.x; acc[4 * k + 1] += w * v.y; acc[4 * k + 2] += w * v.z; acc[4 * k + 3] += w * v.w;
+            }
+        }
+    }
+    float inv = l > 0.f ? 1.f / l : 0.f;
+    if (sequence_flagged(p, b)) {  // by assignment: what came from a stand-in page may be inf or NaN
+        inv = 0.f;
+#pragma unroll
+        for (int k = 0; k < D / 2; ++k) acc[k] = 0.f;
+    }
+    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + s * (D / 2);
+#pragma unroll
+    for (int ch = 0; ch < D / 64; ++ch) store_cols_bf16<32>(dst + ch * 32, acc + ch * 32, inv);
+}
+
+// The two softmax groups (256 threads).
+template <int D, int MODE>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, int* s_cs, const CtaStarts cs, const Piece* ring,
-                                             uint32_t tmem, int s_c, int e_c, volatile int* abort) {
+                                             uint32_t tmem, const Range rg, uint32_t recv_addr, int cl_rank, volatile int* abort) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
+    const int s_c = rg.s_c, e_c = rg.e_c;
     const int s = warp >> 2;                  // stream
     const int r = (warp & 3) * 32 + lane;     // query row == TMEM lane
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
     const float c = p.scale_log2e;
     // fill the window of range starts; the barrier below orders it before its first use
-    if (tid < kCsWindow) {
+    if (MODE == kTcPlanned && tid < kCsWindow) {  // (a call that plans for itself has filled it while planning)
         const int cc = cs.base + tid;
-        s_cs[tid] = (cc >= 0 && cc <= p.n_ctas) ? p.plan.cta_start[cc] : 0;
+        s_cs[tid] = (cc >= 0 && cc <= p.n_ctas) ? cs.g[cc] : 0;
     }
+    bool cl_synced = false;
     Walk w = {s_c, 0, {0, 0}, 0, 0};
     while (w.t < e_c) {
         // one thread waits for the descriptor, so that all 256 take the same decision
@@ -546,7 +672,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         constexpr int kChunks = D / 64;  // 32-column chunks per softmax group
         const bool do_read = !leave && warp_active;
         // the load warps of this CTA have seen every page id of the segment by now
-        const bool zero_rows = pc.complete && !__ldcg(p.plan.seq_ok + pc.b);
+        const bool zero_rows = pc.complete && sequence_flagged(p, pc.b);
         float o[kChunks][32];  // this thread's row, its group's half of the columns
 #pragma unroll
         for (int ch = 0; ch < kChunks; ++ch) {
@@ -569,7 +695,17 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 tc_fence_before();
                 mbar_arrive(&bars->o_free);           // O has been read: the next piece may overwrite it
             }
-            if (do_read && r < pc.rows) {
+            if (MODE == kTcCluster) {
+                // one cluster per segment: a row another CTA owns goes straight into that CTA's receive area
+                const int share = kMaxRows / p.cluster, dest = r / share;
+                if (do_read && r < pc.rows && dest != cl_rank) {
+                    const Recv<D> rv = {recv_addr, share};
+                    const int slot = cl_rank < dest ? cl_rank : cl_rank - 1;
+#pragma unroll
+                    for (int k = 0; k < 32; k += 4)
+                        st_peer_v4(peer_addr(rv.o(slot, r % share, (col + k) >> 2), dest), make_float4(o[ch][k], o[ch][k + 1], o[ch][k + 2], o[ch][k + 3]));
+                }
+            } else if (do_read && r < pc.rows) {
                 if (pc.complete) {
                     __nv_bfloat16* dst = p.out + ((long long)(pc.row0 + i) * p.Hq + pc.kvh * p.G + r % p.G) * D + col;
                     if (zero_rows) {  // by assignment: what was computed from a stand-in page may be inf or NaN
@@ -584,11 +720,21 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 }
             }
         }
-        if (do_read && r < pc.rows && !pc.complete && s == 0) {
+        if (MODE == kTcCluster) {
+            const int share = kMaxRows / p.cluster, dest = r / share;
+            const Recv<D> rv = {recv_addr, share};
+            // (m, l) of the row to its owner (which may be this CTA); a row this CTA could not compute (it is giving up)
+            // counts as "saw no key"
+            if (r < pc.rows && s == 0) st_peer_v2(peer_addr(rv.ml(cl_rank, r % share), dest), do_read ? make_float2(mm, L) : make_float2(-INFINITY, 0.f));
+            cluster_sync_all();  // all 256 threads, whatever happened before; the other warps of the CTA wait in the kernel body
+            cl_synced = true;
+            if (r < pc.rows && dest == cl_rank && !leave)
+                cluster_reduce_row<D>(p, rv, cl_rank, r, s, do_read ? &o[0][0] : nullptr, pc.b, pc.kvh, pc.row0);
+        } else if (do_read && r < pc.rows && !pc.complete && s == 0) {
             p.part.m[pc.slot * kMaxRows + r] = mm;
             p.part.l[pc.slot * kMaxRows + r] = L;
         }
-        if (!pc.complete) {
+        if (MODE != kTcCluster && !pc.complete) {
             // Fused split merge: count the delivered pieces of the segment; whoever delivers the last
             // one combines them all (no CTA ever waits for another).  The barrier orders the partial
             // stores of all threads before thread 0's fence, and the fence before the count.
@@ -620,14 +766,72 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         if (leave) break;
         w.advance(pc);
     }
+    // a CTA that gave up before its epilogue still owes the cluster its arrival: the peers must not wait for ever
+    if (MODE == kTcCluster && !cl_synced) cluster_sync_all();
 }
 
-template <int D>
+// ---------------------------------------------------------------------------------------------
+// A call that plans for itself (kTcSelfPlanned, kTcCluster): at most kSelfPlanMaxRb sequences, one row block
+// each.  Warp 0 of every CTA checks the lengths and makes the scans the plan kernel would have made, into
+// shared memory; the roles then read them through the same Plan pointers.  No launch, no dependency.
+// ---------------------------------------------------------------------------------------------
+template <int MODE>
+__device__ __forceinline__ void self_plan(const AttnParams& p, SelfScans* sc, RowBlock* rbs, int* s_cs, int* s_first) {
+    const int lane = threadIdx.x & 31, B = p.batch;
+    const bool live = lane < B;
+    long long n = 0, Lq = 0, M = 0, nb = 1;
+    bool bad = false;
+    if (live) {
+        n = p.prefix_lens[lane]; Lq = p.q_lens[lane]; M = p.n_mask[lane];
+        nb = p.n_blocks ? p.n_blocks[lane] : 1;
+        bad = n < 0 || Lq < 0 || M < 0 || M > Lq || Lq > p.max_q_len || n + Lq > (long long)p.max_pages * 16;
+        bad = bad || nb < 0 || (nb > 1 && (M % nb != 0 || nb > Lq - M));  // equal mask blocks, one hypothesis each
+        if (bad) Lq = 0;
+    }
+    int q = (int)Lq, t = Lq > 0 ? (int)((n + Lq + kTileTokens - 1) / kTileTokens) : 0, ne = t > 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int uq = __shfl_up_sync(0xffffffffu, q, o), ut = __shfl_up_sync(0xffffffffu, t, o), un = __shfl_up_sync(0xffffffffu, ne, o);
+        if (lane >= o) { q += uq; t += ut; ne += un; }
+    }
+    const int rows = __shfl_sync(0xffffffffu, q, 31);
+    const bool fatal = __any_sync(0xffffffffu, bad) || rows != p.total_q_rows;
+    if (live) {
+        sc->cu_q[lane + 1] = q; sc->cu_tiles[lane + 1] = t; sc->cu_ne[lane + 1] = ne;
+        const RowBlock rb = {lane, 0, (int)n, (int)Lq, (int)M, (int)nb, {0, 0}};
+        rbs[lane] = rb;
+    }
+    if (lane == 0) {
+        sc->cu_q[0] = 0; sc->cu_tiles[0] = 0; sc->cu_ne[0] = 0;
+        sc->fatal = fatal;
+        if (fatal && blockIdx.x == 0) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+    }
+    if (MODE == kTcSelfPlanned) {
+        // the range starts of this CTA and its neighbours, a lane each: the cuts the plan kernel would have made
+        // (range_cut is shared with it and with the host), all in one go instead of one after the other
+        __syncwarp();
+        const int tiles = __shfl_sync(0xffffffffu, t, 31), nonempty = __shfl_sync(0xffffffffu, ne, 31);
+        const long long k = p.piece_cost, W = (long long)p.Hkv * (tiles + k * nonempty);
+        const int total = fatal ? 0 : tiles * p.Hkv;
+        const int n_use = ranges_in_use(W, k, p.min_range_tiles, p.n_ctas);
+        const int cc = (int)blockIdx.x - kCsWindow / 2 + 1 + lane;
+        int start = 0, first = 0;
+        if (cc >= 0 && cc <= p.n_ctas) {
+            const int* ct_ = sc->cu_tiles;
+            const int* ne_ = sc->cu_ne;
+            start = (cc >= n_use || total == 0) ? total
+                                                : range_cut(cc, n_use, W, B, p.Hkv, k, [ct_](int b) { return ct_[b]; }, [ne_](int b) { return ne_[b]; }, &first);
+        }
+        s_cs[lane] = start;
+        if (cc == (int)blockIdx.x) *s_first = first;
+    }
+}
+
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap qmap,
-                                                              AttnParams p) {
-    using C = Cfg<D>;
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+                                                              const AttnParams p_in) {
+    using C = Cfg<D, MODE>;
+    extern __shared__ __align__(1024) unsigned char smem[];  // the swizzled tiles need 1024-byte alignment
     unsigned char* sq = smem;
     unsigned char* sk = smem + C::kQBytes;                      // K ring
     unsigned char* sv = sk + C::kStages * C::kKBytes;           // V ring
@@ -635,12 +839,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     float* ex = reinterpret_cast<float*>(smem + C::kExOffset);
     int* s_cs = reinterpret_cast<int*>(smem + C::kCsOffset);
     Piece* ring = reinterpret_cast<Piece*>(smem + C::kDescOffset);
+    SelfScans* scans = reinterpret_cast<SelfScans*>(smem + C::kScanOffset);
+    RowBlock* rbs = reinterpret_cast<RowBlock*>(smem + C::kRbOffset);
     volatile int* abort = &bars->abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if ((smem_u32(smem) & 1023u) != 0u) {  // uniform; cannot happen with the declared alignment: leave before any barrier
+        if (tid == 0) atomicOr(p_in.status, FD_DEV_TIMEOUT);
+        return;
+    }
 
-    // ---- set-up that needs nothing from the plan kernel: it overlaps that kernel's execution
-    //      (programmatic dependent launch); griddepcontrol.wait below is where its results are needed
+    // ---- set-up that needs nothing from earlier kernels: under programmatic dependent launch it overlaps the
+    //      tail of the previous launch on the stream (the plan kernel, or the previous layer's call);
+    //      griddepcontrol.wait below is where that launch's results are needed
     if (tid == 0) {
         for (int i = 0; i < C::kStages; ++i) {
             mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
@@ -667,19 +878,60 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
-    // a dependent launch behind this one (the next layer's call, when the plan is pinned) may bring its
-    // CTAs in as ours retire and do its own set-up; it waits for this grid to complete before reading anything
+    // a dependent launch behind this one (the next layer's call) may bring its CTAs in as ours retire and do its
+    // own set-up; it waits for this grid to complete before reading anything
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    const PlanHeader hdr = *p.plan.hdr;
-    const int total = hdr.total_tiles;
+    // ---- the work of this CTA
+    AttnParams p = p_in;
     const int cta = blockIdx.x;
-    const int s_c = total ? p.plan.cta_start[cta] : 0, e_c = total ? p.plan.cta_start[cta + 1] : 0;
-    // the range starts of the neighbouring CTAs decide who shares a segment with this one (epilogue, merge)
-    const CtaStarts cs = {p.plan.cta_start, s_cs, cta - kCsWindow / 2 + 1};
-    if (s_c >= e_c) {  // uniform: no tile for this CTA (or nothing at all)
-        if (total == 0 && hdr.fatal) {  // inconsistent lengths: a defined output, zeros
+    int total, n_rb, fatal;
+    Range rg = {0, 0, 0};
+    CtaStarts cs = {};
+    cs.s = s_cs;
+    cs.base = cta - kCsWindow / 2 + 1;
+    int cl_rank = 0, cl_rows = 0, cl_b = 0, cl_kvh = 0, cl_row0 = 0;  // kTcCluster: this CTA's place and its segment
+    bool cl_idle = false;
+    if (MODE == kTcPlanned) {
+        const PlanHeader hdr = *p.plan.hdr;
+        total = hdr.total_tiles; n_rb = hdr.n_rb; fatal = hdr.fatal;
+        if (total) { rg.s_c = p.plan.cta_start[cta]; rg.e_c = p.plan.cta_start[cta + 1]; rg.first = p.plan.cta_first[cta]; }
+        cs.g = p.plan.cta_start;
+    } else {
+        if (warp == 0) self_plan<MODE>(p, scans, rbs, s_cs, &bars->first);
+        __syncthreads();
+        p.plan.rb = rbs; p.plan.cu_q = scans->cu_q; p.plan.cu_tiles = scans->cu_tiles; p.plan.cu_ne = scans->cu_ne;
+        n_rb = p.batch;
+        fatal = scans->fatal;
+        const int tiles = scans->cu_tiles[n_rb], nonempty = scans->cu_ne[n_rb];
+        total = fatal ? 0 : tiles * p.Hkv;
+        if (MODE == kTcSelfPlanned) {
+            // the ranges the plan kernel would have cut (range_cut is shared with it and with the host)
+            cs.ct = scans->cu_tiles; cs.ne = scans->cu_ne;
+            cs.n_rb = n_rb; cs.Hkv = p.Hkv; cs.k = p.piece_cost; cs.total = total;
+            cs.W = (long long)p.Hkv * (tiles + (long long)p.piece_cost * nonempty);
+            cs.n_use = ranges_in_use(cs.W, p.piece_cost, p.min_range_tiles, p.n_ctas);
+            if (total) { rg.s_c = s_cs[cta - cs.base]; rg.e_c = s_cs[cta + 1 - cs.base]; rg.first = bars->first; }
+        } else {
+            // segment = cluster number; the cluster's CTAs take equal shares of its tiles, in rank order
+            const int seg = cta / p.cluster, v = seg / p.Hkv;
+            cl_rank = (int)cluster_ctarank();
+            cl_kvh = seg % p.Hkv;
+            cl_b = v;
+            cl_rows = rbs[v].Lq * p.G;
+            cl_row0 = scans->cu_q[v];
+            const int T = total ? scans->cu_tiles[v + 1] - scans->cu_tiles[v] : 0;
+            const int t_base = p.Hkv * scans->cu_tiles[v] + cl_kvh * T;
+            // (T <= 2^23 tiles and at most 16 ranks: the products fit 32 bits)
+            rg.s_c = t_base + (int)((unsigned)T * (unsigned)cl_rank / (unsigned)p.cluster);
+            rg.e_c = t_base + (int)((unsigned)T * (unsigned)(cl_rank + 1) / (unsigned)p.cluster);
+            rg.first = v;
+            cl_idle = rg.s_c >= rg.e_c && T > 0;  // peers have tiles: stay for the merge
+        }
+    }
+    if (rg.s_c >= rg.e_c && !cl_idle) {  // uniform (over the cluster too): no tile for this CTA, or nothing at all
+        if (total == 0 && fatal) {  // inconsistent lengths: a defined output, zeros
             const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
             uint4* o = reinterpret_cast<uint4*>(p.out);
             for (long long i2 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i2 < n16; i2 += (long long)gridDim.x * blockDim.x)
@@ -689,18 +941,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
         return;
     }
-    // Warp-specialised register budgets: the softmax groups keep a whole 128-column row of S in registers.
-    // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168, what the launch allocated: the increase is served exactly by what
-    // the decrease released (a request for more than that does not return).
-    if (warp < 8) {
+    const uint32_t recv_addr = smem_u32(smem) + (uint32_t)C::kRecvOffset;
+    if (MODE == kTcCluster && cl_idle) {
+        // fewer tiles than CTAs in the cluster: this one tells every owner "saw no key" and combines the rows it owns
+        const Recv<D> rv = {recv_addr, kMaxRows / p.cluster};
+        if (tid < cl_rows) st_peer_v2(peer_addr(rv.ml(cl_rank, tid % rv.share), tid / rv.share), make_float2(-INFINITY, 0.f));
+        cluster_sync_all();
+        const int r = tid & (kMaxRows - 1);
+        if (tid < 2 * kMaxRows && r < cl_rows && r / rv.share == cl_rank)
+            cluster_reduce_row<D>(p, rv, cl_rank, r, tid >> 7, nullptr, cl_b, cl_kvh, cl_row0);
+    } else if (warp < 8) {
+        // Warp-specialised register budgets: the softmax groups keep a whole 128-column row of S in registers.
+        // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168, what the launch allocated: the increase is served exactly by what
+        // the decrease released (a request for more than that does not return).
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        softmax_role<D>(p, bars, ex, s_cs, cs, ring, tmem, s_c, e_c, abort);
+        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, recv_addr, cl_rank, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        if (warp == kKWarp) load_role<D>(tmap, p, hdr.n_rb, sk, bars->k_full, bars->k_empty, 0, s_c, e_c, abort);
-        else if (warp == kVWarp) load_role<D>(tmap, p, hdr.n_rb, sv, bars->v_full, bars->v_empty, 1, s_c, e_c, abort);
-        else if (warp == kMmaWarp) mma_role<D>(p, sq, sk, sv, bars, ring, tmem, s_c, e_c, abort);
-        else q_role<D>(qmap, p, hdr.n_rb, sq, bars, ring, s_c, e_c, abort);
+        if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, abort);
+        else if (warp == kVWarp) load_role<D, MODE>(tmap, p, n_rb, sv, bars->v_full, bars->v_empty, 1, rg, abort);
+        else if (warp == kMmaWarp) mma_role<D, MODE>(p, sq, sk, sv, bars, ring, tmem, rg, abort);
+        else q_role<D, MODE>(qmap, p, n_rb, sq, bars, ring, rg, abort);
+        if (MODE == kTcCluster) cluster_sync_all();  // the cluster barrier of the merge counts every thread
     }
     // ---- common tail: everything of this CTA has completed, or it is giving up
     if (*abort && tid == 0) atomicOr(p.status, FD_DEV_TIMEOUT);
@@ -745,7 +1007,56 @@ struct TcState {
     int d, hkv;
     const CUtensorMap* current;
     const CUtensorMap* qcurrent;
+    int max_clusters[kMaxCluster + 1];  // [C]: clusters of C CTAs of the cluster kernel the device holds at once (0 = not launchable)
 };
+
+template <int D, int MODE>
+cudaError_t configure_kernel() {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D, MODE>::kSmemBytes);
+    if (e == cudaSuccess && MODE == kTcCluster)
+        e = cudaFuncSetAttribute(attn_tc_kernel<D, MODE>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    return e;
+}
+
+// How many clusters of `c` CTAs of the cluster kernel can be resident together (0 if such a launch is refused).
+template <int D>
+int query_clusters(int c, int n_sms) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((n_sms / c) * c);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = Cfg<D, kTcCluster>::kSmemBytes;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<D, kTcCluster>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
+template <int D, int MODE>
+void launch_mode(const TcState* st, const AttnParams& p, cudaStream_t s) {
+    // Programmatic dependent launch: the CTAs may start while the previous launch on the stream (the plan kernel,
+    // or the previous layer's call) is still running; they do their set-up and then wait for it inside the kernel.
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.dynamicSmemBytes = Cfg<D, MODE>::kSmemBytes;
+    if (MODE == kTcCluster) {
+        cfg.gridDim = dim3(p.batch * p.Hkv * p.cluster);  // one cluster per (sequence, kv-head) segment
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, MODE>, *st->current, *st->qcurrent, p);
+}
 
 }  // namespace
 
@@ -765,9 +1076,21 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
         cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", reinterpret_cast<void**>(&st->encode), cudaEnableDefault, &qres);
         if (e != cudaSuccess || !st->encode) { delete st; return e != cudaSuccess ? e : cudaErrorNotSupported; }
         st->d = p.d; st->hkv = p.Hkv;
-        if (p.d == 64) e = cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
-        else e = cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+        if (p.d == 64) {
+            e = configure_kernel<64, kTcPlanned>();
+            if (e == cudaSuccess) e = configure_kernel<64, kTcSelfPlanned>();
+            if (e == cudaSuccess) e = configure_kernel<64, kTcCluster>();
+        } else {
+            e = configure_kernel<128, kTcPlanned>();
+            if (e == cudaSuccess) e = configure_kernel<128, kTcSelfPlanned>();
+            if (e == cudaSuccess) e = configure_kernel<128, kTcCluster>();
+        }
         if (e != cudaSuccess) { delete st; return e; }
+        int n_sms = 0, dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+        for (int c = 0; c <= kMaxCluster; ++c) st->max_clusters[c] = 0;
+        for (int c = 2; c <= kMaxCluster; c *= 2) st->max_clusters[c] = p.d == 64 ? query_clusters<64>(c, n_sms) : query_clusters<128>(c, n_sms);
         *state = st;
     }
     // q: a 3-D view [T][Hq][d], box = 64 elements x G q-heads (one kv-head) x q_box_t block rows
@@ -809,26 +1132,27 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
     return cudaSuccess;
 }
 
-void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s) {
+// CTAs per cluster for a call with one cluster per segment: the largest power of two for which all clusters of the
+// call are resident together (so every SM it can use streams at once); 0 if there is none.
+int attn_tc_cluster_size(const void* state, int n_segments, int n_sms) {
+    const TcState* st = static_cast<const TcState*>(state);
+    if (!st || n_segments <= 0) return 0;
+    for (int c = kMaxCluster; c >= 2; c /= 2)
+        if (n_segments * c <= n_sms && st->max_clusters[c] >= n_segments) return c;
+    return 0;
+}
+
+void launch_attn_tc(void* state, const AttnParams& p, int mode, cudaStream_t s) {
     if (p.batch == 0) return;
     const TcState* st = static_cast<const TcState*>(state);
-    // Programmatic dependent launch: the CTAs may start while the plan kernel (the previous launch on the
-    // stream) is still running; they do their set-up and then wait for it inside the kernel.
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.n_ctas);
-    cfg.blockDim = dim3(kThreads);
-    cfg.stream = s;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     if (p.d == 64) {
-        cfg.dynamicSmemBytes = Cfg<64>::kSmemBytes;
-        cudaLaunchKernelEx(&cfg, attn_tc_kernel<64>, *st->current, *st->qcurrent, p);
+        if (mode == kTcCluster) launch_mode<64, kTcCluster>(st, p, s);
+        else if (mode == kTcSelfPlanned) launch_mode<64, kTcSelfPlanned>(st, p, s);
+        else launch_mode<64, kTcPlanned>(st, p, s);
     } else {
-        cfg.dynamicSmemBytes = Cfg<128>::kSmemBytes;
-        cudaLaunchKernelEx(&cfg, attn_tc_kernel<128>, *st->current, *st->qcurrent, p);
+        if (mode == kTcCluster) launch_mode<128, kTcCluster>(st, p, s);
+        else if (mode == kTcSelfPlanned) launch_mode<128, kTcSelfPlanned>(st, p, s);
+        else launch_mode<128, kTcPlanned>(st, p, s);
     }
 }
 

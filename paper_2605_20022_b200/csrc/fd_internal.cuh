@@ -11,6 +11,8 @@ namespace fd {
 
 constexpr int kTileTokens = 128;   // KV tokens per work tile (8 pages of 16)
 constexpr int kMaxRows = 128;      // query rows of one MMA tile: a row block has kMaxRows / G block rows
+constexpr int kClusterMaxSegments = 18; // most (sequence, kv-head) segments for which the kernel runs one cluster per segment
+constexpr int kSelfPlanMaxRb = 24; // most row blocks for which the tensor-core kernel plans for itself (no plan launch)
 constexpr int kAcceptChunk = 4096; // logits per CTA of the vocab sweep (smaller chunks measured faster: shorter CTA tails)
 
 // Written by the plan kernel, read by the attention and merge kernels.
@@ -38,7 +40,8 @@ struct Plan {
     int* cu_q;      // [n_rb+1] first query row of each row block
     int* cu_tiles;  // [n_rb+1] exclusive scan of the row blocks' tiles (per kv-head)
     int* cu_ne;     // [n_rb+1] exclusive scan of (tiles > 0)
-    int* seq_ok;    // [B]   0 = a page id of the sequence was outside the pool: its rows are zeroed
+    int* seq_bad;   // [B]   number (AttnParams::epoch) of the last call that met a page id outside the pool in the sequence:
+                    //       equal to the running call's number = flagged, the sequence's rows are zeroed
     int* seg_count; // [n_rb * Hkv] partial pieces of a segment that have been written (fused merge)
     int* cta_first; // [n_ctas] row block that owns the first tile of each attention CTA's range
     int* cta_start; // [n_ctas + 1] first tile of each attention CTA's range (non-decreasing; [n_ctas] = total)
@@ -82,8 +85,18 @@ struct AttnParams {
     int q_box_t;      // block rows per Q load box of the tensor-core kernel (see q_box_rows)
     int min_range_tiles;  // least tiles worth giving a CTA a range of its own
     int piece_cost;   // fixed cost of starting a segment in a range, in tiles (balances ranges with many short segments)
+    int epoch;        // number of this attention call on its context, never 0 (see Plan::seq_bad)
+    int cluster;      // CTAs per cluster when every segment is split over one cluster, else 0
     int* status;
 };
+
+// A sequence in which this call met a page id outside the pool: its rows are written as zeros.  The flag is the
+// call's own number, so nothing has to be cleared between calls.
+__device__ __forceinline__ void flag_sequence(const AttnParams& p, int b) {
+    p.plan.seq_bad[b] = p.epoch;
+    atomicOr(p.status, FD_DEV_BAD_PAGE);
+}
+__device__ __forceinline__ bool sequence_flagged(const AttnParams& p, int b) { return __ldcg(p.plan.seq_bad + b) == p.epoch; }
 
 // Hybrid mask of one query row, never materialised: key position j is visible iff
 //     j < limit  ||  (blk_lo <= j && j < blk_hi).
@@ -123,14 +136,17 @@ __host__ __device__ inline int q_box_rows(int G) {
 // per kv-head and of "has tiles".  Returns the first tile of range c; *first_seq = the sequence it lies in.
 __host__ __device__ inline int ranges_in_use(long long W, long long k, int min_range_tiles, int n_ranges) {
     const long long per = k + (min_range_tiles > 1 ? min_range_tiles : 1);
-    long long n = W / per;
+    long long n = ((unsigned long long)W >> 32) == 0 ? (long long)((unsigned)W / (unsigned)per) : W / per;
     if (n > n_ranges) n = n_ranges;
     return (int)(n < 1 ? 1 : n);
 }
 template <class CtAt, class NeAt>
 __host__ __device__ inline int range_cut(int c, int n_use, long long W, int B, int Hkv, long long k, CtAt ct_at, NeAt ne_at,
                                          int* first_seq) {
-    const long long x = ((long long)c * W) / n_use;
+    // (64-bit division is a long dependent instruction sequence on the device: the 32-bit form serves every call
+    // whose cost total fits, with the same result)
+    const unsigned long long cw = (unsigned long long)c * (unsigned long long)W;
+    const long long x = (cw >> 32) == 0 ? (long long)((unsigned)cw / (unsigned)n_use) : (long long)(cw / (unsigned long long)n_use);
     int lo = 0, hi = B;  // last b whose span starts at or before x (of equal starts the last: the non-empty one)
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -139,20 +155,41 @@ __host__ __device__ inline int range_cut(int c, int n_use, long long W, int B, i
     }
     const long long ct = ct_at(lo), nt = (long long)ct_at(lo + 1) - ct;
     const long long rem = x - (long long)Hkv * (ct + k * (long long)ne_at(lo));
-    const long long kvh = rem / (nt + k), r = rem % (nt + k);
+    long long kvh, r;
+    if (((unsigned long long)rem >> 32) == 0 && ((unsigned long long)(nt + k) >> 32) == 0) {
+        kvh = (unsigned)rem / (unsigned)(nt + k);
+        r = (unsigned)rem - (unsigned)kvh * (unsigned)(nt + k);
+    } else {
+        kvh = rem / (nt + k);
+        r = rem % (nt + k);
+    }
     *first_seq = lo;
     return (int)(Hkv * ct + kvh * nt + (r > k ? r - k : 0));
 }
 
-// View of cta_start: a window of it around the reading CTA may be cached in shared memory.
+// View of the range starts cta_start[c]: a window around the reading CTA may be cached in shared memory; an entry
+// outside the window comes from the plan kernel's array in global memory, or -- in a call that plans for itself
+// and has no such array -- is cut again from the scans (ct, ne: tiles and non-empty row blocks, exclusive).
 constexpr int kCsWindow = 32;
 struct CtaStarts {
-    const int* g;   // [n_ctas + 1] in global memory
+    const int* g;   // [n_ctas + 1] in global memory, or nullptr
     const int* s;   // entries [base, base + kCsWindow) in shared memory, or nullptr
     int base;
+    const int* ct;  // self-planned call: [n_rb + 1] scans, and what range_cut needs beside them
+    const int* ne;
+    int n_rb, Hkv, n_use, k, total;
+    long long W;
+    __device__ __forceinline__ int cut(int c) const {
+        if (c >= n_use) return total;
+        int first;
+        const int* ct_ = ct;
+        const int* ne_ = ne;
+        return range_cut(c, n_use, W, n_rb, Hkv, (long long)k, [ct_](int b) { return ct_[b]; }, [ne_](int b) { return ne_[b]; }, &first);
+    }
     __device__ __forceinline__ int at(int c) const {
         const unsigned i = (unsigned)(c - base);
-        return (s && i < (unsigned)kCsWindow) ? s[i] : g[c];
+        if (s && i < (unsigned)kCsWindow) return s[i];
+        return g ? g[c] : cut(c);
     }
 };
 
@@ -207,7 +244,7 @@ __device__ inline void merge_row(const AttnParams& p, const CtaStarts& cs, int c
     float acc[CW];
 #pragma unroll
     for (int c = 0; c < CW; ++c) acc[c] = 0.f;
-    if (!__ldcg(p.plan.seq_ok + b)) {  // a page id of this sequence was bad: defined output, zeros
+    if (sequence_flagged(p, b)) {  // a page id of this sequence was bad: defined output, zeros
         store_cols_bf16<CW>(dst, acc, 0.f);
         return;
     }
@@ -247,13 +284,18 @@ __device__ inline void merge_row(const AttnParams& p, const CtaStarts& cs, int c
     store_cols_bf16<CW>(dst, acc, 1.f / l);
 }
 
+// How a tensor-core attention call finds its work: from the plan kernel's arrays; from scans each CTA makes
+// itself (few row blocks); or one cluster per segment, merged through distributed shared memory.
+enum { kTcPlanned = 0, kTcSelfPlanned = 1, kTcCluster = 2 };
+
 // Launchers (defined next to their kernels).
 void launch_plan(const AttnParams& p, cudaStream_t s);
 cudaError_t attn_simt_prepare(int d);
 void launch_attn_simt(const AttnParams& p, cudaStream_t s);
 bool attn_tc_supported(int d, int G, int max_q_len);
 cudaError_t attn_tc_prepare(void** state, const AttnParams& p);  // tensor map for this kv pool
-void launch_attn_tc(void* state, const AttnParams& p, cudaStream_t s);
+void launch_attn_tc(void* state, const AttnParams& p, int mode, cudaStream_t s);  // mode: kTcPlanned, kTcSelfPlanned, kTcCluster
+int attn_tc_cluster_size(const void* state, int n_segments, int n_sms);    // CTAs per cluster for a call of n_segments, or 0
 void attn_tc_free(void* state);
 void launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);
 void launch_merge(const AttnParams& p, cudaStream_t s);

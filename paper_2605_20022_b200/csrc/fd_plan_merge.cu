@@ -12,7 +12,7 @@
 // many short segments gets fewer tiles.
 //
 // The plan kernel checks the lengths (O(B) work, one CTA).  Page ids are checked where they are
-// used, by the attention kernels: a sequence with an id outside the pool is flagged in seq_ok,
+// used, by the attention kernels: a sequence with an id outside the pool is flagged in seq_bad,
 // read from page 0 instead, and has its output rows zeroed by the merge kernel.
 #include <algorithm>
 
@@ -86,7 +86,6 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
             bad = bad || nb < 0 || (nb > 1 && (M % nb != 0 || nb > Lq - M));
             if (bad) { atomicOr(&s_fatal, 1); Lq = 0; }
             cnt = Lq > 0 ? (int)((Lq + p.rb_rows - 1) / p.rb_rows) : 1;  // an empty sequence keeps one (empty) row block
-            p.plan.seq_ok[b] = 1;
         }
         if (one_each) {
             if (b < B) {
@@ -178,10 +177,11 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(AttnParams p) {
     if (ntiles == 0) return;
     const int b = p.plan.rb[v].b;
     const int t0 = p.Hkv * p.plan.cu_tiles[v] + kvh * ntiles, t1 = t0 + ntiles;
-    const CtaStarts cs = {p.plan.cta_start, nullptr, 0};
+    CtaStarts cs = {};
+    cs.g = p.plan.cta_start;
     const int c_first = range_owner(cs.g, p.n_ctas, t0), c_last = range_owner(cs.g, p.n_ctas, t1 - 1);
     // an unsplit segment was written by the attention kernel itself; it is revisited only to zero it
-    if (segment_pieces(cs, c_first, c_last, t0, t1) <= 1 && p.plan.seq_ok[b]) return;
+    if (segment_pieces(cs, c_first, c_last, t0, t1) <= 1 && !sequence_flagged(p, b)) return;
     merge_row<D, D / 4>(p, cs, c_first, c_last, b, kvh, p.plan.cu_q[v], t0, t1, r, cg);
 }
 

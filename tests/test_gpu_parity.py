@@ -13,7 +13,9 @@ from helpers import Ctx, assert_close, gpu_accept, gpu_attn, gpu_commit
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [fd.FD_ATTN_SIMT, fd.FD_ATTN_AUTO]
+# the CUDA-core kernel; the tensor-core kernel as a call is routed by default (one cluster per segment, self-planned
+# or planned, by size); the tensor-core kernel always on the plan kernel's work list; and always self-planned where legal
+PATHS = [fd.FD_ATTN_SIMT, fd.FD_ATTN_AUTO, fd.FD_ATTN_TCGEN05_PLANNED, fd.FD_ATTN_TCGEN05_SELF_PLANNED]
 
 
 def oracle_attn(step, q, kv):
@@ -31,6 +33,25 @@ def test_attention_workloads(idx, path):
         got, status = gpu_attn(ctx, step, q, kv)
     assert status == 0
     assert_close(got.numpy(), oracle_attn(step, q, kv), step.name)
+
+
+def test_tensor_core_call_routing():
+    """Which form of the tensor-core kernel a call takes: few segments -> one cluster per segment; few sequences ->
+    self-planned; otherwise (or under a pinned plan) the plan kernel's work list.  All forms agree with the oracle."""
+    want = {1: fd.FD_TC_CLUSTER, 2: fd.FD_TC_SELF_PLANNED, 3: fd.FD_TC_PLANNED}
+    for idx, mode in want.items():
+        step = wl.workload(idx)
+        q, kv = wl.make_q(step), wl.make_kv(step)
+        ref = oracle_attn(step, q, kv)
+        for path, expect in ((fd.FD_ATTN_AUTO, mode), (fd.FD_ATTN_TCGEN05_PLANNED, fd.FD_TC_PLANNED),
+                             (fd.FD_ATTN_TCGEN05_SELF_PLANNED, fd.FD_TC_SELF_PLANNED if step.batch <= 24 else fd.FD_TC_PLANNED)):
+            with Ctx(step, path) as ctx:
+                assert fd.fd_attn_last_mode(ctx.h) == -1
+                before = fd.fd_launch_count(ctx.h)
+                got, status = gpu_attn(ctx, step, q, kv)
+                assert status == 0 and fd.fd_attn_last_mode(ctx.h) == expect, (idx, path, fd.fd_attn_last_mode(ctx.h))
+                assert fd.fd_launch_count(ctx.h) - before == (2 if expect == fd.FD_TC_PLANNED else 1)   # one launch unless planned
+                assert_close(got.numpy(), ref, f"{step.name} path {path}")
 
 
 EDGE = {
@@ -257,6 +278,14 @@ def test_long_context_full_size_every_element(path):
                     again = torch.empty_like(q)
                     fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, q, kv, step.num_pages, dpt, dpl, dql, dnm, again)
                     assert torch.equal(out, again), "two runs on the same inputs differ bitwise"
+                # without the pin the tensor-core kernel cuts the same ranges for itself (16 sequences): same bits
+                fd.fd_plan_unpin(ctx.h)
+                again.fill_(0)
+                fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, q, kv, step.num_pages, dpt, dpl, dql, dnm, again)
+                if path in (fd.FD_ATTN_AUTO, fd.FD_ATTN_TCGEN05_SELF_PLANNED):
+                    assert fd.fd_attn_last_mode(ctx.h) == fd.FD_TC_SELF_PLANNED
+                assert torch.equal(out, again), "planned and self-planned calls differ bitwise"
+                fd.fd_plan_pin(ctx.h, step.batch, step.total_q_rows, dpl, dql, dnm)
                 del again
             outc = out.float().cpu().numpy()
             del q, kv, out
