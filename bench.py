@@ -153,10 +153,41 @@ def oracle_sample(step, heads: int, layers: int = 1):
     return est * 1e6, desc, oracle.num_threads()
 
 
+def oracle_full(step):
+    """Time the oracle on the WHOLE step (every layer's attention, accept, commit): no sampling, no scaling.
+    For the workloads whose oracle finishes in about a second."""
+    import numpy as np
+    import oracle
+    from paper_2605_20022_b200 import workload as wl
+    t_total = 0.0
+    for layer in range(step.shape.n_layers):
+        q, kv = wl.make_q(step, layer), wl.make_kv(step, layer)
+        t0 = time.perf_counter()
+        if step.n_blocks is not None:
+            oracle.attn_blocks(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, step.n_blocks)
+        else:
+            oracle.attn(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask)
+        t_total += time.perf_counter() - t0
+    logits, drafts, _ = wl.make_logits(step)
+    t0 = time.perf_counter()
+    acc, _, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    oracle.commit(step.page_table, step.prefix_lens, step.q_lens, acc)
+    t_total += time.perf_counter() - t0
+    return t_total * 1e6, "the whole step (attention of every layer, accept over every candidate row, commit), not scaled", oracle.num_threads()
+
+
+def oracle_time(step, heads=None, layers=4):
+    """The oracle's time for one step: in full where that takes about a second, else on a bounded sample
+    (>= 2 s of oracle work: one sequence, all q-heads, 4 layers), scaled."""
+    if step.attn_bytes() * step.shape.n_layers < 4e9:
+        return oracle_full(step)
+    return oracle_sample(step, heads or step.shape.n_q_heads, layers=layers)
+
+
 def run_reference(args, step):
     vals = []
     for i in range(args.warmup + args.steps):
-        us, desc, cores = oracle_sample(step, args.ref_heads)
+        us, desc, cores = oracle_time(step)
         if i >= args.warmup:
             vals.append(us)
     v = statistics.mean(vals)
@@ -164,7 +195,7 @@ def run_reference(args, step):
         "metric": METRIC, "value": v, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": v / 1e3, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": step.name, "note": "CPU oracle timed on a bounded sample and scaled to one step"},
+        "config": {"workload": step.name, "note": "CPU oracle, as it stands, on the host cores: " + desc},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -217,11 +248,14 @@ class DeviceStep:
             pt.copy_(self.pt0); pl.copy_(self.pl0)
         self.cur = 0
 
-    def run(self, time_attn=False, restore_inline=False):
+    def run(self, time_attn=False, restore_inline=False, attn_only=False):
         """One step on the current stream, on the next restored copy of the page table and lengths.  With
-        restore_inline the copy is refreshed inside the step (a replayed CUDA graph has no other way)."""
+        restore_inline the copy is refreshed inside the step (a replayed CUDA graph has no other way); with
+        attn_only just the attention calls of the step, one per layer (nothing is rewritten, nothing to restore)."""
         fd, torch, st = self.fd, self.torch, self.step
-        if restore_inline:
+        if attn_only:
+            self.pt, self.pl = self.slots[0]
+        elif restore_inline:
             self.pt, self.pl = self.slots[0]
             self.pt.copy_(self.pt0); self.pl.copy_(self.pl0)
         else:
@@ -243,6 +277,8 @@ class DeviceStep:
                 e1.record(); self.attn_events.append((e0, e1))
         if self.L > 1:
             fd.fd_plan_unpin(self.ctx)   # the commit below changes prefix_lens
+        if attn_only:
+            return
         fd.fd_verify_accept(self.ctx, st.batch, st.total_cand_rows, self.logits, self.drafts, self.ql, self.nm,
                             self.acc, self.bon)
         fd.fd_kv_commit(self.ctx, st.batch, self.pt, self.pl, self.ql, self.acc, self.freed, self.n_freed)
@@ -309,17 +345,18 @@ def timed_region(torch, dist, fn, steps, flush=None, prepare=None):
     return ms
 
 
-def capture_step_graph(torch, ds):
+def capture_step_graph(torch, ds, attn_only=False):
     """The whole step (attention x layers, accept, commit) as one CUDA graph on a side stream.  Only
     used after warm-up, so every first-call set-up inside the library has already happened."""
     g = torch.cuda.CUDAGraph()
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
+    run = (lambda: ds.run(attn_only=True)) if attn_only else (lambda: ds.run(restore_inline=True))
     with torch.cuda.stream(side):
-        ds.run(restore_inline=True)
+        run()
         side.synchronize()
         with torch.cuda.graph(g, stream=side):
-            ds.run(restore_inline=True)
+            run()
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     return g
@@ -356,6 +393,109 @@ def check_against_oracle(ds: DeviceStep, n_rows=6):
     return ok_attn and ok_acc
 
 
+def check_full(ds: DeviceStep):
+    """Every attention output element of every layer, the accept result and the commit of the benchmarked tensors
+    against the oracle (for the workloads whose oracle finishes in about a second)."""
+    import numpy as np
+    import oracle
+    torch, st = ds.torch, ds.step
+    ds.restore(); ds.run(); torch.cuda.synchronize()
+    ok = True
+    for l in range(ds.L):
+        qc, kvc = ds.q[l].cpu(), ds.kv[l].cpu()
+        if st.n_blocks is not None:
+            ref = oracle.attn_blocks(qc, kvc, st.page_table, st.prefix_lens, st.q_lens, st.n_mask, st.n_blocks)
+        else:
+            ref = oracle.attn(qc, kvc, st.page_table, st.prefix_lens, st.q_lens, st.n_mask)
+        outc = ds.out[l].float().cpu().numpy()
+        ok = ok and bool(np.isfinite(outc).all() and (np.abs(outc - ref) <= 2e-2 + 2e-2 * np.abs(ref)).all())
+    e_acc, e_bon, _ = oracle.accept(ds.logits.cpu(), ds.drafts.cpu(), st.q_lens, st.n_mask)
+    ok = ok and bool((ds.acc.cpu().numpy() == e_acc).all() and (ds.bon.cpu().numpy() == e_bon).all())
+    ept, epl, efreed = oracle.commit(st.page_table, st.prefix_lens, st.q_lens, e_acc)
+    n = int(ds.n_freed.item())
+    ok = ok and bool((ds.pt.cpu().numpy() == ept).all() and (ds.pl.cpu().numpy() == epl).all() and n == len(efreed)
+                     and (ds.freed[:n].cpu().numpy() == efreed).all())
+    return ok
+
+
+def decode_step_many_layers(torch, step, device, peak, attn_path, layers, reps):
+    """The same workload as the step of a `layers`-layer model: one attention call per layer over distinct KV
+    pools (together larger than L2 for every workload but the tiny one), the work list pinned once per step, then
+    accept and commit.  Timed stream-launched and as a CUDA-graph replay; and the attention calls alone, which is
+    what the roofline figure of a small workload is taken from (a single call bracketed by events measures the
+    event pair as much as the kernel)."""
+    import dataclasses
+    import paper_2605_20022_b200 as fd
+    st = dataclasses.replace(step, shape=dataclasses.replace(step.shape, n_layers=layers))
+    ds = DeviceStep(st, device, attn_path, n_slots=reps + 4)
+    try:
+        ds.restore()
+        for _ in range(3):
+            ds.run()
+        ms_step = timed_region(torch, None, ds.run, reps, prepare=ds.restore) / reps
+        g = capture_step_graph(torch, ds)
+        g.replay()
+        ms_step_g = timed_region(torch, None, g.replay, reps) / reps
+        del g
+        ds.restore()                       # the steps above committed: the attention alone runs on the original lengths
+        attn = lambda: ds.run(attn_only=True)
+        attn()
+        ms_attn = timed_region(torch, None, attn, reps) / reps
+        g = capture_step_graph(torch, ds, attn_only=True)
+        g.replay()
+        ms_attn_g = timed_region(torch, None, g.replay, reps) / reps
+        del g
+        mode = fd.fd_attn_last_mode(ds.ctx)
+        status = fd.fd_last_device_status(ds.ctx)
+    finally:
+        ds.close()
+    nbytes = step.attn_bytes()
+    per_call, per_call_g = ms_attn * 1e3 / layers, ms_attn_g * 1e3 / layers
+    return {"layers": layers, "us_per_step": ms_step * 1e3, "us_per_step_cuda_graph_replay": ms_step_g * 1e3,
+            "us_per_attn_call": per_call, "us_per_attn_call_cuda_graph_replay": per_call_g,
+            "attn_GBps": nbytes / per_call_g / 1e3, "frac_of_measured_peak": nbytes / per_call_g / 1e3 / peak,
+            "frac_of_8TBps_nominal": nbytes / per_call_g / 1e3 / 8000.0,
+            "tensor_core_call_form": {0: "planned", 1: "self-planned", 2: "cluster per segment", -1: "n/a"}[mode],
+            "device_status": status}
+
+
+def small_workload_record(torch, idx, device, peak, attn_path, steps, layers=36):
+    """One line of config.per_workload: a benchmark workload other than the headline one, measured in the same
+    process: the one-layer step as the benchmark spec states it (L2 flushed between steps), the step of a 36-layer model
+    over distinct pools, full parity against the oracle, and the oracle timed in full on the host cores."""
+    import paper_2605_20022_b200 as fd
+    from paper_2605_20022_b200 import workload as wl
+    step = wl.workload(idx)
+    flush = torch.empty((512 << 20,), dtype=torch.uint8, device=device)
+    ds = DeviceStep(step, device, attn_path, n_slots=steps + 4)
+    try:
+        ds.restore()
+        for _ in range(3):
+            ds.run()
+        parity = check_full(ds)
+        ds.attn_events = []
+        ms = timed_region(torch, None, lambda: ds.run(time_attn=True), steps, flush, prepare=ds.restore) / steps
+        attn_us = statistics.mean(a.elapsed_time(b) for a, b in ds.attn_events) * 1e3
+        g = capture_step_graph(torch, ds)
+        g.replay()
+        ms_g = timed_region(torch, None, g.replay, steps, flush) / steps
+        del g
+        status = fd.fd_last_device_status(ds.ctx)
+    finally:
+        ds.close()
+    del flush
+    many = decode_step_many_layers(torch, step, device, peak, attn_path, layers, reps=max(5, min(steps, 10)))
+    cpu_us, cpu_desc, cores = oracle_full(step)
+    return {"workload": step.name, "batch": step.batch, "q_rows": step.total_q_rows, "kv_tokens": int(step.kv_lens.sum()),
+            "attn_bytes": step.attn_bytes(), "logits_bytes": step.logits_bytes(),
+            "us_per_step": ms * 1e3, "us_per_step_cuda_graph_replay": ms_g * 1e3,
+            "us_per_attn_call_alone_event_bracketed": attn_us,
+            "us_per_attn_call": many["us_per_attn_call_cuda_graph_replay"], "attn_GBps": many["attn_GBps"],
+            "frac_of_measured": many["frac_of_measured_peak"], "parity": parity, "device_status": status,
+            "step_of_36_layer_model": many,
+            "cpu_oracle_us_per_step": cpu_us, "cpu_oracle_cores": cores, "cpu_oracle_sample": cpu_desc}
+
+
 def run_ours(args, step, rank, world, dist):
     import torch
     import paper_2605_20022_b200 as fd
@@ -371,7 +511,9 @@ def run_ours(args, step, rank, world, dist):
     ds.restore()
     for _ in range(args.warmup):
         ds.run()
-    parity_ok = check_against_oracle(ds) if rank == 0 else True
+    # small workloads: every element against the full oracle; the 78 GB workload: sampled rows here (its every-element
+    # comparison is the GPU test test_long_context_full_size_every_element)
+    parity_ok = (check_full(ds) if small else check_against_oracle(ds)) if rank == 0 else True
     status = fd.fd_last_device_status(ds.ctx)
 
     sampler = ClockSampler(dev_index)
@@ -472,7 +614,18 @@ def run_ours(args, step, rank, world, dist):
     for _ in range(2):
         hs.run()
     ms_e2e = timed_region(torch, dist, hs.run, args.steps)
+    h2d_bytes, d2h_bytes = hs.h2d, hs.d2h
     ds.close()
+    del hs, ds
+    torch.cuda.empty_cache()
+
+    # The step of a 36-layer model for a one-layer workload (its roofline figure comes from there), and, beside the
+    # headline workload, one record per other benchmark workload, measured in this same process.
+    many, per_workload = None, None
+    if rank == 0 and small:
+        many = decode_step_many_layers(torch, step, device, peak, args.attn_path, 36, reps=max(5, min(args.steps, 10)))
+    if rank == 0 and not small and not args.no_per_workload:
+        per_workload = [small_workload_record(torch, i, device, peak, args.attn_path, steps=10) for i in (0, 1, 2, 3, 5, 6, 7)]
 
     from paper_2605_20022_b200 import replicas
     ms, ms_e2e, ms_graph_r = replicas.max_over_ranks([ms, ms_e2e, ms_graph or 0.0], dist, device)
@@ -484,8 +637,14 @@ def run_ours(args, step, rank, world, dist):
     us_graph = replicas.whole_job_us_per_step(ms_graph_r, args.steps, world) if ms_graph is not None else None
     attn_bytes = step.attn_bytes()
     attn_avg_ms = statistics.mean(attn_ms)
+    how_timed = "CUDA events around each fd_attn_draft_verify call of the timed steps"
+    if many is not None:
+        # one small call bracketed by events measures the event pair as much as the kernel: the launch duration of a
+        # small workload is the average over 36 back-to-back calls on distinct pools (CUDA-graph replay)
+        attn_avg_ms = many["us_per_attn_call_cuda_graph_replay"] * 1e-3
+        how_timed = "CUDA events around 36 back-to-back calls over distinct KV pools (CUDA-graph replay), per call"
     achieved = attn_bytes / (attn_avg_ms * 1e-3) / 1e9
-    cpu_us, cpu_desc, cores = oracle_sample(step, step.shape.n_q_heads, layers=4)
+    cpu_us, cpu_desc, cores = oracle_time(step)
     return {
         "metric": METRIC, "value": us_step, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
@@ -501,14 +660,16 @@ def run_ours(args, step, rank, world, dist):
                    "parity_vs_oracle_sampled": parity_ok, "device_status": status,
                    "us_per_step_cuda_graph_replay": us_graph, "draft_tail_fd_draft_select": draft_tail,
                    "sampling_fd_verify_accept_sample": sample_row,
-                   "mask_rows_in_last_10_layers_only": layer_split},
+                   "mask_rows_in_last_10_layers_only": layer_split,
+                   "us_per_attn_call_alone_event_bracketed": statistics.mean(attn_ms) * 1e3,
+                   "step_of_36_layer_model": many, "per_workload": per_workload},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(step.name) if resolved == "tcgen05" else None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
                      "kernel": "fd_attn_draft_verify (plan launch + split-KV attention launch, merge fused)",
                      "algorithmic_bytes_per_launch": attn_bytes, "avg_launch_ms": attn_avg_ms,
-                     "launches_timed": len(attn_ms)},
+                     "launches_timed": len(attn_ms) if many is None else 36 * max(5, min(args.steps, 10)), "how_timed": how_timed},
         "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": cpu_desc},
-        "e2e": {"value": us_e2e, "unit": UNIT, "h2d_bytes_per_step": hs.h2d, "d2h_bytes_per_step": hs.d2h},
+        "e2e": {"value": us_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "paper_context": paper_context(),
@@ -523,9 +684,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=4, help="0..7, see workload.WORKLOAD_NAMES")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count of workload 4")
-    ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel")
-    ap.add_argument("--ref-heads", type=int, default=8, help="q-heads in the oracle's timed sample")
+    ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel, 3 tcgen05 always planned, 4 tcgen05 self-planned")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
+    ap.add_argument("--no-per-workload", action="store_true", help="headline workload only: skip the records of the other workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

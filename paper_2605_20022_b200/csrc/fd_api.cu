@@ -162,7 +162,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     const size_t o_cuq = take((NR + 1) * sizeof(int));
     const size_t o_cut = take((NR + 1) * sizeof(int));
     const size_t o_ok = take(B * sizeof(int));
-    const size_t o_sc = take(NR * cfg->n_kv_heads * sizeof(int));
+    const size_t o_sc = take(2 * NR * cfg->n_kv_heads * sizeof(int));
     const size_t o_cf = take((size_t)c->n_ctas * sizeof(int));
     const size_t o_cs = take(((size_t)c->n_ctas + 1) * sizeof(int));
     const size_t o_cne = take((NR + 1) * sizeof(int));
@@ -631,7 +631,7 @@ fd_status fd_last_device_status(fd_ctx* c, int32_t* code, void* stream) {
     if (*code & FD_DEV_TIMEOUT) {
         // a call that gave up may have left pieces counted on segments nobody merged: start the next call clean
         c->pinned = false;
-        if (cudaMemsetAsync(c->plan.seg_count, 0, (size_t)c->max_rb * c->cfg.n_kv_heads * sizeof(int), s) != cudaSuccess) return FD_ERR_CUDA;
+        if (cudaMemsetAsync(c->plan.seg_count, 0, 2 * (size_t)c->max_rb * c->cfg.n_kv_heads * sizeof(int), s) != cudaSuccess) return FD_ERR_CUDA;
     }
     return FD_OK;
 }

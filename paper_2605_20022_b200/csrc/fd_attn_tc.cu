@@ -647,15 +647,31 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         //      last one to deliver a piece of the segment -- the merge of all its partials.
         //      All 256 threads take every named barrier, whatever happened before; decisions that must be
         //      uniform (leave, merge) are taken by thread 0 alone and published through shared memory.
+        // A piece of a split segment: who merges is settled by a ticket.  Thread 0 draws it as soon as its own last
+        // tile is done -- the atomic's round trip then hides behind the rest of the piece -- and the CTA that draws
+        // the last ticket of the segment is the merger: every other piece of the segment belongs to a CTA that has
+        // drawn before it, hence is running and will deliver its partial without depending on anyone.  The merger
+        // keeps its own part in registers, waits (bounded) for the others' delivery count, and combines.
+        const int seg_t0 = w.t - pc.tile0, seg_t1 = seg_t0 + pc.seg_nt;
+        int c_first = cta, c_last = cta, n_pieces = 1, ticket = -1;  // (no ticket drawn: never the merger)
+        int* seg_cnt = p.plan.seg_count + 2 * (pc.v * p.Hkv + pc.kvh);  // [0] tickets drawn, [1] partials delivered
+        if (MODE != kTcCluster && !pc.complete) {
+            segment_ctas(cs, p.n_ctas, cta, seg_t0, seg_t1, c_first, c_last);
+            if (tid == 0 && !*abort) {
+                n_pieces = segment_pieces(cs, c_first, c_last, seg_t0, seg_t1);
+                ticket = atomicAdd(seg_cnt, 1);
+            }
+        }
         if (warp_active) ok = ok && wait_all(&bars->all_done, w.piece & 1, abort);
         tc_fence_after();
         const bool two = pc.nt >= 2;
         // Stream exchange: group 1 hands its (m, l) to group 0, which answers with the two scale factors.
         // A thread only ever touches the two slots of its own row, so one barrier each way is enough.
         if (s == 1) { ex[r] = m; ex[kMaxRows + r] = l; }
-        if (tid == 0) bars->epi_flag = *abort ? 2 : 0;
+        if (tid == 0) bars->epi_flag = (*abort ? 2 : 0) | ((MODE != kTcCluster && !pc.complete && ticket == n_pieces - 1) ? 1 : 0);
         named_bar_sync(1, 256);
         const bool leave = (bars->epi_flag & 2) != 0;
+        const bool merger = (bars->epi_flag & 1) != 0;
         float a0 = 0.f, a1 = 0.f, mm = -INFINITY, L = 0.f;
         if (s == 0) {
             const float m1 = two ? ex[r] : -INFINITY, l1 = ex[kMaxRows + r];
@@ -713,7 +729,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                         for (int k = 0; k < 32; ++k) o[ch][k] = 0.f;
                     }
                     store_cols_bf16<32>(dst, o[ch], 1.f);
-                } else {
+                } else if (!merger) {
                     float4* dst = partial_o4(p.part, D, pc.slot, col, r);
 #pragma unroll
                     for (int k = 0; k < 32; k += 4) dst[(k >> 2) * kMaxRows] = make_float4(o[ch][k], o[ch][k + 1], o[ch][k + 2], o[ch][k + 3]);
@@ -731,36 +747,42 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             if (r < pc.rows && dest == cl_rank && !leave)
                 cluster_reduce_row<D>(p, rv, cl_rank, r, s, do_read ? &o[0][0] : nullptr, pc.b, pc.kvh, pc.row0);
         } else if (do_read && r < pc.rows && !pc.complete && s == 0) {
+            // (the merger too: both column halves of its row need them, and only this thread has them)
             p.part.m[pc.slot * kMaxRows + r] = mm;
             p.part.l[pc.slot * kMaxRows + r] = L;
         }
         if (MODE != kTcCluster && !pc.complete) {
-            // Fused split merge: count the delivered pieces of the segment; whoever delivers the last
-            // one combines them all (no CTA ever waits for another).  The barrier orders the partial
-            // stores of all threads before thread 0's fence, and the fence before the count.
-            const int t0 = w.t - pc.tile0, t1 = t0 + pc.seg_nt;
-            int c_first, c_last;
-            segment_ctas(cs, p.n_ctas, cta, t0, t1, c_first, c_last);
-            named_bar_sync(1, 256);
-            if (tid == 0) {
-                int last = 0;
-                if (!leave && !*abort) {
-                    const int n = segment_pieces(cs, c_first, c_last, t0, t1);
+            if (!merger) {
+                // deliver: the barrier orders the partial stores of all threads before thread 0's fence, the fence
+                // before the count.  Nobody waits for the count's result: the CTA goes straight on to its next piece.
+                named_bar_sync(1, 256);
+                if (tid == 0 && !leave && !*abort) {
                     __threadfence();
-                    int* count = p.plan.seg_count + pc.v * p.Hkv + pc.kvh;
-                    last = atomicAdd(count, 1) + 1 == n;
-                    if (last) {
-                        *count = 0;  // everyone has been counted: ready for the next call that uses this plan
-                        __threadfence();
+                    atomicAdd(seg_cnt + 1, 1);
+                }
+            } else {
+                if (tid == 0) {
+                    // the n - 1 other pieces: all drawn before ours, so their CTAs are past their last tile
+                    const unsigned long long t_start = global_ns();
+                    bool there = false;
+                    for (uint32_t it = 0; !there; ++it) {
+                        int v;
+                        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(seg_cnt + 1) : "memory");
+                        there = v >= n_pieces - 1;
+                        if (!there && (it & 15u) == 15u && (*abort || global_ns() - t_start > kWaitLimitNs)) break;
+                    }
+                    if (there) {
+                        seg_cnt[0] = 0;  // everyone has drawn and delivered: ready for the next call
+                        seg_cnt[1] = 0;
+                    } else {
+                        *abort = 1;
                     }
                 }
-                bars->epi_flag = last;
-            }
-            named_bar_sync(1, 256);
-            if (bars->epi_flag & 1) {
+                named_bar_sync(1, 256);  // orders the acquire before every thread's loads of the partials
                 const int rr = tid & (kMaxRows - 1), cg = tid >> 7;
-                // rr == r and cg == s: the columns a thread merges are the ones it has just produced
-                if (rr < pc.rows) merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, t0, t1, rr, cg, &o[0][0], cta);
+                // rr == r and cg == s: the columns a thread merges are the ones it holds in registers
+                if (!*abort && !leave && rr < pc.rows)
+                    merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, seg_t0, seg_t1, rr, cg, &o[0][0], cta);
             }
         }
         if (leave) break;

@@ -42,7 +42,7 @@ struct Plan {
     int* cu_ne;     // [n_rb+1] exclusive scan of (tiles > 0)
     int* seq_bad;   // [B]   number (AttnParams::epoch) of the last call that met a page id outside the pool in the sequence:
                     //       equal to the running call's number = flagged, the sequence's rows are zeroed
-    int* seg_count; // [n_rb * Hkv] partial pieces of a segment that have been written (fused merge)
+    int* seg_count; // [n_rb * Hkv][2] per segment: merge tickets drawn, partial pieces delivered (zero between calls)
     int* cta_first; // [n_ctas] row block that owns the first tile of each attention CTA's range
     int* cta_start; // [n_ctas + 1] first tile of each attention CTA's range (non-decreasing; [n_ctas] = total)
 };

@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(256) plan_kernel(AttnParams p) {
     }
     if (n_rb > p.max_rb) { if (tid == 0) atomicOr(&s_fatal, 1); n_rb = p.max_rb; }
     __syncthreads();
-    for (int i = tid; i < n_rb * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
+    for (int i = tid; i < 2 * n_rb * p.Hkv; i += blockDim.x) p.plan.seg_count[i] = 0;
     // ---- pass 2, over row blocks (only where some block was cut)
     for (int base = 0; base < n_rb && !one_each; base += blockDim.x) {
         const int v = base + tid;
