@@ -57,7 +57,7 @@ constexpr int kThreads = 384;  // warps 0-3 softmax group 0, 4-7 softmax group 1
 constexpr int kKWarp = 8, kVWarp = 9, kMmaWarp = 10;  // warp 11 loads Q
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
-// How Q K^T(j) is kept from overwriting P(j - 2) before the P V that reads it has completed (see mma_role).
+// 1: Q K^T(j) waits for the completion of the P V whose P it overwrites; 0: it does not (see mma_role).
 #ifndef FD_QK_MODE
 #define FD_QK_MODE 1
 #endif
@@ -96,6 +96,7 @@ struct Bars {
     uint64_t q_full, q_free;   // Q tile of a piece landed / no longer read by any MMA
     uint64_t all_done;         // every MMA of a piece has completed
     uint64_t o_free;           // the epilogue of a piece has read O out of TMEM
+    uint64_t merge_bar;        // the other pieces of a segment have been copied into shared memory (merger, last piece)
     uint32_t tmem_base;
     int abort;
     int epi_flag;              // per-epilogue decisions of thread 0: bit 0 merge, bit 1 leave
@@ -335,10 +336,9 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
     using C = Cfg<D, MODE>;
     const int lane = threadIdx.x & 31;
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
-    constexpr uint32_t idesc_qk_half = make_idesc_bf16(128, kTileTokens / 2, false);
     constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
-    const uint32_t q_addr = smem_u32(sq);
+    const uint64_t qd0 = make_smem_desc(smem_u32(sq), 16, 1024);
     const int s_c = rg.s_c, e_c = rg.e_c;
     Walk w = {s_c, 0, {0, 0}, 0, rg.first};
     bool ok = true;
@@ -364,15 +364,16 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
             }
             // the first P V of a stream in a piece overwrites O: the previous piece's epilogue must have read it
             if (jj < 2 && w.piece > 0 && !wait_all(&bars->o_free, (w.piece - 1) & 1, abort)) { ok = false; return; }
+            // (descriptors are made before the last wait: what follows it is the MMA instructions alone.  The address
+            // field of a descriptor is its low 14 bits, in 16-byte units, so a K step is an addition.)
+            const uint64_t vd0 = make_smem_desc(smem_u32(vt), 1024, C::kGroupBytes);
             if (!wait_all(&bars->p_full[s], u & 1, abort)) { ok = false; return; }
             tc_fence_after();
             if (lane == 0) {
-                const uint32_t v_addr = smem_u32(vt);
 #pragma unroll
                 for (int kk = 0; kk < kTileTokens / 16; ++kk)
                     // one page per K step: its two 8-token groups lie kGroupBytes apart, the two halves of d 1 KB apart
-                    umma_ts(tmem + col_o[s], tmem + col_s[s] + kk * 8,
-                            make_smem_desc(v_addr + kk * C::kPageBytes, 1024, C::kGroupBytes), idesc_pv, jj >= 2 || kk > 0);
+                    umma_ts(tmem + col_o[s], tmem + col_s[s] + kk * 8, vd0 + (uint64_t)((kk * C::kPageBytes) >> 4), idesc_pv, jj >= 2 || kk > 0);
                 umma_commit(&bars->v_empty[st]);
                 umma_commit(&bars->pv_done[s]);
             }
@@ -384,36 +385,23 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
             if (!wait_all(&bars->k_full[st], use & 1, abort)) { ok = false; break; }
             // S_s is written over P_s (its first 64 columns), which the P V of tile j - 2 of this stream reads, and
             // nothing orders two MMAs with different accumulators but the completion of the first: Q K^T waits for
-            // that P V's completion barrier (FD_QK_MODE 1, the default).  Measured alternatives, kept for
-            // measurements only: 2 = Q K^T as two N = 64 halves, the tokens 64..127 (columns the P V does not read)
-            // ahead of the wait (11 % slower: the half-width MMAs cost more than the wait); 0 = no wait, relying on
-            // one thread's MMAs executing in issue order (5 % faster than the default, not a documented guarantee).
+            // that P V's completion barrier.  (FD_QK_MODE 0 drops the wait, relying on one thread's MMAs executing in
+            // issue order: 3-5 % faster, but not a documented guarantee; kept for measurements only.  Tried as well:
+            // Q K^T as two N = 64 halves with only the aliasing half behind the wait, 11 % slower; issuing whichever
+            // MMA is ready first from a polling loop, 8 % slower -- the polling warp takes issue slots from the
+            // softmax warps of its scheduler.)
             [[maybe_unused]] const int u_prev = w.u_base[s] + (j >> 1) - 1;  // the stream's previous tile, over all pieces
-            tc_fence_after();
-            const uint32_t k_addr = smem_u32(sk + st * C::kKBytes);
-#if FD_QK_MODE == 2
-            if (lane == 0) {
-#pragma unroll
-                for (int kk = 0; kk < C::kKSteps; ++kk) {
-                    const uint32_t q_off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
-                    const uint32_t k_off = (kk >> 2) * 1024 + (kk & 3) * 32 + 8 * C::kGroupBytes;
-                    umma_ss(tmem + col_s[s] + 64, make_smem_desc(q_addr + q_off, 16, 1024), make_smem_desc(k_addr + k_off, 16, C::kGroupBytes),
-                            idesc_qk_half, kk > 0);
-                }
-            }
-            __syncwarp();
-#endif
+            const uint64_t kd0 = make_smem_desc(smem_u32(sk + st * C::kKBytes), 16, C::kGroupBytes);
 #if FD_QK_MODE != 0
             if (u_prev >= 0 && !wait_all(&bars->pv_done[s], u_prev & 1, abort)) { ok = false; break; }
-            tc_fence_after();
 #endif
+            tc_fence_after();
             if (lane == 0) {
 #pragma unroll
                 for (int kk = 0; kk < C::kKSteps; ++kk) {
-                    const uint32_t q_off = (kk >> 2) * (kMaxRows * 128) + (kk & 3) * 32;
-                    const uint32_t k_off = (kk >> 2) * 1024 + (kk & 3) * 32;
-                    umma_ss(tmem + col_s[s], make_smem_desc(q_addr + q_off, 16, 1024), make_smem_desc(k_addr + k_off, 16, C::kGroupBytes),
-                            FD_QK_MODE == 2 ? idesc_qk_half : idesc_qk, kk > 0);
+                    constexpr int kQHalf = kMaxRows * 128;
+                    umma_ss(tmem + col_s[s], qd0 + (uint64_t)(((kk >> 2) * kQHalf + (kk & 3) * 32) >> 4),
+                            kd0 + (uint64_t)(((kk >> 2) * 1024 + (kk & 3) * 32) >> 4), idesc_qk, kk > 0);
                 }
                 umma_commit(&bars->k_empty[st]);
                 umma_commit(&bars->s_full[s]);
@@ -525,10 +513,58 @@ __device__ __forceinline__ void cluster_reduce_row(const AttnParams& p, const Re
     for (int ch = 0; ch < D / 64; ++ch) store_cols_bf16<32>(dst + ch * 32, acc + ch * 32, inv);
 }
 
+// Merge of a split segment from shared memory (the merger at the last piece of its range, when the rings are idle).
+// The n_other other pieces, in CTA order, lie one after the other at `stage`, each as the O array of a partial slot
+// ([D / 4][128 rows][4 floats]) followed by its m[128] and l[128]; this CTA's own piece -- the own_pos-th of the
+// segment in CTA order -- is in registers (own: the thread's D / 2 columns) with its (m, l) at own_ml[r], own_ml[128 + r].
+// Same arithmetic, same order as merge_row: the result does not depend on who merges.
+template <int D>
+__device__ __forceinline__ void merge_staged(const AttnParams& p, const unsigned char* stage, int n_other, int own_pos, const float* own,
+                                             const float* own_ml, int r, int cg, bool flagged, int kvh, int row0) {
+    constexpr int CW = D / 2;
+    constexpr uint32_t kBlock = kMaxRows * D * 4 + 2 * kMaxRows * 4;
+    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
+    float acc[CW];
+#pragma unroll
+    for (int c = 0; c < CW; ++c) acc[c] = 0.f;
+    if (flagged) {  // a page id of this sequence was bad: defined output, zeros
+        store_cols_bf16<CW>(dst, acc, 0.f);
+        return;
+    }
+    float m = own_ml[r];
+    for (int k = 0; k < n_other; ++k) m = fmaxf(m, reinterpret_cast<const float*>(stage + k * kBlock + kMaxRows * D * 4)[r]);
+    float l = 0.f;
+    for (int pos = 0; pos <= n_other; ++pos) {
+        if (pos == own_pos) {
+            const float mp = own_ml[r], lp = own_ml[kMaxRows + r];
+            const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
+            l += w * lp;
+#pragma unroll
+            for (int k = 0; k < CW; ++k) acc[k] += w * own[k];
+            continue;
+        }
+        const unsigned char* blk = stage + (pos < own_pos ? pos : pos - 1) * kBlock;
+        const float* ml = reinterpret_cast<const float*>(blk + kMaxRows * D * 4);
+        const float mp = ml[r], lp = ml[kMaxRows + r];
+        const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
+        l += w * lp;
+        const float4* o = reinterpret_cast<const float4*>(blk) + ((cg * CW) >> 2) * kMaxRows + r;
+#pragma unroll
+        for (int k = 0; k < CW / 4; ++k) {
+            const float4 v = o[k * kMaxRows];
+            acc[4 * k] += w * v.x;
+            acc[4 * k + 1] += w * v.y;
+            acc[4 * k + 2] += w * v.z;
+            acc[4 * k + 3] += w * v.w;
+        }
+    }
+    store_cols_bf16<CW>(dst, acc, 1.f / l);
+}
+
 // The two softmax groups (256 threads).
 template <int D, int MODE>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, int* s_cs, const CtaStarts cs, const Piece* ring,
-                                             uint32_t tmem, const Range rg, uint32_t recv_addr, int cl_rank, volatile int* abort) {
+                                             uint32_t tmem, const Range rg, uint32_t recv_addr, int cl_rank, unsigned char* stage, volatile int* abort) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     const int s_c = rg.s_c, e_c = rg.e_c;
     const int s = warp >> 2;                  // stream
@@ -655,6 +691,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         const int seg_t0 = w.t - pc.tile0, seg_t1 = seg_t0 + pc.seg_nt;
         int c_first = cta, c_last = cta, n_pieces = 1, ticket = -1;  // (no ticket drawn: never the merger)
         int* seg_cnt = p.plan.seg_count + 2 * (pc.v * p.Hkv + pc.kvh);  // [0] tickets drawn, [1] partials delivered
+        constexpr uint32_t kPieceBytes = kMaxRows * D * 4;                // the O array of a partial slot
+        constexpr uint32_t kStageBlock = kPieceBytes + 2 * kMaxRows * 4;  // ... followed by its m and l
+        // (the staging area also holds this CTA's own (m, l), behind the last block)
+        // (the staging area: the Q tile and both rings, idle at the last piece of a range)
+        constexpr int kMaxStaged = (Cfg<D, MODE>::kQBytes + 2 * Cfg<D, MODE>::kStages * Cfg<D, MODE>::kKBytes - 2 * kMaxRows * 4) / kStageBlock;
         if (MODE != kTcCluster && !pc.complete) {
             segment_ctas(cs, p.n_ctas, cta, seg_t0, seg_t1, c_first, c_last);
             if (tid == 0 && !*abort) {
@@ -668,10 +709,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         // Stream exchange: group 1 hands its (m, l) to group 0, which answers with the two scale factors.
         // A thread only ever touches the two slots of its own row, so one barrier each way is enough.
         if (s == 1) { ex[r] = m; ex[kMaxRows + r] = l; }
-        if (tid == 0) bars->epi_flag = (*abort ? 2 : 0) | ((MODE != kTcCluster && !pc.complete && ticket == n_pieces - 1) ? 1 : 0);
+        if (tid == 0) bars->epi_flag = (*abort ? 2 : 0) | ((MODE != kTcCluster && !pc.complete && ticket == n_pieces - 1) ? 1 : 0) | ((n_pieces - 1) << 8);
         named_bar_sync(1, 256);
         const bool leave = (bars->epi_flag & 2) != 0;
         const bool merger = (bars->epi_flag & 1) != 0;
+        const bool stage_ok = merger && w.t + pc.nt == e_c && (bars->epi_flag >> 8) <= kMaxStaged;  // uniform: from shared memory
         float a0 = 0.f, a1 = 0.f, mm = -INFINITY, L = 0.f;
         if (s == 0) {
             const float m1 = two ? ex[r] : -INFINITY, l1 = ex[kMaxRows + r];
@@ -748,8 +790,14 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 cluster_reduce_row<D>(p, rv, cl_rank, r, s, do_read ? &o[0][0] : nullptr, pc.b, pc.kvh, pc.row0);
         } else if (do_read && r < pc.rows && !pc.complete && s == 0) {
             // (the merger too: both column halves of its row need them, and only this thread has them)
-            p.part.m[pc.slot * kMaxRows + r] = mm;
-            p.part.l[pc.slot * kMaxRows + r] = L;
+            if (stage_ok) {
+                float* own_ml = reinterpret_cast<float*>(stage + kMaxStaged * kStageBlock);
+                own_ml[r] = mm;
+                own_ml[kMaxRows + r] = L;
+            } else {
+                p.part.m[pc.slot * kMaxRows + r] = mm;
+                p.part.l[pc.slot * kMaxRows + r] = L;
+            }
         }
         if (MODE != kTcCluster && !pc.complete) {
             if (!merger) {
@@ -774,15 +822,48 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     if (there) {
                         seg_cnt[0] = 0;  // everyone has drawn and delivered: ready for the next call
                         seg_cnt[1] = 0;
+                        bars->epi_flag |= 4;  // go: read after the barrier below, so that all 256 threads decide alike
                     } else {
                         *abort = 1;
+                    }
+                    // At the last piece of the range the Q tile and the K and V rings are idle (every load of this CTA has
+                    // been consumed): the other pieces (O, m, l) are brought there by bulk copies, all in flight together, and
+                    // the merge reads shared memory.  Read straight from L2 the merge is a chain of dependent round trips
+                    // (row maxima, then piece after piece), each 1-2 us while the other SMs still stream: measured 7-9 us
+                    // for two or three pieces.
+                    if (there && stage_ok) {
+                        fence_proxy_async_all();
+                        mbar_arrive_expect_tx(&bars->merge_bar, (uint32_t)(n_pieces - 1) * kStageBlock);
+                        int k = 0, own_pos = 0;
+                        for (int c = c_first; c <= c_last; ++c) {
+                            const int sc = cs.at(c), ec = cs.at(c + 1);
+                            if (c == cta || max(sc, seg_t0) >= min(ec, seg_t1)) continue;
+                            if (c < cta) ++own_pos;
+                            const int slot = 2 * c + (sc >= seg_t0 ? 0 : 1);
+                            unsigned char* blk = stage + (size_t)k * kStageBlock;
+                            bulk_load(blk, p.part.o + (size_t)slot * (kPieceBytes / 4), kPieceBytes, &bars->merge_bar);
+                            bulk_load(blk + kPieceBytes, p.part.m + slot * kMaxRows, kMaxRows * 4, &bars->merge_bar);
+                            bulk_load(blk + kPieceBytes + kMaxRows * 4, p.part.l + slot * kMaxRows, kMaxRows * 4, &bars->merge_bar);
+                            ++k;
+                        }
+                        // (after the acquire: every CTA of the segment has looked up its page ids by now)
+                        bars->epi_flag |= (own_pos << 16) | (sequence_flagged(p, pc.b) ? 8 : 0);
                     }
                 }
                 named_bar_sync(1, 256);  // orders the acquire before every thread's loads of the partials
                 const int rr = tid & (kMaxRows - 1), cg = tid >> 7;
                 // rr == r and cg == s: the columns a thread merges are the ones it holds in registers
-                if (!*abort && !leave && rr < pc.rows)
-                    merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, seg_t0, seg_t1, rr, cg, &o[0][0], cta);
+                if ((bars->epi_flag & 4) && !leave) {
+                    if (!stage_ok) {
+                        if (rr < pc.rows)
+                            merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, seg_t0, seg_t1, rr, cg, &o[0][0], cta);
+                    } else if (wait_all(&bars->merge_bar, 0, abort)) {  // (used at most once per CTA: phase 0)
+                        if (rr < pc.rows)
+                            merge_staged<D>(p, stage, (int)((bars->epi_flag >> 8) & 0xff), (int)(bars->epi_flag >> 16), &o[0][0],
+                                            reinterpret_cast<const float*>(stage + kMaxStaged * kStageBlock), rr, cg,
+                                            (bars->epi_flag & 8) != 0, pc.kvh, pc.row0);
+                    }
+                }
             }
         }
         if (leave) break;
@@ -888,6 +969,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         mbar_init(&bars->q_free, 1);
         mbar_init(&bars->all_done, 1);
         mbar_init(&bars->o_free, 256);
+        mbar_init(&bars->merge_bar, 1);
         bars->abort = 0;
         bars->epi_flag = 0;
         bars->desc_n = 0;
@@ -977,7 +1059,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168, what the launch allocated: the increase is served exactly by what
         // the decrease released (a request for more than that does not return).
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, recv_addr, cl_rank, abort);
+        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, recv_addr, cl_rank, sq, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, abort);
