@@ -427,7 +427,9 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     int mode = fd::kTcPlanned;
     if (tc && p.rb_per_seq == 1 && c->tc_choice != FD_ATTN_TCGEN05_PLANNED) {
         const int n_seg = batch * p.Hkv;
-        const int cl = (c->tc_choice == FD_ATTN_TCGEN05 && batch <= fd::kSelfPlanMaxRb && n_seg <= fd::kClusterMaxSegments)
+        // (a table too narrow for four tiles per sequence leaves a cluster nothing to split)
+        const bool splittable = (long long)p.max_pages * 16 >= 4 * fd::kTileTokens;
+        const int cl = (c->tc_choice == FD_ATTN_TCGEN05 && batch <= fd::kSelfPlanMaxRb && n_seg <= fd::kClusterMaxSegments && splittable)
                            ? fd::attn_tc_cluster_size(c->tc_state, n_seg, c->n_sms) : 0;
         if (cl >= 2) { mode = fd::kTcCluster; p.cluster = cl; }
         else if (batch <= fd::kSelfPlanMaxRb && !reuse) mode = fd::kTcSelfPlanned;

@@ -62,6 +62,8 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units
 #define FD_QK_MODE 1
 #endif
 
+constexpr int cluster_recv_bytes(int d) { return d == 128 ? 2 * kTileTokens * 128 * 2 : 2 * kTileTokens * 64 * 2; }  // one K and one V stage
+
 template <int D, int MODE>
 struct Cfg {
     static constexpr int kFullStages = (D == 128) ? 3 : 6;
@@ -70,9 +72,10 @@ struct Cfg {
     static constexpr int kStages = MODE == kTcCluster ? ((D == 128) ? 2 : 5) : kFullStages;
     static constexpr int kQBytes = kMaxRows * D * 2;
     static constexpr int kKBytes = kTileTokens * D * 2;  // one K (or V) tile
-    static constexpr int kRecvOffset = kQBytes + 2 * kStages * kKBytes;        // kTcCluster: (m, l) pairs, then rows of O, from the peers
-    static constexpr int kRecvBytes = 2 * (kFullStages - kStages) * kKBytes;
-    static constexpr int kRecvMlBytes = kMaxRows * 8;                           // [cluster size][rows per CTA] float2
+    // kTcCluster: the receive area, 2 KB of (m, l) pairs [cluster size][rows per CTA], then rows of O, from the peers;
+    // it is what the ring gave up: cluster_recv_bytes(D)
+    static constexpr int kRecvOffset = kQBytes + 2 * kStages * kKBytes;
+    static_assert(MODE != kTcCluster || 2 * (kFullStages - kStages) * kKBytes == cluster_recv_bytes(D), "receive area");
     static constexpr int kBarOffset = kQBytes + 2 * kFullStages * kKBytes;
     static constexpr int kCsOffset = kBarOffset + 320;           // window of the CTA range starts
     static constexpr int kDescOffset = kBarOffset + 448;         // ring of piece descriptors
@@ -81,7 +84,6 @@ struct Cfg {
     static constexpr int kRbOffset = kBarOffset + 2048;          // row blocks of a call that plans for itself
     static constexpr int kSmemBytes = kBarOffset + 3072;         // the dynamic shared memory is declared 1024-byte aligned
     // what a CTA receives: (m, l) of every peer, and O rows of every peer but itself, for its 128 / cluster-size rows
-    static_assert(MODE != kTcCluster || kRecvMlBytes + (kMaxRows * D * 4) / 2 <= kRecvBytes, "receive area too small for a cluster of 2");
     static constexpr int kKSteps = D / 16;
     static constexpr int kHalves = D / 64;
     // A K or V tile in shared memory: [8-token group][half of d][8 rows][128 B] -- what one TMA box per page
@@ -103,6 +105,7 @@ struct Bars {
     int desc_n;                // piece descriptors published so far (written by the Q load warp)
     int piece_ok;              // thread 0 of the softmax groups: the descriptor of the next piece is there
     int first;                 // a call that plans for itself: the row block that owns the first tile of this CTA's range
+    int bad;                   // a load warp of this CTA met a page id outside the pool
 };
 constexpr int kDescSlots = 4;
 
@@ -229,7 +232,7 @@ struct Walk {
 // K (which = 0) or V (which = 1) load warp.
 template <int D, int MODE>
 __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnParams& p, int n_rb, unsigned char* ring, uint64_t* full,
-                                          uint64_t* empty, int which, const Range rg, volatile int* abort) {
+                                          uint64_t* empty, int which, const Range rg, volatile int* bad, volatile int* abort) {
     using C = Cfg<D, MODE>;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     constexpr int kOps = 8;  // pages of a tile: one box each
@@ -254,6 +257,7 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             int id = table[pos >> 4];
             if ((unsigned)id >= (unsigned)p.num_pages) {  // never form an address from a bad id
                 flag_sequence(p, pc.b);
+                *bad = 1;
                 id = 0;
             }
             return id;
@@ -457,6 +461,12 @@ __device__ __forceinline__ float4 lds_v4(uint32_t addr) {
     return v;
 }
 constexpr int kMaxCluster = 16;
+// Rows a CTA of a cluster of c owns (the last CTA may own fewer, or none).
+__host__ __device__ constexpr int cluster_share(int c) { return (kMaxRows + c - 1) / c; }
+// Does the receive area (recv_bytes) hold what a CTA of a cluster of c gets: (m, l) from all, O rows from all but itself?
+__host__ __device__ constexpr bool cluster_fits(int c, int d, int recv_bytes) {
+    return c * cluster_share(c) <= 2 * kMaxRows && 2 * kMaxRows * 8 + (c - 1) * cluster_share(c) * d * 4 <= recv_bytes;
+}
 
 // The receive area of a CTA: (m, l) of source CTA c for owned row rl at ml[c * share + rl]; the O row of source c
 // (c != own rank; slot = c, less one past the own rank) as D / 4 16-byte words, word w at position w ^ (rl & 31):
@@ -467,7 +477,7 @@ struct Recv {
     int share;
     __device__ __forceinline__ uint32_t ml(int c, int rl) const { return base + (uint32_t)(c * share + rl) * 8; }
     __device__ __forceinline__ uint32_t o(int slot, int rl, int word) const {
-        return base + kMaxRows * 8 + (uint32_t)((slot * share + rl) * (D / 4) + (word ^ (rl & (D / 4 - 1)))) * 16;
+        return base + 2 * kMaxRows * 8 + (uint32_t)((slot * share + rl) * (D / 4) + (word ^ (rl & (D / 4 - 1)))) * 16;
     }
 };
 
@@ -478,7 +488,12 @@ __device__ __forceinline__ void cluster_reduce_row(const AttnParams& p, const Re
                                                    int kvh, int row0) {
     const int C = p.cluster, rl = r % rv.share;
     float m = -INFINITY;
-    for (int c = 0; c < C; ++c) m = fmaxf(m, lds_v2(rv.ml(c, rl)).x);
+    bool flagged = false;  // some CTA of the cluster met a page id outside the pool (it sent l < 0)
+    for (int c = 0; c < C; ++c) {
+        const float2 ml = lds_v2(rv.ml(c, rl));
+        m = fmaxf(m, ml.x);
+        flagged = flagged || ml.y < 0.f;
+    }
     float acc[D / 2];
 #pragma unroll
     for (int k = 0; k < D / 2; ++k) acc[k] = 0.f;
@@ -503,7 +518,7 @@ __device__ __forceinline__ void cluster_reduce_row(const AttnParams& p, const Re
         }
     }
     float inv = l > 0.f ? 1.f / l : 0.f;
-    if (sequence_flagged(p, b)) {  // by assignment: what came from a stand-in page may be inf or NaN
+    if (flagged) {  // by assignment: what came from a stand-in page may be inf or NaN
         inv = 0.f;
 #pragma unroll
         for (int k = 0; k < D / 2; ++k) acc[k] = 0.f;
@@ -513,50 +528,76 @@ __device__ __forceinline__ void cluster_reduce_row(const AttnParams& p, const Re
     for (int ch = 0; ch < D / 64; ++ch) store_cols_bf16<32>(dst + ch * 32, acc + ch * 32, inv);
 }
 
-// Merge of a split segment from shared memory (the merger at the last piece of its range, when the rings are idle).
-// The n_other other pieces, in CTA order, lie one after the other at `stage`, each as the O array of a partial slot
-// ([D / 4][128 rows][4 floats]) followed by its m[128] and l[128]; this CTA's own piece -- the own_pos-th of the
-// segment in CTA order -- is in registers (own: the thread's D / 2 columns) with its (m, l) at own_ml[r], own_ml[128 + r].
-// Same arithmetic, same order as merge_row: the result does not depend on who merges.
-template <int D>
-__device__ __forceinline__ void merge_staged(const AttnParams& p, const unsigned char* stage, int n_other, int own_pos, const float* own,
-                                             const float* own_ml, int r, int cg, bool flagged, int kvh, int row0) {
+// Merge of a split segment from shared memory (the merger at the last piece of its range, when the Q tile and the
+// rings are idle).  The staging area holds kRound O arrays of partial slots ([D / 4][128 rows][4 floats]) and behind
+// them the (m[128], l[128]) pairs: first this CTA's own, then those of the n_other other pieces in CTA order.  The O
+// arrays come in rounds of kRound pieces (bulk copies issued by thread 0 through issue_round, completion on merge_bar);
+// this CTA's own piece -- the own_pos-th of the segment in CTA order -- is in registers (own: the thread's D / 2
+// columns).  Same arithmetic, same order as merge_row: the result does not depend on who merges.  Called by all 256
+// threads of the softmax groups (it holds barriers); `active`: the thread has a row to write.
+template <int D, int MODE>
+struct Stage {
+    static constexpr uint32_t kBytes = Cfg<D, MODE>::kQBytes + 2 * Cfg<D, MODE>::kStages * Cfg<D, MODE>::kKBytes;
+    static constexpr uint32_t kPieceBytes = kMaxRows * D * 4;
+    static constexpr int kRound = (kBytes - 8192) / kPieceBytes;
+    static constexpr uint32_t kMlOffset = kRound * kPieceBytes;
+    static constexpr int kMaxOthers = (kBytes - kMlOffset) / (2 * kMaxRows * 4) - 1;
+};
+
+template <int D, int MODE, class IssueRound>
+__device__ __forceinline__ void merge_staged(const AttnParams& p, Bars* bars, const unsigned char* stage, int n_other, int own_pos,
+                                             const float* own, int r, int cg, bool active, bool flagged, int kvh, int row0,
+                                             volatile int* abort, IssueRound issue_round) {
+    using S = Stage<D, MODE>;
     constexpr int CW = D / 2;
-    constexpr uint32_t kBlock = kMaxRows * D * 4 + 2 * kMaxRows * 4;
-    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
+    const float* ml = reinterpret_cast<const float*>(stage + S::kMlOffset);  // [1 + n_other][2][128]
     float acc[CW];
 #pragma unroll
     for (int c = 0; c < CW; ++c) acc[c] = 0.f;
-    if (flagged) {  // a page id of this sequence was bad: defined output, zeros
-        store_cols_bf16<CW>(dst, acc, 0.f);
-        return;
-    }
-    float m = own_ml[r];
-    for (int k = 0; k < n_other; ++k) m = fmaxf(m, reinterpret_cast<const float*>(stage + k * kBlock + kMaxRows * D * 4)[r]);
-    float l = 0.f;
-    for (int pos = 0; pos <= n_other; ++pos) {
-        if (pos == own_pos) {
-            const float mp = own_ml[r], lp = own_ml[kMaxRows + r];
-            const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
-            l += w * lp;
-#pragma unroll
-            for (int k = 0; k < CW; ++k) acc[k] += w * own[k];
-            continue;
-        }
-        const unsigned char* blk = stage + (pos < own_pos ? pos : pos - 1) * kBlock;
-        const float* ml = reinterpret_cast<const float*>(blk + kMaxRows * D * 4);
+    float m = -INFINITY, l = 0.f;
+    auto add_own = [&]() {
         const float mp = ml[r], lp = ml[kMaxRows + r];
         const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
         l += w * lp;
-        const float4* o = reinterpret_cast<const float4*>(blk) + ((cg * CW) >> 2) * kMaxRows + r;
 #pragma unroll
-        for (int k = 0; k < CW / 4; ++k) {
-            const float4 v = o[k * kMaxRows];
-            acc[4 * k] += w * v.x;
-            acc[4 * k + 1] += w * v.y;
-            acc[4 * k + 2] += w * v.z;
-            acc[4 * k + 3] += w * v.w;
+        for (int k = 0; k < CW; ++k) acc[k] += w * own[k];
+    };
+    for (int round = 0, k0 = 0;; ++round, k0 += S::kRound) {
+        if (!wait_all(&bars->merge_bar, round & 1, abort)) return;  // uniform: every thread sees the same outcome or leaves
+        if (round == 0 && active) {
+            m = ml[r];
+            for (int k = 0; k < n_other; ++k) m = fmaxf(m, ml[(1 + k) * 2 * kMaxRows + r]);
         }
+        const int k1 = min(n_other, k0 + S::kRound);
+        if (active) {
+            for (int k = k0; k < k1; ++k) {
+                if (k == own_pos) add_own();
+                const float mp = ml[(1 + k) * 2 * kMaxRows + r], lp = ml[(1 + k) * 2 * kMaxRows + kMaxRows + r];
+                const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
+                l += w * lp;
+                const float4* o = reinterpret_cast<const float4*>(stage + (size_t)(k - k0) * S::kPieceBytes) + ((cg * CW) >> 2) * kMaxRows + r;
+#pragma unroll
+                for (int q = 0; q < CW / 4; ++q) {
+                    const float4 v = o[q * kMaxRows];
+                    acc[4 * q] += w * v.x;
+                    acc[4 * q + 1] += w * v.y;
+                    acc[4 * q + 2] += w * v.z;
+                    acc[4 * q + 3] += w * v.w;
+                }
+            }
+        }
+        if (k1 == n_other) break;
+        named_bar_sync(1, 256);  // everyone has read this round's O arrays: the next round may land on them
+        if (threadIdx.x == 0) issue_round(round + 1);
+    }
+    if (!active) return;
+    if (own_pos == n_other) add_own();
+    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + cg * CW;
+    if (flagged) {  // a page id of this sequence was bad: defined output, zeros (by assignment)
+#pragma unroll
+        for (int c = 0; c < CW; ++c) acc[c] = 0.f;
+        store_cols_bf16<CW>(dst, acc, 0.f);
+        return;
     }
     store_cols_bf16<CW>(dst, acc, 1.f / l);
 }
@@ -691,11 +732,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         const int seg_t0 = w.t - pc.tile0, seg_t1 = seg_t0 + pc.seg_nt;
         int c_first = cta, c_last = cta, n_pieces = 1, ticket = -1;  // (no ticket drawn: never the merger)
         int* seg_cnt = p.plan.seg_count + 2 * (pc.v * p.Hkv + pc.kvh);  // [0] tickets drawn, [1] partials delivered
-        constexpr uint32_t kPieceBytes = kMaxRows * D * 4;                // the O array of a partial slot
-        constexpr uint32_t kStageBlock = kPieceBytes + 2 * kMaxRows * 4;  // ... followed by its m and l
-        // (the staging area also holds this CTA's own (m, l), behind the last block)
-        // (the staging area: the Q tile and both rings, idle at the last piece of a range)
-        constexpr int kMaxStaged = (Cfg<D, MODE>::kQBytes + 2 * Cfg<D, MODE>::kStages * Cfg<D, MODE>::kKBytes - 2 * kMaxRows * 4) / kStageBlock;
+        using St = Stage<D, MODE>;
         if (MODE != kTcCluster && !pc.complete) {
             segment_ctas(cs, p.n_ctas, cta, seg_t0, seg_t1, c_first, c_last);
             if (tid == 0 && !*abort) {
@@ -713,7 +750,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         named_bar_sync(1, 256);
         const bool leave = (bars->epi_flag & 2) != 0;
         const bool merger = (bars->epi_flag & 1) != 0;
-        const bool stage_ok = merger && w.t + pc.nt == e_c && (bars->epi_flag >> 8) <= kMaxStaged;  // uniform: from shared memory
+        const bool stage_ok = merger && w.t + pc.nt == e_c && (bars->epi_flag >> 8) <= St::kMaxOthers;  // uniform: from shared memory
         float a0 = 0.f, a1 = 0.f, mm = -INFINITY, L = 0.f;
         if (s == 0) {
             const float m1 = two ? ex[r] : -INFINITY, l1 = ex[kMaxRows + r];
@@ -755,7 +792,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             }
             if (MODE == kTcCluster) {
                 // one cluster per segment: a row another CTA owns goes straight into that CTA's receive area
-                const int share = kMaxRows / p.cluster, dest = r / share;
+                const int share = cluster_share(p.cluster), dest = r / share;
                 if (do_read && r < pc.rows && dest != cl_rank) {
                     const Recv<D> rv = {recv_addr, share};
                     const int slot = cl_rank < dest ? cl_rank : cl_rank - 1;
@@ -779,11 +816,13 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             }
         }
         if (MODE == kTcCluster) {
-            const int share = kMaxRows / p.cluster, dest = r / share;
+            const int share = cluster_share(p.cluster), dest = r / share;
             const Recv<D> rv = {recv_addr, share};
             // (m, l) of the row to its owner (which may be this CTA); a row this CTA could not compute (it is giving up)
-            // counts as "saw no key"
-            if (r < pc.rows && s == 0) st_peer_v2(peer_addr(rv.ml(cl_rank, r % share), dest), do_read ? make_float2(mm, L) : make_float2(-INFINITY, 0.f));
+            // counts as "saw no key"; a CTA whose load warps met a page id outside the pool says so with a negative l
+            if (r < pc.rows && s == 0)
+                st_peer_v2(peer_addr(rv.ml(cl_rank, r % share), dest),
+                           !do_read ? make_float2(-INFINITY, 0.f) : make_float2(mm, bars->bad ? -1.f : L));
             cluster_sync_all();  // all 256 threads, whatever happened before; the other warps of the CTA wait in the kernel body
             cl_synced = true;
             if (r < pc.rows && dest == cl_rank && !leave)
@@ -791,7 +830,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         } else if (do_read && r < pc.rows && !pc.complete && s == 0) {
             // (the merger too: both column halves of its row need them, and only this thread has them)
             if (stage_ok) {
-                float* own_ml = reinterpret_cast<float*>(stage + kMaxStaged * kStageBlock);
+                float* own_ml = reinterpret_cast<float*>(stage + St::kMlOffset);
                 own_ml[r] = mm;
                 own_ml[kMaxRows + r] = L;
             } else {
@@ -826,29 +865,38 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     } else {
                         *abort = 1;
                     }
-                    // At the last piece of the range the Q tile and the K and V rings are idle (every load of this CTA has
-                    // been consumed): the other pieces (O, m, l) are brought there by bulk copies, all in flight together, and
-                    // the merge reads shared memory.  Read straight from L2 the merge is a chain of dependent round trips
-                    // (row maxima, then piece after piece), each 1-2 us while the other SMs still stream: measured 7-9 us
-                    // for two or three pieces.
-                    if (there && stage_ok) {
-                        fence_proxy_async_all();
-                        mbar_arrive_expect_tx(&bars->merge_bar, (uint32_t)(n_pieces - 1) * kStageBlock);
-                        int k = 0, own_pos = 0;
-                        for (int c = c_first; c <= c_last; ++c) {
-                            const int sc = cs.at(c), ec = cs.at(c + 1);
-                            if (c == cta || max(sc, seg_t0) >= min(ec, seg_t1)) continue;
-                            if (c < cta) ++own_pos;
-                            const int slot = 2 * c + (sc >= seg_t0 ? 0 : 1);
-                            unsigned char* blk = stage + (size_t)k * kStageBlock;
-                            bulk_load(blk, p.part.o + (size_t)slot * (kPieceBytes / 4), kPieceBytes, &bars->merge_bar);
-                            bulk_load(blk + kPieceBytes, p.part.m + slot * kMaxRows, kMaxRows * 4, &bars->merge_bar);
-                            bulk_load(blk + kPieceBytes + kMaxRows * 4, p.part.l + slot * kMaxRows, kMaxRows * 4, &bars->merge_bar);
-                            ++k;
+                }
+                // At the last piece of the range the Q tile and the K and V rings are idle (every load of this CTA has
+                // been consumed): the other pieces (m, l, and the O arrays in rounds) are brought there by bulk copies, all
+                // of a round in flight together, and the merge reads shared memory.  Read straight from L2 the merge is
+                // a chain of dependent round trips (row maxima, then piece after piece), each 1-2 us while the other SMs
+                // still stream: measured 7-9 us for two or three pieces.
+                auto issue_round = [&](int round) {  // thread 0
+                    const int k0 = round * St::kRound, k1 = min(n_pieces - 1, k0 + St::kRound);
+                    mbar_arrive_expect_tx(&bars->merge_bar, (uint32_t)(k1 - k0) * St::kPieceBytes + (round == 0 ? (uint32_t)(n_pieces - 1) * 2 * kMaxRows * 4 : 0u));
+                    int k = 0;
+                    for (int c = c_first; c <= c_last; ++c) {
+                        const int sc = cs.at(c), ec = cs.at(c + 1);
+                        if (c == cta || max(sc, seg_t0) >= min(ec, seg_t1)) continue;
+                        const int slot = 2 * c + (sc >= seg_t0 ? 0 : 1);
+                        if (round == 0) {
+                            unsigned char* mlk = stage + St::kMlOffset + (size_t)(1 + k) * 2 * kMaxRows * 4;
+                            bulk_load(mlk, p.part.m + slot * kMaxRows, kMaxRows * 4, &bars->merge_bar);
+                            bulk_load(mlk + kMaxRows * 4, p.part.l + slot * kMaxRows, kMaxRows * 4, &bars->merge_bar);
                         }
-                        // (after the acquire: every CTA of the segment has looked up its page ids by now)
-                        bars->epi_flag |= (own_pos << 16) | (sequence_flagged(p, pc.b) ? 8 : 0);
+                        if (k >= k0 && k < k1)
+                            bulk_load(stage + (size_t)(k - k0) * St::kPieceBytes, p.part.o + (size_t)slot * (St::kPieceBytes / 4), St::kPieceBytes,
+                                      &bars->merge_bar);
+                        ++k;
                     }
+                };
+                if (tid == 0 && (bars->epi_flag & 4) && stage_ok) {
+                    fence_proxy_async_all();
+                    issue_round(0);
+                    int own_pos = 0;
+                    for (int c = c_first; c < cta; ++c) own_pos += max(cs.at(c), seg_t0) < min(cs.at(c + 1), seg_t1);
+                    // (after the acquire: every CTA of the segment has looked up its page ids by now)
+                    bars->epi_flag |= (own_pos << 16) | (sequence_flagged(p, pc.b) ? 8 : 0);
                 }
                 named_bar_sync(1, 256);  // orders the acquire before every thread's loads of the partials
                 const int rr = tid & (kMaxRows - 1), cg = tid >> 7;
@@ -857,11 +905,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                     if (!stage_ok) {
                         if (rr < pc.rows)
                             merge_row<D, D / 2>(p, cs, c_first, c_last, pc.b, pc.kvh, pc.row0, seg_t0, seg_t1, rr, cg, &o[0][0], cta);
-                    } else if (wait_all(&bars->merge_bar, 0, abort)) {  // (used at most once per CTA: phase 0)
-                        if (rr < pc.rows)
-                            merge_staged<D>(p, stage, (int)((bars->epi_flag >> 8) & 0xff), (int)(bars->epi_flag >> 16), &o[0][0],
-                                            reinterpret_cast<const float*>(stage + kMaxStaged * kStageBlock), rr, cg,
-                                            (bars->epi_flag & 8) != 0, pc.kvh, pc.row0);
+                    } else {
+                        merge_staged<D, MODE>(p, bars, stage, (int)((bars->epi_flag >> 8) & 0xff), (int)(bars->epi_flag >> 16), &o[0][0], rr, cg,
+                                              rr < pc.rows, (bars->epi_flag & 8) != 0, pc.kvh, pc.row0, abort, issue_round);
                     }
                 }
             }
@@ -974,6 +1020,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         bars->epi_flag = 0;
         bars->desc_n = 0;
         bars->piece_ok = 0;
+        bars->bad = 0;
         mbar_fence_init();
     }
     if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
@@ -1048,7 +1095,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     const uint32_t recv_addr = smem_u32(smem) + (uint32_t)C::kRecvOffset;
     if (MODE == kTcCluster && cl_idle) {
         // fewer tiles than CTAs in the cluster: this one tells every owner "saw no key" and combines the rows it owns
-        const Recv<D> rv = {recv_addr, kMaxRows / p.cluster};
+        const Recv<D> rv = {recv_addr, cluster_share(p.cluster)};
         if (tid < cl_rows) st_peer_v2(peer_addr(rv.ml(cl_rank, tid % rv.share), tid / rv.share), make_float2(-INFINITY, 0.f));
         cluster_sync_all();
         const int r = tid & (kMaxRows - 1);
@@ -1062,8 +1109,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, recv_addr, cl_rank, sq, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, abort);
-        else if (warp == kVWarp) load_role<D, MODE>(tmap, p, n_rb, sv, bars->v_full, bars->v_empty, 1, rg, abort);
+        if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, &bars->bad, abort);
+        else if (warp == kVWarp) load_role<D, MODE>(tmap, p, n_rb, sv, bars->v_full, bars->v_empty, 1, rg, &bars->bad, abort);
         else if (warp == kMmaWarp) mma_role<D, MODE>(p, sq, sk, sv, bars, ring, tmem, rg, abort);
         else q_role<D, MODE>(qmap, p, n_rb, sq, bars, ring, rg, abort);
         if (MODE == kTcCluster) cluster_sync_all();  // the cluster barrier of the merge counts every thread
@@ -1194,7 +1241,10 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
         for (int c = 0; c <= kMaxCluster; ++c) st->max_clusters[c] = 0;
-        for (int c = 2; c <= kMaxCluster; c *= 2) st->max_clusters[c] = p.d == 64 ? query_clusters<64>(c, n_sms) : query_clusters<128>(c, n_sms);
+        for (int c = 2; c <= kMaxCluster; ++c) {
+            const bool fits = cluster_fits(c, p.d, cluster_recv_bytes(p.d));
+            st->max_clusters[c] = !fits ? 0 : p.d == 64 ? query_clusters<64>(c, n_sms) : query_clusters<128>(c, n_sms);
+        }
         *state = st;
     }
     // q: a 3-D view [T][Hq][d], box = 64 elements x G q-heads (one kv-head) x q_box_t block rows
@@ -1236,12 +1286,13 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
     return cudaSuccess;
 }
 
-// CTAs per cluster for a call with one cluster per segment: the largest power of two for which all clusters of the
-// call are resident together (so every SM it can use streams at once); 0 if there is none.
+// CTAs per cluster for a call with one cluster per segment: the largest size (any, not only powers of two: a GPC holds
+// a limited number of clusters of each size) for which all clusters of the call are resident together, so every SM it
+// can use streams at once and a CTA has the fewest tiles; 0 if there is none.
 int attn_tc_cluster_size(const void* state, int n_segments, int n_sms) {
     const TcState* st = static_cast<const TcState*>(state);
     if (!st || n_segments <= 0) return 0;
-    for (int c = kMaxCluster; c >= 2; c /= 2)
+    for (int c = kMaxCluster; c >= 2; --c)
         if (n_segments * c <= n_sms && st->max_clusters[c] >= n_segments) return c;
     return 0;
 }
