@@ -218,6 +218,9 @@ class DeviceStep:
         self.q = [wl.make_q(step, l, device) for l in range(self.L)]
         self.kv = [wl.make_kv(step, l, device) for l in range(self.L)]
         self.out = [torch.empty_like(t) for t in self.q]
+        # the K/V of the query block as the projections of the step would hand them over: read out of the cache that
+        # already holds them, so that appending them (run(append=True)) leaves every byte of the cache as it was
+        self.k_new, self.v_new = zip(*[wl.query_block_kv(step, kv) for kv in self.kv])
         logits, drafts, self.target = wl.make_logits(step, device)
         self.logits, self.drafts = logits, drafts.to(device)
         self.pt0, self.pl0 = step.page_table.to(device), step.prefix_lens.to(device)
@@ -248,7 +251,7 @@ class DeviceStep:
             pt.copy_(self.pt0); pl.copy_(self.pl0)
         self.cur = 0
 
-    def run(self, time_attn=False, restore_inline=False, attn_only=False):
+    def run(self, time_attn=False, restore_inline=False, attn_only=False, append=False):
         """One step on the current stream, on the next restored copy of the page table and lengths.  With
         restore_inline the copy is refreshed inside the step (a replayed CUDA graph has no other way); with
         attn_only just the attention calls of the step, one per layer (nothing is rewritten, nothing to restore)."""
@@ -264,6 +267,9 @@ class DeviceStep:
         if self.L > 1:   # every layer of the step has the same lengths: one work list serves them all
             fd.fd_plan_pin(self.ctx, st.batch, st.total_q_rows, self.pl, self.ql, self.nm, self.nb)
         for l in range(self.L):
+            if append:   # the step with the KV append inside: write the block's K/V of this layer, then attend
+                fd.fd_kv_append(self.ctx, st.batch, st.total_q_rows, self.k_new[l], self.v_new[l], self.kv[l], st.num_pages,
+                                self.pt, self.pl, self.ql)
             if time_attn:
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record()
@@ -345,13 +351,13 @@ def timed_region(torch, dist, fn, steps, flush=None, prepare=None):
     return ms
 
 
-def capture_step_graph(torch, ds, attn_only=False):
+def capture_step_graph(torch, ds, attn_only=False, append=False):
     """The whole step (attention x layers, accept, commit) as one CUDA graph on a side stream.  Only
     used after warm-up, so every first-call set-up inside the library has already happened."""
     g = torch.cuda.CUDAGraph()
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
-    run = (lambda: ds.run(attn_only=True)) if attn_only else (lambda: ds.run(restore_inline=True))
+    run = (lambda: ds.run(attn_only=True)) if attn_only else (lambda: ds.run(restore_inline=True, append=append))
     with torch.cuda.stream(side):
         run()
         side.synchronize()
@@ -437,6 +443,14 @@ def decode_step_many_layers(torch, step, device, peak, attn_path, layers, reps):
         g.replay()
         ms_step_g = timed_region(torch, None, g.replay, reps) / reps
         del g
+        ds.restore()
+        step_app = lambda: ds.run(append=True)
+        step_app()
+        ms_app = timed_region(torch, None, step_app, reps, prepare=ds.restore) / reps
+        g = capture_step_graph(torch, ds, append=True)
+        g.replay()
+        ms_app_g = timed_region(torch, None, g.replay, reps) / reps
+        del g
         ds.restore()                       # the steps above committed: the attention alone runs on the original lengths
         attn = lambda: ds.run(attn_only=True)
         attn()
@@ -452,6 +466,7 @@ def decode_step_many_layers(torch, step, device, peak, attn_path, layers, reps):
     nbytes = step.attn_bytes()
     per_call, per_call_g = ms_attn * 1e3 / layers, ms_attn_g * 1e3 / layers
     return {"layers": layers, "us_per_step": ms_step * 1e3, "us_per_step_cuda_graph_replay": ms_step_g * 1e3,
+            "us_per_step_with_kv_append": ms_app * 1e3, "us_per_step_with_kv_append_cuda_graph_replay": ms_app_g * 1e3,
             "us_per_attn_call": per_call, "us_per_attn_call_cuda_graph_replay": per_call_g,
             "attn_GBps": nbytes / per_call_g / 1e3, "frac_of_measured_peak": nbytes / per_call_g / 1e3 / peak,
             "frac_of_8TBps_nominal": nbytes / per_call_g / 1e3 / 8000.0,
@@ -610,6 +625,12 @@ def run_ours(args, step, rank, world, dist):
                       "frac_of_measured_peak": nbytes / ms_sv / 1e6 / peak}
         del dlg, fl
 
+    # the same step with the KV append inside (append of the layer's block K/V, then its attention, per layer)
+    n_app = max(2, min(args.steps, 5))
+    ds.restore()
+    ds.run(append=True)
+    ms_append = timed_region(torch, None, lambda: ds.run(append=True), n_app, flush, prepare=ds.restore) / n_app
+
     hs = HostStep(ds)
     for _ in range(2):
         hs.run()
@@ -662,6 +683,7 @@ def run_ours(args, step, rank, world, dist):
                    "sampling_fd_verify_accept_sample": sample_row,
                    "mask_rows_in_last_10_layers_only": layer_split,
                    "us_per_attn_call_alone_event_bracketed": statistics.mean(attn_ms) * 1e3,
+                   "us_per_step_with_kv_append": ms_append * 1e3,
                    "step_of_36_layer_model": many, "per_workload": per_workload},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(step.name) if resolved == "tcgen05" else None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,

@@ -358,7 +358,7 @@ fd_status fd_kv_commit(fd_ctx* ctx, int batch, int32_t* page_table, int32_t* pre
  * layer l-1 comes back while layer l computes; one cudaMemcpyAsync per buffer.
  *
  * fd_host_reserve(ctx, max_total_q_rows, max_total_cand_rows) allocates the device staging
- * (2 x q, 2 x out, logits, small arrays) and the copy streams once; it is the only part that
+ * (2 x q, 2 x out, 2 x the block's K and V, logits, small arrays) and the copy streams once; it is the only part that
  * allocates and must precede fd_step_host.  A second call with sizes within the first is a
  * no-op; larger sizes return FD_ERR_INVALID_ARG.
  *
@@ -384,6 +384,23 @@ fd_status fd_step_host(fd_ctx* ctx, int batch, int total_q_rows, int total_cand_
                        const int32_t* n_blocks_host,
                        int32_t* accepted_len_host, int32_t* bonus_token_host,
                        int32_t* freed_pages_host, int32_t* n_freed_host, void* stream);
+
+/*
+ * The same step with the KV append inside (Sec. 4.1 "Inference": the K/V that the target's own forward pass
+ * computes for the query block go into the cache, where this step's attention and every later step find them).
+ * Per layer the block's K/V go up with its q, fd_kv_append writes them into the layer's pages, and the attention
+ * call follows on the same stream under programmatic dependent launch (its set-up overlaps the append's tail).
+ *
+ *   k_new_host, v_new_host   [n_layers][T, Hkv, d] bf16, rows sequence-major as q; both NULL = fd_step_host
+ *   kv_caches                as above, but written: positions n_b .. n_b + Lq_b - 1 of every sequence
+ */
+fd_status fd_step_host_append(fd_ctx* ctx, int batch, int total_q_rows, int total_cand_rows, int n_layers,
+                              void* const* kv_caches, int num_pages, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, void* out_host, const float* logits_host,
+                              const int32_t* draft_tokens_host, int32_t* page_table_host, int32_t* prefix_lens_host,
+                              const int32_t* q_lens_host, const int32_t* n_mask_host, const int32_t* n_blocks_host,
+                              int32_t* accepted_len_host, int32_t* bonus_token_host, int32_t* freed_pages_host,
+                              int32_t* n_freed_host, void* stream);
 
 /*
  * fd_verify_accept without any allocation.  (The paper has no counterpart; this entry point

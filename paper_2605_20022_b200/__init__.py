@@ -25,7 +25,7 @@ FD_TC_PLANNED, FD_TC_SELF_PLANNED, FD_TC_CLUSTER = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_attn_last_mode", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_verify_accept_sample", "fd_plan_ranges_host"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_step_host_append", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_verify_accept_sample", "fd_plan_ranges_host"]
 
 
 class fd_config(ctypes.Structure):
@@ -73,6 +73,7 @@ def load() -> ctypes.CDLL:
         lib.fd_kv_append.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp]
         lib.fd_draft_select.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
         lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 14
+        lib.fd_step_host_append.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 16
         lib.fd_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         lib.fd_attn_path.argtypes = [vp]
         lib.fd_attn_last_mode.argtypes = [vp]
@@ -234,6 +235,21 @@ def fd_step_host(ctx, batch, total_q_rows, total_cand_rows, kv_caches, num_pages
                                _ptr(accepted_len_host),
                                _ptr(bonus_token_host), _ptr(freed_pages_host), _ptr(n_freed_host), _stream(stream))
     return _check("fd_step_host", code, raise_on_error)
+
+
+def fd_step_host_append(ctx, batch, total_q_rows, total_cand_rows, kv_caches, num_pages, q_host, k_new_host, v_new_host, out_host,
+                        logits_host, draft_tokens_host, page_table_host, prefix_lens_host, q_lens_host, n_mask_host,
+                        accepted_len_host, bonus_token_host, freed_pages_host, n_freed_host, stream=None, raise_on_error=True,
+                        n_blocks_host=None) -> int:
+    """fd_step_host with the KV append inside: `k_new_host` / `v_new_host` are [n_layers, T, Hkv, d] CPU tensors."""
+    n_layers = len(kv_caches)
+    arr = (ctypes.c_void_p * n_layers)(*[_ptr(t) for t in kv_caches])
+    code = load().fd_step_host_append(ctx, batch, total_q_rows, total_cand_rows, n_layers, arr, num_pages, _ptr(q_host),
+                                      _ptr(k_new_host), _ptr(v_new_host), _ptr(out_host), _ptr(logits_host),
+                                      _ptr(draft_tokens_host), _ptr(page_table_host), _ptr(prefix_lens_host),
+                                      _ptr(q_lens_host), _ptr(n_mask_host), _ptr(n_blocks_host), _ptr(accepted_len_host),
+                                      _ptr(bonus_token_host), _ptr(freed_pages_host), _ptr(n_freed_host), _stream(stream))
+    return _check("fd_step_host_append", code, raise_on_error)
 
 
 def fd_selftest_wait_timeout(ctx, limit_ms, stream=None) -> None:

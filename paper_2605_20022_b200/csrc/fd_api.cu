@@ -50,7 +50,7 @@ struct HostStage {
     cudaStream_t h2d, d2h;
     cudaEvent_t start, meta, logits, done, fin, q_ready[2], attn_done[2], out_copied[2];
     unsigned char* pool;
-    void *q[2], *out[2];
+    void *q[2], *out[2], *kn[2], *vn[2];
     float* lg;
     int32_t *drafts, *pt, *pl, *ql, *nm, *nb, *acc, *bon, *freed, *nfreed;
 };
@@ -248,6 +248,8 @@ fd_status fd_host_reserve(fd_ctx* c, int max_total_q_rows, int max_total_cand_ro
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     const size_t o_q0 = take(qb), o_q1 = take(qb), o_o0 = take(qb), o_o1 = take(qb);
+    const size_t kb = (size_t)max_total_q_rows * c->cfg.n_kv_heads * c->cfg.head_dim * 2;
+    const size_t o_k0 = take(kb), o_k1 = take(kb), o_v0 = take(kb), o_v1 = take(kb);
     const size_t o_lg = take((size_t)max_total_cand_rows * c->cfg.vocab * 4);
     const size_t o_dr = take((size_t)max_total_cand_rows * 4);
     const size_t o_pt = take((size_t)B * c->cfg.max_pages_per_seq * 4);
@@ -262,6 +264,7 @@ fd_status fd_host_reserve(fd_ctx* c, int max_total_q_rows, int max_total_cand_ro
     for (cudaEvent_t* e : evs) ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); cudaFree(h->pool); delete h; return FD_ERR_CUDA; }
     h->q[0] = h->pool + o_q0; h->q[1] = h->pool + o_q1; h->out[0] = h->pool + o_o0; h->out[1] = h->pool + o_o1;
+    h->kn[0] = h->pool + o_k0; h->kn[1] = h->pool + o_k1; h->vn[0] = h->pool + o_v0; h->vn[1] = h->pool + o_v1;
     h->lg = reinterpret_cast<float*>(h->pool + o_lg);
     h->drafts = reinterpret_cast<int32_t*>(h->pool + o_dr); h->pt = reinterpret_cast<int32_t*>(h->pool + o_pt);
     h->pl = reinterpret_cast<int32_t*>(h->pool + o_pl); h->ql = reinterpret_cast<int32_t*>(h->pool + o_ql);
@@ -279,7 +282,22 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
                        int32_t* prefix_lens_host, const int32_t* q_lens_host, const int32_t* n_mask_host,
                        const int32_t* n_blocks_host, int32_t* accepted_len_host, int32_t* bonus_token_host, int32_t* freed_pages_host,
                        int32_t* n_freed_host, void* stream) {
+    return fd_step_host_append(c, batch, total_q_rows, total_cand_rows, n_layers, const_cast<void* const*>(kv_caches), num_pages, q_host,
+                               nullptr, nullptr, out_host, logits_host, draft_tokens_host, page_table_host, prefix_lens_host, q_lens_host,
+                               n_mask_host, n_blocks_host, accepted_len_host, bonus_token_host, freed_pages_host, n_freed_host, stream);
+}
+
+fd_status fd_step_host_append(fd_ctx* c, int batch, int total_q_rows, int total_cand_rows, int n_layers,
+                              void* const* kv_caches, int num_pages, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, void* out_host, const float* logits_host,
+                              const int32_t* draft_tokens_host, int32_t* page_table_host, int32_t* prefix_lens_host,
+                              const int32_t* q_lens_host, const int32_t* n_mask_host, const int32_t* n_blocks_host,
+                              int32_t* accepted_len_host, int32_t* bonus_token_host, int32_t* freed_pages_host,
+                              int32_t* n_freed_host, void* stream) {
     if (!c || !c->host) return FD_ERR_INVALID_ARG;
+    if ((k_new_host == nullptr) != (v_new_host == nullptr)) return FD_ERR_INVALID_ARG;
+    const bool append = k_new_host != nullptr;
+    const size_t knb = (size_t)total_q_rows * c->cfg.n_kv_heads * c->cfg.head_dim * 2;
     HostStage* h = c->host;
     if (batch <= 0 || batch > c->cfg.max_batch || n_layers <= 0 || total_q_rows < 0 || total_cand_rows < 0 ||
         total_q_rows > h->max_q_rows || total_cand_rows > h->max_cand_rows)
@@ -313,6 +331,10 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         // q of layer l goes up while layer l-1 computes; the staging pair is reused every other layer
         if (l >= 2) chk(cudaStreamWaitEvent(h->h2d, h->attn_done[b], 0));
         chk(cudaMemcpyAsync(h->q[b], static_cast<const unsigned char*>(q_host) + (size_t)l * qb, qb, H2D, h->h2d));
+        if (append) {  // the block's K/V of this layer ride with its q
+            chk(cudaMemcpyAsync(h->kn[b], static_cast<const unsigned char*>(k_new_host) + (size_t)l * knb, knb, H2D, h->h2d));
+            chk(cudaMemcpyAsync(h->vn[b], static_cast<const unsigned char*>(v_new_host) + (size_t)l * knb, knb, H2D, h->h2d));
+        }
         chk(cudaEventRecord(h->q_ready[b], h->h2d));
         if (l >= 1 && total_cand_rows > 0) {
             // the logits go up in n_layers - 1 slices, one behind each later q block, so that no q block ever
@@ -332,6 +354,8 @@ fd_status fd_step_host(fd_ctx* c, int batch, int total_q_rows, int total_cand_ro
         if (l >= 2) chk(cudaStreamWaitEvent(s, h->out_copied[b], 0));
         if (l == 0 && n_layers > 1)  // one work list for all layers of the step
             st = fd_plan_pin(c, batch, total_q_rows, h->pl, h->ql, h->nm, n_blocks_host ? h->nb : nullptr, s);
+        if (st == FD_OK && append)
+            st = fd_kv_append(c, batch, total_q_rows, h->kn[b], h->vn[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, s);
         if (st == FD_OK)
             st = fd_attn_draft_verify_blocks(c, batch, total_q_rows, h->q[b], kv_caches[l], num_pages, h->pt, h->pl, h->ql, h->nm,
                                              n_blocks_host ? h->nb : nullptr, h->out[b], s);
@@ -573,7 +597,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
     if (!aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(kv_cache, 16)) return FD_ERR_INVALID_ARG;
     fd::AppendParams p;
     p.batch = batch; p.total_rows = total_q_rows; p.num_pages = num_pages; p.Hkv = c->cfg.n_kv_heads; p.d = c->cfg.head_dim;
-    p.max_pages = c->cfg.max_pages_per_seq;
+    p.max_pages = c->cfg.max_pages_per_seq; p.max_q_len = c->cfg.max_q_len;
     p.k_new = static_cast<const __nv_bfloat16*>(k_new); p.v_new = static_cast<const __nv_bfloat16*>(v_new);
     p.kv = static_cast<__nv_bfloat16*>(kv_cache);
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.status = c->status;

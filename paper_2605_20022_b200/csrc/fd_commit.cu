@@ -1,4 +1,6 @@
 // KV commit / rollback: length truncation and page release, one CTA.
+#include <algorithm>
+
 #include "fd_internal.cuh"
 
 namespace fd {
@@ -59,11 +61,17 @@ void launch_commit(const CommitParams& p, cudaStream_t s) {
     commit_kernel<<<1, 256, 0, s>>>(p);
 }
 
-// KV append: K/V of the query block -> its pages ("append, then attend").  One CTA per sequence; 16-byte copies.
-__global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p) {
+// KV append: K/V of the query block -> its pages ("append, then attend").  A CTA per (sequence, group of block rows);
+// 16-byte copies, one page lookup per row.  (One CTA per sequence took 15 us for a 32-row block: 32 dependent rounds.)
+__global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p, int rows_per_cta) {
+    // the attention call that follows on the stream may start its set-up now; it waits for this grid to complete
+    // before it reads the cache
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ int s_red[8];
     __shared__ long long s_row0;
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x, i0 = blockIdx.y * rows_per_cta, tid = threadIdx.x;
+    const int n = p.prefix_lens[b], Lq = p.q_lens[b];
+    if (i0 >= Lq) return;  // uniform (an empty or negative length too)
     // first query row of this sequence = sum of the lengths before it (block-parallel; negative lengths count as 0)
     int part = 0;
     for (int s = tid; s < b; s += blockDim.x) part += max(p.q_lens[s], 0);
@@ -78,32 +86,36 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p) {
     }
     __syncthreads();
     const long long row0 = s_row0;
-    const int n = p.prefix_lens[b], Lq = p.q_lens[b];
-    if (Lq <= 0) return;
     if (n < 0 || row0 + Lq > p.total_rows || (long long)n + Lq > (long long)p.max_pages * 16) {
-        if (tid == 0) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
+        if (tid == 0 && i0 == 0) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         return;
     }
     const int vec_per_head = p.d / 8;                    // 16-byte pieces of one head's row
     const int per_row = p.Hkv * vec_per_head;
-    for (int e = tid; e < Lq * per_row * 2; e += blockDim.x) {
-        const int which = e / (Lq * per_row), rem = e % (Lq * per_row);
-        const int i = rem / per_row, h = (rem % per_row) / vec_per_head, v = rem % vec_per_head;
+    const int i1 = min(Lq, i0 + rows_per_cta);
+    for (int i = i0; i < i1; ++i) {
         const int j = n + i;
         const int page = p.page_table[(long long)b * p.max_pages + (j >> 4)];
         if ((unsigned)page >= (unsigned)p.num_pages) {   // never form an address from a bad id
-            if (h == 0 && v == 0) atomicOr(p.status, FD_DEV_BAD_PAGE);
+            if (tid == 0) atomicOr(p.status, FD_DEV_BAD_PAGE);
             continue;
         }
-        const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + ((row0 + i) * p.Hkv + h) * p.d + v * 8;
-        __nv_bfloat16* dst = p.kv + ((((long long)page * 2 + which) * p.Hkv + h) * 16 + (j & 15)) * p.d + v * 8;
-        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        for (int e = tid; e < 2 * per_row; e += blockDim.x) {
+            const int which = e / per_row, rem = e % per_row;
+            const int h = rem / vec_per_head, v = rem % vec_per_head;
+            const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + ((row0 + i) * p.Hkv + h) * p.d + v * 8;
+            __nv_bfloat16* dst = p.kv + ((((long long)page * 2 + which) * p.Hkv + h) * 16 + (j & 15)) * p.d + v * 8;
+            *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        }
     }
 }
 
 void launch_kv_append(const AppendParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
-    kv_append_kernel<<<p.batch, 256, 0, s>>>(p);
+    // a handful of rows per CTA; long query blocks (up to 4096 rows) get more rows per CTA instead of more CTAs
+    const int rows_per_cta = std::max(4, (p.max_q_len + 63) / 64);
+    const int groups = (p.max_q_len + rows_per_cta - 1) / rows_per_cta;
+    kv_append_kernel<<<dim3(p.batch, groups), 256, 0, s>>>(p, rows_per_cta);
 }
 
 // Branch selection after verification (parallel drafting with one prepared branch per hypothesis):

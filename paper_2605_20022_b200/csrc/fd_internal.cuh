@@ -372,7 +372,7 @@ struct SampleParams {
 int launch_accept_sample(const SampleParams& p, cudaStream_t s);  // returns the number of kernels launched
 
 struct AppendParams {
-    int batch, total_rows, num_pages, Hkv, d, max_pages;
+    int batch, total_rows, num_pages, Hkv, d, max_pages, max_q_len;
     const __nv_bfloat16* k_new;
     const __nv_bfloat16* v_new;
     __nv_bfloat16* kv;

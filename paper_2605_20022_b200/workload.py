@@ -265,3 +265,15 @@ def make_logits(step: Step, device="cpu"):
             drafts[r + j + 1] = target[r + j] if bool(match[r + j]) else other[r + j]
         r += C
     return logits, drafts.to(torch.int32), target.to(torch.int32)
+
+
+def query_block_kv(step: Step, kv: torch.Tensor):
+    """(k_new, v_new) [T, Hkv, d]: the K/V rows of every sequence's query block, read out of a cache that already
+    holds them (positions n_b .. n_b + Lq_b - 1, through the page table) -- what the projections of the step would hand
+    to the KV append.  Pure indexing; `kv` may live on any device."""
+    seq = torch.repeat_interleave(torch.arange(step.batch), step.q_lens.long())
+    start = torch.cumsum(step.q_lens.long(), 0) - step.q_lens.long()
+    pos = step.prefix_lens.long()[seq] + (torch.arange(step.total_q_rows) - start[seq])
+    pages = step.page_table.long()[seq, pos // step.shape.page_size].to(kv.device)
+    slots = (pos % step.shape.page_size).to(kv.device)
+    return kv[pages, 0, :, slots, :].contiguous(), kv[pages, 1, :, slots, :].contiguous()

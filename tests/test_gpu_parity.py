@@ -333,6 +333,50 @@ def test_host_buffer_step_matches_oracle():
             np.testing.assert_array_equal(h_freed.numpy()[:len(efreed)], efreed)
 
 
+def test_host_buffer_step_with_the_kv_append_inside():
+    """fd_step_host_append: the caches start WITHOUT the query block's K/V (NaN there); the step writes them per layer
+    and attends.  Outputs, accept and commit as the oracle on the complete caches; the caches end up bit-exact."""
+    shape = wl.Shape(32, 8, 128, 5000, n_layers=3)
+    step = wl.make_step("host_append", shape, [700, 130, 2049, 0], [32, 9, 20, 16], [16, 0, 8, 0], seed=19, p_match=0.7,
+                        extra_table_cols=1)
+    L, B, T, R = 3, step.batch, step.total_q_rows, step.total_cand_rows
+    qs = [wl.make_q(step, l) for l in range(L)]
+    kvs = [wl.make_kv(step, l) for l in range(L)]
+    blocks = [wl.query_block_kv(step, kv) for kv in kvs]
+    logits, drafts, _ = wl.make_logits(step)
+    holes = []
+    for kv in kvs:                                             # the same caches with the block's slots blanked
+        h = kv.clone()
+        for b in range(B):
+            for j in range(int(step.prefix_lens[b]), int(step.kv_lens[b])):
+                h[int(step.page_table[b, j // 16]), :, :, j % 16, :] = float("nan")
+        holes.append(h.cuda())
+    pin = lambda t: t.contiguous().pin_memory()
+    q_host, out_host = pin(torch.stack(qs)), pin(torch.zeros((L, T, 32, 128), dtype=torch.bfloat16))
+    k_host, v_host = pin(torch.stack([b_[0] for b_ in blocks])), pin(torch.stack([b_[1] for b_ in blocks]))
+    h_logits, h_drafts = pin(logits), pin(drafts)
+    h_pt, h_pl, h_ql, h_nm = pin(step.page_table.clone()), pin(step.prefix_lens.clone()), pin(step.q_lens), pin(step.n_mask)
+    h_acc, h_bon = pin(torch.zeros(B, dtype=torch.int32)), pin(torch.zeros(B, dtype=torch.int32))
+    h_freed, h_nf = pin(torch.full((B * 3,), -7, dtype=torch.int32)), pin(torch.zeros(1, dtype=torch.int32))
+    with Ctx(step) as ctx:
+        fd.fd_host_reserve(ctx.h, T, R)
+        assert fd.fd_step_host_append(ctx.h, B, T, R, holes, step.num_pages, q_host, k_host, None, out_host, h_logits, h_drafts, h_pt,
+                                      h_pl, h_ql, h_nm, h_acc, h_bon, h_freed, h_nf, raise_on_error=False) == fd.FD_ERR_INVALID_ARG
+        fd.fd_step_host_append(ctx.h, B, T, R, holes, step.num_pages, q_host, k_host, v_host, out_host, h_logits, h_drafts, h_pt, h_pl,
+                               h_ql, h_nm, h_acc, h_bon, h_freed, h_nf)
+        torch.cuda.current_stream().synchronize()
+        assert fd.fd_last_device_status(ctx.h) == 0
+    for l in range(L):
+        assert torch.equal(holes[l].cpu().view(torch.int16), kvs[l].view(torch.int16)), f"cache of layer {l}"
+        ref = oracle.attn(qs[l], kvs[l], step.page_table, step.prefix_lens, step.q_lens, step.n_mask)
+        assert_close(out_host[l].float().numpy(), ref, f"layer {l}")
+    e_acc, e_bon, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    np.testing.assert_array_equal(h_acc.numpy(), e_acc); np.testing.assert_array_equal(h_bon.numpy(), e_bon)
+    ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, e_acc)
+    np.testing.assert_array_equal(h_pt.numpy(), ept); np.testing.assert_array_equal(h_pl.numpy(), epl)
+    np.testing.assert_array_equal(h_freed.numpy()[:int(h_nf)], efreed)
+
+
 def test_bounded_wait_times_out_cleanly_and_context_survives():
     """A device-side wait that nothing will ever satisfy gives up after its limit, raises FD_DEV_TIMEOUT and
     the kernel returns; the same context then computes a correct result."""

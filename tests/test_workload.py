@@ -71,3 +71,17 @@ def test_draft_match_rate():
     d, t = drafts.view(4000, 5), target.view(4000, 5)
     rate = (d[:, 1:] == t[:, :-1]).float().mean().item()
     assert abs(rate - 0.75) < 0.02
+
+
+def test_query_block_kv_reads_the_block_through_the_page_table():
+    step = wl.make_step("blk", wl.Shape(8, 2, 64, 100), [0, 15, 33], [5, 17, 1], [2, 16, 0], seed=3)
+    kv = wl.make_kv(step)
+    k_new, v_new = wl.query_block_kv(step, kv)
+    assert k_new.shape == (step.total_q_rows, 2, 64) and v_new.shape == k_new.shape
+    row = 0
+    for b in range(step.batch):
+        for i in range(int(step.q_lens[b])):
+            j = int(step.prefix_lens[b]) + i
+            page = int(step.page_table[b, j // 16])
+            assert torch.equal(k_new[row], kv[page, 0, :, j % 16, :]) and torch.equal(v_new[row], kv[page, 1, :, j % 16, :])
+            row += 1
