@@ -61,29 +61,23 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units
 #ifndef FD_QK_MODE
 #define FD_QK_MODE 1
 #endif
-
-constexpr int cluster_recv_bytes(int d) { return d == 128 ? 2 * kTileTokens * 128 * 2 : 2 * kTileTokens * 64 * 2; }  // one K and one V stage
+// 1: the first fill of the K and V rings is staggered (see load_role)
+#ifndef FD_STAGGER
+#define FD_STAGGER 1
+#endif
 
 template <int D, int MODE>
 struct Cfg {
-    static constexpr int kFullStages = (D == 128) ? 3 : 6;
-    // buffers in the K ring, and again in the V ring.  With one cluster per segment a CTA has few tiles and gives a
-    // third of the ring space to the partial results its peers send it (see the epilogue of softmax_role).
-    static constexpr int kStages = MODE == kTcCluster ? ((D == 128) ? 2 : 5) : kFullStages;
+    static constexpr int kStages = (D == 128) ? 3 : 6;   // buffers in the K ring, and again in the V ring
     static constexpr int kQBytes = kMaxRows * D * 2;
     static constexpr int kKBytes = kTileTokens * D * 2;  // one K (or V) tile
-    // kTcCluster: the receive area, 2 KB of (m, l) pairs [cluster size][rows per CTA], then rows of O, from the peers;
-    // it is what the ring gave up: cluster_recv_bytes(D)
-    static constexpr int kRecvOffset = kQBytes + 2 * kStages * kKBytes;
-    static_assert(MODE != kTcCluster || 2 * (kFullStages - kStages) * kKBytes == cluster_recv_bytes(D), "receive area");
-    static constexpr int kBarOffset = kQBytes + 2 * kFullStages * kKBytes;
+    static constexpr int kBarOffset = kQBytes + 2 * kStages * kKBytes;
     static constexpr int kCsOffset = kBarOffset + 320;           // window of the CTA range starts
     static constexpr int kDescOffset = kBarOffset + 448;         // ring of piece descriptors
     static constexpr int kScanOffset = kBarOffset + 720;         // SelfScans: the scans of a call that plans for itself
     static constexpr int kExOffset = kBarOffset + 1024;          // [2][128] floats: stream exchange in the epilogue
     static constexpr int kRbOffset = kBarOffset + 2048;          // row blocks of a call that plans for itself
     static constexpr int kSmemBytes = kBarOffset + 3072;         // the dynamic shared memory is declared 1024-byte aligned
-    // what a CTA receives: (m, l) of every peer, and O rows of every peer but itself, for its 128 / cluster-size rows
     static constexpr int kKSteps = D / 16;
     static constexpr int kHalves = D / 64;
     // A K or V tile in shared memory: [8-token group][half of d][8 rows][128 B] -- what one TMA box per page
@@ -232,7 +226,7 @@ struct Walk {
 // K (which = 0) or V (which = 1) load warp.
 template <int D, int MODE>
 __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnParams& p, int n_rb, unsigned char* ring, uint64_t* full,
-                                          uint64_t* empty, int which, const Range rg, volatile int* bad, volatile int* abort) {
+                                          uint64_t* empty, int which, const Range rg, uint64_t* k0_full, volatile int* bad, volatile int* abort) {
     using C = Cfg<D, MODE>;
     const int lane = threadIdx.x & 31, cta = blockIdx.x;
     constexpr int kOps = 8;  // pages of a tile: one box each
@@ -268,6 +262,18 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             if (j > 0 && (j & 3) == 0) { ids_cur = ids_next; ids_next = load_ids((j >> 2) + 1); }
             const int phys = __shfl_sync(0xffffffffu, ids_cur, (j & 3) * 8 + pg);
             if (!wait_all(&empty[st], (use & 1) ^ 1, abort)) { ok = false; break; }
+#if FD_STAGGER
+            // The first fill of the rings is not issued all at once: every CTA of the grid starts at the same moment,
+            // and 224 KB per SM in one burst makes the first K tile -- all the MMA warp needs to begin -- land with
+            // the last of it.  K tiles 0 and 1 go out at once; the V tiles and the third K tile follow when K tile 0
+            // has landed (V tile 0 is not needed before the first softmax is through).  A delay, not a dependency:
+            // it ends by itself after a few microseconds.
+            if (g == (which ? 0 : 2) && k0_full != nullptr) {
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(k0_full, 0) && global_ns() - t0 < 4000ull) {}
+                __syncwarp();
+            }
+#endif
             const int pos0 = (pc.tile0 + j) * kTileTokens;
             const int npg = min(8, (pc.kv_len - pos0 + 15) >> 4);
             if (lane == 0) mbar_arrive_expect_tx(&full[st], npg * (16 * D * 2));
@@ -423,12 +429,14 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
 
 // ---------------------------------------------------------------------------------------------
 // One cluster per segment (kTcCluster).  The CTAs of a cluster split the segment's tiles evenly.  Query row r of the
-// segment is owned by CTA r / share of the cluster (share = 128 / cluster size): every CTA sends the unnormalised
-// partial result of the rows it does not own -- O in fp32 and (m, l) -- straight into the owner's shared memory
-// (st.shared::cluster: stores need no round trip), keeps the rows it owns in registers, and after ONE cluster
-// barrier each owner combines what it received with its own part, in rank order (fixed, so the result does not
-// depend on timing), and writes the bf16 rows.  After the barrier nobody touches a peer's memory again, so a CTA
-// may leave as soon as its own rows are written.  No global scratch, no counters, no waiting on flags.
+// segment is owned by CTA r / share of the cluster (share = ceil(128 / cluster size)).  Every CTA writes the
+// unnormalised partial result of the rows it does not own -- O in fp32 and (m, l) -- to its two scratch slots in
+// global memory, one block per owner, keeps the rows it owns in registers, and after ONE cluster barrier each owner
+// brings the c - 1 blocks meant for it into its shared memory with bulk copies, combines them with its own part in
+// rank order (fixed, so the result does not depend on timing) and writes the bf16 rows.  The cluster is there for the
+// barrier and the co-scheduling; the bytes go through L2, because that is the faster carrier: an SM stores 64 KB to
+// global memory in 0.9 us and a bulk copy lands it in 0.3 us, while the SM-to-SM path moved the same rows at about
+// 20 GB/s per SM (3.5-5 us), with st.shared::cluster pushes as with ld.shared::cluster pulls.  No counters, no polling.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -439,93 +447,98 @@ __device__ __forceinline__ void cluster_sync_all() {  // every thread of every C
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ uint32_t peer_addr(uint32_t saddr, uint32_t rank) {  // the same offset in CTA `rank` of the cluster
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void st_peer_v4(uint32_t addr, float4 v) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-__device__ __forceinline__ void st_peer_v2(uint32_t addr, float2 v) {
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v.x), "f"(v.y) : "memory");
-}
-__device__ __forceinline__ float2 lds_v2(uint32_t addr) {
-    float2 v;
-    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ float4 lds_v4(uint32_t addr) {
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
-    return v;
-}
 constexpr int kMaxCluster = 16;
 // Rows a CTA of a cluster of c owns (the last CTA may own fewer, or none).
 __host__ __device__ constexpr int cluster_share(int c) { return (kMaxRows + c - 1) / c; }
-// Does the receive area (recv_bytes) hold what a CTA of a cluster of c gets: (m, l) from all, O rows from all but itself?
-__host__ __device__ constexpr bool cluster_fits(int c, int d, int recv_bytes) {
-    return c * cluster_share(c) <= 2 * kMaxRows && 2 * kMaxRows * 8 + (c - 1) * cluster_share(c) * d * 4 <= recv_bytes;
+// What one CTA hands one owner: the O rows as [d / 4 words][share rows][16 bytes], then (m, l) per row.
+__host__ __device__ constexpr uint32_t cluster_block_bytes(int c, int d) { return (uint32_t)((cluster_share(c) * (d * 4 + 8) + 15) / 16 * 16); }
+// Do the two scratch slots of a CTA, and the K ring where the blocks land, hold the c blocks of a cluster of c?
+__host__ __device__ constexpr bool cluster_fits(int c, int d) {
+    return (uint32_t)c * cluster_block_bytes(c, d) <= 2u * kMaxRows * d * 4 &&
+           (uint32_t)c * cluster_block_bytes(c, d) <= (uint32_t)(d == 128 ? 3 : 6) * kTileTokens * d * 2;
 }
 
-// The receive area of a CTA: (m, l) of source CTA c for owned row rl at ml[c * share + rl]; the O row of source c
-// (c != own rank; slot = c, less one past the own rank) as D / 4 16-byte words, word w at position w ^ (rl & 31):
-// the thread-per-row stores of the senders and of the owner's reads then both spread over all banks.
+// Addresses of the exchange.  In global memory: CTA `cta` of the grid owns scratch slots 2 cta and 2 cta + 1, one block
+// per owner rank.  In shared memory: after the cluster barrier the K ring (idle by then) takes the c blocks meant for
+// this CTA, block c from rank c; its own block it has written there itself.
 template <int D>
-struct Recv {
-    uint32_t base;  // shared-memory address (the same offset in every CTA of the cluster)
+struct Exchange {
+    unsigned char* g_base;  // scratch of this CTA
+    unsigned char* land;    // the K ring (generic address)
+    uint32_t land_s;        // ... and its shared-memory address
     int share;
-    __device__ __forceinline__ uint32_t ml(int c, int rl) const { return base + (uint32_t)(c * share + rl) * 8; }
-    __device__ __forceinline__ uint32_t o(int slot, int rl, int word) const {
-        return base + 2 * kMaxRows * 8 + (uint32_t)((slot * share + rl) * (D / 4) + (word ^ (rl & (D / 4 - 1)))) * 16;
-    }
+    uint32_t block;
+    __device__ __forceinline__ unsigned char* g_block(int dest) const { return g_base + (size_t)dest * block; }
+    __device__ __forceinline__ static uint32_t o_off(int share_, int rl, int word) { return (uint32_t)(word * share_ + rl) * 16; }
+    __device__ __forceinline__ uint32_t ml_off(int rl) const { return (uint32_t)share * D * 4 + (uint32_t)rl * 8; }
 };
 
-// Owner side, after the cluster barrier: thread (row r, half s of the columns) combines the C parts of its row.
-// `own`: this CTA's own part of the row, the thread's D / 2 columns (nullptr: it had no tiles).
+// Owner side, after the cluster barrier: warp 0 brings the peers' blocks in, a lane per peer.
 template <int D>
-__device__ __forceinline__ void cluster_reduce_row(const AttnParams& p, const Recv<D> rv, int rank, int r, int s, const float* own, int b,
-                                                   int kvh, int row0) {
-    const int C = p.cluster, rl = r % rv.share;
-    float m = -INFINITY;
-    bool flagged = false;  // some CTA of the cluster met a page id outside the pool (it sent l < 0)
-    for (int c = 0; c < C; ++c) {
-        const float2 ml = lds_v2(rv.ml(c, rl));
-        m = fmaxf(m, ml.x);
-        flagged = flagged || ml.y < 0.f;
+__device__ __forceinline__ void cluster_fetch(const AttnParams& p, const Exchange<D>& ex, Bars* bars, int rank) {
+    const int C = p.cluster, c = threadIdx.x & 31;
+    if (c == 0) mbar_arrive_expect_tx(&bars->merge_bar, (uint32_t)(C - 1) * ex.block);
+    __syncwarp();
+    if (c < C && c != rank) {
+        fence_proxy_async_all();  // the peers' plain stores, acquired at the barrier, before the bulk copy that reads them
+        const long long cta_stride = (long long)2 * kMaxRows * D * 4;  // two scratch slots per CTA
+        bulk_load(ex.land + (size_t)c * ex.block, ex.g_base + (c - rank) * cta_stride + (long long)rank * ex.block, ex.block, &bars->merge_bar);
     }
-    float acc[D / 2];
+}
+
+// Owner side, once the blocks have landed: the eight warps of the softmax groups share the rows this CTA owns, a row
+// per D / 4 lanes, a lane per 16-byte word (its 8-byte bf16 stores form one contiguous run per row).  Lane c of a row's
+// group holds part c's (m, l) and weight, handed round by shuffles; the c parts are combined in rank order.
+template <int D>
+__device__ __forceinline__ void cluster_reduce(const AttnParams& p, const Exchange<D>& ex, int rank, int rows, int kvh, int row0) {
+    constexpr int kLpr = D / 4;              // lanes per row (>= the largest cluster)
+    constexpr int kRowsPerWarp = 32 / kLpr;
+    static_assert(kLpr >= kMaxCluster, "one lane per part");
+    const int C = p.cluster, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int word = lane % kLpr;
+    const int r_lo = rank * ex.share, n_own = min(ex.share, rows - r_lo);  // rows [r_lo, r_lo + n_own) are this CTA's
+    for (int rl0 = 0; rl0 < n_own; rl0 += 8 * kRowsPerWarp) {              // uniform over the warp: it shuffles
+        const int rl = rl0 + warp * kRowsPerWarp + lane / kLpr;
+        const bool act = rl < n_own;
+        const int rl_c = act ? rl : 0;
+        float2 q = make_float2(-INFINITY, 0.f);
+        if (act && word < C) q = *reinterpret_cast<const float2*>(ex.land + (size_t)word * ex.block + ex.ml_off(rl_c));
+        float m = q.x;
+        int flagged = q.y < 0.f;  // some CTA of the cluster met a page id outside the pool (it sent l < 0)
 #pragma unroll
-    for (int k = 0; k < D / 2; ++k) acc[k] = 0.f;
-    float l = 0.f;
-    for (int c = 0; c < C; ++c) {
-        const float2 ml = lds_v2(rv.ml(c, rl));
-        if (ml.x == -INFINITY) continue;  // that CTA saw no visible key for the row: it sent no O
-        const float w = exp2f(ml.x - m);
-        l += w * ml.y;
-        if (c == rank) {
-            if (own) {
+        for (int o = kLpr / 2; o > 0; o >>= 1) {
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o, kLpr));
+            flagged |= __shfl_xor_sync(0xffffffffu, flagged, o, kLpr);
+        }
+        const float w = q.x == -INFINITY ? 0.f : exp2f(q.x - m);  // a part that saw no visible key for the row counts nothing
+        float l = w * q.y;
 #pragma unroll
-                for (int k = 0; k < D / 2; ++k) acc[k] += w * own[k];
-            }
-        } else {
-            const int slot = c < rank ? c : c - 1;
+        for (int o = kLpr / 2; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o, kLpr);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const unsigned char* o0 = ex.land + Exchange<D>::o_off(ex.share, rl_c, word);
+        for (int c0 = 0; c0 < C; c0 += 4) {
+            float4 v[4];
 #pragma unroll
-            for (int k = 0; k < D / 8; ++k) {
-                const float4 v = lds_v4(rv.o(slot, rl, s * (D / 8) + k));
-                acc[4 * k] += w * v.x; acc[4 * k + 1] += w * v.y; acc[4 * k + 2] += w * v.z; acc[4 * k + 3] += w * v.w;
+            for (int k = 0; k < 4; ++k) v[k] = *reinterpret_cast<const float4*>(o0 + (size_t)min(c0 + k, C - 1) * ex.block);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float wc = __shfl_sync(0xffffffffu, w, min(c0 + k, C - 1), kLpr);
+                if (c0 + k < C && wc != 0.f) {  // (by selection: the O rows of a part without weight may hold anything)
+                    acc.x += wc * v[k].x; acc.y += wc * v[k].y; acc.z += wc * v[k].z; acc.w += wc * v[k].w;
+                }
             }
         }
+        if (!act) continue;
+        float inv = l > 0.f ? 1.f / l : 0.f;
+        if (flagged) {  // by assignment: what came from a stand-in page may be inf or NaN
+            inv = 0.f;
+            acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const int r = r_lo + rl;
+        __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + word * 4;
+        __align__(8) __nv_bfloat162 v2[2] = {__floats2bfloat162_rn(acc.x * inv, acc.y * inv), __floats2bfloat162_rn(acc.z * inv, acc.w * inv)};
+        *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(v2);
     }
-    float inv = l > 0.f ? 1.f / l : 0.f;
-    if (flagged) {  // by assignment: what came from a stand-in page may be inf or NaN
-        inv = 0.f;
-#pragma unroll
-        for (int k = 0; k < D / 2; ++k) acc[k] = 0.f;
-    }
-    __nv_bfloat16* dst = p.out + ((long long)(row0 + r / p.G) * p.Hq + kvh * p.G + r % p.G) * D + s * (D / 2);
-#pragma unroll
-    for (int ch = 0; ch < D / 64; ++ch) store_cols_bf16<32>(dst + ch * 32, acc + ch * 32, inv);
 }
 
 // Merge of a split segment from shared memory (the merger at the last piece of its range, when the Q tile and the
@@ -605,7 +618,7 @@ __device__ __forceinline__ void merge_staged(const AttnParams& p, Bars* bars, co
 // The two softmax groups (256 threads).
 template <int D, int MODE>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, int* s_cs, const CtaStarts cs, const Piece* ring,
-                                             uint32_t tmem, const Range rg, uint32_t recv_addr, int cl_rank, unsigned char* stage, volatile int* abort) {
+                                             uint32_t tmem, const Range rg, const Exchange<D> exch, int cl_rank, unsigned char* stage, volatile int* abort) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     const int s_c = rg.s_c, e_c = rg.e_c;
     const int s = warp >> 2;                  // stream
@@ -791,14 +804,16 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 mbar_arrive(&bars->o_free);           // O has been read: the next piece may overwrite it
             }
             if (MODE == kTcCluster) {
-                // one cluster per segment: a row another CTA owns goes straight into that CTA's receive area
-                const int share = cluster_share(p.cluster), dest = r / share;
-                if (do_read && r < pc.rows && dest != cl_rank) {
-                    const Recv<D> rv = {recv_addr, share};
-                    const int slot = cl_rank < dest ? cl_rank : cl_rank - 1;
+                // one cluster per segment: a row another CTA owns goes to this CTA's scratch block for that owner, a row
+                // this CTA owns to its own block in the K ring, idle since the last MMA (consecutive rows of a block
+                // are consecutive 16-byte words: the warp's stores coalesce, and spread over the banks)
+                const int dest = r / exch.share;
+                if (do_read && r < pc.rows) {
+                    unsigned char* blk = dest != cl_rank ? exch.g_block(dest) : exch.land + (size_t)cl_rank * exch.block;
 #pragma unroll
                     for (int k = 0; k < 32; k += 4)
-                        st_peer_v4(peer_addr(rv.o(slot, r % share, (col + k) >> 2), dest), make_float4(o[ch][k], o[ch][k + 1], o[ch][k + 2], o[ch][k + 3]));
+                        *reinterpret_cast<float4*>(blk + Exchange<D>::o_off(exch.share, r % exch.share, (col + k) >> 2)) =
+                            make_float4(o[ch][k], o[ch][k + 1], o[ch][k + 2], o[ch][k + 3]);
                 }
             } else if (do_read && r < pc.rows) {
                 if (pc.complete) {
@@ -816,17 +831,20 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             }
         }
         if (MODE == kTcCluster) {
-            const int share = cluster_share(p.cluster), dest = r / share;
-            const Recv<D> rv = {recv_addr, share};
-            // (m, l) of the row to its owner (which may be this CTA); a row this CTA could not compute (it is giving up)
-            // counts as "saw no key"; a CTA whose load warps met a page id outside the pool says so with a negative l
-            if (r < pc.rows && s == 0)
-                st_peer_v2(peer_addr(rv.ml(cl_rank, r % share), dest),
-                           !do_read ? make_float2(-INFINITY, 0.f) : make_float2(mm, bars->bad ? -1.f : L));
+            const int dest = r / exch.share, rl = r % exch.share;
+            // (m, l) of the row for its owner (which may be this CTA: then into its own shared memory); a row this CTA
+            // could not compute (it is giving up) counts as "saw no key"; a CTA whose load warps met a page id outside
+            // the pool says so with a negative l
+            if (r < pc.rows && s == 0) {
+                const float2 ml = !do_read ? make_float2(-INFINITY, 0.f) : make_float2(mm, bars->bad ? -1.f : L);
+                unsigned char* blk = dest != cl_rank ? exch.g_block(dest) : exch.land + (size_t)cl_rank * exch.block;
+                *reinterpret_cast<float2*>(blk + exch.ml_off(rl)) = ml;
+            }
             cluster_sync_all();  // all 256 threads, whatever happened before; the other warps of the CTA wait in the kernel body
             cl_synced = true;
-            if (r < pc.rows && dest == cl_rank && !leave)
-                cluster_reduce_row<D>(p, rv, cl_rank, r, s, do_read ? &o[0][0] : nullptr, pc.b, pc.kvh, pc.row0);
+            // (the cluster barrier is a barrier of this CTA's threads as well: its own block in the K ring is complete)
+            if (warp == 0) cluster_fetch<D>(p, exch, bars, cl_rank);
+            if (wait_all(&bars->merge_bar, 0, abort) && !leave) cluster_reduce<D>(p, exch, cl_rank, pc.rows, pc.kvh, pc.row0);
         } else if (do_read && r < pc.rows && !pc.complete && s == 0) {
             // (the merger too: both column halves of its row need them, and only this thread has them)
             if (stage_ok) {
@@ -1092,25 +1110,36 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
         return;
     }
-    const uint32_t recv_addr = smem_u32(smem) + (uint32_t)C::kRecvOffset;
+    Exchange<D> exch = {};
+    if (MODE == kTcCluster) {
+        exch.g_base = reinterpret_cast<unsigned char*>(p.part.o) + (size_t)cta * 2 * kMaxRows * D * 4;
+        exch.land = sk;
+        exch.land_s = smem_u32(sk);
+        exch.share = cluster_share(p.cluster);
+        exch.block = cluster_block_bytes(p.cluster, D);
+    }
     if (MODE == kTcCluster && cl_idle) {
         // fewer tiles than CTAs in the cluster: this one tells every owner "saw no key" and combines the rows it owns
-        const Recv<D> rv = {recv_addr, cluster_share(p.cluster)};
-        if (tid < cl_rows) st_peer_v2(peer_addr(rv.ml(cl_rank, tid % rv.share), tid / rv.share), make_float2(-INFINITY, 0.f));
-        cluster_sync_all();
-        const int r = tid & (kMaxRows - 1);
-        if (tid < 2 * kMaxRows && r < cl_rows && r / rv.share == cl_rank)
-            cluster_reduce_row<D>(p, rv, cl_rank, r, tid >> 7, nullptr, cl_b, cl_kvh, cl_row0);
+        if (tid < cl_rows) {
+            const int dest = tid / exch.share, rl = tid % exch.share;
+            unsigned char* blk = dest != cl_rank ? exch.g_block(dest) : exch.land + (size_t)cl_rank * exch.block;
+            *reinterpret_cast<float2*>(blk + exch.ml_off(rl)) = make_float2(-INFINITY, 0.f);
+        }
+        cluster_sync_all();  // (a CTA-wide barrier as well: the own block is complete)
+        if (warp == 0) cluster_fetch<D>(p, exch, bars, cl_rank);
+        if (tid < 2 * kMaxRows) {  // whole warps: the wait is warp-uniform
+            if (wait_all(&bars->merge_bar, 0, abort)) cluster_reduce<D>(p, exch, cl_rank, cl_rows, cl_kvh, cl_row0);
+        }
     } else if (warp < 8) {
         // Warp-specialised register budgets: the softmax groups keep a whole 128-column row of S in registers.
         // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168, what the launch allocated: the increase is served exactly by what
         // the decrease released (a request for more than that does not return).
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, recv_addr, cl_rank, sq, abort);
+        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, exch, cl_rank, sq, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, &bars->bad, abort);
-        else if (warp == kVWarp) load_role<D, MODE>(tmap, p, n_rb, sv, bars->v_full, bars->v_empty, 1, rg, &bars->bad, abort);
+        if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, &bars->k_full[0], &bars->bad, abort);
+        else if (warp == kVWarp) load_role<D, MODE>(tmap, p, n_rb, sv, bars->v_full, bars->v_empty, 1, rg, &bars->k_full[0], &bars->bad, abort);
         else if (warp == kMmaWarp) mma_role<D, MODE>(p, sq, sk, sv, bars, ring, tmem, rg, abort);
         else q_role<D, MODE>(qmap, p, n_rb, sq, bars, ring, rg, abort);
         if (MODE == kTcCluster) cluster_sync_all();  // the cluster barrier of the merge counts every thread
@@ -1242,7 +1271,7 @@ cudaError_t attn_tc_prepare(void** state, const AttnParams& p) {
         cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
         for (int c = 0; c <= kMaxCluster; ++c) st->max_clusters[c] = 0;
         for (int c = 2; c <= kMaxCluster; ++c) {
-            const bool fits = cluster_fits(c, p.d, cluster_recv_bytes(p.d));
+            const bool fits = cluster_fits(c, p.d);
             st->max_clusters[c] = !fits ? 0 : p.d == 64 ? query_clusters<64>(c, n_sms) : query_clusters<128>(c, n_sms);
         }
         *state = st;
