@@ -27,10 +27,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) of ONE attention-kernel launch on the long-context workload, from the
-# ncu capture summarised in profiles/attn_tc_and_accept_kernels_long_context_1layer.md
-# (dram__bytes_read.sum 2 158 917 000 + dram__bytes_write.sum 7 709 696; one layer = one full-size launch).
-NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_162_654_160}
+# DRAM bytes (read + write) of ONE attention-kernel launch on the long-context workload, from the ncu capture
+# summarised in profiles/attn_tc_and_accept_kernels_long_context_1layer.md
+# (dram__bytes_read.sum 2 154 169 000 + dram__bytes_write.sum 7 170 560; one layer = one full-size launch).
+NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_161_339_560}
 
 METRIC = "draft-verify attn+accept us/step"
 UNIT = "us/step"

@@ -1019,7 +1019,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     // ---- set-up that needs nothing from earlier kernels: under programmatic dependent launch it overlaps the
     //      tail of the previous launch on the stream (the plan kernel, or the previous layer's call);
     //      griddepcontrol.wait below is where that launch's results are needed
-    if (tid == 0) {
+    if (warp == 1 && lane == 0) {
         for (int i = 0; i < C::kStages; ++i) {
             mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
             mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
@@ -1043,6 +1043,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     }
     if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, 512);
     if (warp == kKWarp && lane == 0) { prefetch_tmap(&tmap); prefetch_tmap(&qmap); }
+    // a call that plans for itself: warp 0 does so meanwhile (it needs the earlier kernels' results -- the lengths --
+    // and waits for them on its own; its global loads then overlap the set-up of the other warps)
+    if (MODE != kTcPlanned && warp == 0) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        self_plan<MODE>(p_in, scans, rbs, s_cs, &bars->first);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1068,8 +1074,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         if (total) { rg.s_c = p.plan.cta_start[cta]; rg.e_c = p.plan.cta_start[cta + 1]; rg.first = p.plan.cta_first[cta]; }
         cs.g = p.plan.cta_start;
     } else {
-        if (warp == 0) self_plan<MODE>(p, scans, rbs, s_cs, &bars->first);
-        __syncthreads();
         p.plan.rb = rbs; p.plan.cu_q = scans->cu_q; p.plan.cu_tiles = scans->cu_tiles; p.plan.cu_ne = scans->cu_ne;
         n_rb = p.batch;
         fatal = scans->fatal;
