@@ -159,8 +159,9 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * until fd_plan_unpin, every fd_attn_draft_verify[_blocks] call with the same batch, total_q_rows and the
  * same four length pointers reuses it instead of recomputing it (a call with anything else that needs the plan
  * kernel recomputes and drops the pin; calls that plan for themselves, FD_TC_SELF_PLANNED and FD_TC_CLUSTER,
- * leave it alone).  The caller must not change the contents of the length arrays while the pin holds, and
- * must unpin after a FD_DEV_TIMEOUT status (fd_last_device_status does so
+ * leave it alone).  The caller must not change the contents of the length arrays or of the page table while the
+ * pin holds (from the second call it serves on, the kernel looks up its work and its first pages while the launch
+ * before it on the stream is still running), and must unpin after a FD_DEV_TIMEOUT status (fd_last_device_status does so
  * itself when it reports that bit).  fd_kv_commit rewrites prefix_lens and therefore drops the pin
  * itself: the first attention call of the next step plans afresh (or is preceded by a new fd_plan_pin).
  * fd_kv_append leaves the lengths alone and keeps the pin.

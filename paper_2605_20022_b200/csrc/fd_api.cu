@@ -41,6 +41,7 @@ struct fd_ctx {
     bool pinned;
     int pin_batch, pin_rows;
     const int32_t *pin_pl, *pin_ql, *pin_nm, *pin_nb;
+    bool pin_chain;    // the context's last launch was an attention or append call under the pinned plan (see AttnParams::early)
     struct HostStage* host;  // staging for fd_step_host, nullptr until fd_host_reserve
 };
 
@@ -130,6 +131,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->tc_state = nullptr;
     c->host = nullptr;
     c->pinned = false;
+    c->pin_chain = false;
     if (cudaGetDevice(&c->device) != cudaSuccess ||
         cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
         delete c;
@@ -463,6 +465,10 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
         fd::launch_plan(p, s);
         c->launches += 1;
     }
+    // under a pinned plan, behind another call it served: the plan, the lengths and the page table are not what the
+    // launch before this one writes, and may be read while it still runs
+    p.early = (reuse && c->pinned && c->pin_chain) ? 1 : 0;
+    c->pin_chain = reuse && c->pinned;
     if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
     } else if (tc) {
         fd::launch_attn_tc(c->tc_state, p, mode, s);  // merges split segments in its own epilogue
@@ -485,6 +491,7 @@ fd_status fd_plan_pin(fd_ctx* c, int batch, int total_q_rows, const int32_t* pre
     fd::launch_plan(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
     c->pinned = true;
+    c->pin_chain = false;  // the first call it serves comes right behind the plan kernel and waits for it
     c->pin_batch = batch; c->pin_rows = total_q_rows;
     c->pin_pl = prefix_lens; c->pin_ql = q_lens; c->pin_nm = n_mask; c->pin_nb = n_blocks;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
@@ -523,12 +530,14 @@ fd_status fd_plan_ranges_host(int batch, int n_kv_heads, const int32_t* prefix_l
 fd_status fd_plan_unpin(fd_ctx* c) {
     if (!c) return FD_ERR_INVALID_ARG;
     c->pinned = false;
+    c->pin_chain = false;
     return FD_OK;
 }
 
 fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const float* logits,
                            const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask,
                            int32_t* accepted_len, int32_t* bonus_token, void* stream) {
+    if (c) c->pin_chain = false;  // (not an attention or append call)
     if (!c || batch < 0 || total_cand_rows < 0) return FD_ERR_INVALID_ARG;
     if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
     if (batch == 0) return total_cand_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
@@ -551,6 +560,7 @@ fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, con
                                   const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask, float temperature,
                                   const float* u_accept, const float* u_bonus, int32_t* accepted_len, int32_t* bonus_token,
                                   void* stream) {
+    if (c) c->pin_chain = false;  // (not an attention or append call)
     if (!c || batch < 0 || total_cand_rows < 0 || !(temperature > 0.f)) return FD_ERR_INVALID_ARG;
     if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
     if (batch == 0) return total_cand_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
@@ -573,6 +583,7 @@ fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, con
 
 fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefix_lens, const int32_t* q_lens,
                        const int32_t* accepted_len, int32_t* freed_pages, int32_t* n_freed, void* stream) {
+    if (c) c->pin_chain = false;  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || !n_freed) return FD_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (batch == 0) return cudaMemsetAsync(n_freed, 0, sizeof(int32_t), s) == cudaSuccess ? FD_OK : FD_ERR_CUDA;
@@ -609,6 +620,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
 fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blocks, const float* draft_logits,
                           const float* bias, const int32_t* n_mask, const int32_t* n_blocks, float threshold,
                           int32_t* mask_tokens, float* mask_probs, int32_t* keep_len, void* stream) {
+    if (c) c->pin_chain = false;  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || total_mask_rows < 0 || total_mask_rows > c->max_rows || max_blocks < 1)
         return FD_ERR_INVALID_ARG;
     if (batch == 0) return total_mask_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
@@ -629,6 +641,7 @@ fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blo
 fd_status fd_select_branch(fd_ctx* c, int batch, int max_block_len, const int32_t* mask_tokens, const int32_t* q_lens,
                            const int32_t* n_mask, const int32_t* n_blocks, const int32_t* accepted_len,
                            int32_t* next_draft, int32_t* next_len, void* stream) {
+    if (c) c->pin_chain = false;  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || max_block_len < 1) return FD_ERR_INVALID_ARG;
     if (batch == 0) return FD_OK;
     if (!q_lens || !n_mask || !accepted_len || !next_draft || !next_len) return FD_ERR_INVALID_ARG;
@@ -642,6 +655,7 @@ fd_status fd_select_branch(fd_ctx* c, int batch, int max_block_len, const int32_
 }
 
 fd_status fd_selftest_wait_timeout(fd_ctx* c, int limit_ms, void* stream) {
+    if (c) c->pin_chain = false;  // (not an attention or append call)
     if (!c || limit_ms < 1 || limit_ms > 1000) return FD_ERR_INVALID_ARG;
     fd::launch_wait_timeout_selftest(c->status, (unsigned long long)limit_ms * 1000000ull, static_cast<cudaStream_t>(stream));
     c->launches += 1;

@@ -169,6 +169,10 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// Under programmatic dependent launch: block until the launch before this one on the stream has completed and its
+// writes are visible.  Returns at once when that has happened already (or the launch was an ordinary one).
+__device__ __forceinline__ void wait_prior_launch() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Warp-uniform bounded wait.
 __device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, volatile int* abort) {
     const bool ok = mbar_wait(bar, parity, abort);
@@ -238,6 +242,9 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     const int s_c = rg.s_c, e_c = rg.e_c;
     Walk w = {s_c, 0, {0, 0}, 0, rg.first};
     bool ok = true;
+    // p.early: the first piece and its first page ids are looked up while the launch before this one may still run
+    bool waited = !p.early;
+    int bad_early = -1;
     while (w.t < e_c && ok) {
         const Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
         const int32_t* table = p.page_table + (long long)pc.b * p.max_pages;
@@ -250,7 +257,7 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             if (!(j < pc.nt && pos < pc.kv_len)) return -1;
             int id = table[pos >> 4];
             if ((unsigned)id >= (unsigned)p.num_pages) {  // never form an address from a bad id
-                flag_sequence(p, pc.b);
+                if (waited) flag_sequence(p, pc.b); else bad_early = pc.b;  // (no global write ahead of the prior launch)
                 *bad = 1;
                 id = 0;
             }
@@ -261,6 +268,11 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             const int g = w.g0 + j, st = g % C::kStages, use = g / C::kStages;
             if (j > 0 && (j & 3) == 0) { ids_cur = ids_next; ids_next = load_ids((j >> 2) + 1); }
             const int phys = __shfl_sync(0xffffffffu, ids_cur, (j & 3) * 8 + pg);
+            if (!waited) {  // the KV pool may be written by the launch before this one (the KV append)
+                wait_prior_launch();
+                waited = true;
+                if (bad_early >= 0) flag_sequence(p, bad_early);
+            }
             if (!wait_all(&empty[st], (use & 1) ^ 1, abort)) { ok = false; break; }
 #if FD_STAGGER
             // The first fill of the rings is not issued all at once: every CTA of the grid starts at the same moment,
@@ -312,6 +324,7 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
     int issued = 0;
     Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
     if (lane == 0) publish_piece(bars, ring, 0, pc);
+    if (p.early) wait_prior_launch();  // q may be written by it
     while (w.t < e_c) {
         if (w.piece > 0 && !wait_all(&bars->q_free, (w.piece - 1) & 1, abort)) break;
         const int nbox = (pc.Lv + bt - 1) / bt;
@@ -348,6 +361,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
     constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
+    if (p.early) wait_prior_launch();
     const uint64_t qd0 = make_smem_desc(smem_u32(sq), 16, 1024);
     const int s_c = rg.s_c, e_c = rg.e_c;
     Walk w = {s_c, 0, {0, 0}, 0, rg.first};
@@ -632,6 +646,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
         s_cs[tid] = (cc >= 0 && cc <= p.n_ctas) ? cs.g[cc] : 0;
     }
     bool cl_synced = false;
+    if (p.early) wait_prior_launch();  // before any global write of this role (scratch, counters, out)
     Walk w = {s_c, 0, {0, 0}, 0, 0};
     while (w.t < e_c) {
         // one thread waits for the descriptor, so that all 256 take the same decision
@@ -1046,7 +1061,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     // a call that plans for itself: warp 0 does so meanwhile (it needs the earlier kernels' results -- the lengths --
     // and waits for them on its own; its global loads then overlap the set-up of the other warps)
     if (MODE != kTcPlanned && warp == 0) {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (!p_in.early) wait_prior_launch();
         self_plan<MODE>(p_in, scans, rbs, s_cs, &bars->first);
     }
     tc_fence_before();
@@ -1056,7 +1071,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     // a dependent launch behind this one (the next layer's call) may bring its CTAs in as ours retire and do its
     // own set-up; it waits for this grid to complete before reading anything
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Everything below the plan needs the results of the launch before this one.  Under a pinned plan that launch is
+    // normally the previous layer's call (p.early): it writes neither the plan nor the lengths nor the page table, so
+    // the work of this CTA, its first piece and its first page ids are looked up while it still runs -- three to five
+    // dependent L2 round trips, 2.4 us -- and each role waits for it just before its first access to anything else.
+    if (!p_in.early) wait_prior_launch();
 
     // ---- the work of this CTA
     AttnParams p = p_in;
@@ -1104,6 +1123,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         }
     }
     if (rg.s_c >= rg.e_c && !cl_idle) {  // uniform (over the cluster too): no tile for this CTA, or nothing at all
+        if (p.early) wait_prior_launch();
         if (total == 0 && fatal) {  // inconsistent lengths: a defined output, zeros
             const long long n16 = (long long)p.total_q_rows * p.Hq * D / 8;
             uint4* o = reinterpret_cast<uint4*>(p.out);
@@ -1124,6 +1144,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     }
     if (MODE == kTcCluster && cl_idle) {
         // fewer tiles than CTAs in the cluster: this one tells every owner "saw no key" and combines the rows it owns
+        if (p.early) wait_prior_launch();
         if (tid < cl_rows) {
             const int dest = tid / exch.share, rl = tid % exch.share;
             unsigned char* blk = dest != cl_rank ? exch.g_block(dest) : exch.land + (size_t)cl_rank * exch.block;

@@ -87,6 +87,9 @@ struct AttnParams {
     int piece_cost;   // fixed cost of starting a segment in a range, in tiles (balances ranges with many short segments)
     int epoch;        // number of this attention call on its context, never 0 (see Plan::seq_bad)
     int cluster;      // CTAs per cluster when every segment is split over one cluster, else 0
+    int early;        // 1: the launch before this one on the stream is an attention or append call served by the same pinned
+                      //    plan, which writes neither the plan nor the lengths nor the page table: they may be read
+                      //    before that launch has completed (everything else waits for it)
     int* status;
 };
 
