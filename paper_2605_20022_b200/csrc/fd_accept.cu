@@ -12,72 +12,15 @@ namespace fd {
 
 constexpr int kVecPerThread = kAcceptChunk / (4 * 256);  // float4 loads in flight per thread
 
-__global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_per_row) {
-    const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
-    const float* base = p.logits + (long long)row * p.vocab;
-    const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
+// The accept scan: one CTA of 256 threads, after every row key is final.  `sm`: 2 * batch + 1 ints of shared memory.
+__device__ __forceinline__ void accept_scan(const AcceptParams& p, int* sm) {
     const int tid = threadIdx.x;
-
-    // A thread meets its elements in index order (head, body, tail), so "greater wins" keeps the lowest index of
-    // equal values; a thread whose elements are all -inf falls back to the first one it owns.
-    float bv = -INFINITY;
-    unsigned bi = 0xffffffffu, first = 0xffffffffu;
-    // scalar head up to the first 16-byte boundary, float4 body, scalar tail
-    const int mis = (int)((reinterpret_cast<uintptr_t>(base + c0) >> 2) & 3);
-    const int head = min(c1 - c0, (4 - mis) & 3);
-    const int nvec = (c1 - c0 - head) >> 2;
-    if (tid < head) { first = c0 + tid; const float v0 = base[c0 + tid]; if (v0 > bv) { bv = v0; bi = c0 + tid; } }
-    const float4* vp = reinterpret_cast<const float4*>(base + c0 + head);
-    float4 v[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int e = tid + k * 256;
-        v[k] = (e < nvec) ? __ldcs(vp + e) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-    }
-    if (first == 0xffffffffu && tid < nvec) first = c0 + head + 4 * tid;
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {  // padding is -inf and never wins
-        const unsigned i0 = c0 + head + 4 * (tid + k * 256);
-        if (v[k].x > bv) { bv = v[k].x; bi = i0; }
-        if (v[k].y > bv) { bv = v[k].y; bi = i0 + 1; }
-        if (v[k].z > bv) { bv = v[k].z; bi = i0 + 2; }
-        if (v[k].w > bv) { bv = v[k].w; bi = i0 + 3; }
-    }
-    const int tail0 = c0 + head + 4 * nvec;
-    if (tail0 + tid < c1) {
-        if (first == 0xffffffffu) first = tail0 + tid;
-        const float vt = base[tail0 + tid];
-        if (vt > bv) { bv = vt; bi = tail0 + tid; }
-    }
-    if (bi == 0xffffffffu) bi = first;
-
-    unsigned long long key = (bi == 0xffffffffu) ? 0ull : make_key(bv, bi);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-        key = other > key ? other : key;
-    }
-    __shared__ unsigned long long wkey[8];
-    __shared__ bool last;
-    if ((tid & 31) == 0) wkey[tid >> 5] = key;
-    __syncthreads();
-    if (tid == 0) {
-#pragma unroll
-        for (int w = 1; w < 8; ++w) key = wkey[w] > key ? wkey[w] : key;
-        atomicMax(p.keys + row, key);
-        __threadfence();
-        last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
-    }
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
 
     // ---- accept scan, one CTA, after every row key is final.  Everything is one parallel round of
     //      loads per step (serial walks over global memory would cost a DRAM/L2 latency per element):
     //      (1) block scan of the candidate-row counts, (2) one thread per candidate row compares its
     //      argmax with the next draft and lowers the sequence's first-mismatch index, (3) one thread
     //      per sequence reads the argmax at that index.
-    extern __shared__ int sm[];            // cu_c [B+1], then first_mismatch [B]
     int* cu_c = sm;
     int* first_bad = sm + p.batch + 1;
     __shared__ int s_bad, s_carry, s_wsum[8];
@@ -139,6 +82,69 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_
     __syncthreads();
     for (int r = tid; r < p.total_rows; r += blockDim.x) p.keys[r] = 0ull;
     if (tid == 0) *p.ticket = 0u;
+}
+
+__global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_per_row) {
+    const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
+    const float* base = p.logits + (long long)row * p.vocab;
+    const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
+    const int tid = threadIdx.x;
+
+    // A thread meets its elements in index order (head, body, tail), so "greater wins" keeps the lowest index of
+    // equal values; a thread whose elements are all -inf falls back to the first one it owns.
+    float bv = -INFINITY;
+    unsigned bi = 0xffffffffu, first = 0xffffffffu;
+    // scalar head up to the first 16-byte boundary, float4 body, scalar tail
+    const int mis = (int)((reinterpret_cast<uintptr_t>(base + c0) >> 2) & 3);
+    const int head = min(c1 - c0, (4 - mis) & 3);
+    const int nvec = (c1 - c0 - head) >> 2;
+    if (tid < head) { first = c0 + tid; const float v0 = base[c0 + tid]; if (v0 > bv) { bv = v0; bi = c0 + tid; } }
+    const float4* vp = reinterpret_cast<const float4*>(base + c0 + head);
+    float4 v[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int e = tid + k * 256;
+        v[k] = (e < nvec) ? __ldcs(vp + e) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+    if (first == 0xffffffffu && tid < nvec) first = c0 + head + 4 * tid;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {  // padding is -inf and never wins
+        const unsigned i0 = c0 + head + 4 * (tid + k * 256);
+        if (v[k].x > bv) { bv = v[k].x; bi = i0; }
+        if (v[k].y > bv) { bv = v[k].y; bi = i0 + 1; }
+        if (v[k].z > bv) { bv = v[k].z; bi = i0 + 2; }
+        if (v[k].w > bv) { bv = v[k].w; bi = i0 + 3; }
+    }
+    const int tail0 = c0 + head + 4 * nvec;
+    if (tail0 + tid < c1) {
+        if (first == 0xffffffffu) first = tail0 + tid;
+        const float vt = base[tail0 + tid];
+        if (vt > bv) { bv = vt; bi = tail0 + tid; }
+    }
+    if (bi == 0xffffffffu) bi = first;
+
+    unsigned long long key = (bi == 0xffffffffu) ? 0ull : make_key(bv, bi);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+    }
+    __shared__ unsigned long long wkey[8];
+    __shared__ bool last;
+    if ((tid & 31) == 0) wkey[tid >> 5] = key;
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll
+        for (int w = 1; w < 8; ++w) key = wkey[w] > key ? wkey[w] : key;
+        atomicMax(p.keys + row, key);
+        __threadfence();
+        last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    extern __shared__ int sm[];            // cu_c [B+1], then first_mismatch [B]
+    accept_scan(p, sm);
 }
 
 // R = 0: nothing to sweep, but the outputs are still defined (-1 everywhere).

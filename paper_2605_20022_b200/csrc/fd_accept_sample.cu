@@ -83,26 +83,9 @@ __device__ __forceinline__ float2 fold_stats(const float2* sh, float kt) {
     return make_float2(m, s);
 }
 
-__global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunks) {
-    __shared__ float2 sh_t[8], sh_d[8];
-    __shared__ bool row_last, last;
-    const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks, tid = threadIdx.x;
-    const int c0 = chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
-    const long long off = (long long)row * p.vocab + c0;
-    float x[4 * kVec], d[4 * kVec];
-    load_chunk(p.logits + off, n, tid, x);                        // both rows' loads are in flight together
-    if (p.draft_logits) load_chunk(p.draft_logits + off, n, tid, d);
-    warp_stats(x, p.kt, sh_t);
-    if (p.draft_logits) warp_stats(d, p.kt, sh_d);
-    __syncthreads();
-    if (tid == 0) {
-        p.part[((long long)row * chunks + chunk) * 2] = fold_stats(sh_t, p.kt);
-        p.part[((long long)row * chunks + chunk) * 2 + 1] = p.draft_logits ? fold_stats(sh_d, p.kt) : make_float2(0.f, 1.f);
-        __threadfence();
-        row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks - 1;
-    }
-    __syncthreads();
-    if (!row_last) return;  // only the CTA that completes a row goes on: one fence + count per chunk, not two
+// Warps 0 and 1 of the CTA that delivered the last chunk of `row` fold the row's chunk partials into (max, Z).
+__device__ __forceinline__ void sv_finish_row(const SampleParams& p, int row, int chunks) {
+    const int tid = threadIdx.x;
     if (tid < 64) {  // warp 0: target row, warp 1: draft row
         __threadfence();
         const int which = tid >> 5;
@@ -124,15 +107,11 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
             if (which == 0) p.row_ticket[row] = 0u;
         }
     }
-    __syncthreads();
-    if (tid == 0) {  // rows completed so far: whoever completes the last row finishes the call
-        __threadfence();
-        last = atomicAdd(p.ticket, 1u) == (unsigned)p.total_rows - 1;
-    }
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
+}
 
+// The CTA that finished last of all: accept tests, accepted lengths, and which row each bonus token is drawn from.
+__device__ __forceinline__ void sv_final(const SampleParams& p) {
+    const int tid = threadIdx.x;
     // ---- one CTA.  First the accept test of every row against the draft fed at the next row, all rows in
     //      parallel (each test reads single logits that no cache holds); a sequence's last row has no draft
     //      to test and its flag is never looked at.
@@ -205,6 +184,38 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
         if (bad) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         *p.ticket = 0u;
     }
+}
+
+__global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunks) {
+    __shared__ float2 sh_t[8], sh_d[8];
+    __shared__ bool row_last, last;
+    const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks, tid = threadIdx.x;
+    const int c0 = chunk * kAcceptChunk, n = min(p.vocab, c0 + kAcceptChunk) - c0;
+    const long long off = (long long)row * p.vocab + c0;
+    float x[4 * kVec], d[4 * kVec];
+    load_chunk(p.logits + off, n, tid, x);                        // both rows' loads are in flight together
+    if (p.draft_logits) load_chunk(p.draft_logits + off, n, tid, d);
+    warp_stats(x, p.kt, sh_t);
+    if (p.draft_logits) warp_stats(d, p.kt, sh_d);
+    __syncthreads();
+    if (tid == 0) {
+        p.part[((long long)row * chunks + chunk) * 2] = fold_stats(sh_t, p.kt);
+        p.part[((long long)row * chunks + chunk) * 2 + 1] = p.draft_logits ? fold_stats(sh_d, p.kt) : make_float2(0.f, 1.f);
+        __threadfence();
+        row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks - 1;
+    }
+    __syncthreads();
+    if (!row_last) return;  // only the CTA that completes a row goes on: one fence + count per chunk, not two
+    sv_finish_row(p, row, chunks);
+    __syncthreads();
+    if (tid == 0) {  // rows completed so far: whoever completes the last row finishes the call
+        __threadfence();
+        last = atomicAdd(p.ticket, 1u) == (unsigned)p.total_rows - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    sv_final(p);
 }
 
 // Weight of token y in the distribution the bonus token is drawn from.  ts / ds: (row maximum, 1 / Z) of the target

@@ -672,6 +672,16 @@ fd_status fd_last_device_status(fd_ctx* c, int32_t* code, void* stream) {
         // a call that gave up may have left pieces counted on segments nobody merged: start the next call clean
         c->pinned = false;
         if (cudaMemsetAsync(c->plan.seg_count, 0, 2 * (size_t)c->max_rb * c->cfg.n_kv_heads * sizeof(int), s) != cudaSuccess) return FD_ERR_CUDA;
+        // ... and a sweep that gave up leaves its running maxima and its row / call counters behind
+        const size_t R = (size_t)c->max_rows, B = (size_t)c->cfg.max_batch;
+        if (cudaMemsetAsync(c->keys, 0, R * sizeof(unsigned long long), s) != cudaSuccess ||
+            cudaMemsetAsync(c->ticket, 0, sizeof(unsigned int), s) != cudaSuccess ||
+            cudaMemsetAsync(c->ds_ticket, 0, sizeof(unsigned int), s) != cudaSuccess ||
+            cudaMemsetAsync(c->ds_row_ticket, 0, R * sizeof(unsigned int), s) != cudaSuccess ||
+            cudaMemsetAsync(c->sv_row_ticket, 0, R * sizeof(unsigned int), s) != cudaSuccess ||
+            cudaMemsetAsync(c->sv_ticket, 0, sizeof(unsigned int), s) != cudaSuccess ||
+            cudaMemsetAsync(c->sv_seq_ticket, 0, B * sizeof(unsigned int), s) != cudaSuccess)
+            return FD_ERR_CUDA;
     }
     return FD_OK;
 }

@@ -19,28 +19,12 @@ __device__ __forceinline__ float exp_neg(float x) {
     return y;
 }
 
-__global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams p, int chunks_per_row) {
-    const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
-    const long long rbase = (long long)row * p.vocab;
-    const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
-    const int tid = threadIdx.x, n = c1 - c0;
-    const float* lg = p.logits + rbase + c0;
-    const float* bs = p.bias ? p.bias + rbase + c0 : nullptr;
-    const bool vec = (((reinterpret_cast<uintptr_t>(lg) | (bs ? reinterpret_cast<uintptr_t>(bs) : 0)) & 15) == 0);
-
-    float x[4 * kDsVec];
-#pragma unroll
-    for (int k = 0; k < kDsVec; ++k) {
-        const int e = 4 * (tid + k * 256);
-        if (vec && e + 3 < n) {
-            float4 a = __ldcs(reinterpret_cast<const float4*>(lg + e));
-            if (bs) { const float4 b = __ldcs(reinterpret_cast<const float4*>(bs + e)); a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
-            x[4 * k] = a.x; x[4 * k + 1] = a.y; x[4 * k + 2] = a.z; x[4 * k + 3] = a.w;
-        } else {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) x[4 * k + q] = (e + q < n) ? (bs ? lg[e + q] + bs[e + q] : lg[e + q]) : -INFINITY;
-        }
-    }
+// A chunk's partial from the 4 * kDsVec values each thread holds (thread t: elements 4 * (t + 256 * k) + q of the
+// chunk [c0, c0 + n), -inf past the end): (max, argmax) as a key and sum exp(x - max), folded in a fixed order; thread
+// 0 stores them.  `wkey`, `wsum`: 8 entries of shared memory each.  Holds one barrier.
+__device__ __forceinline__ void ds_chunk_partial(const DraftSelectParams& p, const float (&x)[4 * kDsVec], int row, int chunk,
+                                                 int chunks_per_row, int c0, int n, unsigned long long* wkey, float* wsum) {
+    const int tid = threadIdx.x;
     // a thread meets its elements in index order, so "greater wins" keeps the lowest index of equal values;
     // padding (-inf) never wins, and a thread whose real elements are all -inf falls back to its first one
     float bv = -INFINITY;
@@ -59,10 +43,10 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
     }
     // every warp: its maximum (as a key) and the sum of exp(x - that maximum); thread 0 folds the eight
     // pairs in warp order -- one barrier for the whole chunk
-    __shared__ unsigned long long wkey[8];
-    __shared__ float wsum[8];
-    __shared__ bool last;
-    const float mw = key ? key_value(key) : 0.f;  // a warp wholly past the end of the row has key 0 and adds nothing
+    // a warp wholly past the end of the row has key 0 and adds nothing; neither does one whose logits are all -inf
+    // (a masked-out stretch of the vocabulary): its maximum must not enter a difference, -inf - -inf is NaN
+    float mw = key ? key_value(key) : 0.f;
+    if (mw == -INFINITY) mw = 0.f;
     float s = 0.f;
 #pragma unroll
     for (int k = 0; k < kDsVec; ++k)
@@ -73,7 +57,6 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if ((tid & 31) == 0) { wkey[tid >> 5] = key; wsum[tid >> 5] = s; }
     __syncthreads();
-    __shared__ bool row_last;
     if (tid == 0) {
         key = wkey[0];
 #pragma unroll
@@ -82,14 +65,15 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
         float t = 0.f;
 #pragma unroll
         for (int w = 0; w < 8; ++w)
-            if (wkey[w]) t += wsum[w] * exp_neg(key_value(wkey[w]) - m);
+            if (wkey[w] && key_value(wkey[w]) > -INFINITY) t += wsum[w] * exp_neg(key_value(wkey[w]) - m);
         p.part_key[(long long)row * chunks_per_row + chunk] = key;
         p.part_sum[(long long)row * chunks_per_row + chunk] = t;
-        __threadfence();
-        row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks_per_row - 1;
     }
-    __syncthreads();
-    if (!row_last) return;  // only the CTA that completes a row goes on: one fence + count per chunk, not two
+}
+
+// Warp 0 of the CTA that delivered the last chunk of `row` finishes the row.
+__device__ __forceinline__ void ds_finish_row(const DraftSelectParams& p, int row, int chunks_per_row) {
+    const int tid = threadIdx.x;
     if (tid < 32) {
         // the CTA that delivers the last chunk of a row finishes the row: lanes over chunks, maximum by an
         // exact reduction, sum of the rescaled chunk sums by a fixed shuffle tree (deterministic)
@@ -114,17 +98,12 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
             p.row_ticket[row] = 0u;
         }
     }
-    __syncthreads();
-    if (tid == 0) {  // rows completed so far: whoever completes the last row finishes the call
-        __threadfence();
-        last = atomicAdd(p.ticket, 1u) == (unsigned)p.total_rows - 1;
-    }
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
+}
 
+// The CTA that finished last of all.  `m0`: batch + 1 ints of shared memory.
+__device__ __forceinline__ void ds_final(const DraftSelectParams& p, int* m0) {
+    const int tid = threadIdx.x;
     // ---- one CTA: rows -> (token, confidence), then blocks -> verify length
-    extern __shared__ int m0[];  // [B+1] first mask row of each sequence
     __shared__ int carry, wcnt[8], s_bad;
     if (tid == 0) { carry = 0; m0[0] = 0; s_bad = 0; }
     __syncthreads();
@@ -181,6 +160,51 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
         p.keep_len[e] = keep;
     }
     if (tid == 0) *p.ticket = 0u;
+}
+
+__global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams p, int chunks_per_row) {
+    const int row = blockIdx.x / chunks_per_row, chunk = blockIdx.x % chunks_per_row;
+    const long long rbase = (long long)row * p.vocab;
+    const int c0 = chunk * kAcceptChunk, c1 = min(p.vocab, c0 + kAcceptChunk);
+    const int tid = threadIdx.x, n = c1 - c0;
+    const float* lg = p.logits + rbase + c0;
+    const float* bs = p.bias ? p.bias + rbase + c0 : nullptr;
+    const bool vec = (((reinterpret_cast<uintptr_t>(lg) | (bs ? reinterpret_cast<uintptr_t>(bs) : 0)) & 15) == 0);
+
+    float x[4 * kDsVec];
+#pragma unroll
+    for (int k = 0; k < kDsVec; ++k) {
+        const int e = 4 * (tid + k * 256);
+        if (vec && e + 3 < n) {
+            float4 a = __ldcs(reinterpret_cast<const float4*>(lg + e));
+            if (bs) { const float4 b = __ldcs(reinterpret_cast<const float4*>(bs + e)); a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+            x[4 * k] = a.x; x[4 * k + 1] = a.y; x[4 * k + 2] = a.z; x[4 * k + 3] = a.w;
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) x[4 * k + q] = (e + q < n) ? (bs ? lg[e + q] + bs[e + q] : lg[e + q]) : -INFINITY;
+        }
+    }
+    __shared__ unsigned long long wkey[8];
+    __shared__ float wsum[8];
+    __shared__ bool row_last, last;
+    ds_chunk_partial(p, x, row, chunk, chunks_per_row, c0, n, wkey, wsum);
+    if (tid == 0) {
+        __threadfence();
+        row_last = atomicAdd(p.row_ticket + row, 1u) == (unsigned)chunks_per_row - 1;
+    }
+    __syncthreads();
+    if (!row_last) return;  // only the CTA that completes a row goes on: one fence + count per chunk, not two
+    ds_finish_row(p, row, chunks_per_row);
+    __syncthreads();
+    if (tid == 0) {  // rows completed so far: whoever completes the last row finishes the call
+        __threadfence();
+        last = atomicAdd(p.ticket, 1u) == (unsigned)p.total_rows - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    extern __shared__ int m0[];  // [B+1] first mask row of each sequence
+    ds_final(p, m0);
 }
 
 // No mask rows at all: outputs are still defined.

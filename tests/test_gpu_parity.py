@@ -9,13 +9,22 @@ import torch
 import oracle
 import paper_2605_20022_b200 as fd
 from paper_2605_20022_b200 import workload as wl
-from helpers import Ctx, assert_close, gpu_accept, gpu_attn, gpu_commit
+from helpers import Ctx, assert_close, dev, gpu_accept, gpu_attn, gpu_commit
 
 pytestmark = pytest.mark.gpu
 
 # the CUDA-core kernel; the tensor-core kernel as a call is routed by default (one cluster per segment, self-planned
 # or planned, by size); the tensor-core kernel always on the plan kernel's work list; and always self-planned where legal
 PATHS = [fd.FD_ATTN_SIMT, fd.FD_ATTN_AUTO, fd.FD_ATTN_TCGEN05_PLANNED, fd.FD_ATTN_TCGEN05_SELF_PLANNED]
+
+
+def _one_float_off(t):
+    """A device copy of `t` that starts 4 bytes past a 16-byte boundary: the sweeps cannot use their aligned vector loads."""
+    buf = torch.empty(t.numel() + 1, dtype=t.dtype, device="cuda")
+    v = buf[1:].view(t.shape)
+    v.copy_(t)
+    assert v.data_ptr() % 16 == 4
+    return v
 
 
 def oracle_attn(step, q, kv):
@@ -200,6 +209,39 @@ def test_accept_vocab_sizes_ties_and_alignment(V):
             assert status == 0
             np.testing.assert_array_equal(acc, e_acc)
             np.testing.assert_array_equal(bon, e_bon)
+
+
+@pytest.mark.parametrize("V,B", [(20004, 48), (8192, 96), (12292, 48)])
+def test_accept_many_rows_ties_ragged_chunks_and_alignment(V, B):
+    """Several hundred rows: last chunk of a row ragged (V % 4096 != 0) or full, ties across chunk boundaries, flat /
+    -inf / +inf rows; the same logits one float off a 16-byte boundary (scalar head and tail around the vector loads)
+    must give the same answer."""
+    g = torch.Generator().manual_seed(V)
+    ql = torch.randint(12, 17, (B,), generator=g).tolist()
+    nm = [0] * B
+    step = wl.make_step("acc", wl.Shape(4, 2, 64, V), [5] * B, ql, nm, seed=V, p_match=0.9)
+    logits, drafts, _ = wl.make_logits(step)
+    logits = torch.round(logits * 2) / 2                       # coarse grid: many exact ties, planted peak kept
+    R = logits.shape[0]
+    logits[0] = 0.25                                           # flat row -> index 0
+    logits[1, V - 1] = 9.0; logits[1, 4096] = 9.0; logits[1, 4095] = 9.0   # tie across a chunk boundary -> 4095
+    logits[2, :] = -float("inf"); logits[2, V - 2] = -3e38
+    logits[3, 5000] = float("inf"); logits[3, V - 1] = float("inf")
+    logits[4, :] = -float("inf")                               # nothing finite -> index 0
+    logits[5, 0] = -0.0; logits[5, 1:] = -1.0; logits[5, V - 1] = 0.0      # -0.0 ties with +0.0
+    logits[R - 1] = 1.5; logits[R - 1, V - 1] = 2.0            # the last chunk of the last row decides
+    exp_acc, exp_bon, exp_am = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    assert exp_am[1] == 4095 and exp_am[4] == 0 and exp_am[R - 1] == V - 1
+    with Ctx(step) as ctx:
+        for _ in range(2):                                     # second call: keys and ticket were re-zeroed
+            acc, bon, status = gpu_accept(ctx, step, logits, drafts)
+            assert status == 0
+            np.testing.assert_array_equal(acc, exp_acc); np.testing.assert_array_equal(bon, exp_bon)
+        off = _one_float_off(logits)
+        acc_t = torch.full((B,), -99, dtype=torch.int32, device="cuda"); bon_t = torch.full_like(acc_t, -99)
+        fd.fd_verify_accept(ctx.h, B, R, off, dev(drafts), dev(step.q_lens), dev(step.n_mask), acc_t, bon_t)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        np.testing.assert_array_equal(acc_t.cpu().numpy(), exp_acc); np.testing.assert_array_equal(bon_t.cpu().numpy(), exp_bon)
 
 
 def test_accept_bad_lengths_and_no_candidates():
@@ -510,6 +552,60 @@ def test_draft_select_matches_oracle(V, with_bias):
         bad = torch.tensor([16, 0, 28, 6, 32, 12, 2], dtype=torch.int32)                             # rows do not add up
         fd.fd_draft_select(ctx.h, B, Rm, 8, logits.cuda(), None, bad.cuda(), n_blocks.cuda(), 0.5, tok, pr, keep)
         assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS and (tok == -1).all() and (keep == 0).all()
+
+
+@pytest.mark.parametrize("V,with_second,B", [(20004, True, 40), (20004, False, 40), (8192, True, 100), (12292, False, 48)])
+def test_sweeps_aligned_and_one_float_off_agree_bit_for_bit(V, with_second, B):
+    """Draft-side tail and sampling verification over several hundred rows, once on 16-byte aligned arrays (vector
+    loads) and once on the same data one float off alignment (scalar loads): a chunk's partial and the order the
+    partials are combined in do not depend on how the chunk was loaded, so every output must be identical -- tokens,
+    confidences (bitwise), verify lengths, accepted lengths, bonus tokens -- and both must agree with the oracle.
+    Row 7 has one finite logit, in the last chunk: every other chunk of it is -inf throughout."""
+    g = torch.Generator().manual_seed(V + int(with_second))
+    M = torch.randint(14, 17, (B,), generator=g).tolist()
+    Rm = sum(M)
+    logits = torch.randn((Rm, V), generator=g) * 2
+    logits[torch.arange(Rm), torch.randint(0, V, (Rm,), generator=g)] += 9.0 * torch.rand((Rm,), generator=g) + 3.0
+    logits[7, :] = -float("inf"); logits[7, V - 1] = 0.5        # one finite logit, in the ragged last chunk
+    second = torch.randn((Rm, V), generator=g) if with_second else None
+    n_mask = torch.tensor(M, dtype=torch.int32); n_blocks = torch.ones((B,), dtype=torch.int32)
+    step = wl.make_step("ds", wl.Shape(32, 8, 128, V), [5] * B, [32] * B, M, seed=1)
+    with Ctx(step) as ctx:
+        res = []
+        for mk in (lambda t: t.cuda(), _one_float_off):
+            tok = torch.full((Rm,), -9, dtype=torch.int32, device="cuda"); pr = torch.zeros((Rm,), device="cuda")
+            keep = torch.full((B, 2), -9, dtype=torch.int32, device="cuda")
+            fd.fd_draft_select(ctx.h, B, Rm, 2, mk(logits), None if second is None else mk(second), n_mask.cuda(), n_blocks.cuda(),
+                               0.3, tok, pr, keep)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            res.append((tok.cpu(), pr.cpu(), keep.cpu()))
+        assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][2], res[1][2])
+        assert torch.equal(res[0][1].view(torch.int32), res[1][1].view(torch.int32))
+        e_tok, e_pr, _, _, e_gap = oracle.draft_select(logits, second, n_mask, n_blocks, 0.3, max_blocks=2, want_gap=True)
+        x_abs = float((logits[torch.isfinite(logits)].abs().max() + (second.abs().max() if second is not None else 0)))
+        same = res[0][0].numpy() == e_tok
+        assert (same | (e_gap <= 2 * np.spacing(np.float32(x_abs)))).all()
+        np.testing.assert_allclose(res[0][1].numpy()[same], e_pr[same], rtol=1e-4, atol=1e-30)
+
+        # sampling verification over the same rows taken as candidate rows (draft logits = `second`)
+        ql = torch.tensor(M, dtype=torch.int32); nm0 = torch.zeros((B,), dtype=torch.int32)
+        drafts = torch.randint(0, V, (Rm,), generator=g, dtype=torch.int32)
+        am = logits.argmax(dim=1).to(torch.int32)
+        drafts[1:] = torch.where(torch.rand((Rm - 1,), generator=g) < 0.8, am[:-1], drafts[1:])
+        ua = torch.rand((Rm,), generator=g); ub = torch.rand((B,), generator=g)
+        out = []
+        for mk in (lambda t: t.cuda(), _one_float_off):
+            acc = torch.full((B,), -7, dtype=torch.int32, device="cuda"); bon = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+            for _ in range(2):                                  # twice: the counters must come back to zero
+                fd.fd_verify_accept_sample(ctx.h, B, Rm, mk(logits), None if second is None else mk(second), drafts.cuda(), ql.cuda(),
+                                           nm0.cuda(), 0.7, ua.cuda(), ub.cuda(), acc, bon)
+                assert fd.fd_last_device_status(ctx.h) == 0
+            out.append((acc.cpu(), bon.cpu()))
+        assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1])
+        acc_ref, _, ratio = oracle.accept_stochastic(logits.numpy(), None if second is None else second.numpy(), drafts.numpy(),
+                                                     ql.numpy(), nm0.numpy(), 0.7, ua.numpy(), ub.numpy())
+        differ = int((out[0][0].numpy() != acc_ref).sum())
+        assert differ <= max(1, B // 10), differ                # fp32 probabilities: only near-ties may part
 
 
 def test_kv_append_matches_oracle_and_feeds_the_attention():
