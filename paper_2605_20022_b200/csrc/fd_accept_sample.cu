@@ -65,8 +65,9 @@ __device__ __forceinline__ void warp_stats(const float (&x)[4 * kVec], float kt,
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     float s = 0.f;
     if (m > -INFINITY) {  // a warp whose share lies wholly past the end of the row has nothing
+        const float nm = -m * kt;
 #pragma unroll
-        for (int k = 0; k < 4 * kVec; ++k) s += ex2f((x[k] - m) * kt);  // -inf padding adds 0
+        for (int k = 0; k < 4 * kVec; ++k) s += ex2f(fmaf(x[k], kt, nm));  // one FMA per element; -inf padding adds 0
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);

@@ -13,6 +13,12 @@ constexpr int kDsVec = kAcceptChunk / (4 * 256);
 
 // exp(x) for x <= 0 through one MUFU instruction (relative error about 2^-22: far inside the 1e-4 the
 // confidences are compared at; the sweep is HBM-bound only if the per-element work stays this small)
+constexpr float kLog2e = 1.4426950408889634f;
+__device__ __forceinline__ float exp2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float exp_neg(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x * 1.4426950408889634f));
@@ -48,11 +54,12 @@ __device__ __forceinline__ void ds_chunk_partial(const DraftSelectParams& p, con
     float mw = key ? key_value(key) : 0.f;
     if (mw == -INFINITY) mw = 0.f;
     float s = 0.f;
+    const float nmw = -mw * kLog2e;
 #pragma unroll
     for (int k = 0; k < kDsVec; ++k)
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-            s += exp_neg(x[4 * k + q] - mw);  // padding is -inf and adds 0
+            s += exp2_approx(fmaf(x[4 * k + q], kLog2e, nmw));  // one FMA per element; padding is -inf and adds 0
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if ((tid & 31) == 0) { wkey[tid >> 5] = key; wsum[tid >> 5] = s; }
