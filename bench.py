@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) of ONE attention-kernel launch on the long-context workload, from the ncu capture
 # summarised in profiles/attn_tc_and_accept_kernels_long_context_1layer.md
 # (dram__bytes_read.sum 2 154 169 000 + dram__bytes_write.sum 7 170 560; one layer = one full-size launch).
-NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_161_339_560}
+NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_161_364_480}
 
 METRIC = "draft-verify attn+accept us/step"
 UNIT = "us/step"
@@ -619,7 +619,7 @@ def run_ours(args, step, rank, world, dist):
     small = step.attn_bytes() * step.shape.n_layers < 4 * 126e6      # fits (mostly) in the 126 MB L2
     flush = torch.empty((512 << 20,), dtype=torch.uint8, device=device) if small else None
 
-    draft_tail, accept_row, sample_row = vocabulary_sweeps(torch, fd, ds, step, device, peak, flush, rank)
+    draft_tail, accept_row, sample_row = (None, None, None) if args.no_sweeps else vocabulary_sweeps(torch, fd, ds, step, device, peak, flush, rank)
 
     ds.restore()
     for _ in range(args.warmup):
@@ -769,6 +769,7 @@ def main():
     ap.add_argument("--attn-path", type=int, default=0, help="0 auto, 1 SIMT kernel, 2 tcgen05 kernel, 3 tcgen05 always planned, 4 tcgen05 self-planned")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--no-per-workload", action="store_true", help="headline workload only: skip the records of the other workloads")
+    ap.add_argument("--no-sweeps", action="store_true", help="skip the separate timings of the three vocabulary sweeps (for profiling the step alone)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
