@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 
 # DRAM bytes (read + write) of ONE attention-kernel launch on the long-context workload, from the ncu capture
 # summarised in profiles/attn_tc_and_accept_kernels_long_context_1layer.md
-# (dram__bytes_read.sum 2 154 169 000 + dram__bytes_write.sum 7 170 560; one layer = one full-size launch).
+# (dram__bytes_read.sum 2 154 089 216 + dram__bytes_write.sum 7 275 264; one layer = one full-size launch).
 NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_161_364_480}
 
 METRIC = "draft-verify attn+accept us/step"
