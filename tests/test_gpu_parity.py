@@ -44,6 +44,54 @@ def test_attention_workloads(idx, path):
     assert_close(got.numpy(), oracle_attn(step, q, kv), step.name)
 
 
+def _random_step(seed):
+    """A seeded random shape and batch: heads, group size, head dimension, ragged prefixes (some empty, some a few
+    tiles long), block lengths up to what one 128-row tile holds, any number of mask rows, sometimes several mask blocks."""
+    g = torch.Generator().manual_seed(seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))
+    G = [1, 2, 4, 8][ri(0, 3)]
+    Hkv = [1, 2, 4, 8][ri(0, 3)]
+    while G * Hkv > 32:
+        Hkv //= 2
+    d = [64, 128][ri(0, 1)]
+    B = ri(1, 7)
+    max_rows = min(32, 128 // G)
+    pl, ql, nm, nb = [], [], [], []
+    for _ in range(B):
+        kind = ri(0, 9)
+        pl.append(0 if kind == 0 else ri(1, 40) if kind == 1 else ri(100, 140) if kind == 2 else ri(0, 1500))
+        L = 0 if ri(0, 11) == 0 else ri(1, max_rows)
+        M = ri(0, L) if L else 0
+        C = L - M
+        blocks = 1
+        if M > 1 and C >= 2 and ri(0, 2) == 0:             # several branches: M = blocks * tokens, at most one per candidate row
+            cands = [k for k in range(2, min(M, C) + 1) if M % k == 0]
+            if cands:
+                blocks = cands[ri(0, len(cands) - 1)]
+        ql.append(L); nm.append(M); nb.append(blocks)
+    step = wl.make_step(f"fuzz{seed}", wl.Shape(G * Hkv, Hkv, d, 1000), pl, ql, nm, seed=seed, extra_table_cols=ri(0, 2))
+    return step, torch.tensor(nb, dtype=torch.int32)
+
+
+@pytest.mark.parametrize("seed", list(range(40)))
+def test_random_shapes_against_the_oracle(seed):
+    """Forty seeded random batches through the default routing and through the plan kernel's work list: every output
+    element against the oracle, poisoned slots beyond every sequence's length, NaN in the output buffer beforehand."""
+    step, n_blocks = _random_step(seed)
+    if step.total_q_rows == 0:
+        pytest.skip("all blocks empty")
+    s = step.shape
+    q, kv = wl.make_q(step), wl.make_kv(step)
+    ref = oracle.attn_blocks(q, kv, step.page_table, step.prefix_lens, step.q_lens, step.n_mask, n_blocks)
+    for path in (fd.FD_ATTN_AUTO, fd.FD_ATTN_TCGEN05_PLANNED):
+        with Ctx(step, path) as ctx:
+            out = torch.full((step.total_q_rows, s.n_q_heads, s.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+            fd.fd_attn_draft_verify_blocks(ctx.h, step.batch, step.total_q_rows, q.cuda(), kv.cuda(), step.num_pages, step.page_table.cuda(),
+                                           step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda(), n_blocks.cuda(), out)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            assert_close(out.float().cpu().numpy(), ref, f"{step.name} path {path}")
+
+
 def test_tensor_core_call_routing():
     """Which form of the tensor-core kernel a call takes: few segments -> one cluster per segment; few sequences ->
     self-planned; otherwise (or under a pinned plan) the plan kernel's work list.  All forms agree with the oracle."""
