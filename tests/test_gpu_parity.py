@@ -292,6 +292,37 @@ def test_accept_many_rows_ties_ragged_chunks_and_alignment(V, B):
         np.testing.assert_array_equal(acc_t.cpu().numpy(), exp_acc); np.testing.assert_array_equal(bon_t.cpu().numpy(), exp_bon)
 
 
+@pytest.mark.parametrize("seed", list(range(30)))
+def test_accept_then_commit_random_batches(seed):
+    """Thirty seeded random batches: vocabulary of any size (aligned or not, below and above one chunk), any mix of
+    candidate and mask rows, sequences without candidates, coarse logits (ties); accept and the commit that follows
+    it, bit-exact against the oracle, twice in a row on the same context."""
+    g = torch.Generator().manual_seed(1000 + seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))
+    V = [ri(1, 40), ri(41, 4096), ri(4097, 9000), 4096, 8192][seed % 5]
+    B = ri(1, 40)
+    ql, nm, pl = [], [], []
+    for _ in range(B):
+        L = 0 if ri(0, 9) == 0 else ri(1, 32)
+        M = ri(0, L) if ri(0, 3) else 0
+        ql.append(L); nm.append(M); pl.append(ri(0, 300))
+    step = wl.make_step(f"ac{seed}", wl.Shape(4, 2, 64, V), pl, ql, nm, seed=2000 + seed, p_match=[0.5, 0.8, 0.95][seed % 3],
+                        extra_table_cols=ri(0, 2))
+    logits, drafts, _ = wl.make_logits(step)
+    if seed % 2:
+        logits = torch.round(logits * 2) / 2
+    exp_acc, exp_bon, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, exp_acc)
+    with Ctx(step) as ctx:
+        for _ in range(2):
+            acc, bon, status = gpu_accept(ctx, step, logits, drafts)
+            assert status == 0
+            np.testing.assert_array_equal(acc, exp_acc); np.testing.assert_array_equal(bon, exp_bon)
+            pt, pl2, freed, status = gpu_commit(ctx, step, acc)
+            assert status == 0
+            np.testing.assert_array_equal(pt, ept); np.testing.assert_array_equal(pl2, epl); np.testing.assert_array_equal(freed, efreed)
+
+
 def test_accept_bad_lengths_and_no_candidates():
     step = wl.make_step("acc", wl.Shape(4, 2, 64, 500), [5, 5], [4, 16], [0, 16], seed=3)
     logits, drafts, _ = wl.make_logits(step)
