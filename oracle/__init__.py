@@ -26,8 +26,10 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "fd_oracle.c")
-_SO = os.path.join(_HERE, "libfd_oracle.so")
+# FD_ORACLE_SRC: a test hook.  tests/test_oracle_mutants.py points it at a copy of the source with one mistake planted
+# in it and checks that the pins notice; nothing else sets it.
+_SRC = os.environ.get("FD_ORACLE_SRC") or os.path.join(_HERE, "fd_oracle.c")
+_SO = (_SRC + ".so") if os.environ.get("FD_ORACLE_SRC") else os.path.join(_HERE, "libfd_oracle.so")
 _lib = None
 
 

@@ -29,6 +29,21 @@ def test_tokens_and_confidence_against_library_softmax():
     assert (tok0 != tok).any()                                   # the calibration changes some drafts
 
 
+def test_first_token_as_the_calibrated_argmax():
+    """Index 0 wins only because of its bias (and, in the second row, loses only because of it): the first element
+    of a row takes part in Eq. 4's sum like every other."""
+    V = 50
+    g = torch.Generator().manual_seed(5)
+    logits = torch.randn((2, V), generator=g); bias = torch.zeros((2, V))
+    logits[0, 0] = logits[0].max() - 1.0; bias[0, 0] = 4.0       # wins by its bias
+    logits[1, 0] = logits[1].max() + 1.0; bias[1, 0] = -6.0      # would win without it
+    tok, pr, _, _ = oracle.draft_select(logits, bias, np.array([2], np.int32), None, 0.5, max_blocks=1)
+    x = logits.double() + bias.double()
+    assert tok[0] == 0 and tok[1] == int(x[1].argmax()) != 0
+    ref = torch.softmax(x, dim=1)[torch.arange(2), torch.from_numpy(tok).long()]
+    np.testing.assert_allclose(pr, ref.numpy(), rtol=1e-12)
+
+
 def test_sum_is_not_rounded_to_float32():
     """Two calibrated logits that a float32 sum makes equal (lower index would win) but whose exact sums differ."""
     V = 8
