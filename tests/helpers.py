@@ -50,6 +50,14 @@ def assert_close(got, ref, what=""):
     assert worst <= 0, f"{what}: max |err| {err.max():.4g}, worst excess over tolerance {worst:.4g}"
 
 
+def worst_vector_error(got, ref):
+    """Largest error of a (row, head) output vector relative to the vector's own length.  At long contexts an output
+    element averages tens of thousands of values and is small against the elementwise tolerance, which a lost tile would
+    pass; the vector's relative error shows it (tests/test_comparison_bounds.py measures both)."""
+    got = np.asarray(got, dtype=np.float64)
+    return float((np.linalg.norm(got - ref, axis=-1) / np.linalg.norm(ref, axis=-1)).max())
+
+
 def gpu_accept(ctx, step, logits, drafts, lens=None):
     ql, nm = lens if lens is not None else (step.q_lens, step.n_mask)
     B = int(ql.numel())
