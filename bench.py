@@ -413,8 +413,10 @@ def capture_step_graph(torch, ds, attn_only=False, append=False):
     return g
 
 
-def check_against_oracle(ds: DeviceStep, n_rows=6):
-    """A few sampled attention rows + the accept result of the benchmarked tensors vs the oracle."""
+def check_against_oracle(ds: DeviceStep, n_rows=16):
+    """Sampled attention rows (one per sequence in turn, random block row and head) + the accept result of the
+    benchmarked tensors vs the oracle.  A sampled (row, head) vector must meet the elementwise tolerance and agree to
+    2 % of its own length: at tens of thousands of keys only the second notices a lost tile."""
     import numpy as np
     import oracle
     torch, st = ds.torch, ds.step
@@ -429,8 +431,9 @@ def check_against_oracle(ds: DeviceStep, n_rows=6):
         return ok_attn and bool((ds.acc.cpu().numpy() == e_acc).all() and (ds.bon.cpu().numpy() == e_bon).all())
     cu = torch.cumsum(st.q_lens, 0) - st.q_lens
     worst = 0.0
-    for _ in range(n_rows):
-        b = int(torch.randint(0, st.batch, (1,), generator=g))
+    worst_vec = 0.0
+    for k in range(n_rows):
+        b = k % st.batch
         if int(st.q_lens[b]) == 0:
             continue
         i = int(torch.randint(0, int(st.q_lens[b]), (1,), generator=g))
@@ -438,7 +441,8 @@ def check_against_oracle(ds: DeviceStep, n_rows=6):
         ref = oracle.attn_row(qc, kvc, st.page_table, st.prefix_lens, st.q_lens, st.n_mask, b, i, h)
         err = np.abs(outc[int(cu[b]) + i, h] - ref)
         worst = max(worst, float((err - 2e-2 * np.abs(ref)).max()))
-    ok_attn = worst <= 2e-2
+        worst_vec = max(worst_vec, float(np.linalg.norm(err) / np.linalg.norm(ref)))
+    ok_attn = worst <= 2e-2 and worst_vec <= 2e-2
     e_acc, e_bon, _ = oracle.accept(ds.logits.cpu(), ds.drafts.cpu(), st.q_lens, st.n_mask)
     ok_acc = bool((ds.acc.cpu().numpy() == e_acc).all() and (ds.bon.cpu().numpy() == e_bon).all())
     return ok_attn and ok_acc
@@ -460,6 +464,8 @@ def check_full(ds: DeviceStep):
             ref = oracle.attn(qc, kvc, st.page_table, st.prefix_lens, st.q_lens, st.n_mask)
         outc = ds.out[l].float().cpu().numpy()
         ok = ok and bool(np.isfinite(outc).all() and (np.abs(outc - ref) <= 2e-2 + 2e-2 * np.abs(ref)).all())
+        # and every (row, head) vector to 2 % of its own length (what notices a lost tile at long contexts)
+        ok = ok and bool((np.linalg.norm(outc - ref, axis=-1) <= 2e-2 * np.linalg.norm(ref, axis=-1)).all())
     e_acc, e_bon, _ = oracle.accept(ds.logits.cpu(), ds.drafts.cpu(), st.q_lens, st.n_mask)
     ok = ok and bool((ds.acc.cpu().numpy() == e_acc).all() and (ds.bon.cpu().numpy() == e_bon).all())
     ept, epl, efreed = oracle.commit(st.page_table, st.prefix_lens, st.q_lens, e_acc)
