@@ -165,6 +165,13 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * itself when it reports that bit).  fd_kv_commit rewrites prefix_lens and therefore drops the pin
  * itself: the first attention call of the next step plans afresh (or is preceded by a new fd_plan_pin).
  * fd_kv_append leaves the lengths alone and keeps the pin.
+ * Consecutive attention calls under one pin overlap on the device: a call starts while the call before it is still
+ * finishing, and -- where its range of KV tiles is short -- reads its q and its cache ahead of that call's completion,
+ * provided no earlier call since the pin wrote them (the library compares the `out` ranges of those calls with q and
+ * kv_cache of this one; fd_kv_append in between, which writes the cache, switches the read-ahead off for the next
+ * call).  Every write of a call (out, scratch) waits for the call before it, so results are those of calls run one
+ * after the other.  What the library cannot see is a buffer written by the CALLER's own asynchronous work on another
+ * stream: order such work before the call as usual.
  * The calls served by a pin must be ordered after fd_plan_pin (the
  * same stream, or streams the caller has ordered) and must not overlap one another: they share the context's
  * scratch memory, as all attention calls on one context do.

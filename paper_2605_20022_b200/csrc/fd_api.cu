@@ -2,6 +2,7 @@
 #include <math.h>
 #include <algorithm>
 #include <vector>
+#include <utility>
 #include <new>
 
 #include "fd_internal.cuh"
@@ -42,6 +43,8 @@ struct fd_ctx {
     int pin_batch, pin_rows;
     const int32_t *pin_pl, *pin_ql, *pin_nm, *pin_nb;
     bool pin_chain;    // the context's last launch was an attention or append call under the pinned plan (see AttnParams::early)
+    bool chain_append; // ... and it was the append (which writes the cache the next attention call reads)
+    std::vector<std::pair<uintptr_t, uintptr_t>> chain_out;  // [begin, end) of what the attention calls of the chain have written
     struct HostStage* host;  // staging for fd_step_host, nullptr until fd_host_reserve
 };
 
@@ -144,6 +147,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     if (cfg->attn_path >= FD_ATTN_TCGEN05 && !tc_ok) { delete c; return FD_ERR_UNSUPPORTED; }
     c->tc_choice = cfg->attn_path >= FD_ATTN_TCGEN05 ? cfg->attn_path : FD_ATTN_TCGEN05;
     c->last_mode = -1;
+    c->chain_append = false;
     c->epoch = 0;
     c->attn_path = (cfg->attn_path == FD_ATTN_SIMT || !tc_ok) ? FD_ATTN_SIMT : FD_ATTN_TCGEN05;
     // SIMT kernel: two 74 KB CTAs fit an SM; tensor-core kernel: one persistent CTA per SM
@@ -468,6 +472,22 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     // under a pinned plan, behind another call it served: the plan, the lengths and the page table are not what the
     // launch before this one writes, and may be read while it still runs
     p.early = (reuse && c->pinned && c->pin_chain) ? 1 : 0;
+    if (!p.early) c->chain_out.clear();
+    // ... and so may q and the cache, if no call of the chain writes them: the attention calls before this one write
+    // their `out` (several of them may still be running: each starts as the one before it retires CTAs, and waits for
+    // it only before its own first write), the append writes the cache
+    if (p.early && tc && !c->chain_append) {
+        const uintptr_t q0 = reinterpret_cast<uintptr_t>(q), q1 = q0 + (size_t)total_q_rows * p.Hq * p.d * 2;
+        const uintptr_t k0 = reinterpret_cast<uintptr_t>(kv_cache), k1 = k0 + (size_t)num_pages * 2 * p.Hkv * 16 * p.d * 2;
+        bool clash = c->chain_out.size() >= 1024;  // (a chain that long is not a step of a model: stop keeping track)
+        for (const auto& w : c->chain_out) clash = clash || (w.first < q1 && q0 < w.second) || (w.first < k1 && k0 < w.second);
+        if (!clash) p.early = 2;
+    }
+    if (total_q_rows > 0 && c->chain_out.size() < 1024) {
+        const uintptr_t o0 = reinterpret_cast<uintptr_t>(out);
+        c->chain_out.emplace_back(o0, o0 + (size_t)total_q_rows * p.Hq * p.d * 2);
+    }
+    c->chain_append = false;
     c->pin_chain = reuse && c->pinned;
     if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
     } else if (tc) {
@@ -613,6 +633,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
     p.kv = static_cast<__nv_bfloat16*>(kv_cache);
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.status = c->status;
     fd::launch_kv_append(p, static_cast<cudaStream_t>(stream));
+    c->chain_append = true;  // the next attention call must not read the cache ahead of this launch
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }

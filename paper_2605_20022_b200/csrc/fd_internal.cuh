@@ -90,6 +90,8 @@ struct AttnParams {
     int early;        // 1: the launch before this one on the stream is an attention or append call served by the same pinned
                       //    plan, which writes neither the plan nor the lengths nor the page table: they may be read
                       //    before that launch has completed (everything else waits for it)
+                      // 2: nor does any call of that chain write q or the cache of this one: they may be read early too,
+                      //    and the first piece worked through; the call waits before its first write to global memory
     int* status;
 };
 

@@ -716,6 +716,37 @@ def test_kv_append_matches_oracle_and_feeds_the_attention():
         assert fd.fd_last_device_status(ctx.h) == fd.FD_DEV_BAD_LENGTHS
 
 
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_chain_of_calls_whose_output_is_the_next_query(idx):
+    """Under a pinned plan consecutive attention calls overlap: a call may read its q and its cache while the call
+    before it is still running, unless that call writes them.  Here every call's q IS the previous call's out (the
+    buffers start as NaN), interleaved with calls on buffers of their own: reading ahead must happen only where it is
+    safe, so every result has to match the oracle applied layer by layer."""
+    step = wl.workload(idx)
+    s = step.shape
+    L = 6
+    kvs = [wl.make_kv(step, l) for l in range(L)]
+    q0 = wl.make_q(step)
+    with Ctx(step) as ctx:
+        dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
+        dkv = [k.cuda() for k in kvs]
+        dq0 = q0.cuda()
+        for rep in range(2):
+            outs = [torch.full_like(dq0, float("nan")) for _ in range(L)]
+            fd.fd_plan_pin(ctx.h, step.batch, step.total_q_rows, dpl, dql, dnm)
+            q = dq0
+            for l in range(L):
+                fd.fd_attn_draft_verify(ctx.h, step.batch, step.total_q_rows, q, dkv[l], step.num_pages, dpt, dpl, dql, dnm, outs[l])
+                q = outs[l] if l % 2 == 0 else dq0                               # odd layers feed on the even layer's output
+            fd.fd_plan_unpin(ctx.h)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            # the reference of a layer that feeds on an output is computed from what the kernel produced there
+            for l in range(L):
+                fed = q0 if l % 2 == 0 else outs[l - 1].cpu()
+                ref = oracle.attn(fed, kvs[l], step.page_table, step.prefix_lens, step.q_lens, step.n_mask)
+                assert_close(outs[l].float().cpu().numpy(), ref, f"{step.name} layer {l} rep {rep}")
+
+
 def test_pinned_plan_serves_every_layer_and_is_dropped_on_other_lengths():
     """fd_plan_pin: several attention calls reuse one work list; a call with other lengths recomputes it."""
     step = wl.workload(2)
