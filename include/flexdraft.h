@@ -169,7 +169,9 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * finishing, and -- where its range of KV tiles is short -- reads its q and its cache ahead of that call's completion,
  * provided no earlier call since the pin wrote them (the library compares the `out` ranges of those calls with q and
  * kv_cache of this one; fd_kv_append in between, which writes the cache, switches the read-ahead off for the next
- * call).  Every write of a call (out, scratch) waits for the call before it, so results are those of calls run one
+ * call).  fd_kv_append itself, behind an attention call of the chain, copies while that call finishes (its k_new /
+ * v_new are checked against those `out` ranges in the same way).  Every write of an attention call (out, scratch)
+ * waits for the launch before it, and the append waits for it before it ends, so results are those of calls run one
  * after the other.  What the library cannot see is a buffer written by the CALLER's own asynchronous work on another
  * stream: order such work before the call as usual.
  * The calls served by a pin must be ordered after fd_plan_pin (the

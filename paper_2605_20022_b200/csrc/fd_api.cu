@@ -632,6 +632,18 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
     p.k_new = static_cast<const __nv_bfloat16*>(k_new); p.v_new = static_cast<const __nv_bfloat16*>(v_new);
     p.kv = static_cast<__nv_bfloat16*>(kv_cache);
     p.page_table = page_table; p.prefix_lens = prefix_lens; p.q_lens = q_lens; p.status = c->status;
+    // Behind an attention call of a pinned chain the append need not wait for it: it reads the block's K/V, the page
+    // table and the lengths, none of which the calls of the chain write (their `out` ranges are checked), and writes a
+    // cache that only the NEXT attention call reads.  Its copies then run under that call's merge tail; it waits for the
+    // call before it ends, so the attention call behind it, which waits for the append, has waited for both.
+    p.chained = 0;
+    if (c->pin_chain && c->pinned && !c->chain_append) {
+        const size_t nb = (size_t)total_q_rows * p.Hkv * p.d * 2;
+        const uintptr_t a0 = reinterpret_cast<uintptr_t>(k_new), b0 = reinterpret_cast<uintptr_t>(v_new);
+        bool clash = c->chain_out.size() >= 1024;
+        for (const auto& w : c->chain_out) clash = clash || (w.first < a0 + nb && a0 < w.second) || (w.first < b0 + nb && b0 < w.second);
+        p.chained = clash ? 0 : 1;
+    }
     fd::launch_kv_append(p, static_cast<cudaStream_t>(stream));
     c->chain_append = true;  // the next attention call must not read the cache ahead of this launch
     c->launches += 1;

@@ -71,7 +71,12 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p, int rows
     __shared__ long long s_row0;
     const int b = blockIdx.x, i0 = blockIdx.y * rows_per_cta, tid = threadIdx.x;
     const int n = p.prefix_lens[b], Lq = p.q_lens[b];
-    if (i0 >= Lq) return;  // uniform (an empty or negative length too)
+    // (p.chained: the launch before this one may still be running -- it writes nothing this kernel reads; every CTA
+    // waits for it before leaving, so that whoever waits for THIS launch has waited for that one too)
+    if (i0 >= Lq) {  // uniform (an empty or negative length too)
+        if (p.chained) asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     // first query row of this sequence = sum of the lengths before it (block-parallel; negative lengths count as 0)
     int part = 0;
     for (int s = tid; s < b; s += blockDim.x) part += max(p.q_lens[s], 0);
@@ -87,17 +92,19 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p, int rows
     __syncthreads();
     const long long row0 = s_row0;
     if (n < 0 || row0 + Lq > p.total_rows || (long long)n + Lq > (long long)p.max_pages * 16) {
+        if (p.chained) asm volatile("griddepcontrol.wait;" ::: "memory");  // (before the write to the status word, too)
         if (tid == 0 && i0 == 0) atomicOr(p.status, FD_DEV_BAD_LENGTHS);
         return;
     }
     const int vec_per_head = p.d / 8;                    // 16-byte pieces of one head's row
     const int per_row = p.Hkv * vec_per_head;
     const int i1 = min(Lq, i0 + rows_per_cta);
+    bool bad_page = false;
     for (int i = i0; i < i1; ++i) {
         const int j = n + i;
         const int page = p.page_table[(long long)b * p.max_pages + (j >> 4)];
         if ((unsigned)page >= (unsigned)p.num_pages) {   // never form an address from a bad id
-            if (tid == 0) atomicOr(p.status, FD_DEV_BAD_PAGE);
+            bad_page = true;  // (reported at the end: the status word is shared with the launch before this one)
             continue;
         }
         for (int e = tid; e < 2 * per_row; e += blockDim.x) {
@@ -108,6 +115,8 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p, int rows
             *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
         }
     }
+    if (p.chained) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (bad_page && tid == 0) atomicOr(p.status, FD_DEV_BAD_PAGE);
 }
 
 void launch_kv_append(const AppendParams& p, cudaStream_t s) {
@@ -115,7 +124,20 @@ void launch_kv_append(const AppendParams& p, cudaStream_t s) {
     // a handful of rows per CTA; long query blocks (up to 4096 rows) get more rows per CTA instead of more CTAs
     const int rows_per_cta = std::max(4, (p.max_q_len + 63) / 64);
     const int groups = (p.max_q_len + rows_per_cta - 1) / rows_per_cta;
-    kv_append_kernel<<<dim3(p.batch, groups), 256, 0, s>>>(p, rows_per_cta);
+    if (!p.chained) {
+        kv_append_kernel<<<dim3(p.batch, groups), 256, 0, s>>>(p, rows_per_cta);
+        return;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.batch, groups);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kv_append_kernel, p, rows_per_cta);
 }
 
 // Branch selection after verification (parallel drafting with one prepared branch per hypothesis):

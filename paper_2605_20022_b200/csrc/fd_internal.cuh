@@ -385,6 +385,8 @@ struct AppendParams {
     const int32_t* prefix_lens;
     const int32_t* q_lens;
     int* status;
+    int chained;  // 1: launched as a programmatic dependent of an attention call of the same pinned chain, none of whose
+                  //    writes it reads: the copies run while that call finishes, the kernel waits for it before it ends
 };
 void launch_kv_append(const AppendParams& p, cudaStream_t s);
 

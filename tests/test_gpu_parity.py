@@ -747,6 +747,40 @@ def test_chain_of_calls_whose_output_is_the_next_query(idx):
                 assert_close(outs[l].float().cpu().numpy(), ref, f"{step.name} layer {l} rep {rep}")
 
 
+def test_chained_append_whose_input_is_the_previous_output():
+    """Under a pinned plan the append of layer l + 1 runs while the attention call of layer l is finishing, unless it
+    reads what that call writes.  Layer 1's k_new here IS (a part of) layer 0's out, NaN beforehand; layers 2 and 3 have
+    inputs of their own.  Every cache must end up as the oracle's append of what the inputs finally held, every output
+    as the oracle's attention over that cache."""
+    step = wl.workload(2)
+    s = step.shape
+    T, L = step.total_q_rows, 4
+    g = torch.Generator().manual_seed(21)
+    kvs = [wl.make_kv(step, l) for l in range(L)]
+    qs = [wl.make_q(step, l) for l in range(L)]
+    kn = [torch.randn((T, s.n_kv_heads, s.head_dim), generator=g).bfloat16() for _ in range(L)]
+    vn = [torch.randn((T, s.n_kv_heads, s.head_dim), generator=g).bfloat16() for _ in range(L)]
+    with Ctx(step) as ctx:
+        dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
+        for rep in range(2):
+            pools = [k.cuda() for k in kvs]
+            outs = [torch.full((T, s.n_q_heads, s.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+            dkn = [k.cuda() for k in kn]; dvn = [v.cuda() for v in vn]
+            dkn[1] = outs[0].view(-1)[: T * s.n_kv_heads * s.head_dim].view(T, s.n_kv_heads, s.head_dim)   # aliases out of layer 0
+            fd.fd_plan_pin(ctx.h, step.batch, T, dpl, dql, dnm)
+            for l in range(L):
+                fd.fd_kv_append(ctx.h, step.batch, T, dkn[l], dvn[l], pools[l], step.num_pages, dpt, dpl, dql)
+                fd.fd_attn_draft_verify(ctx.h, step.batch, T, qs[l].cuda(), pools[l], step.num_pages, dpt, dpl, dql, dnm, outs[l])
+            fd.fd_plan_unpin(ctx.h)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            for l in range(L):
+                exp_bits = oracle.kv_append(dkn[l].cpu(), dvn[l].cpu(), kvs[l], step.page_table, step.prefix_lens, step.q_lens)
+                np.testing.assert_array_equal(pools[l].cpu().view(torch.int16).numpy().view(np.uint16), exp_bits)
+                kv_ref = torch.from_numpy(exp_bits.view(np.int16)).view(torch.bfloat16)
+                ref = oracle.attn(qs[l], kv_ref, step.page_table, step.prefix_lens, step.q_lens, step.n_mask)
+                assert_close(outs[l].float().cpu().numpy(), ref, f"layer {l} rep {rep}")
+
+
 def test_pinned_plan_serves_every_layer_and_is_dropped_on_other_lengths():
     """fd_plan_pin: several attention calls reuse one work list; a call with other lengths recomputes it."""
     step = wl.workload(2)
