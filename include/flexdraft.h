@@ -168,8 +168,8 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * Consecutive attention calls under one pin overlap on the device: a call starts while the call before it is still
  * finishing, and -- where its range of KV tiles is short -- reads its q and its cache ahead of that call's completion,
  * provided no earlier call since the pin wrote them (the library compares the `out` ranges of those calls with q and
- * kv_cache of this one; fd_kv_append in between, which writes the cache, switches the read-ahead off for the next
- * call).  fd_kv_append itself, behind an attention call of the chain, copies while that call finishes (its k_new /
+ * kv_cache of this one; behind fd_kv_append, which writes the query block's own slots of the cache, the tiles that
+ * lie wholly in the prefix are still read ahead, the ones that reach into the block after the append has completed).  fd_kv_append itself, behind an attention call of the chain, copies while that call finishes (its k_new /
  * v_new are checked against those `out` ranges in the same way).  Every write of an attention call (out, scratch)
  * waits for the launch before it, and the append waits for it before it ends, so results are those of calls run one
  * after the other.  What the library cannot see is a buffer written by the CALLER's own asynchronous work on another

@@ -476,12 +476,13 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     // ... and so may q and the cache, if no call of the chain writes them: the attention calls before this one write
     // their `out` (several of them may still be running: each starts as the one before it retires CTAs, and waits for
     // it only before its own first write), the append writes the cache
-    if (p.early && tc && !c->chain_append) {
+    if (p.early && tc) {
         const uintptr_t q0 = reinterpret_cast<uintptr_t>(q), q1 = q0 + (size_t)total_q_rows * p.Hq * p.d * 2;
         const uintptr_t k0 = reinterpret_cast<uintptr_t>(kv_cache), k1 = k0 + (size_t)num_pages * 2 * p.Hkv * 16 * p.d * 2;
         bool clash = c->chain_out.size() >= 1024;  // (a chain that long is not a step of a model: stop keeping track)
         for (const auto& w : c->chain_out) clash = clash || (w.first < q1 && q0 < w.second) || (w.first < k1 && k0 < w.second);
-        if (!clash) p.early = 2;
+        // (behind the append, which writes the block's own slots of this cache: everything but those is read ahead)
+        if (!clash) p.early = c->chain_append ? 3 : 2;
     }
     if (total_q_rows > 0 && c->chain_out.size() < 1024) {
         const uintptr_t o0 = reinterpret_cast<uintptr_t>(out);

@@ -245,7 +245,9 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
     bool ok = true;
     // p.early: the first piece and its first page ids are looked up while the launch before this one may still run;
     // p.early == 2: so is the KV pool itself -- that launch is known not to write it -- and this warp waits for it
-    // only if it has something to write (a sequence to flag)
+    // only if it has something to write (a sequence to flag); p.early == 3: that launch is the KV append, which
+    // writes the query block's own slots and nothing else: tiles of the prefix are read ahead, the wait comes before
+    // the first tile that reaches into the block (pages are 16 tokens, tiles 128: no page lies in both kinds)
     bool waited = !p.early;
     int bad_early = -1;
     while (w.t < e_c && ok) {
@@ -260,7 +262,7 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             if (!(j < pc.nt && pos < pc.kv_len)) return -1;
             int id = table[pos >> 4];
             if ((unsigned)id >= (unsigned)p.num_pages) {  // never form an address from a bad id
-                if (!waited && p.early == 2) { wait_prior_launch(); waited = true; }
+                if (!waited && p.early >= 2) { wait_prior_launch(); waited = true; }
                 if (waited) flag_sequence(p, pc.b); else bad_early = pc.b;  // (no global write ahead of the prior launch)
                 *bad = 1;
                 id = 0;
@@ -272,7 +274,7 @@ __device__ __forceinline__ void load_role(const CUtensorMap& tmap, const AttnPar
             const int g = w.g0 + j, st = g % C::kStages, use = g / C::kStages;
             if (j > 0 && (j & 3) == 0) { ids_cur = ids_next; ids_next = load_ids((j >> 2) + 1); }
             const int phys = __shfl_sync(0xffffffffu, ids_cur, (j & 3) * 8 + pg);
-            if (!waited && p.early != 2) {  // the KV pool may be written by the launch before this one (the KV append)
+            if (!waited && (p.early == 1 || (p.early == 3 && (pc.tile0 + j + 1) * kTileTokens > pc.n))) {  // the launch before this one may write what this tile holds
                 wait_prior_launch();
                 waited = true;
                 if (bad_early >= 0) flag_sequence(p, bad_early);
@@ -328,7 +330,7 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
     int issued = 0;
     Piece pc = decode_piece(p, n_rb, w.t, s_c, e_c, cta, w.b);
     if (lane == 0) publish_piece(bars, ring, 0, pc);
-    if (p.early == 1) wait_prior_launch();  // q may be written by it (p.early == 2: it is known not to be)
+    if (p.early == 1) wait_prior_launch();  // q may be written by it (p.early >= 2: it is known not to be)
     while (w.t < e_c) {
         if (w.piece > 0 && !wait_all(&bars->q_free, (w.piece - 1) & 1, abort)) break;
         const int nbox = (pc.Lv + bt - 1) / bt;
@@ -365,7 +367,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
     constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
-    if (p.early == 1) wait_prior_launch();  // (this role touches shared and tensor memory only; p.early == 2 lets it run ahead)
+    if (p.early == 1) wait_prior_launch();  // (this role touches shared and tensor memory only; p.early >= 2 lets it run ahead)
     const uint64_t qd0 = make_smem_desc(smem_u32(sq), 16, 1024);
     const int s_c = rg.s_c, e_c = rg.e_c;
     Walk w = {s_c, 0, {0, 0}, 0, rg.first};
@@ -653,7 +655,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
     // before any global write of this role (scratch, counters, out).  p.early == 2: the tiles of the first piece may be
     // worked through meanwhile -- tensor and shared memory only -- and the wait comes before its ticket and epilogue
     if (p.early == 1) wait_prior_launch();
-    bool prior_done = p.early != 2;
+    bool prior_done = p.early < 2;
     Walk w = {s_c, 0, {0, 0}, 0, 0};
     while (w.t < e_c) {
         // one thread waits for the descriptor, so that all 256 take the same decision
@@ -1133,7 +1135,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     // Reading q and the cache ahead of the launch before this one pays where a call is short (its start and the tail
     // of the call before it overlap); a CTA with a long range gains nothing and only takes bandwidth from the
     // stragglers of that call, which everyone then waits for (measured: + 1.5 % on 222 tiles per CTA).
-    if (p.early == 2 && rg.e_c - rg.s_c > kEarlyLoadMaxTiles) p.early = 1;
+    if (p.early >= 2 && rg.e_c - rg.s_c > kEarlyLoadMaxTiles) p.early = 1;
     if (rg.s_c >= rg.e_c && !cl_idle) {  // uniform (over the cluster too): no tile for this CTA, or nothing at all
         if (p.early) wait_prior_launch();
         if (total == 0 && fatal) {  // inconsistent lengths: a defined output, zeros

@@ -92,6 +92,8 @@ struct AttnParams {
                       //    before that launch has completed (everything else waits for it)
                       // 2: nor does any call of that chain write q or the cache of this one: they may be read early too,
                       //    and the first piece worked through; the call waits before its first write to global memory
+                      // 3: as 2, but the launch before this one is the KV append of this cache: tiles of the prefix are
+                      //    read early, a tile that reaches into the query block after the wait
     int* status;
 };
 
