@@ -143,6 +143,8 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptParams p, int chunks_
     __syncthreads();
     if (!last) return;
     __threadfence();
+    // (one CTA that waits is enough to keep this launch from completing before the one it was chained to)
+    if (p.chained) asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ int sm[];            // cu_c [B+1], then first_mismatch [B]
     accept_scan(p, sm);
 }
@@ -159,7 +161,21 @@ void launch_accept(const AcceptParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
     if (p.total_rows == 0) { accept_empty_kernel<<<1, 256, 0, s>>>(p); return; }
     const int chunks = (p.vocab + kAcceptChunk - 1) / kAcceptChunk;
-    accept_kernel<<<p.total_rows * chunks, 256, (2 * p.batch + 1) * sizeof(int), s>>>(p, chunks);
+    if (!p.chained) {
+        accept_kernel<<<p.total_rows * chunks, 256, (2 * p.batch + 1) * sizeof(int), s>>>(p, chunks);
+        return;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.total_rows * chunks);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = (2 * p.batch + 1) * sizeof(int);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, accept_kernel, p, chunks);
 }
 
 }  // namespace fd

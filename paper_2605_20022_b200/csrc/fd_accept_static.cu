@@ -67,6 +67,7 @@ extern "C" fd_status fd_verify_accept_static(int vocab, int batch, int total_can
     p.batch = batch; p.total_rows = total_cand_rows; p.vocab = vocab;
     p.logits = logits; p.drafts = draft_tokens; p.q_lens = q_lens; p.n_mask = n_mask;
     p.accepted = accepted_len; p.bonus = bonus_token;
+    p.chained = 0;
     p.keys = scratch;
     p.ticket = reinterpret_cast<unsigned int*>(scratch + FD_STATIC_MAX_ROWS);
     p.status = device_status ? device_status : reinterpret_cast<int*>(scratch + FD_STATIC_MAX_ROWS + 1);

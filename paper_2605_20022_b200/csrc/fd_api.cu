@@ -44,6 +44,7 @@ struct fd_ctx {
     const int32_t *pin_pl, *pin_ql, *pin_nm, *pin_nb;
     bool pin_chain;    // the context's last launch was an attention or append call under the pinned plan (see AttnParams::early)
     bool chain_append; // ... and it was the append (which writes the cache the next attention call reads)
+    bool after_attn;   // the context's last launch was an attention call of the tensor-core kernel (it lets its dependents in early)
     std::vector<std::pair<uintptr_t, uintptr_t>> chain_out;  // [begin, end) of what the attention calls of the chain have written
     struct HostStage* host;  // staging for fd_step_host, nullptr until fd_host_reserve
 };
@@ -148,6 +149,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->tc_choice = cfg->attn_path >= FD_ATTN_TCGEN05 ? cfg->attn_path : FD_ATTN_TCGEN05;
     c->last_mode = -1;
     c->chain_append = false;
+    c->after_attn = false;
     c->epoch = 0;
     c->attn_path = (cfg->attn_path == FD_ATTN_SIMT || !tc_ok) ? FD_ATTN_SIMT : FD_ATTN_TCGEN05;
     // SIMT kernel: two 74 KB CTAs fit an SM; tensor-core kernel: one persistent CTA per SM
@@ -489,6 +491,7 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
         c->chain_out.emplace_back(o0, o0 + (size_t)total_q_rows * p.Hq * p.d * 2);
     }
     c->chain_append = false;
+    c->after_attn = tc;
     c->pin_chain = reuse && c->pinned;
     if (c->attn_path == FD_ATTN_TCGEN05 && !tc) {
     } else if (tc) {
@@ -513,6 +516,7 @@ fd_status fd_plan_pin(fd_ctx* c, int batch, int total_q_rows, const int32_t* pre
     c->launches += 1;
     c->pinned = true;
     c->pin_chain = false;  // the first call it serves comes right behind the plan kernel and waits for it
+    c->after_attn = false;
     c->pin_batch = batch; c->pin_rows = total_q_rows;
     c->pin_pl = prefix_lens; c->pin_ql = q_lens; c->pin_nm = n_mask; c->pin_nb = n_blocks;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
@@ -558,7 +562,8 @@ fd_status fd_plan_unpin(fd_ctx* c) {
 fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const float* logits,
                            const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask,
                            int32_t* accepted_len, int32_t* bonus_token, void* stream) {
-    if (c) c->pin_chain = false;  // (not an attention or append call)
+    const bool after_attn = c && c->after_attn;  // (read before it is cleared: the sweep may be chained to that call)
+    if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || total_cand_rows < 0) return FD_ERR_INVALID_ARG;
     if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
     if (batch == 0) return total_cand_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
@@ -572,6 +577,10 @@ fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const floa
     p.logits = logits; p.drafts = draft_tokens; p.q_lens = q_lens; p.n_mask = n_mask;
     p.accepted = accepted_len; p.bonus = bonus_token;
     p.keys = c->keys; p.ticket = c->ticket; p.status = c->status;
+    // Right behind an attention call (the last layer's) the sweep need not wait for it: it reads the logits and the
+    // draft tokens, which that call does not write, into scratch of its own; only the scan, which writes the results,
+    // waits.  (Behind anything else this is an ordinary launch.)
+    p.chained = after_attn ? 1 : 0;
     fd::launch_accept(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
@@ -581,7 +590,7 @@ fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, con
                                   const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask, float temperature,
                                   const float* u_accept, const float* u_bonus, int32_t* accepted_len, int32_t* bonus_token,
                                   void* stream) {
-    if (c) c->pin_chain = false;  // (not an attention or append call)
+    if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || total_cand_rows < 0 || !(temperature > 0.f)) return FD_ERR_INVALID_ARG;
     if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
     if (batch == 0) return total_cand_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
@@ -604,7 +613,7 @@ fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, con
 
 fd_status fd_kv_commit(fd_ctx* c, int batch, int32_t* page_table, int32_t* prefix_lens, const int32_t* q_lens,
                        const int32_t* accepted_len, int32_t* freed_pages, int32_t* n_freed, void* stream) {
-    if (c) c->pin_chain = false;  // (not an attention or append call)
+    if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || !n_freed) return FD_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (batch == 0) return cudaMemsetAsync(n_freed, 0, sizeof(int32_t), s) == cudaSuccess ? FD_OK : FD_ERR_CUDA;
@@ -647,6 +656,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
     }
     fd::launch_kv_append(p, static_cast<cudaStream_t>(stream));
     c->chain_append = true;  // the next attention call must not read the cache ahead of this launch
+    c->after_attn = false;
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }
@@ -654,7 +664,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
 fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blocks, const float* draft_logits,
                           const float* bias, const int32_t* n_mask, const int32_t* n_blocks, float threshold,
                           int32_t* mask_tokens, float* mask_probs, int32_t* keep_len, void* stream) {
-    if (c) c->pin_chain = false;  // (not an attention or append call)
+    if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || total_mask_rows < 0 || total_mask_rows > c->max_rows || max_blocks < 1)
         return FD_ERR_INVALID_ARG;
     if (batch == 0) return total_mask_rows == 0 ? FD_OK : FD_ERR_INVALID_ARG;
@@ -675,7 +685,7 @@ fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blo
 fd_status fd_select_branch(fd_ctx* c, int batch, int max_block_len, const int32_t* mask_tokens, const int32_t* q_lens,
                            const int32_t* n_mask, const int32_t* n_blocks, const int32_t* accepted_len,
                            int32_t* next_draft, int32_t* next_len, void* stream) {
-    if (c) c->pin_chain = false;  // (not an attention or append call)
+    if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || max_block_len < 1) return FD_ERR_INVALID_ARG;
     if (batch == 0) return FD_OK;
     if (!q_lens || !n_mask || !accepted_len || !next_draft || !next_len) return FD_ERR_INVALID_ARG;
@@ -689,7 +699,7 @@ fd_status fd_select_branch(fd_ctx* c, int batch, int max_block_len, const int32_
 }
 
 fd_status fd_selftest_wait_timeout(fd_ctx* c, int limit_ms, void* stream) {
-    if (c) c->pin_chain = false;  // (not an attention or append call)
+    if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || limit_ms < 1 || limit_ms > 1000) return FD_ERR_INVALID_ARG;
     fd::launch_wait_timeout_selftest(c->status, (unsigned long long)limit_ms * 1000000ull, static_cast<cudaStream_t>(stream));
     c->launches += 1;

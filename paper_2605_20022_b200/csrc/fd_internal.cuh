@@ -351,6 +351,9 @@ struct AcceptParams {
     unsigned long long* keys;  // [max rows] running (value, index) maxima, zero between calls
     unsigned int* ticket;      // [1] CTAs finished, zero between calls
     int* status;
+    int chained;               // 1: launched as a programmatic dependent of the attention call before it: the sweep -- logits
+                               //    in, private scratch out -- runs while that call finishes; the CTA that finishes last
+                               //    waits for it before the scan writes the results
 };
 void launch_accept(const AcceptParams& p, cudaStream_t s);
 
