@@ -302,7 +302,7 @@ fd_status fd_select_branch(fd_ctx* ctx, int batch, int max_block_len, const int3
  *   accepted_len, bonus_token   device, [B] int32, overwritten
  *
  * Inconsistent lengths: every accepted_len / bonus_token is set to -1 (FD_DEV_BAD_LENGTHS).
-  * Right behind an attention call of the same context the sweep over the logits starts while that call is still
+ * Right behind an attention call of the same context the sweep over the logits starts while that call is still
  * finishing (neither reads what the other writes); the results are written after it has completed.
  */
 fd_status fd_verify_accept(fd_ctx* ctx, int batch, int total_cand_rows,
