@@ -240,6 +240,9 @@ class DeviceStep:
         G = s.n_q_heads // s.n_kv_heads
         self.ctx = fd.fd_create(s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab, B, self.max_q_len,
                                 step.max_pages_per_seq, s.page_size, 0.0, attn_path)
+        # every step below launches its calls back to back on one stream, nothing of the benchmark's own between them
+        # (event records for timing apart): consecutive calls may overlap
+        fd.fd_calls_back_to_back(self.ctx, True)
         self.attn_events = []
 
     def close(self):

@@ -165,7 +165,7 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
  * itself when it reports that bit).  fd_kv_commit rewrites prefix_lens and therefore drops the pin
  * itself: the first attention call of the next step plans afresh (or is preceded by a new fd_plan_pin).
  * fd_kv_append leaves the lengths alone and keeps the pin.
- * Consecutive attention calls under one pin overlap on the device: a call starts while the call before it is still
+ * Consecutive attention calls under one pin overlap on the device (fd_calls_back_to_back): a call starts while the call before it is still
  * finishing, and -- where its range of KV tiles is short -- reads its q and its cache ahead of that call's completion,
  * provided no earlier call since the pin wrote them (the library compares the `out` ranges of those calls with q and
  * kv_cache of this one; behind fd_kv_append, which writes the query block's own slots of the cache, the tiles that
@@ -184,6 +184,19 @@ fd_status fd_attn_draft_verify(fd_ctx* ctx, int batch, int total_q_rows,
 fd_status fd_plan_pin(fd_ctx* ctx, int batch, int total_q_rows, const int32_t* prefix_lens, const int32_t* q_lens,
                       const int32_t* n_mask, const int32_t* n_blocks, void* stream);
 fd_status fd_plan_unpin(fd_ctx* ctx);
+
+/*
+ * The caller's promise that lets consecutive calls overlap (default: off).  While on, the caller launches nothing of
+ * its own on the stream between two calls on this context -- the calls are back to back, as the layers of a
+ * benchmark step are, or as they are where everything between two attention calls is itself ordered before the first
+ * of them.  The library then knows that the launch before a call is its own, and what that launch writes: see
+ * fd_plan_pin (attention calls read q and the cache ahead, fd_kv_append copies under the tail of the attention call
+ * before it) and fd_verify_accept (its sweep runs under the tail of the last attention call).  Off, every call
+ * waits for the launch before it before it reads anything but the pinned plan, the lengths and the page table: a
+ * kernel of the caller's between two calls may then be any kernel, one that releases its dependents early included.
+ * fd_step_host and fd_step_host_append, which launch nothing but this library's kernels, behave as if it were on.
+ */
+fd_status fd_calls_back_to_back(fd_ctx* ctx, int on);
 
 /*
  * Host-side view of the work split, for schedulers and tests: how fd_attn_draft_verify cuts the 128-token KV
@@ -302,8 +315,8 @@ fd_status fd_select_branch(fd_ctx* ctx, int batch, int max_block_len, const int3
  *   accepted_len, bonus_token   device, [B] int32, overwritten
  *
  * Inconsistent lengths: every accepted_len / bonus_token is set to -1 (FD_DEV_BAD_LENGTHS).
- * Right behind an attention call of the same context the sweep over the logits starts while that call is still
- * finishing (neither reads what the other writes); the results are written after it has completed.
+ * Right behind an attention call of the same context (fd_calls_back_to_back) the sweep over the logits starts while that
+ * call is still finishing (neither reads what the other writes); the results are written after it has completed.
  */
 fd_status fd_verify_accept(fd_ctx* ctx, int batch, int total_cand_rows,
                            const float* logits, const int32_t* draft_tokens,

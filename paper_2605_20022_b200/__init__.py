@@ -25,7 +25,7 @@ FD_TC_PLANNED, FD_TC_SELF_PLANNED, FD_TC_CLUSTER = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_attn_last_mode", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_step_host_append", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_verify_accept_sample", "fd_plan_ranges_host"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_step_host_append", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_calls_back_to_back", "fd_verify_accept_sample", "fd_plan_ranges_host"]
 
 
 class fd_config(ctypes.Structure):
@@ -70,6 +70,7 @@ def load() -> ctypes.CDLL:
         lib.fd_plan_ranges_host.argtypes = [ci, ci, vp, vp, ci, vp]
         lib.fd_plan_pin.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp]
         lib.fd_plan_unpin.argtypes = [vp]
+        lib.fd_calls_back_to_back.argtypes = [vp, ci]
         lib.fd_kv_append.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp]
         lib.fd_draft_select.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
         lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 14
@@ -260,6 +261,10 @@ def fd_last_device_status(ctx, stream=None) -> int:
     code = ctypes.c_int32(0)
     _check("fd_last_device_status", load().fd_last_device_status(ctx, ctypes.byref(code), _stream(stream)), True)
     return code.value
+
+
+def fd_calls_back_to_back(ctx, on=True) -> int:
+    return _check("fd_calls_back_to_back", load().fd_calls_back_to_back(ctx, 1 if on else 0), True)
 
 
 def fd_attn_path(ctx) -> int:

@@ -45,6 +45,7 @@ struct fd_ctx {
     bool pin_chain;    // the context's last launch was an attention or append call under the pinned plan (see AttnParams::early)
     bool chain_append; // ... and it was the append (which writes the cache the next attention call reads)
     bool after_attn;   // the context's last launch was an attention call of the tensor-core kernel (it lets its dependents in early)
+    bool back_to_back; // fd_calls_back_to_back: nothing but this context's own launches sits between its calls on the stream
     std::vector<std::pair<uintptr_t, uintptr_t>> chain_out;  // [begin, end) of what the attention calls of the chain have written
     struct HostStage* host;  // staging for fd_step_host, nullptr until fd_host_reserve
 };
@@ -150,6 +151,7 @@ fd_status fd_create(fd_ctx** out, const fd_config* cfg) {
     c->last_mode = -1;
     c->chain_append = false;
     c->after_attn = false;
+    c->back_to_back = false;
     c->epoch = 0;
     c->attn_path = (cfg->attn_path == FD_ATTN_SIMT || !tc_ok) ? FD_ATTN_SIMT : FD_ATTN_TCGEN05;
     // SIMT kernel: two 74 KB CTAs fit an SM; tensor-core kernel: one persistent CTA per SM
@@ -315,6 +317,12 @@ fd_status fd_step_host_append(fd_ctx* c, int batch, int total_q_rows, int total_
         (total_cand_rows > 0 && (!logits_host || !draft_tokens_host)))
         return FD_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // between the calls of this step the stream holds nothing but this library's launches and event waits
+    struct BackToBack {
+        fd_ctx* c; bool saved;
+        explicit BackToBack(fd_ctx* c_) : c(c_), saved(c_->back_to_back) { c->back_to_back = true; }
+        ~BackToBack() { c->back_to_back = saved; }
+    } back_to_back(c);
     const size_t qb = (size_t)total_q_rows * c->cfg.n_q_heads * c->cfg.head_dim * 2;
     const size_t ptb = (size_t)batch * c->cfg.max_pages_per_seq * 4, lb = (size_t)batch * 4;
     const size_t n_fr = (size_t)batch * ((c->cfg.max_q_len + 15) / 16 + 1);
@@ -478,7 +486,7 @@ fd_status fd_attn_draft_verify_blocks(fd_ctx* c, int batch, int total_q_rows, co
     // ... and so may q and the cache, if no call of the chain writes them: the attention calls before this one write
     // their `out` (several of them may still be running: each starts as the one before it retires CTAs, and waits for
     // it only before its own first write), the append writes the cache
-    if (p.early && tc) {
+    if (p.early && tc && c->back_to_back) {
         const uintptr_t q0 = reinterpret_cast<uintptr_t>(q), q1 = q0 + (size_t)total_q_rows * p.Hq * p.d * 2;
         const uintptr_t k0 = reinterpret_cast<uintptr_t>(kv_cache), k1 = k0 + (size_t)num_pages * 2 * p.Hkv * 16 * p.d * 2;
         bool clash = c->chain_out.size() >= 1024;  // (a chain that long is not a step of a model: stop keeping track)
@@ -552,6 +560,12 @@ fd_status fd_plan_ranges_host(int batch, int n_kv_heads, const int32_t* prefix_l
     return FD_OK;
 }
 
+fd_status fd_calls_back_to_back(fd_ctx* c, int on) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    c->back_to_back = on != 0;
+    return FD_OK;
+}
+
 fd_status fd_plan_unpin(fd_ctx* c) {
     if (!c) return FD_ERR_INVALID_ARG;
     c->pinned = false;
@@ -580,7 +594,7 @@ fd_status fd_verify_accept(fd_ctx* c, int batch, int total_cand_rows, const floa
     // Right behind an attention call (the last layer's) the sweep need not wait for it: it reads the logits and the
     // draft tokens, which that call does not write, into scratch of its own; only the scan, which writes the results,
     // waits.  (Behind anything else this is an ordinary launch.)
-    p.chained = after_attn ? 1 : 0;
+    p.chained = (after_attn && c->back_to_back) ? 1 : 0;
     fd::launch_accept(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
@@ -647,7 +661,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
     // cache that only the NEXT attention call reads.  Its copies then run under that call's merge tail; it waits for the
     // call before it ends, so the attention call behind it, which waits for the append, has waited for both.
     p.chained = 0;
-    if (c->pin_chain && c->pinned && !c->chain_append) {
+    if (c->back_to_back && c->pin_chain && c->pinned && !c->chain_append) {
         const size_t nb = (size_t)total_q_rows * p.Hkv * p.d * 2;
         const uintptr_t a0 = reinterpret_cast<uintptr_t>(k_new), b0 = reinterpret_cast<uintptr_t>(v_new);
         bool clash = c->chain_out.size() >= 1024;

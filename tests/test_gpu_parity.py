@@ -728,6 +728,7 @@ def test_chain_of_calls_whose_output_is_the_next_query(idx):
     kvs = [wl.make_kv(step, l) for l in range(L)]
     q0 = wl.make_q(step)
     with Ctx(step) as ctx:
+        fd.fd_calls_back_to_back(ctx.h, True)                      # nothing but the library's launches between the calls below
         dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
         dkv = [k.cuda() for k in kvs]
         dq0 = q0.cuda()
@@ -761,6 +762,7 @@ def test_chained_append_whose_input_is_the_previous_output():
     kn = [torch.randn((T, s.n_kv_heads, s.head_dim), generator=g).bfloat16() for _ in range(L)]
     vn = [torch.randn((T, s.n_kv_heads, s.head_dim), generator=g).bfloat16() for _ in range(L)]
     with Ctx(step) as ctx:
+        fd.fd_calls_back_to_back(ctx.h, True)                      # nothing but the library's launches between the calls below
         dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
         for rep in range(2):
             pools = [k.cuda() for k in kvs]
