@@ -187,9 +187,9 @@ fd_status fd_plan_unpin(fd_ctx* ctx);
 
 /*
  * The caller's promise that lets consecutive calls overlap (default: off).  While on, the caller launches nothing of
- * its own on the stream between two calls on this context -- the calls are back to back, as the layers of a
- * benchmark step are, or as they are where everything between two attention calls is itself ordered before the first
- * of them.  The library then knows that the launch before a call is its own, and what that launch writes: see
+ * its own on the stream between two calls on this context (a call on another context counts as the caller's own) --
+ * the calls are back to back, as the layers of a benchmark step are, or as they are where everything between two
+ * attention calls is itself ordered before the first of them.  The library then knows that the launch before a call is its own, and what that launch writes: see
  * fd_plan_pin (attention calls read q and the cache ahead, fd_kv_append copies under the tail of the attention call
  * before it) and fd_verify_accept (its sweep runs under the tail of the last attention call).  Off, every call
  * waits for the launch before it before it reads anything but the pinned plan, the lengths and the page table: a
