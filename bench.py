@@ -293,6 +293,19 @@ class DeviceStep:
         fd.fd_kv_commit(self.ctx, st.batch, self.pt, self.pl, self.ql, self.acc, self.freed, self.n_freed)
 
 
+    def run_one_call(self, append=False):
+        """The same step through fd_step_device: one C call launches every kernel of it (no Python between launches)."""
+        fd, st = self.fd, self.step
+        self.pt, self.pl = self.slots[self.cur % len(self.slots)]
+        self.cur += 1
+        if not hasattr(self, "_arr"):
+            self._arr = {k: fd.fd_ptr_array(getattr(self, k)) for k in ("q", "kv", "out", "k_new", "v_new")}
+        a = self._arr
+        fd.fd_step_device(self.ctx, st.batch, st.total_q_rows, st.total_cand_rows, a["q"], a["k_new"] if append else None,
+                          a["v_new"] if append else None, a["kv"], a["out"], st.num_pages, self.pt, self.pl, self.ql, self.nm, self.nb,
+                          self.logits, self.drafts, self.acc, self.bon, self.freed, self.n_freed)
+
+
 class HostStep:
     """End-to-end leg: one C-ABI call (fd_step_host) per step, every per-step input in pinned host
     memory and every result back on the host inside the timed region.  The KV cache is decode state
@@ -493,6 +506,10 @@ def decode_step_many_layers(torch, step, device, peak, attn_path, layers, reps):
         for _ in range(3):
             ds.run()
         ms_step = timed_region(torch, None, ds.run, reps, prepare=ds.restore) / reps
+        ds.restore(); ds.run_one_call()
+        ms_one = timed_region(torch, None, ds.run_one_call, reps, prepare=ds.restore) / reps
+        ds.restore(); ds.run_one_call(append=True)
+        ms_one_app = timed_region(torch, None, lambda: ds.run_one_call(append=True), reps, prepare=ds.restore) / reps
         g = capture_step_graph(torch, ds)
         g.replay()
         ms_step_g = timed_region(torch, None, g.replay, reps) / reps
@@ -520,6 +537,7 @@ def decode_step_many_layers(torch, step, device, peak, attn_path, layers, reps):
     nbytes = step.attn_bytes()
     per_call, per_call_g = ms_attn * 1e3 / layers, ms_attn_g * 1e3 / layers
     return {"layers": layers, "us_per_step": ms_step * 1e3, "us_per_step_cuda_graph_replay": ms_step_g * 1e3,
+            "us_per_step_one_call": ms_one * 1e3, "us_per_step_one_call_with_kv_append": ms_one_app * 1e3,
             "us_per_step_with_kv_append": ms_app * 1e3, "us_per_step_with_kv_append_cuda_graph_replay": ms_app_g * 1e3,
             "us_per_attn_call": per_call, "us_per_attn_call_cuda_graph_replay": per_call_g,
             "attn_GBps": nbytes / per_call_g / 1e3, "frac_of_measured_peak": nbytes / per_call_g / 1e3 / peak,
@@ -698,6 +716,10 @@ def run_ours(args, step, rank, world, dist):
     ds.restore()
     ds.run(append=True)
     ms_append = timed_region(torch, None, lambda: ds.run(append=True), n_app, flush, prepare=ds.restore) / n_app
+    # and the step launched by ONE call of the library (fd_step_device: every launch of the step from C)
+    ds.restore()
+    ds.run_one_call()
+    ms_one_call = timed_region(torch, None, ds.run_one_call, n_app, flush, prepare=ds.restore) / n_app
 
     hs = HostStep(ds)
     for _ in range(2):
@@ -753,6 +775,7 @@ def run_ours(args, step, rank, world, dist):
                    "mask_rows_in_last_10_layers_only": layer_split,
                    "us_per_attn_call_alone_event_bracketed": statistics.mean(attn_ms) * 1e3,
                    "us_per_step_with_kv_append": ms_append * 1e3,
+                   "us_per_step_one_call_fd_step_device": ms_one_call * 1e3,
                    "step_of_36_layer_model": many, "per_workload": per_workload},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(step.name) if resolved == "tcgen05" else None, "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,

@@ -186,6 +186,27 @@ fd_status fd_plan_pin(fd_ctx* ctx, int batch, int total_q_rows, const int32_t* p
 fd_status fd_plan_unpin(fd_ctx* ctx);
 
 /*
+ * A whole step on device buffers in one call: for every layer the KV append (if k_new / v_new are given) and the
+ * attention, on one work list (fd_plan_pin), then fd_verify_accept and fd_kv_commit -- the sequence of Sec. 4.1
+ * "Inference" / Sec. 3, launched from C with nothing between the launches, so that consecutive calls overlap as under
+ * fd_calls_back_to_back.  Everything a layer-by-layer caller gets from the single calls, this gives bit for bit.
+ *
+ *   q, k_new, v_new, kv_caches, out   HOST arrays of n_layers DEVICE pointers (k_new and v_new both NULL: no append);
+ *                                     shapes per layer as fd_attn_draft_verify_blocks / fd_kv_append
+ *   page_table, prefix_lens           device, in/out (the commit rewrites them)
+ *   everything else                   device, as in the single calls; n_blocks may be NULL
+ *
+ * Asynchronous on `stream` like the single calls; errors as theirs (the first one is returned, later launches of the
+ * step are skipped).
+ */
+fd_status fd_step_device(fd_ctx* ctx, int batch, int total_q_rows, int total_cand_rows, int n_layers,
+                         const void* const* q, const void* const* k_new, const void* const* v_new,
+                         void* const* kv_caches, void* const* out, int num_pages, int32_t* page_table,
+                         int32_t* prefix_lens, const int32_t* q_lens, const int32_t* n_mask, const int32_t* n_blocks,
+                         const float* logits, const int32_t* draft_tokens, int32_t* accepted_len,
+                         int32_t* bonus_token, int32_t* freed_pages, int32_t* n_freed, void* stream);
+
+/*
  * The caller's promise that lets consecutive calls overlap (default: off).  While on, the caller launches nothing of
  * its own on the stream between two calls on this context (a call on another context counts as the caller's own) --
  * the calls are back to back, as the layers of a benchmark step are, or as they are where everything between two

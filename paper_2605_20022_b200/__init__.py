@@ -25,7 +25,7 @@ FD_TC_PLANNED, FD_TC_SELF_PLANNED, FD_TC_CLUSTER = 0, 1, 2
 
 EXPORTS = ["fd_create", "fd_destroy", "fd_attn_draft_verify", "fd_verify_accept", "fd_kv_commit",
            "fd_last_device_status", "fd_attn_path", "fd_attn_last_mode", "fd_launch_count", "fd_status_string",
-           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_step_host_append", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_calls_back_to_back", "fd_verify_accept_sample", "fd_plan_ranges_host"]
+           "fd_verify_accept_static", "fd_host_reserve", "fd_step_host", "fd_step_host_append", "fd_step_device", "fd_selftest_wait_timeout", "fd_attn_draft_verify_blocks", "fd_select_branch", "fd_draft_select", "fd_kv_append", "fd_plan_pin", "fd_plan_unpin", "fd_calls_back_to_back", "fd_verify_accept_sample", "fd_plan_ranges_host"]
 
 
 class fd_config(ctypes.Structure):
@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
         lib.fd_plan_pin.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp]
         lib.fd_plan_unpin.argtypes = [vp]
         lib.fd_calls_back_to_back.argtypes = [vp, ci]
+        lib.fd_step_device.argtypes = [vp, ci, ci, ci, ci] + [ctypes.POINTER(vp)] * 5 + [ci] + [vp] * 12
         lib.fd_kv_append.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp]
         lib.fd_draft_select.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
         lib.fd_step_host.argtypes = [vp, ci, ci, ci, ci, ctypes.POINTER(vp), ci] + [vp] * 14
@@ -251,6 +252,23 @@ def fd_step_host_append(ctx, batch, total_q_rows, total_cand_rows, kv_caches, nu
                                       _ptr(q_lens_host), _ptr(n_mask_host), _ptr(n_blocks_host), _ptr(accepted_len_host),
                                       _ptr(bonus_token_host), _ptr(freed_pages_host), _ptr(n_freed_host), _stream(stream))
     return _check("fd_step_host_append", code, raise_on_error)
+
+
+def fd_ptr_array(tensors):
+    """A host array of the device addresses of `tensors` (for fd_step_device: build once, pass every step)."""
+    return (ctypes.c_void_p * len(tensors))(*[_ptr(t) for t in tensors])
+
+
+def fd_step_device(ctx, batch, total_q_rows, total_cand_rows, q, k_new, v_new, kv_caches, out, num_pages, page_table, prefix_lens,
+                   q_lens, n_mask, n_blocks, logits, draft_tokens, accepted_len, bonus_token, freed_pages, n_freed, stream=None,
+                   raise_on_error=True) -> int:
+    """One step on device buffers.  q, k_new, v_new, kv_caches, out: lists of per-layer tensors, or arrays from fd_ptr_array."""
+    arr = lambda x: None if x is None else (x if isinstance(x, ctypes.Array) else fd_ptr_array(x))
+    qa, ka, va, kva, oa = arr(q), arr(k_new), arr(v_new), arr(kv_caches), arr(out)
+    code = load().fd_step_device(ctx, batch, total_q_rows, total_cand_rows, len(kva), qa, ka, va, kva, oa, num_pages, _ptr(page_table),
+                                 _ptr(prefix_lens), _ptr(q_lens), _ptr(n_mask), _ptr(n_blocks), _ptr(logits), _ptr(draft_tokens),
+                                 _ptr(accepted_len), _ptr(bonus_token), _ptr(freed_pages), _ptr(n_freed), _stream(stream))
+    return _check("fd_step_device", code, raise_on_error)
 
 
 def fd_selftest_wait_timeout(ctx, limit_ms, stream=None) -> None:

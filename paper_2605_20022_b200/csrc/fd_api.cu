@@ -560,6 +560,37 @@ fd_status fd_plan_ranges_host(int batch, int n_kv_heads, const int32_t* prefix_l
     return FD_OK;
 }
 
+fd_status fd_step_device(fd_ctx* c, int batch, int total_q_rows, int total_cand_rows, int n_layers, const void* const* q,
+                         const void* const* k_new, const void* const* v_new, void* const* kv_caches, void* const* out,
+                         int num_pages, int32_t* page_table, int32_t* prefix_lens, const int32_t* q_lens, const int32_t* n_mask,
+                         const int32_t* n_blocks, const float* logits, const int32_t* draft_tokens, int32_t* accepted_len,
+                         int32_t* bonus_token, int32_t* freed_pages, int32_t* n_freed, void* stream) {
+    if (!c || n_layers <= 0 || !q || !kv_caches || !out || (k_new == nullptr) != (v_new == nullptr)) return FD_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l)
+        if (!kv_caches[l] || (total_q_rows > 0 && (!q[l] || !out[l])) || (k_new && total_q_rows > 0 && (!k_new[l] || !v_new[l])))
+            return FD_ERR_INVALID_ARG;
+    // the stream holds nothing but this library's launches between the calls below
+    struct BackToBack {
+        fd_ctx* c; bool saved;
+        explicit BackToBack(fd_ctx* c_) : c(c_), saved(c_->back_to_back) { c->back_to_back = true; }
+        ~BackToBack() { c->back_to_back = saved; }
+    } back_to_back(c);
+    fd_status st = FD_OK;
+    if (n_layers > 1) st = fd_plan_pin(c, batch, total_q_rows, prefix_lens, q_lens, n_mask, n_blocks, stream);  // one work list for all layers
+    for (int l = 0; l < n_layers && st == FD_OK; ++l) {
+        if (k_new && total_q_rows > 0)
+            st = fd_kv_append(c, batch, total_q_rows, k_new[l], v_new[l], kv_caches[l], num_pages, page_table, prefix_lens, q_lens, stream);
+        if (st == FD_OK)
+            st = fd_attn_draft_verify_blocks(c, batch, total_q_rows, q[l], kv_caches[l], num_pages, page_table, prefix_lens, q_lens, n_mask,
+                                             n_blocks, out[l], stream);
+    }
+    if (n_layers > 1) fd_plan_unpin(c);  // (no launch; the commit below would drop the pin anyway)
+    if (st != FD_OK) return st;
+    st = fd_verify_accept(c, batch, total_cand_rows, logits, draft_tokens, q_lens, n_mask, accepted_len, bonus_token, stream);
+    if (st != FD_OK) return st;
+    return fd_kv_commit(c, batch, page_table, prefix_lens, q_lens, accepted_len, freed_pages, n_freed, stream);
+}
+
 fd_status fd_calls_back_to_back(fd_ctx* c, int on) {
     if (!c) return FD_ERR_INVALID_ARG;
     c->back_to_back = on != 0;

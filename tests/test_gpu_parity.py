@@ -417,6 +417,60 @@ def test_long_context_full_size_every_element(path):
             assert worst <= 2e-2, f"layer {layer}: worst (row, head) vector off by {worst:.3e} of its length"
 
 
+@pytest.mark.parametrize("append", [False, True])
+def test_device_buffer_step_in_one_call(append):
+    """fd_step_device: a 4-layer step -- (append,) attention per layer on one work list, accept, commit -- launched by
+    one C call, against the oracle; twice on the same context."""
+    shape = wl.Shape(32, 8, 128, 5000, n_layers=4)
+    step = wl.make_step("dev", shape, [700, 130, 2049, 0, 31], [32, 9, 20, 16, 1], [16, 0, 8, 0, 0], seed=19, p_match=0.7, extra_table_cols=1)
+    L, B, T, R = 4, step.batch, step.total_q_rows, step.total_cand_rows
+    g = torch.Generator().manual_seed(23)
+    qs = [wl.make_q(step, l) for l in range(L)]
+    kvs = [wl.make_kv(step, l) for l in range(L)]
+    kn = [torch.randn((T, 8, 128), generator=g).bfloat16() for _ in range(L)]
+    vn = [torch.randn((T, 8, 128), generator=g).bfloat16() for _ in range(L)]
+    logits, drafts, _ = wl.make_logits(step)
+    refs, pools_ref = [], []
+    for l in range(L):
+        kv_l = kvs[l]
+        if append:
+            bits = oracle.kv_append(kn[l], vn[l], kvs[l], step.page_table, step.prefix_lens, step.q_lens)
+            kv_l = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+            pools_ref.append(bits)
+        refs.append(oracle.attn(qs[l], kv_l, step.page_table, step.prefix_lens, step.q_lens, step.n_mask))
+    e_acc, e_bon, _ = oracle.accept(logits, drafts, step.q_lens, step.n_mask)
+    ept, epl, efreed = oracle.commit(step.page_table, step.prefix_lens, step.q_lens, e_acc)
+    with Ctx(step) as ctx:
+        dq = [t.cuda() for t in qs]; dk = [t.cuda() for t in kn]; dv = [t.cuda() for t in vn]
+        pools = [t.cuda() for t in kvs]
+        outs = [torch.full((T, 32, 128), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+        dpt, dpl = step.page_table.cuda(), step.prefix_lens.cuda()
+        dql, dnm = step.q_lens.cuda(), step.n_mask.cuda()
+        acc = torch.full((B,), -9, dtype=torch.int32, device="cuda"); bon = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+        freed = torch.full((B * 3,), -7, dtype=torch.int32, device="cuda"); nfr = torch.zeros(1, dtype=torch.int32, device="cuda")
+        before = fd.fd_launch_count(ctx.h)
+        fd.fd_step_device(ctx.h, B, T, R, dq, dk if append else None, dv if append else None, pools, outs, step.num_pages, dpt, dpl, dql, dnm,
+                          None, logits.cuda(), drafts.cuda(), acc, bon, freed, nfr)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        assert fd.fd_launch_count(ctx.h) - before == 1 + L * (2 if append else 1) + 2      # plan, (append,) attention per layer, accept, commit
+        for l in range(L):
+            assert_close(outs[l].float().cpu().numpy(), refs[l], f"layer {l}")
+            if append:
+                np.testing.assert_array_equal(pools[l].cpu().view(torch.int16).numpy().view(np.uint16), pools_ref[l])
+        np.testing.assert_array_equal(acc.cpu().numpy(), e_acc); np.testing.assert_array_equal(bon.cpu().numpy(), e_bon)
+        np.testing.assert_array_equal(dpt.cpu().numpy(), ept); np.testing.assert_array_equal(dpl.cpu().numpy(), epl)
+        n = int(nfr.item())
+        np.testing.assert_array_equal(freed[:n].cpu().numpy(), efreed)
+        # the same step again on restored tables: same bits (plan pinned and dropped inside the call both times)
+        dpt2, dpl2 = step.page_table.cuda(), step.prefix_lens.cuda()
+        outs2 = [torch.empty_like(o) for o in outs]
+        fd.fd_step_device(ctx.h, B, T, R, dq, dk if append else None, dv if append else None, pools, outs2, step.num_pages, dpt2, dpl2, dql,
+                          dnm, None, logits.cuda(), drafts.cuda(), acc, bon, freed, nfr)
+        assert fd.fd_last_device_status(ctx.h) == 0
+        assert all(torch.equal(a, b) for a, b in zip(outs, outs2))
+        np.testing.assert_array_equal(dpt2.cpu().numpy(), ept); np.testing.assert_array_equal(acc.cpu().numpy(), e_acc)
+
+
 def test_host_buffer_step_matches_oracle():
     """fd_step_host: a whole 3-layer step from pinned host buffers (copies pipelined inside the library)."""
     shape = wl.Shape(32, 8, 128, 5000, n_layers=3)
