@@ -212,7 +212,8 @@ fd_status fd_step_device(fd_ctx* ctx, int batch, int total_q_rows, int total_can
  * the calls are back to back, as the layers of a benchmark step are, or as they are where everything between two
  * attention calls is itself ordered before the first of them.  The library then knows that the launch before a call is its own, and what that launch writes: see
  * fd_plan_pin (attention calls read q and the cache ahead, fd_kv_append copies under the tail of the attention call
- * before it) and fd_verify_accept (its sweep runs under the tail of the last attention call).  Off, every call
+ * before it) and fd_verify_accept (its sweep, like those of fd_verify_accept_sample and fd_draft_select, runs under
+ * the tail of the attention call right before it).  Off, every call
  * waits for the launch before it before it reads anything but the pinned plan, the lengths and the page table: a
  * kernel of the caller's between two calls may then be any kernel, one that releases its dependents early included.
  * fd_step_host and fd_step_host_append, which launch nothing but this library's kernels, behave as if it were on.

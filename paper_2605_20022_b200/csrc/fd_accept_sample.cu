@@ -216,6 +216,8 @@ __global__ void __launch_bounds__(256) sv_stats_kernel(SampleParams p, int chunk
     __syncthreads();
     if (!last) return;
     __threadfence();
+    // (behind an attention call the sweep has not waited for it; this one CTA does, before the results are written)
+    if (p.chained) asm volatile("griddepcontrol.wait;" ::: "memory");
     sv_final(p);
 }
 
@@ -368,7 +370,21 @@ int launch_accept_sample(const SampleParams& p, cudaStream_t s) {
     if (p.batch == 0) return 0;
     if (p.total_rows == 0) { sv_empty_kernel<<<1, 256, 0, s>>>(p); return 1; }
     const int chunks = (p.vocab + kAcceptChunk - 1) / kAcceptChunk;
-    sv_stats_kernel<<<p.total_rows * chunks, 256, 0, s>>>(p, chunks);
+    if (!p.chained) {
+        sv_stats_kernel<<<p.total_rows * chunks, 256, 0, s>>>(p, chunks);
+    } else {
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.total_rows * chunks);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = s;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, sv_stats_kernel, p, chunks);
+}
     sv_sample_kernel<<<p.batch * chunks, 256, 0, s>>>(p, chunks);
     return 2;
 }

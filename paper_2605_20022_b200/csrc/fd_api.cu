@@ -635,6 +635,7 @@ fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, con
                                   const int32_t* draft_tokens, const int32_t* q_lens, const int32_t* n_mask, float temperature,
                                   const float* u_accept, const float* u_bonus, int32_t* accepted_len, int32_t* bonus_token,
                                   void* stream) {
+    const bool after_attn = c && c->after_attn;  // (read before it is cleared: the sweep may be chained to that call)
     if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || total_cand_rows < 0 || !(temperature > 0.f)) return FD_ERR_INVALID_ARG;
     if (batch > c->cfg.max_batch || total_cand_rows > c->max_rows) return FD_ERR_INVALID_ARG;
@@ -652,6 +653,7 @@ fd_status fd_verify_accept_sample(fd_ctx* c, int batch, int total_cand_rows, con
     p.part = c->sv_part; p.row_stat = c->sv_row; p.row_ticket = c->sv_row_ticket; p.ticket = c->sv_ticket;
     p.seq_info = c->sv_seq; p.chunk_w = c->sv_chunk_w; p.seq_ticket = c->sv_seq_ticket; p.flags = c->sv_flags;
     p.status = c->status;
+    p.chained = (after_attn && c->back_to_back) ? 1 : 0;
     c->launches += fd::launch_accept_sample(p, static_cast<cudaStream_t>(stream));
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;
 }
@@ -709,6 +711,7 @@ fd_status fd_kv_append(fd_ctx* c, int batch, int total_q_rows, const void* k_new
 fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blocks, const float* draft_logits,
                           const float* bias, const int32_t* n_mask, const int32_t* n_blocks, float threshold,
                           int32_t* mask_tokens, float* mask_probs, int32_t* keep_len, void* stream) {
+    const bool after_attn = c && c->after_attn;  // (read before it is cleared: the sweep may be chained to that call)
     if (c) { c->pin_chain = false; c->after_attn = false; }  // (not an attention or append call)
     if (!c || batch < 0 || batch > c->cfg.max_batch || total_mask_rows < 0 || total_mask_rows > c->max_rows || max_blocks < 1)
         return FD_ERR_INVALID_ARG;
@@ -722,6 +725,7 @@ fd_status fd_draft_select(fd_ctx* c, int batch, int total_mask_rows, int max_blo
     p.logits = draft_logits; p.bias = bias; p.n_mask = n_mask; p.n_blocks = n_blocks; p.threshold = threshold;
     p.tokens = mask_tokens; p.probs = mask_probs; p.keep_len = keep_len;
     p.part_key = c->ds_key; p.part_sum = c->ds_sum; p.ticket = c->ds_ticket; p.row_ticket = c->ds_row_ticket; p.status = c->status;
+    p.chained = (after_attn && c->back_to_back) ? 1 : 0;
     fd::launch_draft_select(p, static_cast<cudaStream_t>(stream));
     c->launches += 1;
     return cudaGetLastError() == cudaSuccess ? FD_OK : FD_ERR_CUDA;

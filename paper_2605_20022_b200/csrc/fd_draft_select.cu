@@ -210,6 +210,8 @@ __global__ void __launch_bounds__(256, 8) draft_select_kernel(DraftSelectParams 
     __syncthreads();
     if (!last) return;
     __threadfence();
+    // (behind an attention call the sweep has not waited for it; this one CTA does, before the call's last writes)
+    if (p.chained) asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ int m0[];  // [B+1] first mask row of each sequence
     ds_final(p, m0);
 }
@@ -226,7 +228,21 @@ void launch_draft_select(const DraftSelectParams& p, cudaStream_t s) {
     if (p.batch == 0) return;
     if (p.total_rows == 0) { draft_select_empty_kernel<<<1, 256, 0, s>>>(p); return; }
     const int chunks = (p.vocab + kAcceptChunk - 1) / kAcceptChunk;
-    draft_select_kernel<<<p.total_rows * chunks, 256, (p.batch + 1) * sizeof(int), s>>>(p, chunks);
+    if (!p.chained) {
+        draft_select_kernel<<<p.total_rows * chunks, 256, (p.batch + 1) * sizeof(int), s>>>(p, chunks);
+        return;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.total_rows * chunks);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = (p.batch + 1) * sizeof(int);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, draft_select_kernel, p, chunks);
 }
 
 }  // namespace fd

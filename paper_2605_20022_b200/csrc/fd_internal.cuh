@@ -332,6 +332,7 @@ struct DraftSelectParams {
     int32_t* tokens;
     float* probs;
     int32_t* keep_len;        // [B, max_blocks]
+    int chained;                   // 1: behind an attention call, as AcceptParams::chained (the sweep runs ahead)
     unsigned long long* part_key;  // [rows][chunks] per-chunk (max, argmax)
     float* part_sum;               // [rows][chunks] per-chunk sum of exp(x - chunk max)
     unsigned int* ticket;
@@ -378,6 +379,7 @@ struct SampleParams {
     unsigned int* seq_ticket;      // [B], zero between calls
     unsigned char* flags;          // [rows] accept test passed
     int* status;
+    int chained;                   // 1: behind an attention call, as AcceptParams::chained (the statistics sweep runs ahead)
 };
 int launch_accept_sample(const SampleParams& p, cudaStream_t s);  // returns the number of kernels launched
 

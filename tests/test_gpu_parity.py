@@ -323,6 +323,53 @@ def test_accept_then_commit_random_batches(seed):
             np.testing.assert_array_equal(pt, ept); np.testing.assert_array_equal(pl2, epl); np.testing.assert_array_equal(freed, efreed)
 
 
+def test_sweeps_right_behind_an_attention_call():
+    """With fd_calls_back_to_back on, a sweep launched right behind an attention call starts under that call's tail
+    and writes its results after it: the greedy accept, the sampling accept and the draft tail must give exactly what
+    they give on their own."""
+    step = wl.workload(2)
+    s = step.shape
+    B, T, R, Rm = step.batch, step.total_q_rows, step.total_cand_rows, int(step.n_mask.sum())
+    g = torch.Generator().manual_seed(31)
+    q, kv = wl.make_q(step).cuda(), wl.make_kv(step).cuda()
+    logits, drafts, _ = wl.make_logits(step)
+    dlg = (logits + 0.5 * torch.randn(logits.shape, generator=g)).cuda()
+    ua, ub = torch.rand((R,), generator=g).cuda(), torch.rand((B,), generator=g).cuda()
+    ml, mb = torch.randn((Rm, s.vocab), generator=g).cuda(), torch.randn((Rm, s.vocab), generator=g).cuda()
+    logits, drafts = logits.cuda(), drafts.cuda()
+    with Ctx(step) as ctx:
+        dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
+        out = torch.empty_like(q)
+        attend = lambda: fd.fd_attn_draft_verify(ctx.h, B, T, q, kv, step.num_pages, dpt, dpl, dql, dnm, out)
+        def accept():
+            a = torch.full((B,), -9, dtype=torch.int32, device="cuda"); b = torch.full_like(a, -9)
+            fd.fd_verify_accept(ctx.h, B, R, logits, drafts, dql, dnm, a, b)
+            return a, b
+        def sample():
+            a = torch.full((B,), -9, dtype=torch.int32, device="cuda"); b = torch.full_like(a, -9)
+            fd.fd_verify_accept_sample(ctx.h, B, R, logits, dlg, drafts, dql, dnm, 0.8, ua, ub, a, b)
+            return a, b
+        def tail():
+            tok = torch.full((Rm,), -9, dtype=torch.int32, device="cuda"); pr = torch.zeros((Rm,), device="cuda")
+            keep = torch.full((B, 1), -9, dtype=torch.int32, device="cuda")
+            fd.fd_draft_select(ctx.h, B, Rm, 1, ml, mb, dnm, None, 0.3, tok, pr, keep)
+            return tok, pr.view(torch.int32), keep
+        alone = [f() for f in (accept, sample, tail)]
+        torch.cuda.synchronize()
+        fd.fd_calls_back_to_back(ctx.h, True)
+        for rep in range(3):
+            behind = []
+            for f in (accept, sample, tail):
+                attend()
+                behind.append(f())
+            torch.cuda.synchronize()
+            assert fd.fd_last_device_status(ctx.h) == 0
+            for x, y in zip(alone, behind):
+                assert all(torch.equal(u, v) for u, v in zip(x, y))
+        e_acc, e_bon, _ = oracle.accept(logits.cpu(), drafts.cpu(), step.q_lens, step.n_mask)
+        np.testing.assert_array_equal(alone[0][0].cpu().numpy(), e_acc); np.testing.assert_array_equal(alone[0][1].cpu().numpy(), e_bon)
+
+
 def test_accept_bad_lengths_and_no_candidates():
     step = wl.make_step("acc", wl.Shape(4, 2, 64, 500), [5, 5], [4, 16], [0, 16], seed=3)
     logits, drafts, _ = wl.make_logits(step)
