@@ -753,7 +753,8 @@ def run_ours(args, step, rank, world, dist):
         # one small call bracketed by events measures the event pair as much as the kernel: the launch duration of a
         # small workload is the average over 36 back-to-back calls on distinct pools (CUDA-graph replay)
         attn_avg_ms = many["us_per_attn_call_cuda_graph_replay"] * 1e-3
-        how_timed = "CUDA events around 36 back-to-back calls over distinct KV pools (CUDA-graph replay), per call"
+        how_timed = ("CUDA events around 36 back-to-back calls over distinct KV pools under one pinned work list (CUDA-graph replay), per call; "
+                     "consecutive calls overlap on the device (fd_calls_back_to_back): the figure is a call inside a multi-layer step")
     achieved = attn_bytes / (attn_avg_ms * 1e-3) / 1e9
     cpu_us, cpu_desc, cores = oracle_time(step)
     return {
