@@ -884,6 +884,58 @@ def test_chained_append_whose_input_is_the_previous_output():
                 assert_close(outs[l].float().cpu().numpy(), ref, f"layer {l} rep {rep}")
 
 
+@pytest.mark.parametrize("seed", list(range(100, 130)))
+def test_random_chains_against_the_oracle(seed):
+    """Thirty seeded random batches (1 to 60 sequences, any head layout) through three layers under one pinned plan --
+    with or without the append of the block's own K/V before each attention call, with or without the caller's promise
+    that lets consecutive launches overlap -- three times over: every cache bit for bit, every output element within
+    tolerance, NaN in the output buffers beforehand."""
+    g = torch.Generator().manual_seed(seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))
+    G = [1, 2, 4, 8][ri(0, 3)]
+    Hkv = [1, 2, 4, 8][ri(0, 3)]
+    while G * Hkv > 32:
+        Hkv //= 2
+    d = [64, 128][ri(0, 1)]
+    B = [ri(1, 3), ri(4, 12), ri(13, 60)][ri(0, 2)]
+    max_rows = min(32, 128 // G)
+    pl = [[0, ri(1, 40), ri(100, 140), ri(0, 1200), ri(0, 1200)][ri(0, 4)] for _ in range(B)]
+    ql = [0 if ri(0, 11) == 0 else ri(1, max_rows) for _ in range(B)]
+    nm = [ri(0, L) for L in ql]
+    overlap, with_append = bool(ri(0, 1)), bool(ri(0, 1))
+    step = wl.make_step(f"chain{seed}", wl.Shape(G * Hkv, Hkv, d, 1000), pl, ql, nm, seed=seed, extra_table_cols=ri(0, 2))
+    T, s, L = step.total_q_rows, step.shape, 3
+    if T == 0:
+        pytest.skip("all blocks empty")
+    qs = [wl.make_q(step, l) for l in range(L)]
+    kvs = [wl.make_kv(step, l) for l in range(L)]
+    kn = [torch.randn((T, Hkv, d), generator=g).bfloat16() for _ in range(L)]
+    vn = [torch.randn((T, Hkv, d), generator=g).bfloat16() for _ in range(L)]
+    caches, refs = [], []
+    for l in range(L):
+        bits = oracle.kv_append(kn[l], vn[l], kvs[l], step.page_table, step.prefix_lens, step.q_lens) if with_append else \
+            kvs[l].view(torch.int16).numpy().view(np.uint16)
+        caches.append(bits)
+        refs.append(oracle_attn(step, qs[l], torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)))
+    with Ctx(step) as ctx:
+        fd.fd_calls_back_to_back(ctx.h, overlap)
+        dpt, dpl, dql, dnm = step.page_table.cuda(), step.prefix_lens.cuda(), step.q_lens.cuda(), step.n_mask.cuda()
+        dq, dkn, dvn = [q.cuda() for q in qs], [k.cuda() for k in kn], [v.cuda() for v in vn]
+        for rep in range(3):
+            pools = [k.cuda() for k in kvs]
+            outs = [torch.full((T, s.n_q_heads, d), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+            fd.fd_plan_pin(ctx.h, B, T, dpl, dql, dnm)
+            for l in range(L):
+                if with_append:
+                    fd.fd_kv_append(ctx.h, B, T, dkn[l], dvn[l], pools[l], step.num_pages, dpt, dpl, dql)
+                fd.fd_attn_draft_verify(ctx.h, B, T, dq[l], pools[l], step.num_pages, dpt, dpl, dql, dnm, outs[l])
+            fd.fd_plan_unpin(ctx.h)
+            assert fd.fd_last_device_status(ctx.h) == 0
+            for l in range(L):
+                np.testing.assert_array_equal(pools[l].cpu().view(torch.int16).numpy().view(np.uint16), caches[l])
+                assert_close(outs[l].float().cpu().numpy(), refs[l], f"{step.name} layer {l} rep {rep} overlap {overlap} append {with_append}")
+
+
 def test_pinned_plan_serves_every_layer_and_is_dropped_on_other_lengths():
     """fd_plan_pin: several attention calls reuse one work list; a call with other lengths recomputes it."""
     step = wl.workload(2)
