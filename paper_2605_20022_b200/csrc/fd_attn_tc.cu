@@ -57,6 +57,14 @@ constexpr int kThreads = 384;  // warps 0-3 softmax group 0, 4-7 softmax group 1
 constexpr int kKWarp = 8, kVWarp = 9, kMmaWarp = 10;  // warp 11 loads Q
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr int kEarlyLoadMaxTiles = 96;     // longest range of a CTA that starts on its KV before the previous launch has completed
+// Who issues the P V of a tile.  In a range of at least kGroupPvMinTiles tiles warp 0 of the softmax group that wrote P
+// issues it, as soon as the group's P is whole: the MMA warp, which takes its waits in program order (K tile, then the
+// P V that last read the S buffer), then never stands between a finished P and its P V (3-10 % per call from batch 8
+// upwards).  In a shorter range -- and in the cluster form, whose CTAs have one to three tiles -- the MMA warp issues
+// it: there the issue sits on the group's critical path for nothing (batch 1: +0.7 us per call when tried).
+constexpr int kGroupPvMinTiles = 6;
+template <int MODE>
+__device__ __forceinline__ bool pv_by_group(int range_tiles) { return MODE != kTcCluster && range_tiles >= kGroupPvMinTiles; }
 
 // 1: Q K^T(j) waits for the completion of the P V whose P it overwrites; 0: it does not (see mma_role).
 #ifndef FD_QK_MODE
@@ -91,7 +99,6 @@ struct Bars {
     uint64_t k_full[6], k_empty[6], v_full[6], v_empty[6];
     uint64_t s_full[2], p_full[2], pv_done[2];
     uint64_t q_full, q_free;   // Q tile of a piece landed / no longer read by any MMA
-    uint64_t all_done;         // every MMA of a piece has completed
     uint64_t o_free;           // the epilogue of a piece has read O out of TMEM
     uint64_t merge_bar;        // the other pieces of a segment have been copied into shared memory (merger, last piece)
     uint32_t tmem_base;
@@ -214,7 +221,7 @@ __device__ __forceinline__ bool wait_piece(Bars* bars, int n, volatile int* abor
 // its own copies of the running counters:
 //   g0        KV tiles pushed through the rings before this piece      (ring slot and phase)
 //   u_base[s] tiles stream s has processed before this piece           (phase of s_full / p_full / pv_done)
-//   piece     pieces before this one                                   (phase of q_full / q_free / all_done / o_free)
+//   piece     pieces before this one                                   (phase of q_full / q_free / o_free)
 // ---------------------------------------------------------------------------------------------
 struct Walk {
     int t, g0, u_base[2], piece, b;
@@ -358,6 +365,20 @@ __device__ __forceinline__ void q_role(const CUtensorMap& qmap, const AttnParams
     }
 }
 
+// A segment's ragged last tile: V rows no token owns may hold NaN or stale data -- P is 0 there, but 0 * NaN is not.
+// The warp that is about to issue the tile's P V zeroes them (the tile has landed) and fences the writes for the MMA.
+template <class C>
+__device__ __forceinline__ void zero_v_tail(unsigned char* vt, int valid, int lane) {
+    if (valid >= kTileTokens) return;
+    const int nbad = kTileTokens - valid;
+    for (int e = lane; e < nbad * 8 * C::kHalves; e += 32) {
+        const int r = valid + e / (8 * C::kHalves), wd = e % (8 * C::kHalves);
+        *reinterpret_cast<uint4*>(vt + (r >> 3) * C::kGroupBytes + (wd >> 3) * 1024 + (r & 7) * 128 + ((wd & 7) << 4)) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+}
+
 // MMA issuing warp.
 template <int D, int MODE>
 __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq, unsigned char* sk, unsigned char* sv, Bars* bars,
@@ -367,6 +388,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, kTileTokens, false);
     constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const uint32_t col_s[2] = {0u, 128u}, col_o[2] = {256u, 384u};
+    const bool group_pv = pv_by_group<MODE>(rg.e_c - rg.s_c);
     if (p.early == 1) wait_prior_launch();  // (this role touches shared and tensor memory only; p.early >= 2 lets it run ahead)
     const uint64_t qd0 = make_smem_desc(smem_u32(sq), 16, 1024);
     const int s_c = rg.s_c, e_c = rg.e_c;
@@ -376,22 +398,11 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
         if (!__all_sync(0xffffffffu, wait_piece(bars, w.piece, abort))) break;
         const Piece pc = ring[w.piece & (kDescSlots - 1)];
         if (!wait_all(&bars->q_full, w.piece & 1, abort)) break;
-        auto issue_pv = [&](int jj) {
+        auto issue_pv = [&](int jj) {  // (ranges whose P V this warp issues: see kGroupPvMinTiles)
             const int gg = w.g0 + jj, s = jj & 1, st = gg % C::kStages, u = w.u_base[s] + (jj >> 1);
             if (!wait_all(&bars->v_full[st], (gg / C::kStages) & 1, abort)) { ok = false; return; }
             unsigned char* vt = sv + st * C::kKBytes;
-            const int valid = pc.kv_len - (pc.tile0 + jj) * kTileTokens;
-            if (valid < kTileTokens) {
-                // V rows no token owns may hold NaN or stale data: P is 0 there, but 0 * NaN is not
-                const int nbad = kTileTokens - valid;
-                for (int e = lane; e < nbad * 8 * C::kHalves; e += 32) {
-                    const int r = valid + e / (8 * C::kHalves), wd = e % (8 * C::kHalves);
-                    *reinterpret_cast<uint4*>(vt + (r >> 3) * C::kGroupBytes + (wd >> 3) * 1024 + (r & 7) * 128 + ((wd & 7) << 4)) =
-                        make_uint4(0, 0, 0, 0);
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-            }
+            zero_v_tail<C>(vt, pc.kv_len - (pc.tile0 + jj) * kTileTokens, lane);
             // the first P V of a stream in a piece overwrites O: the previous piece's epilogue must have read it
             if (jj < 2 && w.piece > 0 && !wait_all(&bars->o_free, (w.piece - 1) & 1, abort)) { ok = false; return; }
             // (descriptors are made before the last wait: what follows it is the MMA instructions alone.  The address
@@ -438,11 +449,9 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, unsigned char* sq,
                 if (j == pc.nt - 1) umma_commit(&bars->q_free);  // the next piece's Q may come in
             }
             __syncwarp();
-            if (j >= 1) issue_pv(j - 1);
+            if (!group_pv && j >= 1) issue_pv(j - 1);
         }
-        if (ok) issue_pv(pc.nt - 1);
-        if (ok && lane == 0) umma_commit(&bars->all_done);
-        __syncwarp();
+        if (!group_pv && ok) issue_pv(pc.nt - 1);
         w.advance(pc);
     }
 }
@@ -638,7 +647,10 @@ __device__ __forceinline__ void merge_staged(const AttnParams& p, Bars* bars, co
 // The two softmax groups (256 threads).
 template <int D, int MODE>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, float* ex, int* s_cs, const CtaStarts cs, const Piece* ring,
-                                             uint32_t tmem, const Range rg, const Exchange<D> exch, int cl_rank, unsigned char* stage, volatile int* abort) {
+                                             uint32_t tmem, const Range rg, const Exchange<D> exch, int cl_rank, unsigned char* stage,
+                                             unsigned char* sv, volatile int* abort) {
+    using C = Cfg<D, MODE>;
+    constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     const int s_c = rg.s_c, e_c = rg.e_c;
     const int s = warp >> 2;                  // stream
@@ -656,6 +668,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
     // worked through meanwhile -- tensor and shared memory only -- and the wait comes before its ticket and epilogue
     if (p.early == 1) wait_prior_launch();
     bool prior_done = p.early < 2;
+    const bool group_pv = pv_by_group<MODE>(e_c - s_c);
     Walk w = {s_c, 0, {0, 0}, 0, 0};
     while (w.t < e_c) {
         // one thread waits for the descriptor, so that all 256 take the same decision
@@ -755,6 +768,29 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
             tc_fence_before();
             mbar_arrive(&bars->p_full[s]);
             if ((warp & 3) == 0 && lane == 0 && n_idle_threads) mbar_arrive_cnt(&bars->p_full[s], n_idle_threads);
+            if ((warp & 3) == 0 && group_pv) {
+                // ---- P V of this tile, issued by warp 0 of the group itself as soon as the group's P is whole: the MMA
+                //      warp issues Q K^T only and never stands between a finished P and its P V
+                const int gg = w.g0 + j, st = gg % C::kStages;
+                unsigned char* vt = sv + st * C::kKBytes;
+                if (!wait_all(&bars->v_full[st], (gg / C::kStages) & 1, abort)) { ok = false; break; }
+                zero_v_tail<C>(vt, pc.kv_len - (pc.tile0 + j) * kTileTokens, lane);
+                // the first P V of a stream in a piece overwrites O: the previous piece's epilogue (both groups) must have read it
+                if (j < 2 && w.piece > 0 && !wait_all(&bars->o_free, (w.piece - 1) & 1, abort)) { ok = false; break; }
+                // (the address field of a descriptor is its low 14 bits, in 16-byte units, so a K step is an addition)
+                const uint64_t vd0 = make_smem_desc(smem_u32(vt), 1024, C::kGroupBytes);
+                if (!wait_all(&bars->p_full[s], u & 1, abort)) { ok = false; break; }
+                tc_fence_after();
+                if (lane == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < kTileTokens / 16; ++kk)
+                        // one page per K step: its two 8-token groups lie kGroupBytes apart, the two halves of d 1 KB apart
+                        umma_ts(tmem + col_o[s], tmem + col_s[s] + kk * 8, vd0 + (uint64_t)((kk * C::kPageBytes) >> 4), idesc_pv, j >= 2 || kk > 0);
+                    umma_commit(&bars->v_empty[st]);
+                    umma_commit(&bars->pv_done[s]);
+                }
+                __syncwarp();
+            }
         }
 
         // ---- epilogue: merge the two streams, then final rows, or a partial plus -- if this CTA is the
@@ -778,7 +814,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Bars* bars, fl
                 ticket = atomicAdd(seg_cnt, 1);
             }
         }
-        if (warp_active) ok = ok && wait_all(&bars->all_done, w.piece & 1, abort);
+        if (warp_active) {  // every P V of the piece has completed: the last one of each stream
+            ok = ok && wait_all(&bars->pv_done[0], (w.u_base[0] + ((pc.nt + 1) >> 1) - 1) & 1, abort);
+            if (pc.nt >= 2) ok = ok && wait_all(&bars->pv_done[1], (w.u_base[1] + (pc.nt >> 1) - 1) & 1, abort);
+        }
         tc_fence_after();
         const bool two = pc.nt >= 2;
         // Stream exchange: group 1 hands its (m, l) to group 0, which answers with the two scale factors.
@@ -1056,7 +1095,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         }
         mbar_init(&bars->q_full, 1);
         mbar_init(&bars->q_free, 1);
-        mbar_init(&bars->all_done, 1);
         mbar_init(&bars->o_free, 256);
         mbar_init(&bars->merge_bar, 1);
         bars->abort = 0;
@@ -1174,7 +1212,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168, what the launch allocated: the increase is served exactly by what
         // the decrease released (a request for more than that does not return).
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, exch, cl_rank, sq, abort);
+        softmax_role<D, MODE>(p, bars, ex, s_cs, cs, ring, tmem, rg, exch, cl_rank, sq, sv, abort);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         if (warp == kKWarp) load_role<D, MODE>(tmap, p, n_rb, sk, bars->k_full, bars->k_empty, 0, rg, &bars->k_full[0], &bars->bad, abort);
