@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 
 # DRAM bytes (read + write) of ONE attention-kernel launch on the long-context workload, from the ncu capture
 # summarised in profiles/attn_tc_and_accept_kernels_long_context_1layer.md
-# (dram__bytes_read.sum 2 154 089 216 + dram__bytes_write.sum 7 275 264; one layer = one full-size launch).
-NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_161_364_480}
+# (dram__bytes_read.sum 2 154 497 024 + dram__bytes_write.sum 7 547 648; one layer = one full-size launch).
+NCU_TRAFFIC_BYTES = {"qwen3_8b_b16_prefix32768_36layers": 2_162_044_672}
 
 METRIC = "draft-verify attn+accept us/step"
 UNIT = "us/step"
