@@ -62,7 +62,10 @@ constexpr int kEarlyLoadMaxTiles = 96;     // longest range of a CTA that starts
 // P V that last read the S buffer), then never stands between a finished P and its P V (3-10 % per call from batch 8
 // upwards).  In a shorter range -- and in the cluster form, whose CTAs have one to three tiles -- the MMA warp issues
 // it: there the issue sits on the group's critical path for nothing (batch 1: +0.7 us per call when tried).
-constexpr int kGroupPvMinTiles = 6;
+#ifndef FD_GROUP_PV_MIN_TILES
+#define FD_GROUP_PV_MIN_TILES 6
+#endif
+constexpr int kGroupPvMinTiles = FD_GROUP_PV_MIN_TILES;
 template <int MODE>
 __device__ __forceinline__ bool pv_by_group(int range_tiles) { return MODE != kTcCluster && range_tiles >= kGroupPvMinTiles; }
 
