@@ -346,9 +346,9 @@ fd_status fd_verify_accept(fd_ctx* ctx, int batch, int total_cand_rows,
                            int32_t* accepted_len, int32_t* bonus_token, void* stream);
 
 /*
- * Verification at temperature > 0 by speculative sampling (Sec. 3: a draft is accepted according to the
- * ratio between the target distribution p and the drafter distribution q; at the first rejected position
- * the bonus token is drawn from the residual target distribution; committed length = accepted + 1).
+ * Verification at temperature > 0 by speculative sampling (Sec. 3: whether a draft is kept depends on how
+ * the target's probability p of the drafted token compares with the drafter's q; where the first draft is
+ * dropped, the bonus token is drawn from what is left of p once q is taken out; committed length = accepted + 1).
  * Rows and draft_tokens as in fd_verify_accept.  With p_j = softmax(logits[row j] / T) and q_j =
  * softmax(draft_logits[row j] / T), draft j + 1 = x is accepted iff u_accept[row j] < min(1, p_j(x) / q_j(x));
  * rejected at j: bonus ~ max(0, p_j - q_j) normalised; all k accepted: bonus ~ p_k.  A token is drawn from
